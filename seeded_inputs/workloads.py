@@ -1,0 +1,139 @@
+"""Workload descriptions: tensor shapes, layer lists and seeded weights.
+
+A model is a list of `Layer` records.  The records only *name* what each layer is
+(kind, filter size, strides, padding mode, activation, output channels); what an op
+computes, and how output sizes follow from input sizes, is decided independently by the
+oracle and by the CUDA library.
+
+Value distributions:
+  * inputs: uniform on a half-open interval;
+  * filters: He-normal, std = sqrt(2 / fan_in) with fan_in = fh*fw*Cin for a conv,
+    fh*fw for a depthwise filter (one input channel feeds each output), K for a dense layer;
+  * biases: N(0, 0.01^2) (BatchNorm is taken as already folded into the bias).
+Tensors of one config are drawn from one seed in a fixed order: stream 0 is the input,
+then layer i uses stream 2*i+1 for its filter and 2*i+2 for its bias.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List, Optional, Tuple
+
+import numpy as np
+
+from .generator import normal, uniform
+
+# layer kinds
+CONV2D = "conv2d"
+DEPTHWISE = "depthwise_conv2d"
+GLOBAL_AVG_POOL = "global_avg_pool"
+DENSE = "dense"
+SOFTMAX = "softmax"
+
+CONFIG_SEEDS = {
+    "matmul512": 1901,
+    "separable_block": 5350,
+    "mobilenet_025_128": 2019,
+    "mobilenet_100_224": 224,
+    "mobilenet_100_224_b128": 128,
+}
+
+
+@dataclass
+class Layer:
+    kind: str
+    filter_hw: Tuple[int, int] = (1, 1)
+    strides: Tuple[int, int] = (1, 1)
+    dilations: Tuple[int, int] = (1, 1)
+    pad: str = "same"  # 'same' | 'valid'
+    act: str = "none"  # 'none' | 'relu' | 'relu6'
+    out_channels: int = 0  # conv2d / dense: Cout ; depthwise: channel multiplier
+    name: str = ""
+    filter: Optional[np.ndarray] = None
+    bias: Optional[np.ndarray] = None
+
+
+_PW_WIDTHS = (64, 128, 128, 256, 256, 512, 512, 512, 512, 512, 512, 1024, 1024)
+_DW_STRIDES = (1, 2, 1, 2, 1, 2, 1, 1, 1, 1, 1, 2, 1)
+
+
+def mobilenet_v1_layers(alpha: float, classes: int = 1000) -> List[Layer]:
+    """MobileNet-v1-style layer list: stem 3x3/2, 13 x (dw 3x3, pw 1x1), pool, dense, softmax."""
+    layers = [
+        Layer(CONV2D, (3, 3), (2, 2), (1, 1), "same", "relu6", int(32 * alpha), "stem")
+    ]
+    for i, (width, stride) in enumerate(zip(_PW_WIDTHS, _DW_STRIDES), start=1):
+        layers.append(
+            Layer(DEPTHWISE, (3, 3), (stride, stride), (1, 1), "same", "relu6", 1, f"dw{i}")
+        )
+        layers.append(
+            Layer(CONV2D, (1, 1), (1, 1), (1, 1), "same", "relu6", int(width * alpha), f"pw{i}")
+        )
+    layers.append(Layer(GLOBAL_AVG_POOL, name="pool"))
+    layers.append(Layer(DENSE, out_channels=classes, name="dense"))
+    layers.append(Layer(SOFTMAX, name="softmax"))
+    return layers
+
+
+def layer_channels(layers: List[Layer], in_channels: int) -> List[Tuple[int, int]]:
+    """(Cin, Cout) of every layer, by following the channel count through the list."""
+    out = []
+    c = in_channels
+    for layer in layers:
+        if layer.kind in (CONV2D, DENSE):
+            out.append((c, layer.out_channels))
+            c = layer.out_channels
+        elif layer.kind == DEPTHWISE:
+            out.append((c, c * layer.out_channels))
+            c = c * layer.out_channels
+        else:
+            out.append((c, c))
+    return out
+
+
+def make_model_weights(layers: List[Layer], in_channels: int, seed: int) -> List[Layer]:
+    """Fill `filter` / `bias` of every weighted layer from the seed (see module docstring)."""
+    chans = layer_channels(layers, in_channels)
+    for i, (layer, (cin, cout)) in enumerate(zip(layers, chans)):
+        fs, bs = 2 * i + 1, 2 * i + 2
+        fh, fw = layer.filter_hw
+        if layer.kind == CONV2D:
+            std = float(np.sqrt(2.0 / (fh * fw * cin)))
+            layer.filter = normal(seed, fs, (fh, fw, cin, cout), 0.0, std)
+            layer.bias = normal(seed, bs, (cout,), 0.0, 0.01)
+        elif layer.kind == DEPTHWISE:
+            std = float(np.sqrt(2.0 / (fh * fw)))
+            layer.filter = normal(seed, fs, (fh, fw, cin, layer.out_channels), 0.0, std)
+            layer.bias = normal(seed, bs, (cout,), 0.0, 0.01)
+        elif layer.kind == DENSE:
+            std = float(np.sqrt(2.0 / cin))
+            layer.filter = normal(seed, fs, (cin, cout), 0.0, std)
+            layer.bias = normal(seed, bs, (cout,), 0.0, 0.01)
+    return layers
+
+
+def config_matmul(size: int = 512, seed: Optional[int] = None):
+    """Config 1: A[size,size] x B[size,size], entries uniform[-1,1), no transpose."""
+    seed = CONFIG_SEEDS["matmul512"] if seed is None else seed
+    a = uniform(seed, 0, (size, size), -1.0, 1.0)
+    b = uniform(seed, 1, (size, size), -1.0, 1.0)
+    return a, b
+
+
+def config_separable_block(hw: int = 112, cin: int = 32, cout: int = 64, batch: int = 1,
+                           seed: Optional[int] = None):
+    """Config 2: x[b,hw,hw,cin] ~ U[0,6); dw 3x3 s1 'same' + bias + relu6; pw 1x1 + bias + relu6."""
+    seed = CONFIG_SEEDS["separable_block"] if seed is None else seed
+    x = uniform(seed, 0, (batch, hw, hw, cin), 0.0, 6.0)
+    layers = [
+        Layer(DEPTHWISE, (3, 3), (1, 1), (1, 1), "same", "relu6", 1, "dw"),
+        Layer(CONV2D, (1, 1), (1, 1), (1, 1), "same", "relu6", cout, "pw"),
+    ]
+    make_model_weights(layers, cin, seed)
+    return x, layers
+
+
+def config_mobilenet(alpha: float, hw: int, batch: int, seed: int, classes: int = 1000):
+    """Configs 3-5: MobileNet-v1-style model, input [batch,hw,hw,3] ~ U[-1,1)."""
+    x = uniform(seed, 0, (batch, hw, hw, 3), -1.0, 1.0)
+    layers = make_model_weights(mobilenet_v1_layers(alpha, classes), 3, seed)
+    return x, layers
