@@ -1,0 +1,206 @@
+/*
+ * tfjsb — op kernels and a small graph executor for a TensorFlow.js-style inference path,
+ * written for NVIDIA B200 (sm_100a).  C ABI of libtfjsb.so.
+ *
+ * The op list follows the ops API of "TensorFlow.js: Machine Learning for the Web and
+ * Beyond" (arxiv 1901.05350): operations are device-independent calls that dispatch to
+ * device kernels (Sec. 3.3); tf.matMul and tf.conv2d are the ops the paper names
+ * (Sec. 3.6, Sec. 4.1, Listing 2); the model the paper times is MobileNet v1 (Table 1,
+ * Sec. 3.9), which also needs depthwiseConv2d, the fused bias + relu/relu6 epilogue,
+ * avgPool and softmax.  The paper does not define those ops' arithmetic; this library
+ * follows TensorFlow's definitions (cross-correlation, NHWC, HWIO filters, 'same' padding
+ * with the odd element after, avgPool dividing by the in-bounds count).
+ *
+ * Conventions shared by every call
+ *   Tensors   fp32, dense, row-major, last dimension contiguous; 4-D tensors are NHWC.
+ *             `tfjsb_tensor.data` is a DEVICE pointer unless a parameter says "host".
+ *             It must be 16-byte aligned.  The caller owns every tensor it passes; `out`
+ *             must be pre-allocated with exactly the inferred shape and must not alias an
+ *             input (tensors are immutable, ops are functional: Sec. 3.7).
+ *             A reshape is the caller changing `rank`/`dims` over the same `data`
+ *             (reshape is free: Sec. 3.4).
+ *   Async     Every op enqueues its kernels on `stream` (a cudaStream_t passed as void*;
+ *             NULL = the legacy default stream) and returns without synchronising, like
+ *             the paper's ops returning a handle before the GPU is done (Sec. 4.1.1).
+ *             Results are valid once the caller synchronises the stream.
+ *   Errors    Every call returns a tfjsb_status.  All argument checks happen on the host
+ *             before anything is launched; on error nothing has been enqueued.
+ *             `tfjsb_last_error` gives a message for the last failing call on that context
+ *             (valid until the next call on the context).  No CPU fallback exists: with no
+ *             usable CUDA device `tfjsb_init` fails with TFJSB_ERR_CUDA.
+ *   Threads   A context may be used from one host thread at a time.
+ */
+#ifndef TFJSB_H_
+#define TFJSB_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tfjsb_ctx tfjsb_ctx;
+typedef struct tfjsb_model tfjsb_model;
+
+typedef struct {
+    void* data;      /* device pointer to fp32 elements, 16-byte aligned */
+    int32_t rank;    /* 1..4 */
+    int64_t dims[4]; /* dims[0..rank-1]; the rest ignored */
+} tfjsb_tensor;
+
+typedef enum {
+    TFJSB_OK = 0,
+    TFJSB_ERR_INVALID_ARG = 1, /* null pointer, bad enum, bad rank, misaligned pointer, aliasing */
+    TFJSB_ERR_SHAPE = 2,       /* dimensions inconsistent with each other or with `out` */
+    TFJSB_ERR_UNSUPPORTED = 3, /* valid in principle, not implemented (e.g. stride>1 with dilation>1) */
+    TFJSB_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed; message holds the CUDA error */
+    TFJSB_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up (reported by tfjsb_check_device_status) */
+    TFJSB_ERR_OOM = 6          /* device allocation failed */
+} tfjsb_status;
+
+typedef enum { TFJSB_PAD_VALID = 0, TFJSB_PAD_SAME = 1 } tfjsb_pad;
+typedef enum { TFJSB_ACT_NONE = 0, TFJSB_ACT_RELU = 1, TFJSB_ACT_RELU6 = 2 } tfjsb_act;
+
+/* Which multiplier the GEMM-shaped ops (matMul, conv2d, dense) use.
+ *   TF32  tensor cores (tcgen05, operands read as TF32, fp32 accumulation in tensor memory)
+ *         wherever the shape allows, CUDA cores otherwise.  Default.
+ *   FP32  CUDA-core FFMA everywhere: the variant kept for exactness checks. */
+typedef enum { TFJSB_MATH_TF32 = 0, TFJSB_MATH_FP32 = 1 } tfjsb_math;
+
+/* ---- context ------------------------------------------------------------------------ */
+
+/* Creates a context on CUDA device `device` (makes it current for the calling thread).
+ * Allocates a small device status word and, lazily, scratch memory for transposes.
+ * Fails with TFJSB_ERR_CUDA when there is no such device or it is not compute capability 10.x. */
+tfjsb_status tfjsb_init(int device, tfjsb_ctx** ctx);
+/* Synchronises the device, frees everything the context owns.  Models must be destroyed first. */
+tfjsb_status tfjsb_shutdown(tfjsb_ctx* ctx);
+tfjsb_status tfjsb_set_math(tfjsb_ctx* ctx, tfjsb_math mode);
+const char* tfjsb_last_error(tfjsb_ctx* ctx);
+/* Synchronises `stream`, then reads the device status word that kernels with bounded waits
+ * write.  Returns TFJSB_ERR_TIMEOUT (and clears the word) if any wait gave up since the last
+ * check, TFJSB_OK otherwise. */
+tfjsb_status tfjsb_check_device_status(tfjsb_ctx* ctx, void* stream);
+/* Number of kernels this context (and its models) has launched since creation. */
+int64_t tfjsb_launch_count(tfjsb_ctx* ctx);
+
+/* ---- shape inference (pure host arithmetic) ------------------------------------------ */
+
+/* One spatial dimension of a convolution or pooling window.
+ *   ek = (k-1)*dilation + 1
+ *   VALID: out = floor((in - ek)/stride) + 1, no padding; in < ek is TFJSB_ERR_SHAPE
+ *   SAME : out = ceil(in/stride); total = max((out-1)*stride + ek - in, 0);
+ *          pad_before = floor(total/2); pad_after = total - pad_before.
+ * Any of out / pad_before / pad_after may be NULL. */
+tfjsb_status tfjsb_window_out_shape(int64_t in, int k, int stride, int dilation, tfjsb_pad pad,
+                                    int64_t* out, int* pad_before, int* pad_after);
+
+/* ---- ops ---------------------------------------------------------------------------- */
+
+/* tf.matMul (Sec. 3.6; Listing 2 is the no-transpose case).
+ *   out[M,N] = op(a) . op(b);  a is [M,K], or [K,M] when transpose_a; b is [K,N], or [N,K]
+ *   when transpose_b.  Rank 2 only.  Inner-dimension or `out` mismatch: TFJSB_ERR_SHAPE.
+ * TF32 mode uses the tensor-core kernel when K % 4 == 0 and N % 4 == 0 (row pitches must be
+ * multiples of 16 bytes for the bulk tensor copies); operands that are not already K-contiguous
+ * are transposed into context-owned scratch first.  Other shapes, and FP32 mode, run on CUDA cores. */
+tfjsb_status tfjsb_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_tensor* b, int transpose_a,
+                          int transpose_b, tfjsb_tensor* out, void* stream);
+
+/* tf.conv2d with an optional fused bias and activation.
+ *   x [N,H,W,Cin], filter [fh,fw,Cin,Cout], bias NULL or [Cout], out [N,Ho,Wo,Cout]
+ *   out[n,oy,ox,co] = act( bias[co] + sum_{ky,kx,ci} x[n, oy*sh - pt + ky*dh, ox*sw - pl + kx*dw, ci]
+ *                                                  * filter[ky,kx,ci,co] ),   outside the image = 0
+ *   strides = {sh, sw}, dilations = {dh, dw}; Ho/Wo/pt/pl from tfjsb_window_out_shape.
+ * A stride > 1 together with a dilation > 1 is TFJSB_ERR_UNSUPPORTED.
+ * 1x1 / stride 1 filters run as a GEMM over x viewed as [N*H*W, Cin]. */
+tfjsb_status tfjsb_conv2d(tfjsb_ctx* ctx, const tfjsb_tensor* x, const tfjsb_tensor* filter, const int strides[2],
+                          tfjsb_pad pad, const int dilations[2], const tfjsb_tensor* bias, tfjsb_act act,
+                          tfjsb_tensor* out, void* stream);
+
+/* tf.depthwiseConv2d with an optional fused bias and activation.
+ *   x [N,H,W,C], filter [fh,fw,C,mult], bias NULL or [C*mult], out [N,Ho,Wo,C*mult]
+ *   out[n,oy,ox,c*mult+q] = act( bias[c*mult+q] + sum_{ky,kx} x[n,iy,ix,c] * filter[ky,kx,c,q] )
+ * Always fp32 CUDA-core arithmetic (not a dense contraction).  Same stride/dilation rule as conv2d. */
+tfjsb_status tfjsb_depthwise_conv2d(tfjsb_ctx* ctx, const tfjsb_tensor* x, const tfjsb_tensor* filter,
+                                    const int strides[2], tfjsb_pad pad, const int dilations[2],
+                                    const tfjsb_tensor* bias, tfjsb_act act, tfjsb_tensor* out, void* stream);
+
+/* tf.avgPool.  x [N,H,W,C] -> out [N,Ho,Wo,C]; each output is the sum of the in-bounds
+ * window elements divided by their number (padding never counts). */
+tfjsb_status tfjsb_avg_pool(tfjsb_ctx* ctx, const tfjsb_tensor* x, const int filter_size[2], const int strides[2],
+                            tfjsb_pad pad, tfjsb_tensor* out, void* stream);
+
+/* tf.softmax over the last dimension of a rank 1..4 tensor:
+ *   out[..., j] = exp(x[..., j] - max_j x) / sum_k exp(x[..., k] - max_j x). */
+tfjsb_status tfjsb_softmax(tfjsb_ctx* ctx, const tfjsb_tensor* logits, tfjsb_tensor* out, void* stream);
+
+/* The elementwise epilogue on its own (the paper's elementwise shader, Fig. 3):
+ *   out[..., c] = act(x[..., c] + bias[c]);  bias NULL or [last dim].
+ *   relu(v) = v > 0 ? v : +0 (so -0 -> +0), NaN stays NaN; relu6(v) = min(relu(v), 6).
+ * One fp32 add and one clamp per element: results are bit-identical to the definition. */
+tfjsb_status tfjsb_bias_act(tfjsb_ctx* ctx, const tfjsb_tensor* x, const tfjsb_tensor* bias, tfjsb_act act,
+                            tfjsb_tensor* out, void* stream);
+
+/* ---- models ------------------------------------------------------------------------- */
+
+typedef enum {
+    TFJSB_LAYER_CONV2D = 0,          /* filter [fh,fw,Cin,out_channels] */
+    TFJSB_LAYER_DEPTHWISE_CONV2D = 1,/* filter [fh,fw,C,out_channels] (out_channels = channel multiplier) */
+    TFJSB_LAYER_AVG_POOL = 2,        /* filter_hw = window; {0,0} = global pool ('valid', window = H x W),
+                                        whose output is viewed as [N, C] */
+    TFJSB_LAYER_DENSE = 3,           /* input viewed as [N, K]; filter [K,out_channels]; bias; act */
+    TFJSB_LAYER_SOFTMAX = 4
+} tfjsb_layer_kind;
+
+typedef struct {
+    int32_t kind;          /* tfjsb_layer_kind */
+    int32_t filter_hw[2];
+    int32_t strides[2];
+    int32_t dilations[2];
+    int32_t pad;           /* tfjsb_pad */
+    int32_t act;           /* tfjsb_act */
+    int32_t out_channels;
+    const float* filter;   /* HOST pointer, copied (and re-laid out) at model creation; NULL for pool/softmax */
+    const float* bias;     /* HOST pointer or NULL */
+} tfjsb_layer_desc;
+
+/* Builds an executor for a straight-line model: shape inference for every layer, weights
+ * copied to the device (1x1-conv and dense filters are also stored K-contiguous for the
+ * tensor-core kernel), one arena for all intermediates (two ping-pong regions, reused across
+ * layers and runs, like the paper's texture recycler, Sec. 4.1.2), tensor maps encoded once.
+ * `input_dims` is the NHWC input shape; the batch size is fixed per model.
+ * The math mode in force on `ctx` at creation is baked into the model. */
+tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, int n_layers,
+                                const int64_t input_dims[4], tfjsb_model** model);
+tfjsb_status tfjsb_model_destroy(tfjsb_model* model);
+/* Shape of the model's final output. */
+tfjsb_status tfjsb_model_output_shape(tfjsb_model* model, int32_t* rank, int64_t dims[4]);
+/* Number of kernels one run launches. */
+int32_t tfjsb_model_launches_per_run(tfjsb_model* model);
+
+/* Runs every layer in order on `stream` and returns without synchronising (Sec. 4.1.1).
+ * `input` and `output` are device tensors with the model's input / output shapes. */
+tfjsb_status tfjsb_run_model(tfjsb_model* model, const tfjsb_tensor* input, tfjsb_tensor* output, void* stream);
+
+/* The same run from HOST memory: copies `host_input` (input-shape fp32, ideally pinned) to the
+ * device, runs the model, copies the output to `host_output`, all on `stream`, and
+ * synchronises the stream before returning (the blocking dataSync() of Sec. 3.6). */
+tfjsb_status tfjsb_run_model_host(tfjsb_model* model, const float* host_input, float* host_output, void* stream);
+
+/* Debug aid (the paper's debug mode downloads every intermediate, Sec. 3.8): a view of the
+ * output of layer `layer` as left by the last run.  With the ping-pong arena only the most
+ * recent layers survive a full run, so call tfjsb_model_set_keep_all(model, 1) before the run
+ * to give every layer its own buffer. */
+tfjsb_status tfjsb_model_set_keep_all(tfjsb_model* model, int keep_all);
+tfjsb_status tfjsb_model_layer_output(tfjsb_model* model, int layer, tfjsb_tensor* view);
+
+/* Per-layer device timing (the paper's per-kernel profile, Sec. 3.8): runs the model `reps`
+ * times with a CUDA event pair around every layer, synchronises, and writes the mean
+ * milliseconds per layer into ms_per_layer[0..n_layers-1] (host). */
+tfjsb_status tfjsb_model_profile(tfjsb_model* model, const tfjsb_tensor* input, tfjsb_tensor* output, int reps,
+                                 float* ms_per_layer, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TFJSB_H_ */

@@ -1,0 +1,120 @@
+// Shared declarations of the CUDA library: context, error helpers, the fused epilogue,
+// and the host-side launchers each kernel file exports to the API layer.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <stdint.h>
+
+#include <string>
+
+#include "tfjsb.h"
+
+namespace tfjsb {
+
+// ---- device status word -------------------------------------------------------------------
+// Kernels with bounded waits OR a code into this word when a wait gives up; the host reads it
+// in tfjsb_check_device_status.
+enum : unsigned int {
+    DEV_STATUS_OK = 0u,
+    DEV_STATUS_TIMEOUT_PRODUCER = 1u,  // TMA producer waited too long for a free stage
+    DEV_STATUS_TIMEOUT_MMA = 2u,       // MMA issuer waited too long for data or for a free accumulator
+    DEV_STATUS_TIMEOUT_EPILOGUE = 4u,  // epilogue waited too long for an accumulator
+    DEV_STATUS_TIMEOUT_DRAIN = 8u      // teardown waited too long for copies in flight
+};
+
+// ---- fused epilogue (bias add, then activation), identical in every kernel -----------------
+//   v = acc + bias ; relu: v > 0 ? v : +0 (NaN stays NaN) ; relu6: min(relu(v), 6)
+__device__ __forceinline__ float apply_act(float v, int act) {
+    if (act == TFJSB_ACT_NONE) return v;
+    if (v != v) return v;
+    float r = v > 0.0f ? v : 0.0f;
+    if (act == TFJSB_ACT_RELU6) r = r > 6.0f ? 6.0f : r;
+    return r;
+}
+
+// ---- context --------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct Scratch {
+    float* ptr = nullptr;
+    size_t bytes = 0;
+};
+
+}  // namespace tfjsb
+
+struct tfjsb_ctx {
+    int device = 0;
+    int sm_count = 0;
+    tfjsb_math math = TFJSB_MATH_TF32;
+    std::string last_error;
+    unsigned int* dev_status = nullptr;  // device status word
+    tfjsb::EncodeTiledFn encode_tiled = nullptr;
+    tfjsb::Scratch scratch_a, scratch_b;  // transposed operands of tfjsb_matmul
+    int64_t launches = 0;
+    int live_models = 0;
+};
+
+namespace tfjsb {
+
+tfjsb_status fail(tfjsb_ctx* ctx, tfjsb_status st, const std::string& msg);
+tfjsb_status cuda_fail(tfjsb_ctx* ctx, cudaError_t err, const char* what);
+// Grows `s` to at least `bytes` (frees and reallocates; callers keep stream order in mind).
+tfjsb_status ensure_scratch(tfjsb_ctx* ctx, Scratch* s, size_t bytes);
+
+// ---- geometry of one convolution / pooling call -----------------------------------------------
+struct ConvGeom {
+    int64_t N;
+    int H, W, C;        // input
+    int fh, fw;         // filter window
+    int Co;             // output channels (conv: Cout; depthwise: C*mult; pool: C)
+    int mult;           // depthwise channel multiplier (1 otherwise)
+    int sh, sw, dh, dw; // strides, dilations
+    int pt, pl;         // padding before (top, left)
+    int Ho, Wo;
+};
+
+// ---- launchers (each returns the CUDA launch error; `launches` is incremented per kernel) -----
+cudaError_t launch_bias_act(const float* x, const float* bias, float* y, int64_t rows, int64_t C, int act,
+                            cudaStream_t s, int64_t* launches);
+cudaError_t launch_avg_pool(const float* x, float* y, const ConvGeom& g, cudaStream_t s, int64_t* launches);
+cudaError_t launch_softmax(const float* x, float* y, int64_t rows, int64_t cols, cudaStream_t s, int64_t* launches);
+// out[c, r] = in[r, c] for in of shape [rows, cols]
+cudaError_t launch_transpose(const float* in, float* out, int64_t rows, int64_t cols, cudaStream_t s,
+                             int64_t* launches);
+
+// C[M,N] = act(A' B' + bias), CUDA-core fp32.  A' element (i,k) at a[i*a_rs + k*a_cs]; B' element
+// (k,j) at b[k*b_rs + j*b_cs]; C row pitch ldc.
+cudaError_t launch_gemm_fp32(const float* a, int64_t a_rs, int64_t a_cs, const float* b, int64_t b_rs, int64_t b_cs,
+                             const float* bias, int act, float* c, int64_t ldc, int64_t M, int64_t N, int64_t K,
+                             cudaStream_t s, int64_t* launches);
+
+// Direct convolution on CUDA cores (any window, stride, dilation).  filter [fh,fw,Cin,Cout].
+cudaError_t launch_conv2d_fp32(const float* x, const float* f, const float* bias, int act, float* y,
+                               const ConvGeom& g, cudaStream_t s, int64_t* launches);
+
+// Depthwise convolution.  filter [fh,fw,C,mult].
+cudaError_t launch_depthwise(const float* x, const float* f, const float* bias, int act, float* y,
+                             const ConvGeom& g, cudaStream_t s, int64_t* launches);
+
+// Tensor-core GEMM: C[M,N] = act(A[M,K] . Bt[N,K]^T + bias); all three row-major with K (resp. N)
+// contiguous.  A plan holds the tensor maps and tile choice; it can be built once and reused while
+// the pointers stay the same.
+struct GemmTf32Plan {
+    CUtensorMap map_a, map_b, map_c;
+    int64_t M, N, K;
+    int block_n;       // 32..256
+    int stages;
+    int num_tiles;
+    int grid;
+    size_t smem_bytes;
+};
+bool gemm_tf32_supported(int64_t M, int64_t N, int64_t K);
+tfjsb_status gemm_tf32_plan(tfjsb_ctx* ctx, const float* a, const float* bt, float* c, int64_t M, int64_t N,
+                            int64_t K, GemmTf32Plan* plan);
+cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int act, unsigned int* dev_status,
+                             cudaStream_t s, int64_t* launches);
+
+}  // namespace tfjsb

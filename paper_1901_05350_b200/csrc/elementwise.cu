@@ -1,0 +1,212 @@
+// Bandwidth-bound helpers: the standalone bias+activation op, avgPool, softmax, and the
+// 2-D transpose used to make matMul operands K-contiguous.
+#include "common.cuh"
+
+namespace tfjsb {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+inline int grid_for(int64_t work_items, int threads, int max_blocks) {
+    int64_t b = (work_items + threads - 1) / threads;
+    if (b < 1) b = 1;
+    if (b > max_blocks) b = max_blocks;
+    return (int)b;
+}
+
+// ---- bias + activation ----------------------------------------------------------------------
+// out[r, c] = act(x[r, c] + bias[c]).  float4 path: C % 4 == 0, so a float4 never straddles rows.
+__global__ void bias_act_vec4_kernel(const float4* __restrict__ x, const float* __restrict__ bias,
+                                     float4* __restrict__ y, int64_t n_vec, int C4, int act) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += stride) {
+        float4 v = x[i];
+        if (bias) {
+            const int c = (int)(i % C4) * 4;
+            const float4 b = *reinterpret_cast<const float4*>(bias + c);
+            v.x = v.x + b.x; v.y = v.y + b.y; v.z = v.z + b.z; v.w = v.w + b.w;
+        }
+        v.x = apply_act(v.x, act); v.y = apply_act(v.y, act);
+        v.z = apply_act(v.z, act); v.w = apply_act(v.w, act);
+        y[i] = v;
+    }
+}
+
+__global__ void bias_act_scalar_kernel(const float* __restrict__ x, const float* __restrict__ bias,
+                                       float* __restrict__ y, int64_t n, int64_t C, int act) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        float v = x[i];
+        if (bias) v = v + bias[i % C];
+        y[i] = apply_act(v, act);
+    }
+}
+
+// ---- avgPool ----------------------------------------------------------------------------------
+// One thread per output element, channel fastest (coalesced).  Padding never counts.
+__global__ void avg_pool_window_kernel(const float* __restrict__ x, float* __restrict__ y, ConvGeom g,
+                                       int64_t n_out) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_out; i += stride) {
+        const int c = (int)(i % g.C);
+        int64_t t = i / g.C;
+        const int ox = (int)(t % g.Wo); t /= g.Wo;
+        const int oy = (int)(t % g.Ho);
+        const int64_t n = t / g.Ho;
+        float acc = 0.0f;
+        int count = 0;
+        for (int ky = 0; ky < g.fh; ++ky) {
+            const int iy = oy * g.sh - g.pt + ky;
+            if (iy < 0 || iy >= g.H) continue;
+            for (int kx = 0; kx < g.fw; ++kx) {
+                const int ix = ox * g.sw - g.pl + kx;
+                if (ix < 0 || ix >= g.W) continue;
+                acc += x[((n * g.H + iy) * (int64_t)g.W + ix) * g.C + c];
+                ++count;
+            }
+        }
+        y[i] = acc / (float)count;
+    }
+}
+
+// Global pool: a block owns (image n, 32 consecutive channels).  Lane = channel (coalesced 128-byte
+// rows), the 8 warps stride over the H*W positions, partial sums meet in shared memory.
+__global__ void avg_pool_global_kernel(const float* __restrict__ x, float* __restrict__ y, int HW, int C) {
+    __shared__ float partial[8][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int c = blockIdx.x * 32 + lane;
+    const int64_t n = blockIdx.y;
+    float acc = 0.0f;
+    if (c < C) {
+        const float* base = x + n * (int64_t)HW * C + c;
+        for (int p = warp; p < HW; p += 8) acc += base[(int64_t)p * C];
+    }
+    partial[warp][lane] = acc;
+    __syncthreads();
+    if (warp == 0 && c < C) {
+        float s = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) s += partial[w][lane];
+        y[n * C + c] = s / (float)HW;
+    }
+}
+
+// ---- softmax ----------------------------------------------------------------------------------
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// One block (kThreads) per row: max, then sum of exp(x - max), then the quotient.
+__global__ void softmax_rows_kernel(const float* __restrict__ x, float* __restrict__ y, int64_t cols) {
+    __shared__ float red[kThreads / 32];
+    __shared__ float bcast;
+    const float* xr = x + (int64_t)blockIdx.x * cols;
+    float* yr = y + (int64_t)blockIdx.x * cols;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    float m = -INFINITY;
+    for (int64_t j = threadIdx.x; j < cols; j += kThreads) m = fmaxf(m, xr[j]);
+    m = warp_max(m);
+    if (lane == 0) red[warp] = m;
+    __syncthreads();
+    if (warp == 0) {
+        float v = lane < kThreads / 32 ? red[lane] : -INFINITY;
+        v = warp_max(v);
+        if (lane == 0) bcast = v;
+    }
+    __syncthreads();
+    m = bcast;
+
+    float sum = 0.0f;
+    for (int64_t j = threadIdx.x; j < cols; j += kThreads) sum += expf(xr[j] - m);
+    sum = warp_sum(sum);
+    __syncthreads();  // red[] and bcast are reused
+    if (lane == 0) red[warp] = sum;
+    __syncthreads();
+    if (warp == 0) {
+        float v = lane < kThreads / 32 ? red[lane] : 0.0f;
+        v = warp_sum(v);
+        if (lane == 0) bcast = v;
+    }
+    __syncthreads();
+    sum = bcast;
+
+    for (int64_t j = threadIdx.x; j < cols; j += kThreads) yr[j] = expf(xr[j] - m) / sum;
+}
+
+// ---- transpose --------------------------------------------------------------------------------
+__global__ void transpose_kernel(const float* __restrict__ in, float* __restrict__ out, int64_t rows,
+                                 int64_t cols) {
+    __shared__ float tile[32][33];
+    const int64_t c0 = (int64_t)blockIdx.x * 32, r0 = (int64_t)blockIdx.y * 32;
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        const int64_t r = r0 + j, c = c0 + threadIdx.x;
+        if (r < rows && c < cols) tile[j][threadIdx.x] = in[r * cols + c];
+    }
+    __syncthreads();
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        const int64_t c = c0 + j, r = r0 + threadIdx.x;
+        if (r < rows && c < cols) out[c * rows + r] = tile[threadIdx.x][j];
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_bias_act(const float* x, const float* bias, float* y, int64_t rows, int64_t C, int act,
+                            cudaStream_t s, int64_t* launches) {
+    const int64_t n = rows * C;
+    if (n == 0) return cudaSuccess;
+    if (C % 4 == 0) {
+        const int64_t n_vec = n / 4;
+        bias_act_vec4_kernel<<<grid_for(n_vec, kThreads, 148 * 16), kThreads, 0, s>>>(
+            reinterpret_cast<const float4*>(x), bias, reinterpret_cast<float4*>(y), n_vec, (int)(C / 4), act);
+    } else {
+        bias_act_scalar_kernel<<<grid_for(n, kThreads, 148 * 16), kThreads, 0, s>>>(x, bias, y, n, C, act);
+    }
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_avg_pool(const float* x, float* y, const ConvGeom& g, cudaStream_t s, int64_t* launches) {
+    const int64_t n_out = g.N * g.Ho * g.Wo * g.C;
+    if (n_out == 0) return cudaSuccess;
+    const bool global = g.Ho == 1 && g.Wo == 1 && g.fh == g.H && g.fw == g.W && g.pt == 0 && g.pl == 0 &&
+                        g.N <= 65535;
+    if (global) {
+        dim3 grid((g.C + 31) / 32, (unsigned)g.N);
+        avg_pool_global_kernel<<<grid, 256, 0, s>>>(x, y, g.H * g.W, g.C);
+    } else {
+        avg_pool_window_kernel<<<grid_for(n_out, kThreads, 148 * 16), kThreads, 0, s>>>(x, y, g, n_out);
+    }
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_softmax(const float* x, float* y, int64_t rows, int64_t cols, cudaStream_t s,
+                           int64_t* launches) {
+    if (rows == 0) return cudaSuccess;
+    // gridDim.x is 2^31-1: enough for any tensor that fits in memory
+    softmax_rows_kernel<<<(unsigned)rows, kThreads, 0, s>>>(x, y, cols);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_transpose(const float* in, float* out, int64_t rows, int64_t cols, cudaStream_t s,
+                             int64_t* launches) {
+    if (rows == 0 || cols == 0) return cudaSuccess;
+    dim3 grid((unsigned)((cols + 31) / 32), (unsigned)((rows + 31) / 32));
+    if (grid.y > 65535) return cudaErrorInvalidConfiguration;
+    transpose_kernel<<<grid, dim3(32, 8), 0, s>>>(in, out, rows, cols);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace tfjsb

@@ -1,0 +1,431 @@
+// Graph executor: a straight-line model (list of layer records) planned once and run as a
+// sequence of kernel launches on one stream.
+//
+// Planning (tfjsb_model_create): shape inference per layer, weights copied to the device (the
+// filters of GEMM-shaped layers are additionally stored [Cout, Cin], K-contiguous, for the
+// tensor-core kernel), one arena holding two ping-pong regions for the intermediates (a layer
+// reads one region and writes the other; the regions are reused by every run, in the spirit of
+// the paper's texture recycler, Sec. 4.1.2), tensor maps encoded once against those fixed
+// addresses.  Running (tfjsb_run_model) therefore does no allocation, no shape arithmetic and
+// no synchronisation: it enqueues the kernels and returns (Sec. 4.1.1).
+#include <vector>
+
+#include "common.cuh"
+
+using namespace tfjsb;
+
+namespace {
+
+enum StepKind { STEP_GEMM_TF32, STEP_GEMM_FP32, STEP_CONV_FP32, STEP_DEPTHWISE, STEP_POOL, STEP_SOFTMAX };
+
+struct Step {
+    StepKind kind;
+    ConvGeom g{};                // conv / depthwise / pool
+    int64_t M = 0, N = 0, K = 0;  // gemm; softmax: M rows, N cols
+    int act = TFJSB_ACT_NONE;
+    float* filter = nullptr;     // device, as given ([fh,fw,Cin,Cout] / [K,N])
+    float* filter_km = nullptr;  // device, [N,K] (tensor-core layers only)
+    float* bias = nullptr;       // device or null
+    GemmTf32Plan plan{};
+    bool plan_built = false;
+    int32_t out_rank = 4;
+    int64_t out_dims[4] = {0, 0, 0, 0};
+    int64_t out_elems = 0;
+    float* out = nullptr;        // where this layer writes (arena or, for the last layer, the caller's output)
+    const float* in = nullptr;   // where it reads (arena or, for the first layer, the caller's input)
+};
+
+}  // namespace
+
+struct tfjsb_model {
+    tfjsb_ctx* ctx = nullptr;
+    std::vector<Step> steps;
+    std::vector<float*> owned;  // every device allocation of this model
+    int64_t in_dims[4] = {0, 0, 0, 0};
+    int64_t in_elems = 0;
+    float* arena = nullptr;
+    size_t region_elems = 0;     // elements per ping-pong region
+    float* keep_all_arena = nullptr;
+    bool keep_all = false;
+    float* staged_in = nullptr;  // device copies used by tfjsb_run_model_host
+    float* staged_out = nullptr;
+    bool use_tf32 = true;
+    // caller buffers the first/last tensor maps were last encoded for
+    const void* bound_in = nullptr;
+    void* bound_out = nullptr;
+};
+
+namespace {
+
+tfjsb_status dev_alloc(tfjsb_model* m, size_t elems, float** out) {
+    *out = nullptr;
+    if (elems == 0) elems = 4;
+    cudaError_t e = cudaMalloc(out, elems * sizeof(float));
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return fail(m->ctx, TFJSB_ERR_OOM, "could not allocate " + std::to_string(elems * 4) + " bytes on the device");
+    }
+    m->owned.push_back(*out);
+    return TFJSB_OK;
+}
+
+tfjsb_status upload(tfjsb_model* m, const float* host, size_t elems, float** out) {
+    tfjsb_status st = dev_alloc(m, elems, out);
+    if (st != TFJSB_OK) return st;
+    cudaError_t e = cudaMemcpy(*out, host, elems * sizeof(float), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) return cuda_fail(m->ctx, e, "copying weights to the device");
+    return TFJSB_OK;
+}
+
+bool window(int64_t in, int k, int s, int d, int pad, int* out, int* before) {
+    int64_t o;
+    int a;
+    if (tfjsb_window_out_shape(in, k, s, d, (tfjsb_pad)pad, &o, before, &a) != TFJSB_OK) return false;
+    *out = (int)o;
+    return true;
+}
+
+// (Re)binds the addresses a step reads and writes; tensor-core plans depend on them.
+tfjsb_status bind_step(tfjsb_model* m, Step& st, const float* in, float* out) {
+    const bool changed = st.in != in || st.out != out;
+    st.in = in;
+    st.out = out;
+    if (st.kind == STEP_GEMM_TF32 && (changed || !st.plan_built)) {
+        tfjsb_status rc = gemm_tf32_plan(m->ctx, in, st.filter_km, out, st.M, st.N, st.K, &st.plan);
+        if (rc != TFJSB_OK) return rc;
+        st.plan_built = true;
+    }
+    return TFJSB_OK;
+}
+
+// Assigns buffers: layer i reads the previous layer's output; intermediates alternate between the
+// two arena regions (or get a region each in keep-all mode); the ends use the caller's tensors.
+tfjsb_status bind_all(tfjsb_model* m, const float* input, float* output) {
+    const int n = (int)m->steps.size();
+    const float* cur = input;
+    size_t keep_off = 0;
+    for (int i = 0; i < n; ++i) {
+        Step& st = m->steps[i];
+        float* dst;
+        if (i == n - 1) dst = output;
+        else if (m->keep_all) {
+            dst = m->keep_all_arena + keep_off;
+            keep_off += (size_t)((st.out_elems + 63) / 64 * 64);
+        } else dst = m->arena + (size_t)(i & 1) * m->region_elems;
+        tfjsb_status rc = bind_step(m, st, cur, dst);
+        if (rc != TFJSB_OK) return rc;
+        cur = dst;
+    }
+    m->bound_in = input;
+    m->bound_out = output;
+    return TFJSB_OK;
+}
+
+cudaError_t launch_step(tfjsb_model* m, const Step& st, cudaStream_t s) {
+    tfjsb_ctx* ctx = m->ctx;
+    switch (st.kind) {
+        case STEP_GEMM_TF32:
+            return launch_gemm_tf32(st.plan, st.bias, st.act, ctx->dev_status, s, &ctx->launches);
+        case STEP_GEMM_FP32:
+            return launch_gemm_fp32(st.in, st.K, 1, st.filter, st.N, 1, st.bias, st.act, st.out, st.N, st.M, st.N, st.K,
+                                    s, &ctx->launches);
+        case STEP_CONV_FP32:
+            return launch_conv2d_fp32(st.in, st.filter, st.bias, st.act, st.out, st.g, s, &ctx->launches);
+        case STEP_DEPTHWISE:
+            return launch_depthwise(st.in, st.filter, st.bias, st.act, st.out, st.g, s, &ctx->launches);
+        case STEP_POOL:
+            return launch_avg_pool(st.in, st.out, st.g, s, &ctx->launches);
+        case STEP_SOFTMAX:
+            return launch_softmax(st.in, st.out, st.M, st.N, s, &ctx->launches);
+    }
+    return cudaErrorUnknown;
+}
+
+tfjsb_status check_io(tfjsb_model* m, const tfjsb_tensor* input, const tfjsb_tensor* output) {
+    tfjsb_ctx* ctx = m->ctx;
+    if (!input || !output || !input->data || !output->data) return fail(ctx, TFJSB_ERR_INVALID_ARG, "input / output is null");
+    if (input->rank != 4) return fail(ctx, TFJSB_ERR_SHAPE, "input must be rank 4 (NHWC)");
+    for (int i = 0; i < 4; ++i)
+        if (input->dims[i] != m->in_dims[i]) return fail(ctx, TFJSB_ERR_SHAPE, "input shape differs from the model's");
+    const Step& last = m->steps.back();
+    if (output->rank != last.out_rank) return fail(ctx, TFJSB_ERR_SHAPE, "output rank differs from the model's");
+    for (int i = 0; i < last.out_rank; ++i)
+        if (output->dims[i] != last.out_dims[i]) return fail(ctx, TFJSB_ERR_SHAPE, "output shape differs from the model's");
+    if ((reinterpret_cast<uintptr_t>(input->data) & 15u) || (reinterpret_cast<uintptr_t>(output->data) & 15u))
+        return fail(ctx, TFJSB_ERR_INVALID_ARG, "input / output must be 16-byte aligned");
+    if (input->data == output->data) return fail(ctx, TFJSB_ERR_INVALID_ARG, "output aliases the input");
+    return TFJSB_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, int n_layers,
+                                const int64_t input_dims[4], tfjsb_model** out) {
+    if (!ctx) return TFJSB_ERR_INVALID_ARG;
+    if (!out) return fail(ctx, TFJSB_ERR_INVALID_ARG, "model out-pointer is null");
+    *out = nullptr;
+    if (!layers || n_layers < 1 || !input_dims) return fail(ctx, TFJSB_ERR_INVALID_ARG, "no layers / no input shape");
+    for (int i = 0; i < 4; ++i)
+        if (input_dims[i] < 1 || input_dims[i] > 0x3fffffff) return fail(ctx, TFJSB_ERR_SHAPE, "input dimensions must be in [1, 2^30]");
+
+    tfjsb_model* m = new tfjsb_model();
+    m->ctx = ctx;
+    m->use_tf32 = ctx->math == TFJSB_MATH_TF32 && ctx->encode_tiled != nullptr;
+    for (int i = 0; i < 4; ++i) m->in_dims[i] = input_dims[i];
+    m->in_elems = input_dims[0] * input_dims[1] * input_dims[2] * input_dims[3];
+
+    // running shape: rank 4 [N,H,W,C] or rank 2 [N,F]
+    int rank = 4;
+    int64_t d[4] = {input_dims[0], input_dims[1], input_dims[2], input_dims[3]};
+    tfjsb_status st = TFJSB_OK;
+    auto bail = [&](tfjsb_status code, const std::string& msg) {
+        fail(ctx, code, msg);
+        for (float* p : m->owned) cudaFree(p);
+        delete m;
+        return code;
+    };
+
+    for (int li = 0; li < n_layers; ++li) {
+        const tfjsb_layer_desc& L = layers[li];
+        const std::string where = "layer " + std::to_string(li) + ": ";
+        Step step;
+        step.act = L.act;
+        if (L.act != TFJSB_ACT_NONE && L.act != TFJSB_ACT_RELU && L.act != TFJSB_ACT_RELU6)
+            return bail(TFJSB_ERR_INVALID_ARG, where + "unknown activation");
+        switch (L.kind) {
+            case TFJSB_LAYER_CONV2D:
+            case TFJSB_LAYER_DEPTHWISE_CONV2D: {
+                if (rank != 4) return bail(TFJSB_ERR_SHAPE, where + "needs a rank-4 input");
+                if (!L.filter) return bail(TFJSB_ERR_INVALID_ARG, where + "filter is null");
+                if (L.filter_hw[0] < 1 || L.filter_hw[1] < 1 || L.strides[0] < 1 || L.strides[1] < 1 ||
+                    L.dilations[0] < 1 || L.dilations[1] < 1 || L.out_channels < 1)
+                    return bail(TFJSB_ERR_INVALID_ARG, where + "window, strides, dilations and out_channels must be >= 1");
+                if ((L.strides[0] > 1 || L.strides[1] > 1) && (L.dilations[0] > 1 || L.dilations[1] > 1))
+                    return bail(TFJSB_ERR_UNSUPPORTED, where + "a stride > 1 together with a dilation > 1 is not supported");
+                if (L.pad != TFJSB_PAD_VALID && L.pad != TFJSB_PAD_SAME) return bail(TFJSB_ERR_INVALID_ARG, where + "unknown padding mode");
+                const bool dw = L.kind == TFJSB_LAYER_DEPTHWISE_CONV2D;
+                ConvGeom g;
+                g.N = d[0]; g.H = (int)d[1]; g.W = (int)d[2]; g.C = (int)d[3];
+                g.fh = L.filter_hw[0]; g.fw = L.filter_hw[1];
+                g.sh = L.strides[0]; g.sw = L.strides[1]; g.dh = L.dilations[0]; g.dw = L.dilations[1];
+                g.mult = dw ? L.out_channels : 1;
+                const int64_t co = dw ? (int64_t)g.C * L.out_channels : L.out_channels;
+                if (co > 0x3fffffff) return bail(TFJSB_ERR_UNSUPPORTED, where + "too many output channels");
+                g.Co = (int)co;
+                if (!window(g.H, g.fh, g.sh, g.dh, L.pad, &g.Ho, &g.pt) || !window(g.W, g.fw, g.sw, g.dw, L.pad, &g.Wo, &g.pl))
+                    return bail(TFJSB_ERR_SHAPE, where + "the filter window does not fit the input under 'valid' padding");
+                step.g = g;
+                const size_t f_elems = (size_t)g.fh * g.fw * g.C * (dw ? g.mult : g.Co);
+                if ((st = upload(m, L.filter, f_elems, &step.filter)) != TFJSB_OK) return bail(st, ctx->last_error);
+                if (L.bias && (st = upload(m, L.bias, (size_t)g.Co, &step.bias)) != TFJSB_OK) return bail(st, ctx->last_error);
+                if (dw) step.kind = STEP_DEPTHWISE;
+                else if (g.fh == 1 && g.fw == 1 && g.sh == 1 && g.sw == 1) {
+                    step.M = g.N * g.H * g.W; step.K = g.C; step.N = g.Co;
+                    step.kind = (m->use_tf32 && gemm_tf32_supported(step.M, step.N, step.K)) ? STEP_GEMM_TF32 : STEP_GEMM_FP32;
+                } else step.kind = STEP_CONV_FP32;
+                step.out_rank = 4;
+                step.out_dims[0] = g.N; step.out_dims[1] = g.Ho; step.out_dims[2] = g.Wo; step.out_dims[3] = g.Co;
+                break;
+            }
+            case TFJSB_LAYER_AVG_POOL: {
+                if (rank != 4) return bail(TFJSB_ERR_SHAPE, where + "needs a rank-4 input");
+                const bool global = L.filter_hw[0] == 0 && L.filter_hw[1] == 0;
+                ConvGeom g;
+                g.N = d[0]; g.H = (int)d[1]; g.W = (int)d[2]; g.C = (int)d[3];
+                g.Co = g.C; g.mult = 1; g.dh = g.dw = 1;
+                if (global) {
+                    g.fh = g.H; g.fw = g.W; g.sh = g.sw = 1; g.pt = g.pl = 0; g.Ho = g.Wo = 1;
+                } else {
+                    if (L.filter_hw[0] < 1 || L.filter_hw[1] < 1 || L.strides[0] < 1 || L.strides[1] < 1)
+                        return bail(TFJSB_ERR_INVALID_ARG, where + "window and strides must be >= 1");
+                    if (L.pad != TFJSB_PAD_VALID && L.pad != TFJSB_PAD_SAME) return bail(TFJSB_ERR_INVALID_ARG, where + "unknown padding mode");
+                    g.fh = L.filter_hw[0]; g.fw = L.filter_hw[1]; g.sh = L.strides[0]; g.sw = L.strides[1];
+                    if (!window(g.H, g.fh, g.sh, 1, L.pad, &g.Ho, &g.pt) || !window(g.W, g.fw, g.sw, 1, L.pad, &g.Wo, &g.pl))
+                        return bail(TFJSB_ERR_SHAPE, where + "the pooling window does not fit the input under 'valid' padding");
+                }
+                step.kind = STEP_POOL;
+                step.g = g;
+                if (global) {
+                    step.out_rank = 2;
+                    step.out_dims[0] = g.N; step.out_dims[1] = g.C;
+                } else {
+                    step.out_rank = 4;
+                    step.out_dims[0] = g.N; step.out_dims[1] = g.Ho; step.out_dims[2] = g.Wo; step.out_dims[3] = g.C;
+                }
+                break;
+            }
+            case TFJSB_LAYER_DENSE: {
+                if (!L.filter) return bail(TFJSB_ERR_INVALID_ARG, where + "filter is null");
+                if (L.out_channels < 1) return bail(TFJSB_ERR_INVALID_ARG, where + "out_channels must be >= 1");
+                int64_t feat = 1;
+                for (int i = 1; i < rank; ++i) feat *= d[i];
+                step.M = d[0]; step.K = feat; step.N = L.out_channels;
+                if ((st = upload(m, L.filter, (size_t)(step.K * step.N), &step.filter)) != TFJSB_OK) return bail(st, ctx->last_error);
+                if (L.bias && (st = upload(m, L.bias, (size_t)step.N, &step.bias)) != TFJSB_OK) return bail(st, ctx->last_error);
+                step.kind = (m->use_tf32 && gemm_tf32_supported(step.M, step.N, step.K)) ? STEP_GEMM_TF32 : STEP_GEMM_FP32;
+                step.out_rank = 2;
+                step.out_dims[0] = step.M; step.out_dims[1] = step.N;
+                break;
+            }
+            case TFJSB_LAYER_SOFTMAX: {
+                step.kind = STEP_SOFTMAX;
+                step.N = d[rank - 1];
+                step.M = 1;
+                for (int i = 0; i < rank - 1; ++i) step.M *= d[i];
+                step.out_rank = rank;
+                for (int i = 0; i < rank; ++i) step.out_dims[i] = d[i];
+                break;
+            }
+            default:
+                return bail(TFJSB_ERR_INVALID_ARG, where + "unknown layer kind");
+        }
+        if (step.kind == STEP_GEMM_TF32) {
+            // weights [K,N] -> [N,K] once, on the device
+            if ((st = dev_alloc(m, (size_t)(step.K * step.N), &step.filter_km)) != TFJSB_OK) return bail(st, ctx->last_error);
+            cudaError_t e = launch_transpose(step.filter, step.filter_km, step.K, step.N, 0, &ctx->launches);
+            if (e != cudaSuccess) return bail(TFJSB_ERR_CUDA, std::string("transposing weights: ") + cudaGetErrorString(e));
+        }
+        step.out_elems = 1;
+        for (int i = 0; i < step.out_rank; ++i) step.out_elems *= step.out_dims[i];
+        rank = step.out_rank;
+        for (int i = 0; i < 4; ++i) d[i] = i < rank ? step.out_dims[i] : 0;
+        m->steps.push_back(step);
+    }
+
+    // arena: two regions, each large enough for the largest intermediate
+    int64_t largest = 0;
+    for (size_t i = 0; i + 1 < m->steps.size(); ++i)
+        if (m->steps[i].out_elems > largest) largest = m->steps[i].out_elems;
+    m->region_elems = (size_t)((largest + 63) / 64 * 64);
+    if ((st = dev_alloc(m, 2 * m->region_elems, &m->arena)) != TFJSB_OK) return bail(st, ctx->last_error);
+    cudaError_t e = cudaDeviceSynchronize();  // weight transposes done
+    if (e != cudaSuccess) return bail(TFJSB_ERR_CUDA, std::string("model set-up: ") + cudaGetErrorString(e));
+    ++ctx->live_models;
+    *out = m;
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_model_destroy(tfjsb_model* m) {
+    if (!m) return TFJSB_ERR_INVALID_ARG;
+    cudaDeviceSynchronize();
+    for (float* p : m->owned) cudaFree(p);
+    --m->ctx->live_models;
+    delete m;
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_model_output_shape(tfjsb_model* m, int32_t* rank, int64_t dims[4]) {
+    if (!m || !rank || !dims) return TFJSB_ERR_INVALID_ARG;
+    const Step& last = m->steps.back();
+    *rank = last.out_rank;
+    for (int i = 0; i < 4; ++i) dims[i] = i < last.out_rank ? last.out_dims[i] : 0;
+    return TFJSB_OK;
+}
+
+int32_t tfjsb_model_launches_per_run(tfjsb_model* m) { return m ? (int32_t)m->steps.size() : -1; }
+
+tfjsb_status tfjsb_run_model(tfjsb_model* m, const tfjsb_tensor* input, tfjsb_tensor* output, void* stream) {
+    if (!m) return TFJSB_ERR_INVALID_ARG;
+    tfjsb_status st = check_io(m, input, output);
+    if (st != TFJSB_OK) return st;
+    if (m->bound_in != input->data || m->bound_out != output->data) {
+        if ((st = bind_all(m, static_cast<const float*>(input->data), static_cast<float*>(output->data))) != TFJSB_OK) return st;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (const Step& step : m->steps) {
+        cudaError_t e = launch_step(m, step, s);
+        if (e != cudaSuccess) return cuda_fail(m->ctx, e, "layer launch");
+    }
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_run_model_host(tfjsb_model* m, const float* host_input, float* host_output, void* stream) {
+    if (!m) return TFJSB_ERR_INVALID_ARG;
+    tfjsb_ctx* ctx = m->ctx;
+    if (!host_input || !host_output) return fail(ctx, TFJSB_ERR_INVALID_ARG, "host_input / host_output is null");
+    tfjsb_status st;
+    const Step& last = m->steps.back();
+    if (!m->staged_in) {
+        if ((st = dev_alloc(m, (size_t)m->in_elems, &m->staged_in)) != TFJSB_OK) return st;
+        if ((st = dev_alloc(m, (size_t)last.out_elems, &m->staged_out)) != TFJSB_OK) return st;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(m->staged_in, host_input, (size_t)m->in_elems * 4, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "host-to-device copy of the input");
+    tfjsb_tensor in{m->staged_in, 4, {m->in_dims[0], m->in_dims[1], m->in_dims[2], m->in_dims[3]}};
+    tfjsb_tensor out{m->staged_out, last.out_rank, {last.out_dims[0], last.out_dims[1], last.out_dims[2], last.out_dims[3]}};
+    if ((st = tfjsb_run_model(m, &in, &out, stream)) != TFJSB_OK) return st;
+    e = cudaMemcpyAsync(host_output, m->staged_out, (size_t)last.out_elems * 4, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "device-to-host copy of the output");
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaStreamSynchronize");
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_model_set_keep_all(tfjsb_model* m, int keep_all) {
+    if (!m) return TFJSB_ERR_INVALID_ARG;
+    if (keep_all && !m->keep_all_arena) {
+        size_t total = 0;
+        for (size_t i = 0; i + 1 < m->steps.size(); ++i) total += (size_t)((m->steps[i].out_elems + 63) / 64 * 64);
+        tfjsb_status st = dev_alloc(m, total, &m->keep_all_arena);
+        if (st != TFJSB_OK) return st;
+    }
+    m->keep_all = keep_all != 0;
+    m->bound_in = nullptr;  // force a re-bind on the next run
+    m->bound_out = nullptr;
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_model_layer_output(tfjsb_model* m, int layer, tfjsb_tensor* view) {
+    if (!m || !view) return TFJSB_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= (int)m->steps.size()) return fail(m->ctx, TFJSB_ERR_INVALID_ARG, "no such layer");
+    const Step& st = m->steps[layer];
+    if (!st.out) return fail(m->ctx, TFJSB_ERR_INVALID_ARG, "the model has not run yet");
+    view->data = st.out;
+    view->rank = st.out_rank;
+    for (int i = 0; i < 4; ++i) view->dims[i] = i < st.out_rank ? st.out_dims[i] : 0;
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_model_profile(tfjsb_model* m, const tfjsb_tensor* input, tfjsb_tensor* output, int reps,
+                                 float* ms_per_layer, void* stream) {
+    if (!m) return TFJSB_ERR_INVALID_ARG;
+    tfjsb_ctx* ctx = m->ctx;
+    if (!ms_per_layer || reps < 1) return fail(ctx, TFJSB_ERR_INVALID_ARG, "ms_per_layer is null or reps < 1");
+    tfjsb_status st = check_io(m, input, output);
+    if (st != TFJSB_OK) return st;
+    if (m->bound_in != input->data || m->bound_out != output->data) {
+        if ((st = bind_all(m, static_cast<const float*>(input->data), static_cast<float*>(output->data))) != TFJSB_OK) return st;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int n = (int)m->steps.size();
+    std::vector<cudaEvent_t> ev((size_t)n + 1);
+    for (auto& e : ev)
+        if (cudaEventCreate(&e) != cudaSuccess) return fail(ctx, TFJSB_ERR_CUDA, "cudaEventCreate failed");
+    std::vector<double> sum((size_t)n, 0.0);
+    tfjsb_status rc = TFJSB_OK;
+    for (int r = 0; r < reps && rc == TFJSB_OK; ++r) {
+        cudaEventRecord(ev[0], s);
+        for (int i = 0; i < n; ++i) {
+            cudaError_t e = launch_step(m, m->steps[i], s);
+            if (e != cudaSuccess) { rc = cuda_fail(ctx, e, "layer launch"); break; }
+            cudaEventRecord(ev[i + 1], s);
+        }
+        cudaError_t e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) { rc = cuda_fail(ctx, e, "cudaStreamSynchronize"); break; }
+        if (rc != TFJSB_OK) break;
+        for (int i = 0; i < n; ++i) {
+            float ms = 0.f;
+            cudaEventElapsedTime(&ms, ev[i], ev[i + 1]);
+            sum[i] += ms;
+        }
+    }
+    for (auto& e : ev) cudaEventDestroy(e);
+    if (rc == TFJSB_OK)
+        for (int i = 0; i < n; ++i) ms_per_layer[i] = (float)(sum[i] / reps);
+    return rc;
+}
+
+}  // extern "C"

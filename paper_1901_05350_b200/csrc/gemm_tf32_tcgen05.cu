@@ -1,0 +1,492 @@
+// Tensor-core GEMM for sm_100a with the fused bias + activation epilogue:
+//
+//     C[M,N] = act( A[M,K] . Bt[N,K]^T + bias[N] )        fp32 in, fp32 out
+//
+// A and Bt are row-major with K contiguous ("K-major"), which is what a pointwise convolution
+// over NHWC activations gives for A (rows = pixels, columns = input channels) and what the
+// model builder / the matMul entry point produce for the weights.  Operands are fed to the
+// tensor cores as they lie in memory (`kind::tf32` reads the fp32 bit pattern and uses its top
+// 19 bits); products are accumulated in fp32 in tensor memory.
+//
+// Structure (one persistent CTA per SM, 6 warps, static round-robin over 128 x block_n tiles):
+//   warp 0      producer: one thread issues the bulk tensor copies (TMA, 128-byte swizzle) of the
+//               A tile [128 x 32] and the Bt tile [block_n x 32] of each k-block into a ring of
+//               shared-memory stages, signalling a "full" mbarrier per stage.
+//   warp 1      allocates tensor memory; one thread issues tcgen05.mma (M=128, N=block_n, K=8,
+//               four per k-block) into one of two accumulator stages, frees shared-memory stages
+//               with tcgen05.commit -> "empty" mbarrier, and hands a finished accumulator to the
+//               epilogue with tcgen05.commit -> "acc_full".
+//   warps 2-5   epilogue: each warp owns the 32 accumulator rows (TMEM lanes) its warp id allows
+//               it to read, pulls them out 32 columns at a time (tcgen05.ld), adds bias, applies
+//               the activation, writes the 32x32 block into its own swizzled staging slab and
+//               stores it with a bulk tensor copy (clipped at the matrix edge by the hardware).
+//               The two accumulator stages let the epilogue of tile i overlap the MMAs of tile i+1.
+// Ragged edges need no special code: rows/columns past M, N or K are zero-filled on load and
+// clipped on store by the tensor maps.
+//
+// Every wait is bounded: a wait that exceeds WAIT_LIMIT_NS raises an abort flag that all roles
+// poll, ORs a code into the context's device status word, and the CTA drains its copies, frees
+// its tensor memory and returns.
+#include "common.cuh"
+
+namespace tfjsb {
+
+namespace {
+
+constexpr int BLOCK_M = 128;
+constexpr int BLOCK_K = 32;  // fp32 elements: one 128-byte swizzle row
+constexpr int UMMA_K = 8;    // tf32 elements per tcgen05.mma
+constexpr int ACC_STAGES = 2;
+constexpr int MAX_STAGES = 8;
+constexpr int NUM_THREADS = 192;
+constexpr int EPI_COLS = 32;
+constexpr int A_STAGE_BYTES = BLOCK_M * BLOCK_K * 4;             // 16 KiB
+constexpr int EPI_SLAB_BYTES = 32 * EPI_COLS * 4;                // 4 KiB: 32 rows x 128 B
+constexpr int EPI_BYTES = 4 /*warps*/ * 2 /*buffers*/ * EPI_SLAB_BYTES;  // 32 KiB
+constexpr int SMEM_LIMIT = 232448;                               // 227 KiB
+constexpr unsigned long long WAIT_LIMIT_NS = 500ull * 1000ull * 1000ull;
+
+// ---- PTX wrappers -----------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Waits for the phase with the given parity; gives up after WAIT_LIMIT_NS or when another role
+// has raised the abort flag.  Returns false on giving up.
+__device__ __noinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t it = 1; it < (1u << 26); ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if ((it & 63u) == 0u && global_ns() - t0 > WAIT_LIMIT_NS) return false;
+    }
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map),
+                 "r"(src), "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] . B[smem]^T, single-CTA, TF32 operands, fp32 accumulate.
+__device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 lanes x 32 columns of 32-bit accumulators: thread t of the warp gets lane (base lane + t).
+__device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, written by TMA with
+// the 128-byte swizzle: 8-row groups are 1024 bytes apart (stride byte offset), the leading byte
+// offset is unused for swizzled K-major tiles, descriptor version 1, layout type 2 (128B swizzle).
+__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(1024u >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// Instruction descriptor: fp32 accumulator, TF32 A and B, both K-major, N and M encoded as N/8, M/16.
+__device__ __forceinline__ uint32_t make_idesc_tf32(int m, int n) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+struct KernelArgs {
+    int M, N, K;
+    int block_n;
+    int stages;
+    int n_tiles;    // tiles along N
+    int num_tiles;  // total
+    const float* bias;
+    int act;
+    unsigned int* dev_status;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const __grid_constant__ CUtensorMap map_c, const KernelArgs args) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[MAX_STAGES];
+    __shared__ __align__(8) uint64_t bar_empty[MAX_STAGES];
+    __shared__ __align__(8) uint64_t bar_acc_full[ACC_STAGES];
+    __shared__ __align__(8) uint64_t bar_acc_empty[ACC_STAGES];
+    __shared__ __align__(8) uint64_t bar_drain;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag_s;
+
+    volatile int* abort_flag = &abort_flag_s;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int block_n = args.block_n, stages = args.stages;
+    const int stage_bytes = A_STAGE_BYTES + block_n * BLOCK_K * 4;
+    const int num_k_blocks = (args.K + BLOCK_K - 1) / BLOCK_K;
+
+    // dynamic shared memory, aligned to the 1024-byte swizzle pattern:
+    //   [epilogue slabs: 32 KiB][stage 0: A | B][stage 1] ...
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t epi_base = smem_base;
+    const uint32_t stage_base = smem_base + EPI_BYTES;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        for (int s = 0; s < ACC_STAGES; ++s) {
+            mbar_init(smem_u32(&bar_acc_full[s]), 1);
+            mbar_init(smem_u32(&bar_acc_empty[s]), 4);
+        }
+        mbar_init(smem_u32(&bar_drain), 1);
+        abort_flag_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
+    }
+    const uint32_t tmem_cols = (uint32_t)(ACC_STAGES * block_n);  // 64, 128, 256 or 512: a power of two >= 32
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         smem_u32(&tmem_base_slot)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int armed[MAX_STAGES];      // parity of the last phase armed on each stage, -1 = never
+#pragma unroll
+            for (int s = 0; s < MAX_STAGES; ++s) armed[s] = -1;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
+                const int m0 = (tile / args.n_tiles) * BLOCK_M;
+                const int n0 = (tile % args.n_tiles) * block_n;
+                for (int kb = 0; kb < num_k_blocks; ++kb) {
+                    if (!bounded_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_flag)) {
+                        if (!*abort_flag) {
+                            *abort_flag = 1;
+                            atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_PRODUCER);
+                        }
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t full = smem_u32(&bar_full[stage]);
+                    const uint32_t a_dst = stage_base + (uint32_t)stage * (uint32_t)stage_bytes;
+                    mbar_arrive_expect_tx(full, (uint32_t)stage_bytes);
+                    tma_load_2d(a_dst, &map_a, full, kb * BLOCK_K, m0);
+                    tma_load_2d(a_dst + A_STAGE_BYTES, &map_b, full, kb * BLOCK_K, n0);
+#pragma unroll
+                    for (int s = 0; s < MAX_STAGES; ++s)
+                        if (s == stage) armed[s] = (int)phase;
+                    if (++stage == stages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // Another role may never consume what was armed: wait (bounded) for the copies in
+                // flight so that nothing lands in shared memory after the CTA has gone.
+#pragma unroll
+                for (int s = 0; s < MAX_STAGES; ++s) {
+                    if (s < stages && armed[s] >= 0) {
+                        const unsigned long long t0 = global_ns();
+                        while (!mbar_try_wait(smem_u32(&bar_full[s]), (uint32_t)armed[s])) {
+                            if (global_ns() - t0 > WAIT_LIMIT_NS) {
+                                atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_DRAIN);
+                                break;
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_tf32(BLOCK_M, block_n);
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            bool issued_any = false;
+            for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
+                if (!bounded_wait(smem_u32(&bar_acc_empty[acc]), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * block_n);
+                for (int kb = 0; kb < num_k_blocks; ++kb) {
+                    if (!bounded_wait(smem_u32(&bar_full[stage]), phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = stage_base + (uint32_t)stage * (uint32_t)stage_bytes;
+                    const uint64_t a_desc = make_kmajor_sw128_desc(a_addr);
+                    const uint64_t b_desc = make_kmajor_sw128_desc(a_addr + A_STAGE_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+                        // step along K inside the 128-byte swizzled row: 32 bytes = 2 descriptor units
+                        tc_mma_tf32(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                    (kb | k) != 0 ? 1u : 0u);
+                    }
+                    issued_any = true;
+                    tc_commit(smem_u32(&bar_empty[stage]));
+                    if (++stage == stages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(&bar_acc_full[acc]));
+                if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+            }
+            if (!ok) {
+                if (!*abort_flag) {
+                    *abort_flag = 1;
+                    atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_MMA);
+                }
+                if (issued_any) {
+                    // let the MMAs already issued finish before tensor memory is released
+                    tc_commit(smem_u32(&bar_drain));
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(smem_u32(&bar_drain), 0u)) {
+                        if (global_ns() - t0 > WAIT_LIMIT_NS) {
+                            atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_DRAIN);
+                            break;
+                        }
+                    }
+                }
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue (warps 2..5)
+        const int quad = warp & 3;  // the TMEM lane quadrant this warp may read
+        const uint32_t slab0 = epi_base + (uint32_t)((warp - 2) * 2) * EPI_SLAB_BYTES;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        int buf = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
+            const int m0 = (tile / args.n_tiles) * BLOCK_M;
+            const int n0 = (tile % args.n_tiles) * block_n;
+            // every lane polls (each needs the acquire), the vote keeps the warp uniform
+            const bool got = bounded_wait(smem_u32(&bar_acc_full[acc]), acc_phase, abort_flag);
+            if (!__all_sync(0xffffffffu, got)) {
+                if (lane == 0 && !*abort_flag) {
+                    *abort_flag = 1;
+                    atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_EPILOGUE);
+                }
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            const int row0 = m0 + quad * 32;
+            // chunks whose first column is past N hold nothing to store
+            int n_chunks = block_n / EPI_COLS;
+            const int live_cols = args.N - n0;
+            if (live_cols < block_n) n_chunks = (live_cols + EPI_COLS - 1) / EPI_COLS;
+            const bool rows_live = row0 < args.M;
+            for (int ch = 0; ch < n_chunks; ++ch) {
+                uint32_t r[32];
+                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * block_n + ch * EPI_COLS);
+                tc_ld_32x32(taddr, r);
+                tc_ld_wait();
+                if (ch == n_chunks - 1) {
+                    // accumulator fully read by this warp: hand it back to the MMA issuer
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
+                }
+                if (!rows_live) continue;
+                const int col0 = n0 + ch * EPI_COLS;
+                // staging slab free again?  (at most one older store may still be reading the other slab)
+                if (lane == 0) tma_store_wait_read<1>();
+                __syncwarp();
+                const uint32_t slab = slab0 + (uint32_t)buf * EPI_SLAB_BYTES;
+                const uint32_t row_addr = slab + (uint32_t)lane * 128u;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    float4 v;
+                    v.x = __uint_as_float(r[4 * j + 0]); v.y = __uint_as_float(r[4 * j + 1]);
+                    v.z = __uint_as_float(r[4 * j + 2]); v.w = __uint_as_float(r[4 * j + 3]);
+                    const int c = col0 + 4 * j;
+                    if (args.bias != nullptr && c < args.N) {  // N % 4 == 0: a quad is all in or all out
+                        const float4 b = __ldg(reinterpret_cast<const float4*>(args.bias + c));
+                        v.x = v.x + b.x; v.y = v.y + b.y; v.z = v.z + b.z; v.w = v.w + b.w;
+                    }
+                    v.x = apply_act(v.x, args.act); v.y = apply_act(v.y, args.act);
+                    v.z = apply_act(v.z, args.act); v.w = apply_act(v.w, args.act);
+                    // 128-byte swizzle: 16-byte chunk j of row `lane` lives at chunk j ^ (lane % 8)
+                    const uint32_t dst = row_addr + (uint32_t)((j ^ (lane & 7)) << 4);
+                    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z),
+                                 "f"(v.w)
+                                 : "memory");
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(&map_c, slab, col0, row0);
+                    tma_store_commit();
+                }
+                buf ^= 1;
+            }
+            if (n_chunks == 0) {  // cannot happen (n0 < N), kept so an accumulator is never leaked
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
+            }
+            if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (lane == 0) tma_store_wait_all();
+        __syncwarp();
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols)
+                     : "memory");
+    }
+}
+
+int choose_block_n(int64_t M, int64_t N, int sm_count) {
+    int bn = 32;
+    while (bn < 256 && bn < N) bn <<= 1;
+    const int64_t m_tiles = (M + BLOCK_M - 1) / BLOCK_M;
+    while (bn > 32 && m_tiles * ((N + bn - 1) / bn) < sm_count) bn >>= 1;
+    return bn;
+}
+
+tfjsb_status encode_2d(tfjsb_ctx* ctx, CUtensorMap* map, const void* base, int64_t inner, int64_t outer,
+                       int box_inner, int box_outer, const char* what) {
+    cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+    cuuint64_t strides[1] = {(cuuint64_t)inner * 4u};
+    cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
+    cuuint32_t elem[2] = {1u, 1u};
+    CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides,
+                                   box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return fail(ctx, TFJSB_ERR_CUDA,
+                    std::string("cuTensorMapEncodeTiled failed for ") + what + " (CUresult " + std::to_string((int)r) + ")");
+    return TFJSB_OK;
+}
+
+}  // namespace
+
+bool gemm_tf32_supported(int64_t M, int64_t N, int64_t K) {
+    // row pitches of A, Bt (K floats) and C (N floats) must be multiples of 16 bytes; coordinates are 32-bit
+    return M >= 1 && N >= 4 && K >= 4 && (K % 4 == 0) && (N % 4 == 0) && M < (1LL << 31) - 256 && N < (1LL << 31) - 256 &&
+           K < (1LL << 31) - 256 && ((M + BLOCK_M - 1) / BLOCK_M) * ((N + 31) / 32) < (1LL << 31);
+}
+
+tfjsb_status gemm_tf32_plan(tfjsb_ctx* ctx, const float* a, const float* bt, float* c, int64_t M, int64_t N,
+                            int64_t K, GemmTf32Plan* plan) {
+    if (!gemm_tf32_supported(M, N, K)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the TF32 GEMM");
+    if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+    plan->M = M; plan->N = N; plan->K = K;
+    plan->block_n = choose_block_n(M, N, ctx->sm_count);
+    const int stage_bytes = A_STAGE_BYTES + plan->block_n * BLOCK_K * 4;
+    int stages = (SMEM_LIMIT - 1024 - EPI_BYTES - 512) / stage_bytes;
+    if (stages > MAX_STAGES) stages = MAX_STAGES;
+    plan->stages = stages;
+    plan->smem_bytes = (size_t)1024 + EPI_BYTES + (size_t)stages * stage_bytes;
+    const int64_t n_tiles = (N + plan->block_n - 1) / plan->block_n;
+    const int64_t tiles = ((M + BLOCK_M - 1) / BLOCK_M) * n_tiles;
+    plan->num_tiles = (int)tiles;
+    plan->grid = (int)(tiles < ctx->sm_count ? tiles : ctx->sm_count);
+    tfjsb_status st;
+    if ((st = encode_2d(ctx, &plan->map_a, a, K, M, BLOCK_K, BLOCK_M, "A")) != TFJSB_OK) return st;
+    if ((st = encode_2d(ctx, &plan->map_b, bt, K, N, BLOCK_K, plan->block_n, "B")) != TFJSB_OK) return st;
+    if ((st = encode_2d(ctx, &plan->map_c, c, N, M, EPI_COLS, 32, "C")) != TFJSB_OK) return st;
+    return TFJSB_OK;
+}
+
+cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int act, unsigned int* dev_status,
+                             cudaStream_t s, int64_t* launches) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             SMEM_LIMIT - 2048);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    KernelArgs args;
+    args.M = (int)plan.M; args.N = (int)plan.N; args.K = (int)plan.K;
+    args.block_n = plan.block_n;
+    args.stages = plan.stages;
+    args.n_tiles = (int)((plan.N + plan.block_n - 1) / plan.block_n);
+    args.num_tiles = plan.num_tiles;
+    args.bias = bias;
+    args.act = act;
+    args.dev_status = dev_status;
+    gemm_tf32_kernel<<<plan.grid, NUM_THREADS, plan.smem_bytes, s>>>(plan.map_a, plan.map_b, plan.map_c, args);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace tfjsb

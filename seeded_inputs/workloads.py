@@ -32,9 +32,13 @@ SOFTMAX = "softmax"
 CONFIG_SEEDS = {
     "matmul512": 1901,
     "separable_block": 5350,
-    "mobilenet_025_128": 2019,
+    # 2019, 2020 and 2021 were tried first for this config: their oracle top-1 / top-2 logit margins
+    # (3.0 %, 0.4 %, 4.7 % of the logit range) are below or too close to four times the whole-model
+    # tolerance, so a top-1 comparison would test luck; 2022 gives 11 %.
+    "mobilenet_025_128": 2022,
     "mobilenet_100_224": 224,
-    "mobilenet_100_224_b128": 128,
+    # the batch-128 config is the same model: same weights, and image 0 is the batch-1 image
+    "mobilenet_100_224_b128": 224,
 }
 
 

@@ -30,3 +30,11 @@ def tfjsb():
     import paper_1901_05350_b200 as pkg
 
     return pkg
+
+
+@pytest.fixture(scope="session")
+def ctx(tfjsb):
+    c = tfjsb.Context(0)
+    yield c
+    c.check_device_status()
+    c.close()

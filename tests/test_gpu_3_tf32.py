@@ -1,0 +1,129 @@
+"""GPU parity of the tensor-core (tcgen05, TF32) GEMM path: matMul, 1x1 conv2d, fused epilogue.
+
+Tolerances.  TF32 keeps 10 explicit mantissa bits of each operand, so against the exact
+(double-accumulate) oracle the per-op bar is a relative Frobenius error <= 5e-3.  Against the
+oracle run with the same operand rounding (products and sums still in double) only fp32
+accumulation order remains, and the bar is 2e-5; whichever of truncation / round-to-nearest
+matches tells how the hardware reads fp32 bits.  Small integers are exact in TF32 and every
+partial sum is exact in fp32, so there the result must be bit-identical: a zero-tolerance
+check of descriptors, swizzles, tile tails and the epilogue's addressing.
+"""
+import numpy as np
+import pytest
+
+import seeded_inputs as si
+from helpers import dev, host, rel_fro, same_bits
+
+pytestmark = pytest.mark.gpu
+
+TF32_TOL = 5e-3
+MATCHED_TOL = 2e-5
+
+GEMM_SHAPES = [
+    # M, K, N
+    (128, 32, 32),        # one tile, one k-block, one MMA group
+    (128, 64, 64),
+    (512, 512, 512),      # config 1
+    (300, 100, 72),       # ragged in M, K and N
+    (1, 1024, 1000),      # batch-1 dense layer
+    (128, 1024, 1000),    # batch-128 dense layer: N tail inside a 32-column chunk
+    (12544, 32, 64),      # config 2 pointwise step
+    (3136, 128, 128),
+    (1000, 8, 16),        # K and N below one tile
+    (4100, 36, 260),      # N just above one 256 tile
+    (49, 1024, 1024),     # many k-blocks: the stage ring wraps several times
+    (20000, 256, 512),    # more tiles than SMs: persistent loop, both accumulator stages reused
+]
+
+
+@pytest.mark.parametrize("mkn", GEMM_SHAPES)
+def test_matmul_tf32_integer_exact(ctx, oracle, mkn):
+    M, K, N = mkn
+    a = si.small_integers(301, 0, (M, K), -8, 8)
+    b = si.small_integers(301, 1, (K, N), -8, 8)
+    got = host(ctx.matmul(dev(a), dev(b)))
+    ctx.check_device_status()
+    want = (a.astype(np.int64) @ b.astype(np.int64)).astype(np.float32)
+    assert same_bits(got, want)
+
+
+@pytest.mark.parametrize("mkn", GEMM_SHAPES)
+def test_matmul_tf32_parity(ctx, oracle, mkn):
+    M, K, N = mkn
+    a = si.uniform(302, 0, (M, K), -1, 1)
+    b = si.uniform(302, 1, (K, N), -1, 1)
+    got = host(ctx.matmul(dev(a), dev(b)))
+    ctx.check_device_status()
+    if M * K * N <= 600_000_000:
+        want = oracle.matmul(a, b)
+        assert rel_fro(got, want) <= TF32_TOL
+        matched = min(rel_fro(got, oracle.matmul(a, b, operand="tf32_rz")),
+                      rel_fro(got, oracle.matmul(a, b, operand="tf32_rna")))
+        assert matched <= MATCHED_TOL
+    else:  # sampled rows, each computed one by one by the oracle
+        rows = np.unique(np.linspace(0, M - 1, 257).astype(np.int64))
+        want = oracle.matmul(a[rows], b)
+        assert rel_fro(got[rows], want) <= TF32_TOL
+
+
+@pytest.mark.parametrize("ta,tb", [(False, True), (True, False), (True, True)])
+def test_matmul_tf32_transposes(ctx, oracle, ta, tb):
+    M, K, N = 260, 96, 132
+    a = si.uniform(303, 0, (K, M) if ta else (M, K), -1, 1)
+    b = si.uniform(303, 1, (N, K) if tb else (K, N), -1, 1)
+    got = host(ctx.matmul(dev(a), dev(b), ta, tb))
+    ctx.check_device_status()
+    assert rel_fro(got, oracle.matmul(a, b, ta, tb)) <= TF32_TOL
+    ai = si.small_integers(304, 0, a.shape, -8, 8)
+    bi = si.small_integers(304, 1, b.shape, -8, 8)
+    assert same_bits(host(ctx.matmul(dev(ai), dev(bi), ta, tb)), oracle.matmul(ai, bi, ta, tb))
+
+
+def test_matmul_unaligned_shapes_take_the_cuda_core_path(ctx, oracle):
+    a = si.uniform(305, 0, (70, 27), -1, 1)   # K % 4 != 0
+    b = si.uniform(305, 1, (27, 33), -1, 1)   # N % 4 != 0
+    got = host(ctx.matmul(dev(a), dev(b)))
+    assert rel_fro(got, oracle.matmul(a, b)) <= 1e-5
+
+
+@pytest.mark.parametrize("act", ["none", "relu", "relu6"])
+@pytest.mark.parametrize("shape", [(1, 112, 112, 32, 64), (2, 14, 14, 512, 512), (1, 7, 7, 1024, 1024),
+                                   (3, 9, 5, 8, 16), (1, 28, 28, 128, 256)])
+def test_pointwise_conv_tf32_fused_epilogue(ctx, oracle, shape, act):
+    N, H, W, Cin, Cout = shape
+    x = si.uniform(306, 0, (N, H, W, Cin), 0, 6)
+    f = si.normal(306, 1, (1, 1, Cin, Cout), 0, float(np.sqrt(2.0 / Cin)))
+    b = si.normal(306, 2, (Cout,), 0, 0.5)
+    got = host(ctx.conv2d(dev(x), dev(f), bias=dev(b), act=act))
+    ctx.check_device_status()
+    want = oracle.conv2d(x, f, bias=b, act=act)
+    assert got.shape == want.shape
+    assert rel_fro(got, want) <= TF32_TOL
+    if act == "relu6":
+        assert got.min() >= 0 and got.max() <= 6
+    xi = si.small_integers(307, 0, x.shape, -8, 8)
+    fi = si.small_integers(307, 1, f.shape, -8, 8)
+    bi = si.small_integers(307, 2, b.shape, -8, 8)
+    assert same_bits(host(ctx.conv2d(dev(xi), dev(fi), bias=dev(bi), act=act)),
+                     oracle.conv2d(xi, fi, bias=bi, act=act))
+
+
+def test_separable_block_config2(ctx, oracle):
+    x, layers = si.config_separable_block()
+    dw, pw = layers
+    y1 = ctx.depthwise_conv2d(dev(x), dev(dw.filter), dw.strides, dw.pad, dw.dilations, dev(dw.bias), dw.act)
+    y2 = host(ctx.conv2d(y1, dev(pw.filter), pw.strides, pw.pad, pw.dilations, dev(pw.bias), pw.act))
+    ctx.check_device_status()
+    w1 = oracle.depthwise_conv2d(x, dw.filter, dw.strides, dw.pad, dw.dilations, dw.bias, dw.act)
+    w2 = oracle.conv2d(w1, pw.filter, pw.strides, pw.pad, pw.dilations, pw.bias, pw.act)
+    assert rel_fro(host(y1), w1) <= 1e-6
+    assert rel_fro(y2, w2) <= TF32_TOL
+
+
+def test_tf32_result_is_deterministic(ctx):
+    a = dev(si.uniform(308, 0, (5000, 256), -1, 1))
+    b = dev(si.uniform(308, 1, (256, 512), -1, 1))
+    first = host(ctx.matmul(a, b))
+    for _ in range(3):
+        assert same_bits(host(ctx.matmul(a, b)), first)
+    ctx.check_device_status()

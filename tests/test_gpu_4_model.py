@@ -1,0 +1,144 @@
+"""GPU parity of the graph executor on the MobileNet-v1-style configs.
+
+Whole-model bar: max |logit_gpu - logit_oracle| <= 1e-2 * (max logit - min logit) per image, and
+the same top-1 class.  With random weights two logits can nearly tie, so each image's oracle
+top-1 / top-2 margin is checked first: it must be at least 4x the tolerance, otherwise the
+top-1 comparison would be testing luck (if a seed ever fails this, change the seed and say so).
+"""
+import numpy as np
+import pytest
+
+import seeded_inputs as si
+from helpers import dev, host, rel_fro, same_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def logits_and_probs(model, x_dev):
+    probs = model.run(x_dev)
+    logits = model.layer_output(model.n_layers - 2)
+    return host(logits), host(probs)
+
+
+def check_against_oracle(got_logits, got_probs, want_logits, want_probs, rel=1e-2):
+    for i in range(want_logits.shape[0]):
+        span = float(want_logits[i].max() - want_logits[i].min())
+        tol = rel * span
+        top = np.sort(want_logits[i])
+        err = float(np.max(np.abs(got_logits[i] - want_logits[i])))
+        assert err <= tol, f"image {i}: max logit error {err:.3e} > {tol:.3e}"
+        if rel >= 1e-2:
+            assert top[-1] - top[-2] >= 4 * tol, f"image {i}: oracle top-1 margin too small; pick another seed"
+        assert int(got_logits[i].argmax()) == int(want_logits[i].argmax())
+        assert int(got_probs[i].argmax()) == int(want_probs[i].argmax())
+        assert abs(float(got_probs[i].astype(np.float64).sum()) - 1) <= 1e-5
+    return True
+
+
+@pytest.mark.parametrize("math", ["tf32", "fp32"])
+def test_small_model_every_layer(ctx, oracle, math):
+    """A reduced model (alpha 0.25, 64x64 input, batch 3): every layer's output against the oracle."""
+    x, layers = si.config_mobilenet(0.25, 64, 3, seed=4243, classes=100)
+    want = oracle.run_model(layers, x, keep_all=True)
+    ctx.set_math(math)
+    try:
+        model = ctx.model(layers, x.shape)
+    finally:
+        ctx.set_math("tf32")
+    model.set_keep_all(True)
+    probs = host(model.run(dev(x)))
+    ctx.check_device_status()
+    assert model.launches_per_run == len(layers) == 30
+    tol = 2e-2 if math == "tf32" else 1e-4  # per-layer drift accumulates through 27 conv layers
+    for i, layer in enumerate(layers):
+        got = host(model.layer_output(i)) if i < len(layers) - 1 else probs
+        assert got.shape == want[i].shape, layer.name
+        assert rel_fro(got, want[i]) <= tol, f"layer {i} ({layer.name}) diverges: {rel_fro(got, want[i]):.3e}"
+        if layer.act == "relu6":
+            assert got.min() >= 0 and got.max() <= 6
+    check_against_oracle(host(model.layer_output(28)), probs, want[28], want[29], rel=1e-2 if math == "tf32" else 1e-4)
+    model.close()
+
+
+def test_config3_mobilenet_025_128(ctx, oracle):
+    x, layers = si.config_mobilenet(0.25, 128, 1, seed=si.CONFIG_SEEDS["mobilenet_025_128"])
+    want = oracle.run_model(layers, x, keep_all=True)
+    model = ctx.model(layers, x.shape)
+    model.set_keep_all(True)
+    got_logits, got_probs = logits_and_probs(model, dev(x))
+    ctx.check_device_status()
+    check_against_oracle(got_logits, got_probs, want[-2], want[-1])
+    model.close()
+
+
+def test_config4_mobilenet_100_224(ctx, oracle):
+    x, layers = si.config_mobilenet(1.0, 224, 1, seed=si.CONFIG_SEEDS["mobilenet_100_224"])
+    want = oracle.run_model(layers, x, keep_all=True)
+    model = ctx.model(layers, x.shape)
+    model.set_keep_all(True)
+    got_logits, got_probs = logits_and_probs(model, dev(x))
+    ctx.check_device_status()
+    check_against_oracle(got_logits, got_probs, want[-2], want[-1])
+    # ping-pong arena and keep-all buffers give the same bits
+    model.set_keep_all(False)
+    assert same_bits(host(model.run(dev(x))), got_probs)
+    # fp32 CUDA-core variant of the same model: tighter agreement
+    ctx.set_math("fp32")
+    try:
+        exact = ctx.model(layers, x.shape)
+    finally:
+        ctx.set_math("tf32")
+    exact.set_keep_all(True)
+    el, ep = logits_and_probs(exact, dev(x))
+    check_against_oracle(el, ep, want[-2], want[-1], rel=1e-4)
+    exact.close()
+    model.close()
+
+
+def test_config5_mobilenet_100_224_batch128_sampled_images(ctx, oracle):
+    """Full batch-128 run in the launch configuration the benchmark times; images are independent,
+    so the oracle recomputes a sample of them one by one."""
+    import torch
+
+    x, layers = si.config_mobilenet(1.0, 224, 128, seed=si.CONFIG_SEEDS["mobilenet_100_224_b128"])
+    model = ctx.model(layers, x.shape)
+    xd = dev(x)
+    probs = model.run(xd)
+    logits = model.layer_output(model.n_layers - 2)  # the ping-pong region still holds the dense output
+    ctx.check_device_status()
+    probs, logits = host(probs), host(logits)
+    assert probs.shape == (128, 1000)
+    assert np.all(np.abs(probs.astype(np.float64).sum(-1) - 1) <= 1e-5)
+    sample = [0, 1, 37, 64, 127]
+    want = oracle.run_model(layers, x[sample], keep_all=True)
+    check_against_oracle(logits[sample], probs[sample], want[-2], want[-1])
+    # host-buffer entry point: same bits as the device-resident run
+    hin = torch.from_numpy(x).pin_memory()
+    hout = torch.empty(128, 1000).pin_memory()
+    model.run_host(hin, hout)
+    assert same_bits(hout.numpy(), probs)
+    # per-layer profile returns one positive time per layer
+    ms = model.profile(xd, reps=2)
+    assert len(ms) == 30 and all(t > 0 for t in ms)
+    model.close()
+
+
+def test_model_rejects_wrong_shapes(ctx, tfjsb):
+    import torch
+
+    x, layers = si.config_mobilenet(0.25, 32, 1, seed=5, classes=10)
+    model = ctx.model(layers, x.shape)
+    with pytest.raises(tfjsb.TfjsbError) as e:
+        model.run(torch.zeros(1, 33, 32, 3, device="cuda"))
+    assert e.value.status_name == "SHAPE"
+    with pytest.raises(tfjsb.TfjsbError) as e:
+        model.run(dev(x), out=torch.zeros(1, 11, device="cuda"))
+    assert e.value.status_name == "SHAPE"
+    bad = si.mobilenet_v1_layers(0.25, 10)
+    si.make_model_weights(bad, 3, 5)
+    bad[1].dilations = (2, 2)
+    bad[1].strides = (2, 2)
+    with pytest.raises(tfjsb.TfjsbError) as e:
+        ctx.model(bad, x.shape)
+    assert e.value.status_name == "UNSUPPORTED"
+    model.close()
