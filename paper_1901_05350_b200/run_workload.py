@@ -1,0 +1,75 @@
+"""Runs one of the synthetic workloads through the library a fixed number of times.
+
+    python -m paper_1901_05350_b200.run_workload --workload mobilenet224 --batch 128 --steps 3
+    python -m paper_1901_05350_b200.run_workload --workload matmul --size 4096 --steps 3
+    python -m paper_1901_05350_b200.run_workload --workload block --batch 32 --steps 3
+
+A plain driver for profilers and quick timing: it builds the inputs, runs `--warmup` untimed and
+`--steps` timed passes on one stream, prints the mean device time per pass, and exits.
+"""
+from __future__ import annotations
+
+import argparse
+import os
+import sys
+
+sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+
+
+def main() -> int:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", choices=["mobilenet224", "mobilenet128_025", "matmul", "block"],
+                    default="mobilenet224")
+    ap.add_argument("--batch", type=int, default=128)
+    ap.add_argument("--size", type=int, default=512, help="matmul: M = K = N")
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=1)
+    ap.add_argument("--math", choices=["tf32", "fp32"], default="tf32")
+    args = ap.parse_args()
+
+    import torch
+
+    import paper_1901_05350_b200 as tfjsb
+    import seeded_inputs as si
+
+    ctx = tfjsb.Context(0, math=args.math)
+    if args.workload == "matmul":
+        a, b = si.config_matmul(args.size)
+        a, b = torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()
+        out = torch.empty(args.size, args.size, device="cuda")
+        step = lambda: ctx.matmul(a, b, out=out)
+    elif args.workload == "block":
+        x, (dw, pw) = si.config_separable_block(batch=args.batch)
+        x = torch.from_numpy(x).cuda()
+        wd, bd = torch.from_numpy(dw.filter).cuda(), torch.from_numpy(dw.bias).cuda()
+        wp, bp = torch.from_numpy(pw.filter).cuda(), torch.from_numpy(pw.bias).cuda()
+        mid = torch.empty(x.shape, device="cuda")
+        out = torch.empty(x.shape[:3] + (pw.out_channels,), device="cuda")
+
+        def step():
+            ctx.depthwise_conv2d(x, wd, dw.strides, dw.pad, dw.dilations, bd, dw.act, out=mid)
+            ctx.conv2d(mid, wp, pw.strides, pw.pad, pw.dilations, bp, pw.act, out=out)
+    else:
+        alpha, hw = (1.0, 224) if args.workload == "mobilenet224" else (0.25, 128)
+        x, layers = si.config_mobilenet(alpha, hw, args.batch, seed=si.CONFIG_SEEDS["mobilenet_100_224"])
+        model = ctx.model(layers, x.shape)
+        x = torch.from_numpy(x).cuda()
+        out = torch.empty(model.output_shape, device="cuda")
+        step = lambda: model.run(x, out=out)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(args.steps):
+        step()
+    stop.record()
+    torch.cuda.synchronize()
+    ctx.check_device_status()
+    print(f"{args.workload}: {start.elapsed_time(stop) / max(args.steps, 1):.4f} ms per pass over {args.steps} passes")
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
