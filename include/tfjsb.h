@@ -106,6 +106,27 @@ tfjsb_status tfjsb_window_out_shape(int64_t in, int k, int stride, int dilation,
 tfjsb_status tfjsb_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_tensor* b, int transpose_a,
                           int transpose_b, tfjsb_tensor* out, void* stream);
 
+/* The same operation as tfjsb_matmul for callers that must not allocate device memory; the
+ * paper has no counterpart of this call.  tfjsb_matmul transposes operands that are not
+ * K-contiguous into scratch memory it takes from cudaMalloc.  Some callers cannot afford that
+ * where they call the library: a real-time loop that may not block on the allocator or on the
+ * device synchronisation an allocation can imply, a service whose device-memory budget was
+ * fixed at start-up, any code that runs at a point where cudaMalloc is not permitted.  Here the
+ * scratch is a fixed 16 MiB array that is part of the library's device image on every GPU that
+ * loads it (held until the process exits), and the call never allocates or frees anything.
+ * Create `ctx` at start-up, while allocating is still allowed.
+ *   Limit     (a's elements if transpose_a) + (b's elements if not transpose_b), each rounded up
+ *             to 64, must not exceed 4 Mi floats; otherwise TFJSB_ERR_UNSUPPORTED with the sizes
+ *             in the message and nothing launched.  Operands already K-contiguous need no scratch.
+ *   Sharing   one array per GPU, shared by all calls and contexts and never cleared (every
+ *             element read is overwritten first).  Calls whose kernels may overlap on the GPU
+ *             race on it: keep them on one stream or order them with events.
+ *   Set-up    the first call on a GPU looks up the array's device address
+ *             (cudaGetSymbolAddress); make that first call before any stream capture starts.
+ * Arguments, results and every other rule are those of tfjsb_matmul. */
+tfjsb_status tfjsb_matmul_static_scratch(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_tensor* b,
+                                         int transpose_a, int transpose_b, tfjsb_tensor* out, void* stream);
+
 /* tf.conv2d with an optional fused bias and activation.
  *   x [N,H,W,Cin], filter [fh,fw,Cin,Cout], bias NULL or [Cout], out [N,Ho,Wo,Cout]
  *   out[n,oy,ox,co] = act( bias[co] + sum_{ky,kx,ci} x[n, oy*sh - pt + ky*dh, ox*sw - pl + kx*dw, ci]

@@ -28,7 +28,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "UNSUPPORTED", 4: "CUD
 
 EXPORTS = [
     "tfjsb_init", "tfjsb_shutdown", "tfjsb_set_math", "tfjsb_last_error", "tfjsb_check_device_status",
-    "tfjsb_launch_count", "tfjsb_window_out_shape", "tfjsb_matmul", "tfjsb_conv2d", "tfjsb_depthwise_conv2d",
+    "tfjsb_launch_count", "tfjsb_window_out_shape", "tfjsb_matmul", "tfjsb_matmul_static_scratch", "tfjsb_conv2d", "tfjsb_depthwise_conv2d",
     "tfjsb_avg_pool", "tfjsb_softmax", "tfjsb_bias_act", "tfjsb_model_create", "tfjsb_model_destroy",
     "tfjsb_model_output_shape", "tfjsb_model_launches_per_run", "tfjsb_run_model", "tfjsb_run_model_host",
     "tfjsb_model_set_keep_all", "tfjsb_model_layer_output", "tfjsb_model_profile",
@@ -76,6 +76,7 @@ def _load_library() -> ctypes.CDLL:
     lib.tfjsb_launch_count.restype = i64
     lib.tfjsb_window_out_shape.argtypes = [i64, i32, i32, i32, i32, ctypes.POINTER(i64), ip, ip]
     lib.tfjsb_matmul.argtypes = [vp, tp, tp, i32, i32, tp, vp]
+    lib.tfjsb_matmul_static_scratch.argtypes = [vp, tp, tp, i32, i32, tp, vp]
     lib.tfjsb_conv2d.argtypes = [vp, tp, tp, ip, i32, ip, tp, i32, tp, vp]
     lib.tfjsb_depthwise_conv2d.argtypes = [vp, tp, tp, ip, i32, ip, tp, i32, tp, vp]
     lib.tfjsb_avg_pool.argtypes = [vp, tp, ip, ip, i32, tp, vp]
@@ -181,6 +182,18 @@ class Context:
         out = self._empty((M, N)) if out is None else out
         self._check(lib.tfjsb_matmul(self._h, _desc(a), _desc(b), int(transpose_a), int(transpose_b), _desc(out),
                                      _stream()))
+        return out
+
+    def matmul_static_scratch(self, a, b, transpose_a: bool = False, transpose_b: bool = False, out=None):
+        """matmul for callers that must not allocate device memory inside the call: operands are
+        transposed into a fixed 16 MiB array in the library instead of cudaMalloc'ed scratch.
+        Pass `out` (the binding would otherwise allocate it); problems whose operands to transpose
+        exceed 4 Mi floats are rejected.  Calls share the array: keep them on one stream."""
+        M = a.shape[1] if transpose_a else a.shape[0]
+        N = b.shape[0] if transpose_b else b.shape[1]
+        out = self._empty((M, N)) if out is None else out
+        self._check(lib.tfjsb_matmul_static_scratch(self._h, _desc(a), _desc(b), int(transpose_a),
+                                                    int(transpose_b), _desc(out), _stream()))
         return out
 
     def _conv_out(self, x, fh, fw, strides, pad, dilations, channels):

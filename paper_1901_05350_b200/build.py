@@ -29,6 +29,7 @@ SOURCES = [
     "gemm_tf32_tcgen05.cu",
     "conv2d_fp32_simt.cu",
     "depthwise.cu",
+    "matmul_static_scratch.cu",
 ]
 
 NVCC_FLAGS = [
