@@ -8,7 +8,7 @@
 // tensor cores as they lie in memory (`kind::tf32` reads the fp32 bit pattern and uses its top
 // 19 bits); products are accumulated in fp32 in tensor memory.
 //
-// Structure (one persistent CTA per SM, 6 warps, static round-robin over 128 x block_n tiles):
+// Structure (one persistent CTA per SM, 10 warps, static round-robin over 128 x block_n tiles):
 //   warp 0      producer: one thread issues the bulk tensor copies (TMA, 128-byte swizzle) of the
 //               A tile [128 x 32] and the Bt tile [block_n x 32] of each k-block into a ring of
 //               shared-memory stages, signalling a "full" mbarrier per stage.
@@ -16,10 +16,12 @@
 //               four per k-block) into one of two accumulator stages, frees shared-memory stages
 //               with tcgen05.commit -> "empty" mbarrier, and hands a finished accumulator to the
 //               epilogue with tcgen05.commit -> "acc_full".
-//   warps 2-5   epilogue: each warp owns the 32 accumulator rows (TMEM lanes) its warp id allows
-//               it to read, pulls them out 32 columns at a time (tcgen05.ld), adds bias, applies
-//               the activation, writes the 32x32 block into its own swizzled staging slab and
-//               stores it with a bulk tensor copy (clipped at the matrix edge by the hardware).
+//   warps 2-9   epilogue: each warp reads the 32 accumulator rows (TMEM lanes) its warp id allows
+//               it to read, 32 columns at a time (tcgen05.ld); the two warps of a lane quadrant
+//               take alternate column chunks.  A chunk gets bias and activation in registers, goes
+//               into the warp's own swizzled staging slab and leaves with a bulk tensor store
+//               (clipped at the matrix edge by the hardware).  One warp per scheduler cannot hide
+//               its own instruction latency, hence eight.
 //               The two accumulator stages let the epilogue of tile i overlap the MMAs of tile i+1.
 // Ragged edges need no special code: rows/columns past M, N or K are zero-filled on load and
 // clipped on store by the tensor maps.
@@ -38,11 +40,11 @@ constexpr int BLOCK_K = 32;  // fp32 elements: one 128-byte swizzle row
 constexpr int UMMA_K = 8;    // tf32 elements per tcgen05.mma
 constexpr int ACC_STAGES = 2;
 constexpr int MAX_STAGES = 8;
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;  // producer warp, MMA warp, 8 epilogue warps
 constexpr int EPI_COLS = 32;
 constexpr int A_STAGE_BYTES = BLOCK_M * BLOCK_K * 4;             // 16 KiB
 constexpr int EPI_SLAB_BYTES = 32 * EPI_COLS * 4;                // 4 KiB: 32 rows x 128 B
-constexpr int EPI_BYTES = 4 /*warps*/ * 2 /*buffers*/ * EPI_SLAB_BYTES;  // 32 KiB
+constexpr int EPI_BYTES = 8 /*epilogue warps*/ * EPI_SLAB_BYTES;      // 32 KiB
 constexpr int SMEM_LIMIT = 232448;                               // 227 KiB
 constexpr unsigned long long WAIT_LIMIT_NS = 500ull * 1000ull * 1000ull;
 
@@ -155,6 +157,36 @@ __device__ __forceinline__ uint32_t make_idesc_tf32(int m, int n) {
     return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+// Fused epilogue of one 32-row x 32-column accumulator block held one row per lane: bias add,
+// activation, and the swizzled store into the staging slab the bulk tensor store reads from
+// (16-byte chunk j of row `lane` lives at chunk j ^ (lane % 8): the 128-byte swizzle).
+template <int ACT>
+__device__ __forceinline__ float act_select(float v) {
+    if (ACT == TFJSB_ACT_NONE) return v;
+    float r = v > 0.0f ? v : 0.0f;
+    if (ACT == TFJSB_ACT_RELU6) r = r > 6.0f ? 6.0f : r;
+    return v != v ? v : r;  // NaN stays NaN
+}
+template <int ACT>
+__device__ __forceinline__ void stage_chunk(const uint32_t (&r)[32], const float* __restrict__ bias, int cols_left,
+                                            uint32_t row_addr, int lane) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        float4 v;
+        v.x = __uint_as_float(r[4 * j + 0]); v.y = __uint_as_float(r[4 * j + 1]);
+        v.z = __uint_as_float(r[4 * j + 2]); v.w = __uint_as_float(r[4 * j + 3]);
+        if (bias != nullptr && 4 * j < cols_left) {  // N % 4 == 0: a quad is all in or all out
+            const float4 b = __ldg(reinterpret_cast<const float4*>(bias + 4 * j));
+            v.x = v.x + b.x; v.y = v.y + b.y; v.z = v.z + b.z; v.w = v.w + b.w;
+        }
+        v.x = act_select<ACT>(v.x); v.y = act_select<ACT>(v.y);
+        v.z = act_select<ACT>(v.z); v.w = act_select<ACT>(v.w);
+        const uint32_t dst = row_addr + (uint32_t)((j ^ (lane & 7)) << 4);
+        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+                     : "memory");
+    }
+}
+
 struct KernelArgs {
     int M, N, K;
     int block_n;
@@ -197,7 +229,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         }
         for (int s = 0; s < ACC_STAGES; ++s) {
             mbar_init(smem_u32(&bar_acc_full[s]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[s]), 4);
+            mbar_init(smem_u32(&bar_acc_empty[s]), 8);
         }
         mbar_init(smem_u32(&bar_drain), 1);
         abort_flag_s = 0;
@@ -321,12 +353,15 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             }
         }
     } else {
-        // ---------------------------------------------------------------- epilogue (warps 2..5)
-        const int quad = warp & 3;  // the TMEM lane quadrant this warp may read
-        const uint32_t slab0 = epi_base + (uint32_t)((warp - 2) * 2) * EPI_SLAB_BYTES;
+        // ---------------------------------------------------------------- epilogue (warps 2..9)
+        // Two warps share each TMEM lane quadrant (a warp may only read lanes 32*(warp%4)..+31):
+        // the first of the pair takes the even 32-column chunks of a tile, the second the odd ones.
+        const int ew = warp - 2;
+        const int quad = warp & 3;
+        const int half = ew >> 2;
+        const uint32_t slab = epi_base + (uint32_t)ew * EPI_SLAB_BYTES;
         int acc = 0;
         uint32_t acc_phase = 0;
-        int buf = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
             const int m0 = (tile / args.n_tiles) * BLOCK_M;
@@ -348,51 +383,38 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const int live_cols = args.N - n0;
             if (live_cols < block_n) n_chunks = (live_cols + EPI_COLS - 1) / EPI_COLS;
             const bool rows_live = row0 < args.M;
-            for (int ch = 0; ch < n_chunks; ++ch) {
+            bool released = false;
+            for (int ch = half; ch < n_chunks; ch += 2) {
                 uint32_t r[32];
                 const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * block_n + ch * EPI_COLS);
                 tc_ld_32x32(taddr, r);
                 tc_ld_wait();
-                if (ch == n_chunks - 1) {
-                    // accumulator fully read by this warp: hand it back to the MMA issuer
+                if (ch + 2 >= n_chunks) {
+                    // this warp has read its share of the accumulator: hand it back to the MMA issuer
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
+                    released = true;
                 }
                 if (!rows_live) continue;
                 const int col0 = n0 + ch * EPI_COLS;
-                // staging slab free again?  (at most one older store may still be reading the other slab)
-                if (lane == 0) tma_store_wait_read<1>();
+                // the slab is free once the previous store issued from it has read it
+                if (lane == 0) tma_store_wait_read<0>();
                 __syncwarp();
-                const uint32_t slab = slab0 + (uint32_t)buf * EPI_SLAB_BYTES;
                 const uint32_t row_addr = slab + (uint32_t)lane * 128u;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    float4 v;
-                    v.x = __uint_as_float(r[4 * j + 0]); v.y = __uint_as_float(r[4 * j + 1]);
-                    v.z = __uint_as_float(r[4 * j + 2]); v.w = __uint_as_float(r[4 * j + 3]);
-                    const int c = col0 + 4 * j;
-                    if (args.bias != nullptr && c < args.N) {  // N % 4 == 0: a quad is all in or all out
-                        const float4 b = __ldg(reinterpret_cast<const float4*>(args.bias + c));
-                        v.x = v.x + b.x; v.y = v.y + b.y; v.z = v.z + b.z; v.w = v.w + b.w;
-                    }
-                    v.x = apply_act(v.x, args.act); v.y = apply_act(v.y, args.act);
-                    v.z = apply_act(v.z, args.act); v.w = apply_act(v.w, args.act);
-                    // 128-byte swizzle: 16-byte chunk j of row `lane` lives at chunk j ^ (lane % 8)
-                    const uint32_t dst = row_addr + (uint32_t)((j ^ (lane & 7)) << 4);
-                    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z),
-                                 "f"(v.w)
-                                 : "memory");
-                }
+                const float* bias = (args.bias != nullptr) ? args.bias + col0 : nullptr;
+                const int cols_left = args.N - col0;
+                if (args.act == TFJSB_ACT_RELU6) stage_chunk<TFJSB_ACT_RELU6>(r, bias, cols_left, row_addr, lane);
+                else if (args.act == TFJSB_ACT_RELU) stage_chunk<TFJSB_ACT_RELU>(r, bias, cols_left, row_addr, lane);
+                else stage_chunk<TFJSB_ACT_NONE>(r, bias, cols_left, row_addr, lane);
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
                     tma_store_2d(&map_c, slab, col0, row0);
                     tma_store_commit();
                 }
-                buf ^= 1;
             }
-            if (n_chunks == 0) {  // cannot happen (n0 < N), kept so an accumulator is never leaked
+            if (!released) {  // no chunk of this tile fell to this warp
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
