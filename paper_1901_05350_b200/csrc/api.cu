@@ -358,9 +358,12 @@ tfjsb_status tfjsb_depthwise_conv2d(tfjsb_ctx* ctx, const tfjsb_tensor* x, const
     g.mult = (int)filter->dims[3];
     if (overlaps(out, x) || overlaps(out, filter) || overlaps(out, bias)) return fail(ctx, TFJSB_ERR_INVALID_ARG, "out aliases an input");
     if (numel(out) == 0) return TFJSB_OK;
-    cudaError_t e = launch_depthwise(static_cast<const float*>(x->data), static_cast<const float*>(filter->data),
+    DepthwisePlan plan;
+    if ((st = depthwise_plan(ctx, static_cast<const float*>(x->data), g, &plan)) != TFJSB_OK) return st;
+    cudaError_t e = launch_depthwise(plan, static_cast<const float*>(x->data), static_cast<const float*>(filter->data),
                                      bias ? static_cast<const float*>(bias->data) : nullptr, act,
-                                     static_cast<float*>(out->data), g, static_cast<cudaStream_t>(stream), &ctx->launches);
+                                     static_cast<float*>(out->data), g, ctx->dev_status,
+                                     static_cast<cudaStream_t>(stream), &ctx->launches);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "depthwise launch");
     return TFJSB_OK;
 }

@@ -20,7 +20,8 @@ enum : unsigned int {
     DEV_STATUS_TIMEOUT_PRODUCER = 1u,  // TMA producer waited too long for a free stage
     DEV_STATUS_TIMEOUT_MMA = 2u,       // MMA issuer waited too long for data or for a free accumulator
     DEV_STATUS_TIMEOUT_EPILOGUE = 4u,  // epilogue waited too long for an accumulator
-    DEV_STATUS_TIMEOUT_DRAIN = 8u      // teardown waited too long for copies in flight
+    DEV_STATUS_TIMEOUT_DRAIN = 8u,     // teardown waited too long for copies in flight
+    DEV_STATUS_TIMEOUT_DEPTHWISE = 16u // depthwise kernel waited too long for an input tile
 };
 
 // ---- fused epilogue (bias add, then activation), identical in every kernel -----------------
@@ -95,9 +96,21 @@ cudaError_t launch_gemm_fp32(const float* a, int64_t a_rs, int64_t a_cs, const f
 cudaError_t launch_conv2d_fp32(const float* x, const float* f, const float* bias, int act, float* y,
                                const ConvGeom& g, cudaStream_t s, int64_t* launches);
 
-// Depthwise convolution.  filter [fh,fw,C,mult].
-cudaError_t launch_depthwise(const float* x, const float* f, const float* bias, int act, float* y,
-                             const ConvGeom& g, cudaStream_t s, int64_t* launches);
+// Depthwise convolution.  filter [fh,fw,C,mult].  A plan picks the kernel and, for the bulk-copy
+// pipelined 3x3 kernel, holds the tensor map of the input; it stays valid while `x` and the
+// geometry stay the same.
+struct DepthwisePlan {
+    int variant = -1;  // -1: register kernel / scalar kernel; >= 0: index of the pipelined instance
+    CUtensorMap map_x;
+    int tiles_x = 0, tiles_y = 0, c_blocks = 0;
+    int64_t num_tiles = 0;
+    int grid = 0, stages = 0;
+    size_t smem_bytes = 0;
+};
+tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const float* x, const ConvGeom& g, DepthwisePlan* plan);
+cudaError_t launch_depthwise(const DepthwisePlan& plan, const float* x, const float* f, const float* bias, int act,
+                             float* y, const ConvGeom& g, unsigned int* dev_status, cudaStream_t s,
+                             int64_t* launches);
 
 // Tensor-core GEMM: C[M,N] = act(A[M,K] . Bt[N,K]^T + bias); all three row-major with K (resp. N)
 // contiguous.  A plan holds the tensor maps and tile choice; it can be built once and reused while

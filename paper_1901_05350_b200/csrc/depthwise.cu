@@ -14,7 +14,17 @@
 //
 // Everything else (other windows, dilation, channel multipliers, odd channel counts) takes the
 // scalar kernel: one thread per output element.
+//
+// Pipelined path (same shapes as the fast path, C >= 32, tensor maps available): the register
+// kernel above is bound by load latency, not bandwidth (its loads sit in registers, ~80 per thread,
+// so few warps fit and few bytes are in flight).  `depthwise3x3_tma_kernel` keeps the bytes in
+// flight in shared memory instead: persistent CTAs walk tiles of TH x TW output pixels x 32
+// channels; one thread issues the bulk tensor copy (TMA) of the next tiles' input patches
+// ((TH-1)*S+3 rows x (TW-1)*S+3 columns x 128 bytes, zero-filled outside the image, which is the
+// 'same' padding) into a ring of stages while all 256 threads compute the current tile from
+// shared memory with the same sliding-row scheme and store float4s straight to global memory.
 #include "common.cuh"
+#include "ptx_sm100.cuh"
 
 namespace tfjsb {
 
@@ -122,6 +132,179 @@ __global__ void depthwise_generic_kernel(const float* __restrict__ x, const floa
     }
 }
 
+// ---- pipelined kernel ---------------------------------------------------------------------------
+constexpr int DW_CB = 32;          // channels per tile: one 128-byte line per pixel
+constexpr int DW_MAX_STAGES = 4;
+
+struct DwTiling {
+    int tiles_x, tiles_y, c_blocks, stages;
+    long long num_tiles;
+};
+
+template <int S, int TW, int R>
+struct DwTile {
+    static constexpr int RG = 32 / TW;                 // row groups of threads: 256 = 8 quads x TW x RG
+    static constexpr int TH = RG * R;                  // output rows per tile
+    static constexpr int TWIN = (TW - 1) * S + 3;      // input patch
+    static constexpr int THIN = (TH - 1) * S + 3;
+    static constexpr int STAGE_FLOATS = THIN * TWIN * DW_CB;
+    static constexpr int STAGE_BYTES = STAGE_FLOATS * 4;
+};
+
+template <int S, int TW, int R>
+__global__ void __launch_bounds__(DW_THREADS, 2)
+depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __restrict__ f,
+                        const float* __restrict__ bias, int act, float* __restrict__ y, ConvGeom g, DwTiling t,
+                        unsigned int* dev_status) {
+    using T = DwTile<S, TW, R>;
+    extern __shared__ uint8_t dw_smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[DW_MAX_STAGES];
+    __shared__ int abort_flag_s;
+    volatile int* abort_flag = &abort_flag_s;
+
+    const uint32_t smem_base = (ptx::smem_u32(dw_smem_raw) + 127u) & ~127u;
+    const float* smem_f = reinterpret_cast<const float*>(dw_smem_raw + (smem_base - ptx::smem_u32(dw_smem_raw)));
+    const int tid = threadIdx.x;
+    const int c4 = tid & 7;
+    const int col = (tid >> 3) % TW;
+    const int rg = tid / (8 * TW);
+
+    if (tid == 0) {
+        for (int s = 0; s < t.stages; ++s) ptx::mbar_init(ptx::smem_u32(&bar_full[s]), 1);
+        abort_flag_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+    }
+    __syncthreads();
+
+    // tile index -> (channel block, tile column, tile row, image); channel block fastest so that CTAs
+    // running side by side touch neighbouring 128-byte lines of the same pixels
+    auto issue = [&](long long tile, int slot) {
+        const int cb = (int)(tile % t.c_blocks);
+        long long q = tile / t.c_blocks;
+        const int tx = (int)(q % t.tiles_x); q /= t.tiles_x;
+        const int ty = (int)(q % t.tiles_y);
+        const int n = (int)(q / t.tiles_y);
+        const uint32_t bar = ptx::smem_u32(&bar_full[slot]);
+        ptx::mbar_arrive_expect_tx(bar, (uint32_t)T::STAGE_BYTES);
+        ptx::tma_load_4d(smem_base + (uint32_t)slot * (uint32_t)T::STAGE_BYTES, &map_x, bar, cb * DW_CB,
+                         tx * TW * S - g.pl, ty * T::TH * S - g.pt, n);
+    };
+
+    const long long first = blockIdx.x, step = gridDim.x;
+    long long issued = 0;  // tiles handed to the copy engine so far (thread 0 only)
+    if (tid == 0) {
+        for (int i = 0; i < t.stages - 1; ++i)
+            if (first + i * step < t.num_tiles) { issue(first + i * step, i); ++issued; }
+    }
+
+    long long i = 0;
+    bool ok = true;
+    for (long long tile = first; tile < t.num_tiles; tile += step, ++i) {
+        const int slot = (int)(i % t.stages);
+        const bool got = ptx::bounded_wait(ptx::smem_u32(&bar_full[slot]), (uint32_t)((i / t.stages) & 1), abort_flag);
+        // also the barrier that says everyone is done with the previous tile's stage
+        if (!__syncthreads_and(got ? 1 : 0)) { ok = false; break; }
+        if (tid == 0) {
+            const long long ahead = i + t.stages - 1;
+            if (first + ahead * step < t.num_tiles) { issue(first + ahead * step, (int)(ahead % t.stages)); ++issued; }
+        }
+
+        const int cb = (int)(tile % t.c_blocks);
+        long long q = tile / t.c_blocks;
+        const int tx = (int)(q % t.tiles_x); q /= t.tiles_x;
+        const int ty = (int)(q % t.tiles_y);
+        const long long n = q / t.tiles_y;
+        const int c = cb * DW_CB + c4 * 4;
+        const int ox = tx * TW + col;
+        const int oy0 = ty * T::TH + rg * R;
+        const bool live = c < g.C && ox < g.Wo && oy0 < g.Ho;
+
+        float4 w[9];
+        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (live) {
+#pragma unroll
+            for (int k = 0; k < 9; ++k) w[k] = __ldg(reinterpret_cast<const float4*>(f + (int64_t)k * g.C + c));
+            if (bias) b = __ldg(reinterpret_cast<const float4*>(bias + c));
+        }
+        float4 acc[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+        if (live) {
+            const float* patch = smem_f + (size_t)slot * T::STAGE_FLOATS + ((rg * R * S) * T::TWIN + col * S) * DW_CB + c4 * 4;
+            constexpr int IN_ROWS = (R - 1) * S + 3;
+#pragma unroll
+            for (int j = 0; j < IN_ROWS; ++j) {
+                const float* row = patch + j * T::TWIN * DW_CB;
+                const float4 v0 = ld4(row), v1 = ld4(row + DW_CB), v2 = ld4(row + 2 * DW_CB);
+#pragma unroll
+                for (int ky = 0; ky < 3; ++ky) {
+                    const int d = j - ky;
+                    if (d >= 0 && d % S == 0 && d / S < R) {
+                        fma4(acc[d / S], v0, w[ky * 3 + 0]);
+                        fma4(acc[d / S], v1, w[ky * 3 + 1]);
+                        fma4(acc[d / S], v2, w[ky * 3 + 2]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const int oy = oy0 + r;
+                if (oy < g.Ho) {
+                    float4 v = acc[r];
+                    v.x = apply_act(v.x + b.x, act); v.y = apply_act(v.y + b.y, act);
+                    v.z = apply_act(v.z + b.z, act); v.w = apply_act(v.w + b.w, act);
+                    *reinterpret_cast<float4*>(y + ((n * g.Ho + oy) * (int64_t)g.Wo + ox) * g.Co + c) = v;
+                }
+            }
+        }
+    }
+
+    if (!ok && tid == 0) {
+        if (!*abort_flag) *abort_flag = 1;
+        atomicOr(dev_status, DEV_STATUS_TIMEOUT_DEPTHWISE);
+        // wait (bounded) for the copies still in flight so nothing lands after the CTA has gone
+        for (long long k = i; k < issued; ++k) {
+            const unsigned long long t0 = ptx::global_ns();
+            while (!ptx::mbar_try_wait(ptx::smem_u32(&bar_full[k % t.stages]), (uint32_t)((k / t.stages) & 1))) {
+                if (ptx::global_ns() - t0 > ptx::WAIT_LIMIT_NS) {
+                    atomicOr(dev_status, DEV_STATUS_TIMEOUT_DRAIN);
+                    break;
+                }
+            }
+        }
+    }
+}
+
+// the instances: {stride, tile width, rows per thread}
+struct DwVariant {
+    int S, TW, TH, stage_bytes;
+};
+constexpr DwVariant kDwVariants[] = {
+    {1, 16, DwTile<1, 16, 4>::TH, DwTile<1, 16, 4>::STAGE_BYTES},  // 0: large stride-1 images
+    {1, 16, DwTile<1, 16, 7>::TH, DwTile<1, 16, 7>::STAGE_BYTES},  // 1: 9..14 output rows in one tile
+    {1, 8, DwTile<1, 8, 2>::TH, DwTile<1, 8, 2>::STAGE_BYTES},     // 2: images up to 8 wide
+    {2, 16, DwTile<2, 16, 2>::TH, DwTile<2, 16, 2>::STAGE_BYTES},  // 3: stride 2
+    {2, 8, DwTile<2, 8, 2>::TH, DwTile<2, 8, 2>::STAGE_BYTES},     // 4: stride 2, outputs up to 8 wide
+};
+constexpr int DW_SMEM_BUDGET = 113 * 1024;  // two CTAs per SM
+
+template <int S, int TW, int R>
+cudaError_t launch_tma_instance(const DepthwisePlan& plan, const float* f, const float* bias, int act, float* y,
+                                const ConvGeom& g, unsigned int* dev_status, cudaStream_t s) {
+    static bool attr_set = false;
+    auto kernel = depthwise3x3_tma_kernel<S, TW, R>;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DW_SMEM_BUDGET);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    DwTiling t{plan.tiles_x, plan.tiles_y, plan.c_blocks, plan.stages, (long long)plan.num_tiles};
+    kernel<<<plan.grid, DW_THREADS, plan.smem_bytes, s>>>(plan.map_x, f, bias, act, y, g, t, dev_status);
+    return cudaGetLastError();
+}
+
 int pow2_at_most(int v, int cap) {
     int p = 1;
     while (p < v && p < cap) p <<= 1;
@@ -130,10 +313,58 @@ int pow2_at_most(int v, int cap) {
 
 }  // namespace
 
-cudaError_t launch_depthwise(const float* x, const float* f, const float* bias, int act, float* y,
-                             const ConvGeom& g, cudaStream_t s, int64_t* launches) {
+tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const float* x, const ConvGeom& g, DepthwisePlan* plan) {
+    plan->variant = -1;
+    const bool shape_ok = g.fh == 3 && g.fw == 3 && g.mult == 1 && g.dh == 1 && g.dw == 1 && g.sh == g.sw &&
+                          (g.sh == 1 || g.sh == 2) && (g.C % 4 == 0) && g.C >= DW_CB && g.N <= 0x7fffffff;
+    if (!shape_ok || !ctx->encode_tiled) return TFJSB_OK;
+    int v;
+    if (g.sh == 1) v = g.Wo <= 8 ? 2 : ((g.Ho > 8 && g.Ho <= 14) ? 1 : 0);
+    else v = g.Wo <= 8 ? 4 : 3;
+    const DwVariant& d = kDwVariants[v];
+    const int twin = (d.TW - 1) * d.S + 3, thin = (d.TH - 1) * d.S + 3;
+    cuuint64_t dims[4] = {(cuuint64_t)g.C, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
+    cuuint64_t strides[3] = {(cuuint64_t)g.C * 4u, (cuuint64_t)g.W * g.C * 4u, (cuuint64_t)g.H * g.W * g.C * 4u};
+    cuuint32_t box[4] = {(cuuint32_t)DW_CB, (cuuint32_t)twin, (cuuint32_t)thin, 1u};
+    cuuint32_t elem[4] = {1u, 1u, 1u, 1u};
+    CUresult r = ctx->encode_tiled(&plan->map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(x), dims, strides,
+                                   box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the depthwise input (CUresult " +
+                                             std::to_string((int)r) + ")");
+    plan->tiles_x = (g.Wo + d.TW - 1) / d.TW;
+    plan->tiles_y = (g.Ho + d.TH - 1) / d.TH;
+    plan->c_blocks = (g.C + DW_CB - 1) / DW_CB;
+    plan->num_tiles = (int64_t)plan->tiles_x * plan->tiles_y * plan->c_blocks * g.N;
+    int stages = (DW_SMEM_BUDGET - 256) / d.stage_bytes;
+    if (stages > DW_MAX_STAGES) stages = DW_MAX_STAGES;
+    if (stages < 2) return TFJSB_OK;  // cannot happen with the instances above
+    plan->stages = stages;
+    plan->smem_bytes = (size_t)stages * d.stage_bytes + 128;
+    const int64_t max_grid = (int64_t)ctx->sm_count * 2;
+    plan->grid = (int)(plan->num_tiles < max_grid ? plan->num_tiles : max_grid);
+    plan->variant = v;
+    return TFJSB_OK;
+}
+
+cudaError_t launch_depthwise(const DepthwisePlan& plan, const float* x, const float* f, const float* bias, int act,
+                             float* y, const ConvGeom& g, unsigned int* dev_status, cudaStream_t s,
+                             int64_t* launches) {
     const int64_t n_out = g.N * g.Ho * g.Wo * g.Co;
     if (n_out == 0) return cudaSuccess;
+    if (plan.variant >= 0) {
+        cudaError_t e;
+        switch (plan.variant) {
+            case 0: e = launch_tma_instance<1, 16, 4>(plan, f, bias, act, y, g, dev_status, s); break;
+            case 1: e = launch_tma_instance<1, 16, 7>(plan, f, bias, act, y, g, dev_status, s); break;
+            case 2: e = launch_tma_instance<1, 8, 2>(plan, f, bias, act, y, g, dev_status, s); break;
+            case 3: e = launch_tma_instance<2, 16, 2>(plan, f, bias, act, y, g, dev_status, s); break;
+            default: e = launch_tma_instance<2, 8, 2>(plan, f, bias, act, y, g, dev_status, s); break;
+        }
+        ++*launches;
+        return e;
+    }
     const bool fast = g.fh == 3 && g.fw == 3 && g.mult == 1 && g.dh == 1 && g.dw == 1 && g.sh == g.sw &&
                       (g.sh == 1 || g.sh == 2) && (g.C % 4 == 0) && g.N <= 65535;
     if (fast) {

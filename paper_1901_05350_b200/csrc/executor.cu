@@ -27,6 +27,7 @@ struct Step {
     float* filter_km = nullptr;  // device, [N,K] (tensor-core layers only)
     float* bias = nullptr;       // device or null
     GemmTf32Plan plan{};
+    DepthwisePlan dw_plan{};
     bool plan_built = false;
     int32_t out_rank = 4;
     int64_t out_dims[4] = {0, 0, 0, 0};
@@ -95,6 +96,11 @@ tfjsb_status bind_step(tfjsb_model* m, Step& st, const float* in, float* out) {
         if (rc != TFJSB_OK) return rc;
         st.plan_built = true;
     }
+    if (st.kind == STEP_DEPTHWISE && (changed || !st.plan_built)) {
+        tfjsb_status rc = depthwise_plan(m->ctx, in, st.g, &st.dw_plan);
+        if (rc != TFJSB_OK) return rc;
+        st.plan_built = true;
+    }
     return TFJSB_OK;
 }
 
@@ -132,7 +138,8 @@ cudaError_t launch_step(tfjsb_model* m, const Step& st, cudaStream_t s) {
         case STEP_CONV_FP32:
             return launch_conv2d_fp32(st.in, st.filter, st.bias, st.act, st.out, st.g, s, &ctx->launches);
         case STEP_DEPTHWISE:
-            return launch_depthwise(st.in, st.filter, st.bias, st.act, st.out, st.g, s, &ctx->launches);
+            return launch_depthwise(st.dw_plan, st.in, st.filter, st.bias, st.act, st.out, st.g, ctx->dev_status, s,
+                                    &ctx->launches);
         case STEP_POOL:
             return launch_avg_pool(st.in, st.out, st.g, s, &ctx->launches);
         case STEP_SOFTMAX:

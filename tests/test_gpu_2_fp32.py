@@ -92,6 +92,13 @@ DW_CASES = [
     (2, 56, 56, 64, 3, 3, 1, (2, 2), "same", (1, 1)),
     (1, 14, 14, 512, 3, 3, 1, (1, 1), "same", (1, 1)),
     (1, 7, 7, 1024, 3, 3, 1, (1, 1), "same", (1, 1)),
+    (2, 20, 37, 48, 3, 3, 1, (1, 1), "same", (1, 1)),     # pipelined kernel: ragged tiles, partial channel block
+    (1, 14, 14, 64, 3, 3, 1, (1, 1), "same", (1, 1)),     # pipelined kernel: whole 14-row image in one tile
+    (3, 7, 7, 96, 3, 3, 1, (1, 1), "same", (1, 1)),       # pipelined kernel: narrow-image instance
+    (2, 29, 31, 32, 3, 3, 1, (2, 2), "same", (1, 1)),     # pipelined kernel: stride 2, odd sizes
+    (1, 14, 14, 160, 3, 3, 1, (2, 2), "same", (1, 1)),    # pipelined kernel: stride 2, narrow output
+    (1, 9, 40, 32, 3, 3, 1, (1, 1), "valid", (1, 1)),     # pipelined kernel: 'valid' (no padding offset)
+    (5, 33, 18, 36, 3, 3, 1, (2, 2), "valid", (1, 1)),
     (3, 13, 11, 24, 3, 3, 1, (1, 1), "same", (1, 1)),     # channel quads not a power of two, ragged rows
     (2, 15, 9, 8, 3, 3, 1, (2, 2), "same", (1, 1)),       # odd sizes at stride 2 (symmetric padding)
     (1, 10, 10, 16, 3, 3, 1, (1, 1), "valid", (1, 1)),
