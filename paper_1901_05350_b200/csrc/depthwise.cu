@@ -159,6 +159,7 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
     using T = DwTile<S, TW, R>;
     extern __shared__ uint8_t dw_smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[DW_MAX_STAGES];
+    __shared__ int4 tile_info[DW_MAX_STAGES];
     __shared__ int abort_flag_s;
     volatile int* abort_flag = &abort_flag_s;
 
@@ -178,43 +179,49 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
     __syncthreads();
 
     // tile index -> (channel block, tile column, tile row, image); channel block fastest so that CTAs
-    // running side by side touch neighbouring 128-byte lines of the same pixels
-    auto issue = [&](long long tile, int slot) {
-        const int cb = (int)(tile % t.c_blocks);
-        long long q = tile / t.c_blocks;
-        const int tx = (int)(q % t.tiles_x); q /= t.tiles_x;
-        const int ty = (int)(q % t.tiles_y);
-        const int n = (int)(q / t.tiles_y);
+    // running side by side touch neighbouring 128-byte lines of the same pixels.  Only the issuing
+    // thread pays for the divisions: it leaves the coordinates beside the stage for everyone else
+    // (written before its mbarrier arrive, read after the wait: release / acquire).
+    auto issue = [&](int tile, int slot) {
+        const int cb = tile % t.c_blocks;
+        int q = tile / t.c_blocks;
+        const int tx = q % t.tiles_x; q /= t.tiles_x;
+        const int ty = q % t.tiles_y;
+        const int n = q / t.tiles_y;
+        tile_info[slot] = make_int4(cb, tx, ty, n);
         const uint32_t bar = ptx::smem_u32(&bar_full[slot]);
         ptx::mbar_arrive_expect_tx(bar, (uint32_t)T::STAGE_BYTES);
         ptx::tma_load_4d(smem_base + (uint32_t)slot * (uint32_t)T::STAGE_BYTES, &map_x, bar, cb * DW_CB,
                          tx * TW * S - g.pl, ty * T::TH * S - g.pt, n);
     };
 
-    const long long first = blockIdx.x, step = gridDim.x;
-    long long issued = 0;  // tiles handed to the copy engine so far (thread 0 only)
+    const int num_tiles = (int)t.num_tiles;
+    const int first = blockIdx.x, step = gridDim.x;
+    const int my_tiles = first < num_tiles ? (num_tiles - first + step - 1) / step : 0;
+    int issued = 0;  // tiles handed to the copy engine so far (thread 0 only)
     if (tid == 0) {
-        for (int i = 0; i < t.stages - 1; ++i)
-            if (first + i * step < t.num_tiles) { issue(first + i * step, i); ++issued; }
+        for (; issued < t.stages - 1 && issued < my_tiles; ++issued) issue(first + issued * step, issued);
     }
 
-    long long i = 0;
+    int i = 0;
+    int slot = 0;
+    uint32_t parity = 0;
     bool ok = true;
-    for (long long tile = first; tile < t.num_tiles; tile += step, ++i) {
-        const int slot = (int)(i % t.stages);
-        const bool got = ptx::bounded_wait(ptx::smem_u32(&bar_full[slot]), (uint32_t)((i / t.stages) & 1), abort_flag);
+    for (; i < my_tiles; ++i) {
+        const bool got = ptx::bounded_wait(ptx::smem_u32(&bar_full[slot]), parity, abort_flag);
         // also the barrier that says everyone is done with the previous tile's stage
         if (!__syncthreads_and(got ? 1 : 0)) { ok = false; break; }
-        if (tid == 0) {
-            const long long ahead = i + t.stages - 1;
-            if (first + ahead * step < t.num_tiles) { issue(first + ahead * step, (int)(ahead % t.stages)); ++issued; }
+        if (tid == 0 && issued < my_tiles) {
+            int ahead_slot = slot + t.stages - 1;
+            if (ahead_slot >= t.stages) ahead_slot -= t.stages;
+            issue(first + issued * step, ahead_slot);
+            ++issued;
         }
-
-        const int cb = (int)(tile % t.c_blocks);
-        long long q = tile / t.c_blocks;
-        const int tx = (int)(q % t.tiles_x); q /= t.tiles_x;
-        const int ty = (int)(q % t.tiles_y);
-        const long long n = q / t.tiles_y;
+        const int4 info = tile_info[slot];
+        const int cb = info.x, tx = info.y, ty = info.z;
+        const long long n = info.w;
+        const int cur_slot = slot;
+        if (++slot == t.stages) { slot = 0; parity ^= 1u; }
         const int c = cb * DW_CB + c4 * 4;
         const int ox = tx * TW + col;
         const int oy0 = ty * T::TH + rg * R;
@@ -232,7 +239,7 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
         for (int r = 0; r < R; ++r) acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
 
         if (live) {
-            const float* patch = smem_f + (size_t)slot * T::STAGE_FLOATS + ((rg * R * S) * T::TWIN + col * S) * DW_CB + c4 * 4;
+            const float* patch = smem_f + (size_t)cur_slot * T::STAGE_FLOATS + ((rg * R * S) * T::TWIN + col * S) * DW_CB + c4 * 4;
             constexpr int IN_ROWS = (R - 1) * S + 3;
 #pragma unroll
             for (int j = 0; j < IN_ROWS; ++j) {
@@ -265,7 +272,7 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
         if (!*abort_flag) *abort_flag = 1;
         atomicOr(dev_status, DEV_STATUS_TIMEOUT_DEPTHWISE);
         // wait (bounded) for the copies still in flight so nothing lands after the CTA has gone
-        for (long long k = i; k < issued; ++k) {
+        for (int k = i; k < issued; ++k) {
             const unsigned long long t0 = ptx::global_ns();
             while (!ptx::mbar_try_wait(ptx::smem_u32(&bar_full[k % t.stages]), (uint32_t)((k / t.stages) & 1))) {
                 if (ptx::global_ns() - t0 > ptx::WAIT_LIMIT_NS) {
@@ -316,7 +323,7 @@ int pow2_at_most(int v, int cap) {
 tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const float* x, const ConvGeom& g, DepthwisePlan* plan) {
     plan->variant = -1;
     const bool shape_ok = g.fh == 3 && g.fw == 3 && g.mult == 1 && g.dh == 1 && g.dw == 1 && g.sh == g.sw &&
-                          (g.sh == 1 || g.sh == 2) && (g.C % 4 == 0) && g.C >= DW_CB && g.N <= 0x7fffffff;
+                          (g.sh == 1 || g.sh == 2) && (g.C % 4 == 0) && g.C >= DW_CB;
     if (!shape_ok || !ctx->encode_tiled) return TFJSB_OK;
     int v;
     if (g.sh == 1) v = g.Wo <= 8 ? 2 : ((g.Ho > 8 && g.Ho <= 14) ? 1 : 0);
@@ -337,6 +344,7 @@ tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const float* x, const ConvGeom& g, D
     plan->tiles_y = (g.Ho + d.TH - 1) / d.TH;
     plan->c_blocks = (g.C + DW_CB - 1) / DW_CB;
     plan->num_tiles = (int64_t)plan->tiles_x * plan->tiles_y * plan->c_blocks * g.N;
+    if (plan->num_tiles > 0x7fffffff) return TFJSB_OK;  // tile indices are 32-bit in the kernel
     int stages = (DW_SMEM_BUDGET - 256) / d.stage_bytes;
     if (stages > DW_MAX_STAGES) stages = DW_MAX_STAGES;
     if (stages < 2) return TFJSB_OK;  // cannot happen with the instances above

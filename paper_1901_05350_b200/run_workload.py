@@ -3,6 +3,8 @@
     python -m paper_1901_05350_b200.run_workload --workload mobilenet224 --batch 128 --steps 3
     python -m paper_1901_05350_b200.run_workload --workload matmul --size 4096 --steps 3
     python -m paper_1901_05350_b200.run_workload --workload block --batch 32 --steps 3
+    python -m paper_1901_05350_b200.run_workload --workload depthwise --batch 128 --hw 14 --channels 512 --stride 1
+    python -m paper_1901_05350_b200.run_workload --workload pointwise --batch 128 --hw 14 --channels 512 --cout 512
 
 A plain driver for profilers and quick timing: it builds the inputs, runs `--warmup` untimed and
 `--steps` timed passes on one stream, prints the mean device time per pass, and exits.
@@ -18,10 +20,14 @@ sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
 
 def main() -> int:
     ap = argparse.ArgumentParser()
-    ap.add_argument("--workload", choices=["mobilenet224", "mobilenet128_025", "matmul", "block"],
+    ap.add_argument("--workload", choices=["mobilenet224", "mobilenet128_025", "matmul", "block", "depthwise", "pointwise"],
                     default="mobilenet224")
     ap.add_argument("--batch", type=int, default=128)
     ap.add_argument("--size", type=int, default=512, help="matmul: M = K = N")
+    ap.add_argument("--hw", type=int, default=112, help="depthwise / pointwise: input height = width")
+    ap.add_argument("--channels", type=int, default=32, help="depthwise / pointwise: input channels")
+    ap.add_argument("--cout", type=int, default=64, help="pointwise: output channels")
+    ap.add_argument("--stride", type=int, default=1, help="depthwise: stride")
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
     ap.add_argument("--math", choices=["tf32", "fp32"], default="tf32")
@@ -49,6 +55,22 @@ def main() -> int:
         def step():
             ctx.depthwise_conv2d(x, wd, dw.strides, dw.pad, dw.dilations, bd, dw.act, out=mid)
             ctx.conv2d(mid, wp, pw.strides, pw.pad, pw.dilations, bp, pw.act, out=out)
+    elif args.workload in ("depthwise", "pointwise"):
+        x = torch.from_numpy(si.uniform(7, 0, (args.batch, args.hw, args.hw, args.channels), 0.0, 6.0)).cuda()
+        if args.workload == "depthwise":
+            w = torch.from_numpy(si.normal(7, 1, (3, 3, args.channels, 1), 0.0, 0.47)).cuda()
+            b = torch.from_numpy(si.normal(7, 2, (args.channels,), 0.0, 0.01)).cuda()
+            strides = (args.stride, args.stride)
+            out = ctx.depthwise_conv2d(x, w, strides, "same", (1, 1), b, "relu6")
+            step = lambda: ctx.depthwise_conv2d(x, w, strides, "same", (1, 1), b, "relu6", out=out)
+        else:
+            from seeded_inputs.workloads import Layer
+
+            layer = Layer("conv2d", (1, 1), (1, 1), (1, 1), "same", "relu6", args.cout, "pw")
+            si.make_model_weights([layer], args.channels, 7)
+            model = ctx.model([layer], x.shape)  # the executor keeps the weights K-contiguous
+            out = torch.empty(model.output_shape, device="cuda")
+            step = lambda: model.run(x, out=out)
     else:
         alpha, hw = (1.0, 224) if args.workload == "mobilenet224" else (0.25, 128)
         x, layers = si.config_mobilenet(alpha, hw, args.batch, seed=si.CONFIG_SEEDS["mobilenet_100_224"])
