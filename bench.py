@@ -120,7 +120,7 @@ def layer_work(layers, in_shape, window_out_shape):
                 co = layer.out_channels
                 flops = 2 * n * ho * wo * co * fh * fw * c
                 weights = fh * fw * c * co
-                kernel = "gemm_tf32" if (fh, fw) == (1, 1) and layer.strides == (1, 1) else "conv2d_fp32"
+                kernel = "gemm_tf32" if (fh, fw) == (1, 1) and layer.strides == (1, 1) else "conv2d_igemm_tf32"
             else:
                 co = c * layer.out_channels
                 flops = 2 * n * ho * wo * co * fh * fw
@@ -147,10 +147,11 @@ def roofline_rows(rows, ms, peaks, fp32_tflops):
     tf32_peak = peaks["bf16_tflops_sustained"] / 2.0  # dense TF32 is nominally half of dense bf16
     out = []
     for row, t_ms in zip(rows, ms):
-        compute_peak = tf32_peak if row["kernel"] == "gemm_tf32" else fp32_tflops
+        on_tensor_cores = row["kernel"] in ("gemm_tf32", "conv2d_igemm_tf32")
+        compute_peak = tf32_peak if on_tensor_cores else fp32_tflops
         t_compute = row["flops"] / (compute_peak * 1e12)
         t_hbm = row["bytes"] / (peaks["hbm_gbs"] * 1e9)
-        bound = "tensor" if (row["kernel"] == "gemm_tf32" and t_compute > t_hbm) else ("alu" if t_compute > t_hbm else "hbm")
+        bound = "tensor" if (on_tensor_cores and t_compute > t_hbm) else ("alu" if t_compute > t_hbm else "hbm")
         t_roof = max(t_compute, t_hbm)
         out.append(dict(row, ms=t_ms, bound=bound, roofline_us=t_roof * 1e6, frac=t_roof / (t_ms * 1e-3) if t_ms > 0 else None,
                         gbs=row["bytes"] / (t_ms * 1e-3) / 1e9 if t_ms > 0 else None,
@@ -403,7 +404,7 @@ def run_ours(args):
 
 # DRAM bytes (read + write) per launch of each kernel from the ncu captures summarised under
 # profiles/; None until a capture of the current kernel exists.
-TRAFFIC_BYTES_PER_LAUNCH = {"gemm_tf32": None, "depthwise3x3": None, "conv2d_fp32": None}
+TRAFFIC_BYTES_PER_LAUNCH = {"gemm_tf32": None, "depthwise3x3": None, "conv2d_igemm_tf32": None}
 
 
 def main():

@@ -331,6 +331,19 @@ tfjsb_status tfjsb_conv2d(tfjsb_ctx* ctx, const tfjsb_tensor* x, const tfjsb_ten
             return cuda_fail(ctx, e, "fp32 gemm launch");
         return TFJSB_OK;
     }
+    if (ctx->math == TFJSB_MATH_TF32 && conv_igemm_supported(g) && ctx->encode_tiled) {
+        // implicit GEMM on the tensor cores: the filter is packed [Cout, k_pad] into scratch first
+        const int64_t k_pad = conv_igemm_k_pad(g);
+        if ((st = ensure_scratch(ctx, &ctx->scratch_b, (size_t)Cout * k_pad * 4)) != TFJSB_OK) return st;
+        if ((e = launch_pack_filter(pf, ctx->scratch_b.ptr, (int64_t)g.fh * g.fw * g.C, Cout, k_pad, s, &ctx->launches)) !=
+            cudaSuccess)
+            return cuda_fail(ctx, e, "filter packing");
+        GemmTf32Plan plan;
+        if ((st = conv_igemm_plan(ctx, px, ctx->scratch_b.ptr, py, g, &plan)) != TFJSB_OK) return st;
+        if ((e = launch_gemm_tf32(plan, pbias, act, ctx->dev_status, s, &ctx->launches)) != cudaSuccess)
+            return cuda_fail(ctx, e, "implicit-GEMM conv2d launch");
+        return TFJSB_OK;
+    }
     if ((e = launch_conv2d_fp32(px, pf, pbias, act, py, g, s, &ctx->launches)) != cudaSuccess)
         return cuda_fail(ctx, e, "conv2d launch");
     return TFJSB_OK;

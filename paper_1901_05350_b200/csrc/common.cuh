@@ -120,13 +120,27 @@ struct GemmTf32Plan {
     int64_t M, N, K;
     int block_n;       // 32..256
     int stages;
+    int acc_stages;
     int num_tiles;
     int grid;
     size_t smem_bytes;
+    // implicit-GEMM convolution: A is gathered from x by the kernel instead of copied
+    bool gather = false;
+    const float* x = nullptr;
+    ConvGeom g{};
 };
 bool gemm_tf32_supported(int64_t M, int64_t N, int64_t K);
 tfjsb_status gemm_tf32_plan(tfjsb_ctx* ctx, const float* a, const float* bt, float* c, int64_t M, int64_t N,
                             int64_t K, GemmTf32Plan* plan);
+// Implicit-GEMM convolution on the same kernel: M = N*Ho*Wo output pixels, K = fh*fw*Cin, N = Cout.
+// `bt` is the filter packed as [Cout, k_pad] (K-contiguous, zero padded to a multiple of 32).
+bool conv_igemm_supported(const ConvGeom& g);
+int64_t conv_igemm_k_pad(const ConvGeom& g);
+tfjsb_status conv_igemm_plan(tfjsb_ctx* ctx, const float* x, const float* bt, float* y, const ConvGeom& g,
+                             GemmTf32Plan* plan);
+// out[n, k] = k < K ? f[k, n] : 0 for f of shape [K, N], out of shape [N, k_pad]
+cudaError_t launch_pack_filter(const float* f, float* out, int64_t K, int64_t N, int64_t k_pad, cudaStream_t s,
+                               int64_t* launches);
 cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int act, unsigned int* dev_status,
                              cudaStream_t s, int64_t* launches);
 

@@ -158,7 +158,27 @@ __global__ void transpose_kernel(const float* __restrict__ in, float* __restrict
     }
 }
 
+// ---- filter packing for the implicit-GEMM convolution ------------------------------------------------
+__global__ void pack_filter_kernel(const float* __restrict__ f, float* __restrict__ out, int64_t K, int64_t N,
+                                   int64_t k_pad) {
+    const int64_t total = N * k_pad;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int64_t n = i / k_pad, k = i - n * k_pad;
+        out[i] = k < K ? f[k * N + n] : 0.0f;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_pack_filter(const float* f, float* out, int64_t K, int64_t N, int64_t k_pad, cudaStream_t s,
+                               int64_t* launches) {
+    const int64_t total = N * k_pad;
+    if (total == 0) return cudaSuccess;
+    pack_filter_kernel<<<grid_for(total, kThreads, 148 * 8), kThreads, 0, s>>>(f, out, K, N, k_pad);
+    ++*launches;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_bias_act(const float* x, const float* bias, float* y, int64_t rows, int64_t C, int act,
                             cudaStream_t s, int64_t* launches) {

@@ -16,7 +16,7 @@ using namespace tfjsb;
 
 namespace {
 
-enum StepKind { STEP_GEMM_TF32, STEP_GEMM_FP32, STEP_CONV_FP32, STEP_DEPTHWISE, STEP_POOL, STEP_SOFTMAX };
+enum StepKind { STEP_GEMM_TF32, STEP_GEMM_FP32, STEP_CONV_TF32, STEP_CONV_FP32, STEP_DEPTHWISE, STEP_POOL, STEP_SOFTMAX };
 
 struct Step {
     StepKind kind;
@@ -96,6 +96,11 @@ tfjsb_status bind_step(tfjsb_model* m, Step& st, const float* in, float* out) {
         if (rc != TFJSB_OK) return rc;
         st.plan_built = true;
     }
+    if (st.kind == STEP_CONV_TF32 && (changed || !st.plan_built)) {
+        tfjsb_status rc = conv_igemm_plan(m->ctx, in, st.filter_km, out, st.g, &st.plan);
+        if (rc != TFJSB_OK) return rc;
+        st.plan_built = true;
+    }
     if (st.kind == STEP_DEPTHWISE && (changed || !st.plan_built)) {
         tfjsb_status rc = depthwise_plan(m->ctx, in, st.g, &st.dw_plan);
         if (rc != TFJSB_OK) return rc;
@@ -131,6 +136,7 @@ cudaError_t launch_step(tfjsb_model* m, const Step& st, cudaStream_t s) {
     tfjsb_ctx* ctx = m->ctx;
     switch (st.kind) {
         case STEP_GEMM_TF32:
+        case STEP_CONV_TF32:
             return launch_gemm_tf32(st.plan, st.bias, st.act, ctx->dev_status, s, &ctx->launches);
         case STEP_GEMM_FP32:
             return launch_gemm_fp32(st.in, st.K, 1, st.filter, st.N, 1, st.bias, st.act, st.out, st.N, st.M, st.N, st.K,
@@ -231,7 +237,7 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
                 else if (g.fh == 1 && g.fw == 1 && g.sh == 1 && g.sw == 1) {
                     step.M = g.N * g.H * g.W; step.K = g.C; step.N = g.Co;
                     step.kind = (m->use_tf32 && gemm_tf32_supported(step.M, step.N, step.K)) ? STEP_GEMM_TF32 : STEP_GEMM_FP32;
-                } else step.kind = STEP_CONV_FP32;
+                } else step.kind = (m->use_tf32 && conv_igemm_supported(g)) ? STEP_CONV_TF32 : STEP_CONV_FP32;
                 step.out_rank = 4;
                 step.out_dims[0] = g.N; step.out_dims[1] = g.Ho; step.out_dims[2] = g.Wo; step.out_dims[3] = g.Co;
                 break;
@@ -287,6 +293,14 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
             }
             default:
                 return bail(TFJSB_ERR_INVALID_ARG, where + "unknown layer kind");
+        }
+        if (step.kind == STEP_CONV_TF32) {
+            // filter [fh*fw*Cin, Cout] -> [Cout, k_pad] once, on the device
+            const int64_t k_pad = conv_igemm_k_pad(step.g);
+            if ((st = dev_alloc(m, (size_t)(k_pad * step.g.Co), &step.filter_km)) != TFJSB_OK) return bail(st, ctx->last_error);
+            cudaError_t e = launch_pack_filter(step.filter, step.filter_km, (int64_t)step.g.fh * step.g.fw * step.g.C,
+                                               step.g.Co, k_pad, 0, &ctx->launches);
+            if (e != cudaSuccess) return bail(TFJSB_ERR_CUDA, std::string("packing weights: ") + cudaGetErrorString(e));
         }
         if (step.kind == STEP_GEMM_TF32) {
             // weights [K,N] -> [N,K] once, on the device

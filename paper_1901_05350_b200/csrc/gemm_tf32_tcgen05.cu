@@ -41,16 +41,18 @@ namespace {
 constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 32;  // fp32 elements: one 128-byte swizzle row
 constexpr int UMMA_K = 8;    // tf32 elements per tcgen05.mma
-constexpr int ACC_STAGES = 2;
+constexpr int MAX_ACC_STAGES = 4;
 constexpr int MAX_STAGES = 8;
-constexpr int NUM_THREADS = 320;  // producer warp, MMA warp, 8 epilogue warps
+constexpr int GEMM_THREADS = 320;    // producer warp, MMA warp, 8 epilogue warps
+constexpr int GATHER_GROUPS = 3;     // implicit-GEMM convolution: groups of 4 warps that build A tiles
+constexpr int CONV_THREADS = GEMM_THREADS + GATHER_GROUPS * 128;
 constexpr int EPI_COLS = 32;
 constexpr int A_STAGE_BYTES = BLOCK_M * BLOCK_K * 4;             // 16 KiB
 constexpr int EPI_SLAB_BYTES = 32 * EPI_COLS * 4;                // 4 KiB: 32 rows x 128 B
 constexpr int EPI_BYTES = 8 /*epilogue warps*/ * EPI_SLAB_BYTES;      // 32 KiB
 constexpr int SMEM_LIMIT = 232448;                               // 227 KiB
 
-// ---- PTX wrappers ----------------------------------------------------w per lane: bias add,
+// Fused epilogue of one 32-row x 32-column accumulator block held one row per lane: bias add,
 // activation, and the swizzled store into the staging slab the bulk tensor store reads from
 // (16-byte chunk j of row `lane` lives at chunk j ^ (lane % 8): the 128-byte swizzle).
 template <int ACT>
@@ -80,32 +82,117 @@ __device__ __forceinline__ void stage_chunk(const uint32_t (&r)[32], const float
     }
 }
 
+// ---- A-row gathers of the implicit-GEMM convolution ---------------------------------------------
+// Each fills v[0..31] with columns k0..k0+31 of one row of the im2col matrix: k = (ky*fw + kx)*Cin + ci
+// -> x[iy0 + ky*dh, ix0 + kx*dw, ci], zero outside the image, for k >= k_total and for dead rows.
+
+// Window and channel count known at compile time and fh*fw*Cin <= 32 (one k-block): no index
+// arithmetic is left at run time beyond three row pointers and six bounds flags.
+template <int FH, int FW, int CIN>
+__device__ __forceinline__ void gather_small(float (&v)[BLOCK_K], const float* __restrict__ xn, const ConvGeom& g,
+                                             int iy0, int ix0, bool live) {
+    static_assert(FH * FW * CIN <= BLOCK_K, "one k-block only");
+    const float* rowp[FH];
+    bool vy[FH], vx[FW];
+#pragma unroll
+    for (int ky = 0; ky < FH; ++ky) {
+        const int iy = iy0 + ky * g.dh;
+        vy[ky] = live && iy >= 0 && iy < g.H;
+        rowp[ky] = xn + ((int64_t)iy * g.W + ix0) * CIN;
+    }
+#pragma unroll
+    for (int kx = 0; kx < FW; ++kx) {
+        const int ix = ix0 + kx * g.dw;
+        vx[kx] = ix >= 0 && ix < g.W;
+    }
+    const int dwc = g.dw * CIN;
+#pragma unroll
+    for (int e = 0; e < BLOCK_K; ++e) {
+        if (e < FH * FW * CIN) {
+            const int ky = e / (FW * CIN), kx = (e / CIN) % FW, ci = e % CIN;
+            v[e] = (vy[ky] && vx[kx]) ? __ldg(rowp[ky] + kx * dwc + ci) : 0.0f;
+        } else {
+            v[e] = 0.0f;
+        }
+    }
+}
+
+// Cin % 4 == 0: four consecutive k share a tap, so each quad is one float4 load.
+__device__ __forceinline__ void gather_vec4(float (&v)[BLOCK_K], const float* __restrict__ xn, const ConvGeom& g,
+                                            int iy0, int ix0, bool live, int k0, int k_total) {
+    int tap = k0 / g.C;
+    int ci = k0 - tap * g.C;
+    int ky = tap / g.fw;
+    int kx = tap - ky * g.fw;
+#pragma unroll
+    for (int e = 0; e < BLOCK_K; e += 4) {
+        float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
+        const int iy = iy0 + ky * g.dh, ix = ix0 + kx * g.dw;
+        if (live && k0 + e < k_total && iy >= 0 && iy < g.H && ix >= 0 && ix < g.W)
+            q = __ldg(reinterpret_cast<const float4*>(xn + ((int64_t)iy * g.W + ix) * g.C + ci));
+        v[e] = q.x; v[e + 1] = q.y; v[e + 2] = q.z; v[e + 3] = q.w;
+        ci += 4;
+        if (ci == g.C) { ci = 0; if (++kx == g.fw) { kx = 0; ++ky; } }
+    }
+}
+
+// Any window and channel count: a pointer walks the tap, re-based when the tap column or row changes.
+__device__ __forceinline__ void gather_scalar(float (&v)[BLOCK_K], const float* __restrict__ xn, const ConvGeom& g,
+                                              int iy0, int ix0, bool live, int k0, int k_total) {
+    int tap = k0 / g.C;
+    int ci = k0 - tap * g.C;
+    int ky = tap / g.fw;
+    int kx = tap - ky * g.fw;
+    int iy = iy0 + ky * g.dh, ix = ix0 + kx * g.dw;
+    const float* p = xn + ((int64_t)iy * g.W + ix) * g.C + ci;
+    bool ok = live && iy >= 0 && iy < g.H && ix >= 0 && ix < g.W;
+    const int left = k_total - k0;
+#pragma unroll
+    for (int e = 0; e < BLOCK_K; ++e) {
+        v[e] = (ok && e < left) ? __ldg(p) : 0.0f;
+        ++p;
+        if (++ci == g.C) {
+            ci = 0;
+            if (++kx == g.fw) { kx = 0; ++ky; }
+            iy = iy0 + ky * g.dh;
+            ix = ix0 + kx * g.dw;
+            p = xn + ((int64_t)iy * g.W + ix) * g.C;
+            ok = live && iy >= 0 && iy < g.H && ix >= 0 && ix < g.W;
+        }
+    }
+}
+
 struct KernelArgs {
     int M, N, K;
     int block_n;
     int stages;
     int n_tiles;    // tiles along N
     int num_tiles;  // total
+    int acc_stages;  // accumulator stages in tensor memory: 2 (block_n 256) or 4
     const float* bias;
     int act;
     unsigned int* dev_status;
+    // implicit-GEMM convolution only: the input tensor and its geometry (A is gathered, not copied)
+    const float* x;
+    ConvGeom g;
 };
 
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+template <bool GATHER>
+__global__ void __launch_bounds__(GATHER ? CONV_THREADS : GEMM_THREADS, 1)
 gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const __grid_constant__ CUtensorMap map_c, const KernelArgs args) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[MAX_STAGES];
     __shared__ __align__(8) uint64_t bar_empty[MAX_STAGES];
-    __shared__ __align__(8) uint64_t bar_acc_full[ACC_STAGES];
-    __shared__ __align__(8) uint64_t bar_acc_empty[ACC_STAGES];
+    __shared__ __align__(8) uint64_t bar_acc_full[MAX_ACC_STAGES];
+    __shared__ __align__(8) uint64_t bar_acc_empty[MAX_ACC_STAGES];
     __shared__ __align__(8) uint64_t bar_drain;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
 
     volatile int* abort_flag = &abort_flag_s;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int block_n = args.block_n, stages = args.stages;
+    const int block_n = args.block_n, stages = args.stages, acc_stages = args.acc_stages;
     const int stage_bytes = A_STAGE_BYTES + block_n * BLOCK_K * 4;
     const int num_k_blocks = (args.K + BLOCK_K - 1) / BLOCK_K;
 
@@ -117,21 +204,23 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
-            mbar_init(smem_u32(&bar_full[s]), 1);
+            // a stage is full when the copy engine has delivered its bytes and, for the convolution,
+            // the four warps of one gather group have written the A tile
+            mbar_init(smem_u32(&bar_full[s]), GATHER ? 5 : 1);
             mbar_init(smem_u32(&bar_empty[s]), 1);
         }
-        for (int s = 0; s < ACC_STAGES; ++s) {
+        for (int s = 0; s < acc_stages; ++s) {
             mbar_init(smem_u32(&bar_acc_full[s]), 1);
             mbar_init(smem_u32(&bar_acc_empty[s]), 8);
         }
         mbar_init(smem_u32(&bar_drain), 1);
         abort_flag_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+        if (!GATHER) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
     }
-    const uint32_t tmem_cols = (uint32_t)(ACC_STAGES * block_n);  // 64, 128, 256 or 512: a power of two >= 32
+    const uint32_t tmem_cols = (uint32_t)(acc_stages * block_n);  // 128, 256 or 512: a power of two >= 32
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                          smem_u32(&tmem_base_slot)),
@@ -156,6 +245,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
                 const int m0 = (tile / args.n_tiles) * BLOCK_M;
                 const int n0 = (tile % args.n_tiles) * block_n;
+                (void)m0;
                 for (int kb = 0; kb < num_k_blocks; ++kb) {
                     if (!bounded_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_flag)) {
                         if (!*abort_flag) {
@@ -167,8 +257,12 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     }
                     const uint32_t full = smem_u32(&bar_full[stage]);
                     const uint32_t a_dst = stage_base + (uint32_t)stage * (uint32_t)stage_bytes;
-                    mbar_arrive_expect_tx(full, (uint32_t)stage_bytes);
-                    tma_load_2d(a_dst, &map_a, full, kb * BLOCK_K, m0);
+                    if (GATHER) {
+                        mbar_arrive_expect_tx(full, (uint32_t)(stage_bytes - A_STAGE_BYTES));
+                    } else {
+                        mbar_arrive_expect_tx(full, (uint32_t)stage_bytes);
+                        tma_load_2d(a_dst, &map_a, full, kb * BLOCK_K, m0);
+                    }
                     tma_load_2d(a_dst + A_STAGE_BYTES, &map_b, full, kb * BLOCK_K, n0);
 #pragma unroll
                     for (int s = 0; s < MAX_STAGES; ++s)
@@ -225,7 +319,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 }
                 if (!ok) break;
                 tc_commit(smem_u32(&bar_acc_full[acc]));
-                if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+                if (++acc == acc_stages) { acc = 0; acc_phase ^= 1u; }
             }
             if (!ok) {
                 if (!*abort_flag) {
@@ -245,10 +339,11 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 }
             }
         }
-    } else {
+    } else if (warp < 10) {
         // ---------------------------------------------------------------- epilogue (warps 2..9)
-        // Two warps share each TMEM lane quadrant (a warp may only read lanes 32*(warp%4)..+31):
-        // the first of the pair takes the even 32-column chunks of a tile, the second the odd ones.
+        // Two warps share each TMEM lane quadrant (a warp may only read lanes 32*(warp%4)..+31) and
+        // take alternate 32-column chunks, counted across tiles so that with one chunk per tile they
+        // alternate tiles.
         const int ew = warp - 2;
         const int quad = warp & 3;
         const int half = ew >> 2;
@@ -256,6 +351,8 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
+        const int chunks_per_tile = block_n / EPI_COLS;
+        int first_chunk = half;  // parity bookkeeping: chunk `ch` of this tile is ours when (ch - first_chunk) is even
         for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
             const int m0 = (tile / args.n_tiles) * BLOCK_M;
             const int n0 = (tile % args.n_tiles) * block_n;
@@ -277,7 +374,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             if (live_cols < block_n) n_chunks = (live_cols + EPI_COLS - 1) / EPI_COLS;
             const bool rows_live = row0 < args.M;
             bool released = false;
-            for (int ch = half; ch < n_chunks; ch += 2) {
+            for (int ch = first_chunk; ch < n_chunks; ch += 2) {
                 uint32_t r[32];
                 const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * block_n + ch * EPI_COLS);
                 tc_ld_32x32(taddr, r);
@@ -312,10 +409,77 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
             }
-            if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+            if (chunks_per_tile & 1) first_chunk ^= 1;
+            if (++acc == acc_stages) { acc = 0; acc_phase ^= 1u; }
         }
         if (lane == 0) tma_store_wait_all();
         __syncwarp();
+    }
+
+    else if (GATHER) {
+        // ---------------------------------------------------------------- A-tile gather (warps 10..)
+        // Implicit GEMM: row p of A is output pixel p = (n, oy, ox); column k = (ky*fw + kx)*Cin + ci
+        // is the input sample that pixel sees through filter tap (ky, kx) at channel ci, zero outside
+        // the image and for k >= fh*fw*Cin.  One thread builds one row of a 128 x 32 tile (32 loads in
+        // flight) and writes it in the 128-byte-swizzled layout the tensor core reads; the groups take
+        // k-blocks in turn so that several tiles' loads are outstanding at once.
+        const ConvGeom& g = args.g;
+        const int gw = warp - 10;
+        const int group = gw >> 2;
+        const int row = ((gw & 3) << 5) + lane;
+        const bool vec4 = (g.C & 3) == 0;
+        const bool small333 = g.fh == 3 && g.fw == 3 && g.C == 3;  // the usual RGB stem: everything compile-time
+        const int k_total = g.fh * g.fw * g.C;
+        int stage = 0;
+        uint32_t phase = 0;
+        int turn = 0;  // which group's turn the next k-block is
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
+            const int m0 = (tile / args.n_tiles) * BLOCK_M;
+            const int p = m0 + row;
+            const bool live = p < args.M;
+            int iy0 = 0, ix0 = 0;
+            const float* xn = args.x;
+            if (live) {
+                const int hw = g.Ho * g.Wo;
+                const int n = p / hw;
+                const int rem = p - n * hw;
+                const int oy = rem / g.Wo, ox = rem - oy * g.Wo;
+                iy0 = oy * g.sh - g.pt;
+                ix0 = ox * g.sw - g.pl;
+                xn = args.x + (int64_t)n * g.H * g.W * g.C;
+            }
+            for (int kb = 0; kb < num_k_blocks; ++kb) {
+                if (turn == group) {
+                    const bool got = bounded_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_flag);
+                    if (!__all_sync(0xffffffffu, got)) {
+                        if (lane == 0 && !*abort_flag) {
+                            *abort_flag = 1;
+                            atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_PRODUCER);
+                        }
+                        ok = false;
+                        break;
+                    }
+                    float v[BLOCK_K];
+                    if (small333) gather_small<3, 3, 3>(v, xn, g, iy0, ix0, live);
+                    else if (vec4) gather_vec4(v, xn, g, iy0, ix0, live, kb * BLOCK_K, k_total);
+                    else gather_scalar(v, xn, g, iy0, ix0, live, kb * BLOCK_K, k_total);
+                    const uint32_t row_addr = stage_base + (uint32_t)stage * (uint32_t)stage_bytes + (uint32_t)row * 128u;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t dst = row_addr + (uint32_t)((j ^ (row & 7)) << 4);
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[4 * j]), "f"(v[4 * j + 1]),
+                                     "f"(v[4 * j + 2]), "f"(v[4 * j + 3])
+                                     : "memory");
+                    }
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bar_full[stage]));
+                }
+                if (++turn == GATHER_GROUPS) turn = 0;
+                if (++stage == stages) { stage = 0; phase ^= 1u; }
+            }
+        }
     }
 
     // ---------------------------------------------------------------- teardown
@@ -359,12 +523,13 @@ bool gemm_tf32_supported(int64_t M, int64_t N, int64_t K) {
            K < (1LL << 31) - 256 && ((M + BLOCK_M - 1) / BLOCK_M) * ((N + 31) / 32) < (1LL << 31);
 }
 
-tfjsb_status gemm_tf32_plan(tfjsb_ctx* ctx, const float* a, const float* bt, float* c, int64_t M, int64_t N,
-                            int64_t K, GemmTf32Plan* plan) {
-    if (!gemm_tf32_supported(M, N, K)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the TF32 GEMM");
-    if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
-    plan->M = M; plan->N = N; plan->K = K;
+namespace {
+
+// tile choice, pipeline depth and the B / C tensor maps shared by the GEMM and the convolution
+tfjsb_status plan_common(tfjsb_ctx* ctx, const float* bt, int64_t k_pitch, float* c, GemmTf32Plan* plan) {
+    const int64_t M = plan->M, N = plan->N;
     plan->block_n = choose_block_n(M, N, ctx->sm_count);
+    plan->acc_stages = plan->block_n == 256 ? 2 : MAX_ACC_STAGES;
     const int stage_bytes = A_STAGE_BYTES + plan->block_n * BLOCK_K * 4;
     int stages = (SMEM_LIMIT - 1024 - EPI_BYTES - 512) / stage_bytes;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
@@ -375,9 +540,50 @@ tfjsb_status gemm_tf32_plan(tfjsb_ctx* ctx, const float* a, const float* bt, flo
     plan->num_tiles = (int)tiles;
     plan->grid = (int)(tiles < ctx->sm_count ? tiles : ctx->sm_count);
     tfjsb_status st;
-    if ((st = encode_2d(ctx, &plan->map_a, a, K, M, BLOCK_K, BLOCK_M, "A")) != TFJSB_OK) return st;
-    if ((st = encode_2d(ctx, &plan->map_b, bt, K, N, BLOCK_K, plan->block_n, "B")) != TFJSB_OK) return st;
+    if ((st = encode_2d(ctx, &plan->map_b, bt, k_pitch, N, BLOCK_K, plan->block_n, "B")) != TFJSB_OK) return st;
     if ((st = encode_2d(ctx, &plan->map_c, c, N, M, EPI_COLS, 32, "C")) != TFJSB_OK) return st;
+    return TFJSB_OK;
+}
+
+}  // namespace
+
+tfjsb_status gemm_tf32_plan(tfjsb_ctx* ctx, const float* a, const float* bt, float* c, int64_t M, int64_t N,
+                            int64_t K, GemmTf32Plan* plan) {
+    if (!gemm_tf32_supported(M, N, K)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the TF32 GEMM");
+    if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+    plan->M = M; plan->N = N; plan->K = K;
+    plan->gather = false;
+    plan->x = nullptr;
+    tfjsb_status st;
+    if ((st = plan_common(ctx, bt, K, c, plan)) != TFJSB_OK) return st;
+    return encode_2d(ctx, &plan->map_a, a, K, M, BLOCK_K, BLOCK_M, "A");
+}
+
+int64_t conv_igemm_k_pad(const ConvGeom& g) {
+    const int64_t k = (int64_t)g.fh * g.fw * g.C;
+    return (k + BLOCK_K - 1) / BLOCK_K * BLOCK_K;
+}
+
+bool conv_igemm_supported(const ConvGeom& g) {
+    const int64_t M = g.N * g.Ho * g.Wo;
+    const int64_t K = (int64_t)g.fh * g.fw * g.C;
+    return M >= 1 && g.Co >= 4 && (g.Co % 4 == 0) && K >= 1 && K < (1 << 24) && M < (1LL << 31) - 256 &&
+           (int64_t)g.H * g.W * g.C < (1LL << 31) && ((M + BLOCK_M - 1) / BLOCK_M) * ((g.Co + 31) / 32) < (1LL << 31);
+}
+
+tfjsb_status conv_igemm_plan(tfjsb_ctx* ctx, const float* x, const float* bt, float* y, const ConvGeom& g,
+                             GemmTf32Plan* plan) {
+    if (!conv_igemm_supported(g)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the implicit-GEMM convolution");
+    if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+    plan->M = g.N * g.Ho * g.Wo;
+    plan->N = g.Co;
+    plan->K = (int64_t)g.fh * g.fw * g.C;
+    plan->gather = true;
+    plan->x = x;
+    plan->g = g;
+    tfjsb_status st = plan_common(ctx, bt, conv_igemm_k_pad(g), y, plan);
+    if (st != TFJSB_OK) return st;
+    plan->map_a = plan->map_b;  // unused by the gathering kernel; kept initialised
     return TFJSB_OK;
 }
 
@@ -385,8 +591,11 @@ cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int ac
                              cudaStream_t s, int64_t* launches) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemm_tf32_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              SMEM_LIMIT - 2048);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(gemm_tf32_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     SMEM_LIMIT - 2048);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -396,10 +605,16 @@ cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int ac
     args.stages = plan.stages;
     args.n_tiles = (int)((plan.N + plan.block_n - 1) / plan.block_n);
     args.num_tiles = plan.num_tiles;
+    args.acc_stages = plan.acc_stages;
     args.bias = bias;
     args.act = act;
     args.dev_status = dev_status;
-    gemm_tf32_kernel<<<plan.grid, NUM_THREADS, plan.smem_bytes, s>>>(plan.map_a, plan.map_b, plan.map_c, args);
+    args.x = plan.x;
+    args.g = plan.g;
+    if (plan.gather)
+        gemm_tf32_kernel<true><<<plan.grid, CONV_THREADS, plan.smem_bytes, s>>>(plan.map_a, plan.map_b, plan.map_c, args);
+    else
+        gemm_tf32_kernel<false><<<plan.grid, GEMM_THREADS, plan.smem_bytes, s>>>(plan.map_a, plan.map_b, plan.map_c, args);
     ++*launches;
     return cudaGetLastError();
 }

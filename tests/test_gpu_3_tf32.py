@@ -108,6 +108,39 @@ def test_pointwise_conv_tf32_fused_epilogue(ctx, oracle, shape, act):
                      oracle.conv2d(xi, fi, bias=bi, act=act))
 
 
+IGEMM_CASES = [
+    # N, H, W, Cin, fh, fw, Cout, strides, pad, dilations: conv2d as an implicit GEMM on the tensor cores
+    (1, 224, 224, 3, 3, 3, 32, (2, 2), "same", (1, 1)),   # the stem of the 224 models (K = 27, scalar gather)
+    (2, 33, 29, 3, 3, 3, 8, (2, 2), "same", (1, 1)),
+    (1, 17, 19, 5, 3, 3, 40, (1, 1), "same", (1, 1)),     # K = 45: two k-blocks, the second mostly padding
+    (1, 20, 20, 16, 3, 3, 36, (2, 2), "valid", (1, 1)),   # Cin % 4 == 0: float4 gather, K = 144
+    (1, 15, 15, 4, 3, 3, 8, (1, 1), "same", (2, 2)),      # dilation
+    (1, 12, 14, 7, 5, 3, 12, (3, 2), "same", (1, 1)),     # 5x3 window, unequal strides
+    (3, 9, 9, 30, 1, 1, 52, (2, 2), "same", (1, 1)),      # strided 1x1
+    (1, 6, 6, 72, 3, 3, 4, (1, 1), "valid", (1, 1)),      # K = 648: the stage ring wraps
+    (5, 40, 40, 8, 3, 3, 260, (1, 1), "same", (1, 1)),    # Cout just above one 256-wide tile, many pixel tiles
+]
+
+
+@pytest.mark.parametrize("case", IGEMM_CASES)
+def test_conv2d_implicit_gemm_tf32(ctx, oracle, case):
+    N, H, W, Cin, fh, fw, Cout, strides, pad, dil = case
+    x = si.uniform(309, 0, (N, H, W, Cin), -1, 1)
+    f = si.normal(309, 1, (fh, fw, Cin, Cout), 0, float(np.sqrt(2.0 / (fh * fw * Cin))))
+    b = si.normal(309, 2, (Cout,), 0, 0.5)
+    got = host(ctx.conv2d(dev(x), dev(f), strides, pad, dil, dev(b), "relu6"))
+    ctx.check_device_status()
+    want = oracle.conv2d(x, f, strides, pad, dil, b, "relu6")
+    assert got.shape == want.shape
+    assert rel_fro(got, want) <= TF32_TOL
+    matched = oracle.conv2d(x, f, strides, pad, dil, b, "relu6", operand="tf32_rz")
+    assert rel_fro(got, matched) <= MATCHED_TOL
+    xi = si.small_integers(310, 0, x.shape, -4, 4)
+    fi = si.small_integers(310, 1, f.shape, -4, 4)
+    assert same_bits(host(ctx.conv2d(dev(xi), dev(fi), strides, pad, dil)), oracle.conv2d(xi, fi, strides, pad, dil))
+    ctx.check_device_status()
+
+
 def test_separable_block_config2(ctx, oracle):
     x, layers = si.config_separable_block()
     dw, pw = layers
