@@ -61,7 +61,9 @@ class LayerDesc(ctypes.Structure):
 
 
 def _load_library() -> ctypes.CDLL:
-    path = _build.build()
+    # TFJSB_LIBRARY points at an already built libtfjsb.so (e.g. an instrumented build); otherwise the
+    # library is (re)built in-tree when its sources are newer
+    path = os.environ.get("TFJSB_LIBRARY") or _build.build()
     lib = ctypes.CDLL(path)
     vp, i32, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
     tp = ctypes.POINTER(Tensor)

@@ -25,13 +25,30 @@ enum : unsigned int {
 };
 
 // ---- fused epilogue (bias add, then activation), identical in every kernel -----------------
-//   v = acc + bias ; relu: v > 0 ? v : +0 (NaN stays NaN) ; relu6: min(relu(v), 6)
-__device__ __forceinline__ float apply_act(float v, int act) {
-    if (act == TFJSB_ACT_NONE) return v;
-    if (v != v) return v;
-    float r = v > 0.0f ? v : 0.0f;
-    if (act == TFJSB_ACT_RELU6) r = r > 6.0f ? 6.0f : r;
+//   v = acc + bias ; relu: v > 0 ? v : +0 (NaN stays NaN, -0 -> +0) ; relu6: min(relu(v), 6)
+// max.NaN / min.NaN return NaN when an input is NaN and order -0 below +0, which is exactly that
+// definition in two instructions (a compare-and-select chain costs four times as many, and the
+// bandwidth-bound kernels turned out to be bound by instruction issue).
+__device__ __forceinline__ float relu_nan(float v) {
+    float r;
+    asm("max.NaN.f32 %0, %1, 0f00000000;" : "=f"(r) : "f"(v));
     return r;
+}
+__device__ __forceinline__ float relu6_nan(float v) {
+    float r;
+    asm("max.NaN.f32 %0, %1, 0f00000000;\n\tmin.NaN.f32 %0, %0, 0f40C00000;" : "=f"(r) : "f"(v));
+    return r;
+}
+__device__ __forceinline__ float apply_act(float v, int act) {
+    const float r = relu_nan(v);
+    const float r6 = relu6_nan(v);
+    return act == TFJSB_ACT_NONE ? v : (act == TFJSB_ACT_RELU6 ? r6 : r);
+}
+template <int ACT>
+__device__ __forceinline__ float apply_act_t(float v) {
+    if (ACT == TFJSB_ACT_NONE) return v;
+    if (ACT == TFJSB_ACT_RELU6) return relu6_nan(v);
+    return relu_nan(v);
 }
 
 // ---- context --------------------------------------------------------------------------------

@@ -19,10 +19,11 @@
 // kernel above is bound by load latency, not bandwidth (its loads sit in registers, ~80 per thread,
 // so few warps fit and few bytes are in flight).  `depthwise3x3_tma_kernel` keeps the bytes in
 // flight in shared memory instead: persistent CTAs walk tiles of TH x TW output pixels x 32
-// channels; one thread issues the bulk tensor copy (TMA) of the next tiles' input patches
+// channels; a producer warp issues the bulk tensor copy (TMA) of the next tiles' input patches
 // ((TH-1)*S+3 rows x (TW-1)*S+3 columns x 128 bytes, zero-filled outside the image, which is the
-// 'same' padding) into a ring of stages while all 256 threads compute the current tile from
-// shared memory with the same sliding-row scheme and store float4s straight to global memory.
+// 'same' padding) into a ring of stages (full / empty mbarriers) while eight compute warps work
+// on the landed tiles from shared memory with the same sliding-row scheme and store float4s
+// straight to global memory.
 #include "common.cuh"
 #include "ptx_sm100.cuh"
 
@@ -151,14 +152,17 @@ struct DwTile {
     static constexpr int STAGE_BYTES = STAGE_FLOATS * 4;
 };
 
+constexpr int DW_TMA_THREADS = DW_THREADS + 32;  // eight compute warps and the warp that issues the copies
+
 template <int S, int TW, int R>
-__global__ void __launch_bounds__(DW_THREADS, 2)
+__global__ void __launch_bounds__(DW_TMA_THREADS, 2)
 depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __restrict__ f,
                         const float* __restrict__ bias, int act, float* __restrict__ y, ConvGeom g, DwTiling t,
                         unsigned int* dev_status) {
     using T = DwTile<S, TW, R>;
     extern __shared__ uint8_t dw_smem_raw[];
-    __shared__ __align__(8) uint64_t bar_full[DW_MAX_STAGES];
+    __shared__ __align__(8) uint64_t bar_full[DW_MAX_STAGES];   // copy landed (1 arrival + bytes)
+    __shared__ __align__(8) uint64_t bar_empty[DW_MAX_STAGES];  // the eight compute warps are done with the stage
     __shared__ int4 tile_info[DW_MAX_STAGES];
     __shared__ int abort_flag_s;
     volatile int* abort_flag = &abort_flag_s;
@@ -166,80 +170,104 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
     const uint32_t smem_base = (ptx::smem_u32(dw_smem_raw) + 127u) & ~127u;
     const float* smem_f = reinterpret_cast<const float*>(dw_smem_raw + (smem_base - ptx::smem_u32(dw_smem_raw)));
     const int tid = threadIdx.x;
-    const int c4 = tid & 7;
-    const int col = (tid >> 3) % TW;
-    const int rg = tid / (8 * TW);
+    const int warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
-        for (int s = 0; s < t.stages; ++s) ptx::mbar_init(ptx::smem_u32(&bar_full[s]), 1);
+        for (int s = 0; s < t.stages; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&bar_full[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&bar_empty[s]), DW_THREADS / 32);
+        }
         abort_flag_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
     }
     __syncthreads();
 
-    // tile index -> (channel block, tile column, tile row, image); channel block fastest so that CTAs
-    // running side by side touch neighbouring 128-byte lines of the same pixels.  Only the issuing
-    // thread pays for the divisions: it leaves the coordinates beside the stage for everyone else
-    // (written before its mbarrier arrive, read after the wait: release / acquire).
-    auto issue = [&](int tile, int slot) {
-        const int cb = tile % t.c_blocks;
-        int q = tile / t.c_blocks;
-        const int tx = q % t.tiles_x; q /= t.tiles_x;
-        const int ty = q % t.tiles_y;
-        const int n = q / t.tiles_y;
-        tile_info[slot] = make_int4(cb, tx, ty, n);
-        const uint32_t bar = ptx::smem_u32(&bar_full[slot]);
-        ptx::mbar_arrive_expect_tx(bar, (uint32_t)T::STAGE_BYTES);
-        ptx::tma_load_4d(smem_base + (uint32_t)slot * (uint32_t)T::STAGE_BYTES, &map_x, bar, cb * DW_CB,
-                         tx * TW * S - g.pl, ty * T::TH * S - g.pt, n);
-    };
-
     const int num_tiles = (int)t.num_tiles;
     const int first = blockIdx.x, step = gridDim.x;
     const int my_tiles = first < num_tiles ? (num_tiles - first + step - 1) / step : 0;
-    int issued = 0;  // tiles handed to the copy engine so far (thread 0 only)
-    if (tid == 0) {
-        for (; issued < t.stages - 1 && issued < my_tiles; ++issued) issue(first + issued * step, issued);
+
+    if (warp == DW_THREADS / 32) {
+        // ------------------------------------------------------------ producer: one thread
+        // tile index -> (channel block, tile column, tile row, image), channel block fastest.  Only this
+        // thread pays for the divisions: it leaves the coordinates beside the stage for the compute
+        // warps (written before its mbarrier arrive, read after their wait: release / acquire).
+        if (lane == 0) {
+            int slot = 0;
+            uint32_t parity = 0;
+            int i = 0;
+            bool ok = true;
+            for (; i < my_tiles; ++i) {
+                if (!ptx::bounded_wait(ptx::smem_u32(&bar_empty[slot]), parity ^ 1u, abort_flag)) { ok = false; break; }
+                const int tile = first + i * step;
+                const int cb = tile % t.c_blocks;
+                int q = tile / t.c_blocks;
+                const int tx = q % t.tiles_x; q /= t.tiles_x;
+                const int ty = q % t.tiles_y;
+                const int n = q / t.tiles_y;
+                tile_info[slot] = make_int4(cb, tx, ty, n);
+                const uint32_t bar = ptx::smem_u32(&bar_full[slot]);
+                ptx::mbar_arrive_expect_tx(bar, (uint32_t)T::STAGE_BYTES);
+                ptx::tma_load_4d(smem_base + (uint32_t)slot * (uint32_t)T::STAGE_BYTES, &map_x, bar, cb * DW_CB,
+                                 tx * TW * S - g.pl, ty * T::TH * S - g.pt, n);
+                if (++slot == t.stages) { slot = 0; parity ^= 1u; }
+            }
+            if (!ok || *abort_flag) {
+                if (!*abort_flag) *abort_flag = 1;
+                atomicOr(dev_status, DEV_STATUS_TIMEOUT_DEPTHWISE);
+                // wait (bounded) for the copies still in flight so nothing lands after the CTA has gone
+                const int lo = i - t.stages > 0 ? i - t.stages : 0;
+                for (int k = lo; k < i; ++k) {
+                    const unsigned long long t0 = ptx::global_ns();
+                    while (!ptx::mbar_try_wait(ptx::smem_u32(&bar_full[k % t.stages]), (uint32_t)((k / t.stages) & 1))) {
+                        if (ptx::global_ns() - t0 > ptx::WAIT_LIMIT_NS) {
+                            atomicOr(dev_status, DEV_STATUS_TIMEOUT_DRAIN);
+                            break;
+                        }
+                    }
+                }
+            }
+        }
+        return;
     }
 
-    int i = 0;
+    // ---------------------------------------------------------------- compute warps
+    // The warps never synchronise with each other: each waits for the stage, does its share of the
+    // tile and reports the stage free, so a fast warp can run up to `stages` tiles ahead of a slow one.
+    const int c4 = tid & 7;
+    const int col = (tid >> 3) % TW;
+    const int rg = tid / (8 * TW);
+    const int64_t row_pitch = (int64_t)g.Wo * g.Co;
+
+    float4 w[9];
+    float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+    int loaded_cb = -1;
     int slot = 0;
     uint32_t parity = 0;
-    bool ok = true;
-    for (; i < my_tiles; ++i) {
+    for (int i = 0; i < my_tiles; ++i) {
         const bool got = ptx::bounded_wait(ptx::smem_u32(&bar_full[slot]), parity, abort_flag);
-        // also the barrier that says everyone is done with the previous tile's stage
-        if (!__syncthreads_and(got ? 1 : 0)) { ok = false; break; }
-        if (tid == 0 && issued < my_tiles) {
-            int ahead_slot = slot + t.stages - 1;
-            if (ahead_slot >= t.stages) ahead_slot -= t.stages;
-            issue(first + issued * step, ahead_slot);
-            ++issued;
+        if (!__all_sync(0xffffffffu, got)) {
+            if (lane == 0) *abort_flag = 1;
+            break;
         }
         const int4 info = tile_info[slot];
         const int cb = info.x, tx = info.y, ty = info.z;
-        const long long n = info.w;
-        const int cur_slot = slot;
-        if (++slot == t.stages) { slot = 0; parity ^= 1u; }
         const int c = cb * DW_CB + c4 * 4;
         const int ox = tx * TW + col;
         const int oy0 = ty * T::TH + rg * R;
         const bool live = c < g.C && ox < g.Wo && oy0 < g.Ho;
 
-        float4 w[9];
-        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
         if (live) {
+            if (cb != loaded_cb) {
 #pragma unroll
-            for (int k = 0; k < 9; ++k) w[k] = __ldg(reinterpret_cast<const float4*>(f + (int64_t)k * g.C + c));
-            if (bias) b = __ldg(reinterpret_cast<const float4*>(bias + c));
-        }
-        float4 acc[R];
+                for (int k = 0; k < 9; ++k) w[k] = __ldg(reinterpret_cast<const float4*>(f + (int64_t)k * g.C + c));
+                if (bias) b = __ldg(reinterpret_cast<const float4*>(bias + c));
+                loaded_cb = cb;
+            }
+            float4 acc[R];
 #pragma unroll
-        for (int r = 0; r < R; ++r) acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-
-        if (live) {
-            const float* patch = smem_f + (size_t)cur_slot * T::STAGE_FLOATS + ((rg * R * S) * T::TWIN + col * S) * DW_CB + c4 * 4;
+            for (int r = 0; r < R; ++r) acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+            const float* patch = smem_f + (size_t)slot * T::STAGE_FLOATS + ((rg * R * S) * T::TWIN + col * S) * DW_CB + c4 * 4;
             constexpr int IN_ROWS = (R - 1) * S + 3;
 #pragma unroll
             for (int j = 0; j < IN_ROWS; ++j) {
@@ -255,32 +283,25 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
                     }
                 }
             }
+            // the stage has been read: hand it back before the stores go out
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bar_empty[slot]));
+            float* yp = y + (((int64_t)info.w * g.Ho + oy0) * g.Wo + ox) * g.Co + c;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                const int oy = oy0 + r;
-                if (oy < g.Ho) {
+                if (oy0 + r < g.Ho) {
                     float4 v = acc[r];
                     v.x = apply_act(v.x + b.x, act); v.y = apply_act(v.y + b.y, act);
                     v.z = apply_act(v.z + b.z, act); v.w = apply_act(v.w + b.w, act);
-                    *reinterpret_cast<float4*>(y + ((n * g.Ho + oy) * (int64_t)g.Wo + ox) * g.Co + c) = v;
+                    *reinterpret_cast<float4*>(yp) = v;
                 }
+                yp += row_pitch;
             }
+        } else {
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bar_empty[slot]));
         }
-    }
-
-    if (!ok && tid == 0) {
-        if (!*abort_flag) *abort_flag = 1;
-        atomicOr(dev_status, DEV_STATUS_TIMEOUT_DEPTHWISE);
-        // wait (bounded) for the copies still in flight so nothing lands after the CTA has gone
-        for (int k = i; k < issued; ++k) {
-            const unsigned long long t0 = ptx::global_ns();
-            while (!ptx::mbar_try_wait(ptx::smem_u32(&bar_full[k % t.stages]), (uint32_t)((k / t.stages) & 1))) {
-                if (ptx::global_ns() - t0 > ptx::WAIT_LIMIT_NS) {
-                    atomicOr(dev_status, DEV_STATUS_TIMEOUT_DRAIN);
-                    break;
-                }
-            }
-        }
+        if (++slot == t.stages) { slot = 0; parity ^= 1u; }
     }
 }
 
@@ -308,7 +329,7 @@ cudaError_t launch_tma_instance(const DepthwisePlan& plan, const float* f, const
         attr_set = true;
     }
     DwTiling t{plan.tiles_x, plan.tiles_y, plan.c_blocks, plan.stages, (long long)plan.num_tiles};
-    kernel<<<plan.grid, DW_THREADS, plan.smem_bytes, s>>>(plan.map_x, f, bias, act, y, g, t, dev_status);
+    kernel<<<plan.grid, DW_TMA_THREADS, plan.smem_bytes, s>>>(plan.map_x, f, bias, act, y, g, t, dev_status);
     return cudaGetLastError();
 }
 

@@ -56,13 +56,6 @@ constexpr int SMEM_LIMIT = 232448;                               // 227 KiB
 // activation, and the swizzled store into the staging slab the bulk tensor store reads from
 // (16-byte chunk j of row `lane` lives at chunk j ^ (lane % 8): the 128-byte swizzle).
 template <int ACT>
-__device__ __forceinline__ float act_select(float v) {
-    if (ACT == TFJSB_ACT_NONE) return v;
-    float r = v > 0.0f ? v : 0.0f;
-    if (ACT == TFJSB_ACT_RELU6) r = r > 6.0f ? 6.0f : r;
-    return v != v ? v : r;  // NaN stays NaN
-}
-template <int ACT>
 __device__ __forceinline__ void stage_chunk(const uint32_t (&r)[32], const float* __restrict__ bias, int cols_left,
                                             uint32_t row_addr, int lane) {
 #pragma unroll
@@ -74,8 +67,8 @@ __device__ __forceinline__ void stage_chunk(const uint32_t (&r)[32], const float
             const float4 b = __ldg(reinterpret_cast<const float4*>(bias + 4 * j));
             v.x = v.x + b.x; v.y = v.y + b.y; v.z = v.z + b.z; v.w = v.w + b.w;
         }
-        v.x = act_select<ACT>(v.x); v.y = act_select<ACT>(v.y);
-        v.z = act_select<ACT>(v.z); v.w = act_select<ACT>(v.w);
+        v.x = apply_act_t<ACT>(v.x); v.y = apply_act_t<ACT>(v.y);
+        v.z = apply_act_t<ACT>(v.z); v.w = apply_act_t<ACT>(v.w);
         const uint32_t dst = row_addr + (uint32_t)((j ^ (lane & 7)) << 4);
         asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
                      : "memory");

@@ -41,9 +41,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 
 // Waits for the phase with the given parity; gives up after WAIT_LIMIT_NS or when another role
-// has raised the abort flag.  Returns false on giving up.
-static __device__ __noinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
+// has raised the abort flag.  Returns false on giving up.  The first probe is inlined: a wait that
+// is already satisfied costs one try_wait (a call here doubled the cost of every pipeline step of
+// the single-thread producer and MMA loops).
+static __device__ __noinline__ bool bounded_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     const unsigned long long t0 = global_ns();
     for (uint32_t it = 1; it < (1u << 26); ++it) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -51,6 +52,10 @@ static __device__ __noinline__ bool bounded_wait(uint32_t bar, uint32_t parity, 
         if ((it & 63u) == 0u && global_ns() - t0 > WAIT_LIMIT_NS) return false;
     }
     return false;
+}
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return bounded_wait_slow(bar, parity, abort_flag);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
