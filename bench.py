@@ -338,12 +338,14 @@ def run_ours(args):
             achieved, peak, unit = sum(r["flops"] for r in sel) / sel_s / 1e12, fp32_tflops, "TFLOP/s"
         line["roofline"] = {
             "bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-            "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(dominant),
+            "traffic": traffic_of([r["name"] for r in sel]),
+            "algorithmic": int(sum(r["bytes"] for r in sel)) if bound == "hbm" else int(sum(r["flops"] for r in sel)),
             "kernel": dominant, "launches": [r["name"] for r in sel],
             "share_of_step": by_kernel[dominant]["ms"] / total_ms,
             "peak_source": peaks["source"] + (" HBM copy bandwidth" if bound == "hbm" else
                                               " bf16 sustained / 2 (nominal TF32:bf16 ratio)" if bound == "tensor" else " derived"),
-            "how": "algorithmic bytes (or flops) of the listed layers / their summed CUDA-event durations, per pass",
+            "how": "algorithmic bytes (or flops) of the listed layers / their summed CUDA-event durations, per pass; "
+                   "traffic = ncu DRAM read+write bytes summed over the same layers",
         }
         line["roofline_step"] = {"sum_roofline_us": sum(r["roofline_us"] for r in rows), "sum_measured_us": total_ms * 1e3,
                                  "frac": sum(r["roofline_us"] for r in rows) / (total_ms * 1e3)}
@@ -402,9 +404,21 @@ def run_ours(args):
     return 0
 
 
-# DRAM bytes (read + write) per launch of each kernel from the ncu captures summarised under
-# profiles/; None until a capture of the current kernel exists.
-TRAFFIC_BYTES_PER_LAUNCH = {"gemm_tf32": None, "depthwise3x3": None, "conv2d_igemm_tf32": None}
+# DRAM bytes (read + write) per layer of one batch-128 pass, from the one-pass ncu capture summarised in
+# profiles/mobilenet224_b128_dram_traffic.md (cold caches; writes of tensors smaller than L2 are partly
+# counted in the following launch).  Set an entry to None when its kernel changes after the capture.
+TRAFFIC_BYTES_PER_LAYER = {
+    "stem": 222781184, "dw1": 354778880, "pw1": 553852416, "dw2": 493160192, "pw2": 244466688, "dw3": 358310400,
+    "pw3": 352247552, "dw4": 234437120, "pw4": 90361088, "dw5": 154387456, "pw5": 146417920, "dw6": 108002816,
+    "pw6": 26323968, "dw7": 53459456, "pw7": 54098944, "dw8": 54950912, "pw8": 54062848, "dw9": 53772800,
+    "pw9": 54500608, "dw10": 53778688, "pw10": 54076160, "dw11": 53393408, "pw11": 54304768, "dw12": 51419392,
+    "pw12": 14978816, "dw13": 25765120, "pw13": 29919232, "dense": 4654592,
+}
+
+
+def traffic_of(layer_names):
+    vals = [TRAFFIC_BYTES_PER_LAYER.get(n) for n in layer_names]
+    return None if any(v is None for v in vals) else int(sum(vals))
 
 
 def main():
