@@ -204,9 +204,19 @@ int32_t tfjsb_model_launches_per_run(tfjsb_model* model);
 tfjsb_status tfjsb_run_model(tfjsb_model* model, const tfjsb_tensor* input, tfjsb_tensor* output, void* stream);
 
 /* The same run from HOST memory: copies `host_input` (input-shape fp32, ideally pinned) to the
- * device, runs the model, copies the output to `host_output`, all on `stream`, and
- * synchronises the stream before returning (the blocking dataSync() of Sec. 3.6). */
+ * device, runs the model, copies the output to `host_output`, and synchronises `stream` before
+ * returning (the blocking dataSync() of Sec. 3.6).  Batches of 32 images or more (a multiple of 4)
+ * are pipelined in 4 slices: slice c+1 is copied on an internal stream while slice c is computed
+ * on `stream` as a graph replay (images are independent, so the result is that of the whole-batch
+ * run). */
 tfjsb_status tfjsb_run_model_host(tfjsb_model* model, const float* host_input, float* host_output, void* stream);
+
+/* Replays one run as a CUDA graph instead of enqueueing the layers one by one (the enqueue cost per
+ * program is what the paper's async design hides, Sec. 4.1.1; a graph removes it from the host).
+ * The graph is captured on a private stream at the next tfjsb_run_model, for the input / output
+ * buffers of that call, and re-captured when they change.  Run the model once without the graph
+ * first.  Off by default. */
+tfjsb_status tfjsb_model_set_graph(tfjsb_model* model, int use_graph);
 
 /* Debug aid (the paper's debug mode downloads every intermediate, Sec. 3.8): a view of the
  * output of layer `layer` as left by the last run.  With the ping-pong arena only the most

@@ -8,6 +8,7 @@
 // the paper's texture recycler, Sec. 4.1.2), tensor maps encoded once against those fixed
 // addresses.  Running (tfjsb_run_model) therefore does no allocation, no shape arithmetic and
 // no synchronisation: it enqueues the kernels and returns (Sec. 4.1.1).
+#include <cstdlib>
 #include <vector>
 
 #include "common.cuh"
@@ -54,6 +55,18 @@ struct tfjsb_model {
     // caller buffers the first/last tensor maps were last encoded for
     const void* bound_in = nullptr;
     void* bound_out = nullptr;
+    // tfjsb_run_model_host pipelines the batch in slices: slice c+1 is copied to the device on a
+    // stream of its own while slice c is computed.  Each slice has a view of this model with a
+    // smaller batch: the same weights and arena, its own shapes, plans and fixed staging addresses.
+    std::vector<tfjsb_model*> slices;
+    std::vector<cudaEvent_t> slice_copied;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t compute_done = nullptr;
+    bool is_view = false;
+    // optional CUDA-graph replay of one run (tfjsb_model_set_graph): captured for the current binding
+    bool use_graph = false;
+    cudaGraphExec_t graph_exec = nullptr;
+    cudaStream_t capture_stream = nullptr;
 };
 
 namespace {
@@ -152,6 +165,66 @@ cudaError_t launch_step(tfjsb_model* m, const Step& st, cudaStream_t s) {
             return launch_softmax(st.in, st.out, st.M, st.N, s, &ctx->launches);
     }
     return cudaErrorUnknown;
+}
+
+// A view of `parent` for a batch of `n` images: steps copied with every batch-proportional size scaled.
+tfjsb_model* make_batch_view(tfjsb_model* parent, int64_t n) {
+    const int64_t pn = parent->in_dims[0];
+    tfjsb_model* v = new tfjsb_model();
+    v->ctx = parent->ctx;
+    v->is_view = true;
+    v->use_tf32 = parent->use_tf32;
+    v->arena = parent->arena;
+    v->region_elems = parent->region_elems;
+    v->steps = parent->steps;
+    for (int i = 0; i < 4; ++i) v->in_dims[i] = parent->in_dims[i];
+    v->in_dims[0] = n;
+    v->in_elems = parent->in_elems / pn * n;
+    for (Step& st : v->steps) {
+        st.g.N = n;
+        st.M = st.M / pn * n;  // GEMM rows and softmax rows are both proportional to the batch
+        st.out_dims[0] = n;
+        st.out_elems = st.out_elems / pn * n;
+        st.plan_built = false;
+        st.in = nullptr;
+        st.out = nullptr;
+    }
+    return v;
+}
+
+void drop_graph(tfjsb_model* m) {
+    if (m->graph_exec) {
+        cudaGraphExecDestroy(m->graph_exec);
+        m->graph_exec = nullptr;
+    }
+}
+
+// Records one run (every layer's launch, in order) into a graph on a private stream.  Nothing
+// executes during the capture; the first launch of every kernel must already have happened
+// outside a capture (function attributes are set then), which a warm-up run guarantees.
+tfjsb_status capture_graph(tfjsb_model* m) {
+    tfjsb_ctx* ctx = m->ctx;
+    cudaError_t e;
+    if (!m->capture_stream && (e = cudaStreamCreateWithFlags(&m->capture_stream, cudaStreamNonBlocking)) != cudaSuccess)
+        return cuda_fail(ctx, e, "cudaStreamCreate");
+    if ((e = cudaStreamBeginCapture(m->capture_stream, cudaStreamCaptureModeRelaxed)) != cudaSuccess)
+        return cuda_fail(ctx, e, "cudaStreamBeginCapture");
+    const int64_t before = ctx->launches;
+    cudaError_t launch_err = cudaSuccess;
+    for (const Step& step : m->steps)
+        if ((launch_err = launch_step(m, step, m->capture_stream)) != cudaSuccess) break;
+    ctx->launches = before;  // recorded, not run
+    cudaGraph_t graph = nullptr;
+    e = cudaStreamEndCapture(m->capture_stream, &graph);
+    if (launch_err != cudaSuccess || e != cudaSuccess) {
+        if (graph) cudaGraphDestroy(graph);
+        (void)cudaGetLastError();
+        return cuda_fail(ctx, launch_err != cudaSuccess ? launch_err : e, "capturing the model into a graph");
+    }
+    e = cudaGraphInstantiate(&m->graph_exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaGraphInstantiate");
+    return TFJSB_OK;
 }
 
 tfjsb_status check_io(tfjsb_model* m, const tfjsb_tensor* input, const tfjsb_tensor* output) {
@@ -331,6 +404,16 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
 tfjsb_status tfjsb_model_destroy(tfjsb_model* m) {
     if (!m) return TFJSB_ERR_INVALID_ARG;
     cudaDeviceSynchronize();
+    drop_graph(m);
+    if (m->capture_stream) cudaStreamDestroy(m->capture_stream);
+    for (tfjsb_model* v : m->slices) {
+        drop_graph(v);
+        if (v->capture_stream) cudaStreamDestroy(v->capture_stream);
+        delete v;
+    }
+    for (cudaEvent_t e : m->slice_copied) cudaEventDestroy(e);
+    if (m->compute_done) cudaEventDestroy(m->compute_done);
+    if (m->copy_stream) cudaStreamDestroy(m->copy_stream);
     for (float* p : m->owned) cudaFree(p);
     --m->ctx->live_models;
     delete m;
@@ -353,12 +436,27 @@ tfjsb_status tfjsb_run_model(tfjsb_model* m, const tfjsb_tensor* input, tfjsb_te
     if (st != TFJSB_OK) return st;
     if (m->bound_in != input->data || m->bound_out != output->data) {
         if ((st = bind_all(m, static_cast<const float*>(input->data), static_cast<float*>(output->data))) != TFJSB_OK) return st;
+        drop_graph(m);  // the captured launches point at the old buffers
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (m->use_graph) {
+        if (!m->graph_exec && (st = capture_graph(m)) != TFJSB_OK) return st;
+        cudaError_t e = cudaGraphLaunch(m->graph_exec, s);
+        if (e != cudaSuccess) return cuda_fail(m->ctx, e, "cudaGraphLaunch");
+        m->ctx->launches += (int64_t)m->steps.size();
+        return TFJSB_OK;
+    }
     for (const Step& step : m->steps) {
         cudaError_t e = launch_step(m, step, s);
         if (e != cudaSuccess) return cuda_fail(m->ctx, e, "layer launch");
     }
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_model_set_graph(tfjsb_model* m, int use_graph) {
+    if (!m) return TFJSB_ERR_INVALID_ARG;
+    m->use_graph = use_graph != 0;
+    if (!m->use_graph) drop_graph(m);
     return TFJSB_OK;
 }
 
@@ -373,11 +471,55 @@ tfjsb_status tfjsb_run_model_host(tfjsb_model* m, const float* host_input, float
         if ((st = dev_alloc(m, (size_t)last.out_elems, &m->staged_out)) != TFJSB_OK) return st;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaMemcpyAsync(m->staged_in, host_input, (size_t)m->in_elems * 4, cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "host-to-device copy of the input");
-    tfjsb_tensor in{m->staged_in, 4, {m->in_dims[0], m->in_dims[1], m->in_dims[2], m->in_dims[3]}};
-    tfjsb_tensor out{m->staged_out, last.out_rank, {last.out_dims[0], last.out_dims[1], last.out_dims[2], last.out_dims[3]}};
-    if ((st = tfjsb_run_model(m, &in, &out, stream)) != TFJSB_OK) return st;
+    cudaError_t e;
+    const int64_t n = m->in_dims[0];
+    // four slices: more of them lose more to per-launch fixed costs than the extra overlap returns
+    int n_slices = (n % 4 == 0 && n >= 32) ? 4 : 1;
+    if (const char* env = getenv("TFJSB_HOST_SLICES")) {  // tuning knob: 1 disables the pipelining
+        const int v = atoi(env);
+        if (v >= 1 && n % v == 0 && m->slices.empty()) n_slices = v;
+        else if (!m->slices.empty()) n_slices = (int)m->slices.size();
+    }
+    if (n_slices > 1 && !m->keep_all) {
+        if (m->slices.empty()) {
+            if ((e = cudaStreamCreateWithFlags(&m->copy_stream, cudaStreamNonBlocking)) != cudaSuccess)
+                return cuda_fail(ctx, e, "cudaStreamCreate");
+            if ((e = cudaEventCreateWithFlags(&m->compute_done, cudaEventDisableTiming)) != cudaSuccess)
+                return cuda_fail(ctx, e, "cudaEventCreate");
+            for (int c = 0; c < n_slices; ++c) {
+                cudaEvent_t ev;
+                if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess)
+                    return cuda_fail(ctx, e, "cudaEventCreate");
+                m->slice_copied.push_back(ev);
+                m->slices.push_back(make_batch_view(m, n / n_slices));
+            }
+        }
+        const int64_t in_slice = m->in_elems / n_slices, out_slice = last.out_elems / n_slices;
+        // the copy stream starts after whatever the caller queued on `stream` before this call
+        if ((e = cudaEventRecord(m->compute_done, s)) != cudaSuccess) return cuda_fail(ctx, e, "cudaEventRecord");
+        if ((e = cudaStreamWaitEvent(m->copy_stream, m->compute_done, 0)) != cudaSuccess) return cuda_fail(ctx, e, "cudaStreamWaitEvent");
+        for (int c = 0; c < n_slices; ++c) {
+            e = cudaMemcpyAsync(m->staged_in + c * in_slice, host_input + c * in_slice, (size_t)in_slice * 4,
+                                cudaMemcpyHostToDevice, m->copy_stream);
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "host-to-device copy of the input");
+            if ((e = cudaEventRecord(m->slice_copied[c], m->copy_stream)) != cudaSuccess) return cuda_fail(ctx, e, "cudaEventRecord");
+        }
+        for (int c = 0; c < n_slices; ++c) {
+            tfjsb_model* v = m->slices[c];
+            if ((e = cudaStreamWaitEvent(s, m->slice_copied[c], 0)) != cudaSuccess) return cuda_fail(ctx, e, "cudaStreamWaitEvent");
+            tfjsb_tensor in{m->staged_in + c * in_slice, 4, {v->in_dims[0], v->in_dims[1], v->in_dims[2], v->in_dims[3]}};
+            const Step& vl = v->steps.back();
+            tfjsb_tensor out{m->staged_out + c * out_slice, vl.out_rank, {vl.out_dims[0], vl.out_dims[1], vl.out_dims[2], vl.out_dims[3]}};
+            if ((st = tfjsb_run_model(v, &in, &out, stream)) != TFJSB_OK) return st;
+            v->use_graph = true;  // the first pass ran launch by launch; later passes replay a graph
+        }
+    } else {
+        e = cudaMemcpyAsync(m->staged_in, host_input, (size_t)m->in_elems * 4, cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "host-to-device copy of the input");
+        tfjsb_tensor in{m->staged_in, 4, {m->in_dims[0], m->in_dims[1], m->in_dims[2], m->in_dims[3]}};
+        tfjsb_tensor out{m->staged_out, last.out_rank, {last.out_dims[0], last.out_dims[1], last.out_dims[2], last.out_dims[3]}};
+        if ((st = tfjsb_run_model(m, &in, &out, stream)) != TFJSB_OK) return st;
+    }
     e = cudaMemcpyAsync(host_output, m->staged_out, (size_t)last.out_elems * 4, cudaMemcpyDeviceToHost, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "device-to-host copy of the output");
     e = cudaStreamSynchronize(s);
@@ -394,6 +536,7 @@ tfjsb_status tfjsb_model_set_keep_all(tfjsb_model* m, int keep_all) {
         if (st != TFJSB_OK) return st;
     }
     m->keep_all = keep_all != 0;
+    drop_graph(m);
     m->bound_in = nullptr;  // force a re-bind on the next run
     m->bound_out = nullptr;
     return TFJSB_OK;

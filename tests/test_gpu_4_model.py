@@ -117,6 +117,15 @@ def test_config5_mobilenet_100_224_batch128_sampled_images(ctx, oracle):
     hout = torch.empty(128, 1000).pin_memory()
     model.run_host(hin, hout)
     assert same_bits(hout.numpy(), probs)
+    model.run_host(hin, hout.zero_())  # second call: the slices replay their captured graphs
+    assert same_bits(hout.numpy(), probs)
+    # graph replay of the whole-batch run gives the same bits as launch-by-launch
+    out2 = torch.empty(128, 1000, device="cuda")
+    model.set_graph(True)
+    model.run(xd, out=out2)
+    model.run(xd, out=out2)
+    assert same_bits(host(out2), probs)
+    model.set_graph(False)
     # per-layer profile returns one positive time per layer
     ms = model.profile(xd, reps=2)
     assert len(ms) == 30 and all(t > 0 for t in ms)
