@@ -278,7 +278,11 @@ class Model:
         odims = (ctypes.c_int64 * 4)()
         ctx._check(lib.tfjsb_model_output_shape(self._h, ctypes.byref(rank), odims))
         self.output_shape = tuple(odims[i] for i in range(rank.value))
-        self.launches_per_run = lib.tfjsb_model_launches_per_run(self._h)
+
+    @property
+    def launches_per_run(self) -> int:
+        """Kernels one run launches in the current mode (fused blocks count once)."""
+        return int(lib.tfjsb_model_launches_per_run(self._h))
 
     def close(self):
         if self._h:

@@ -30,6 +30,7 @@ SOURCES = [
     "conv2d_fp32_simt.cu",
     "depthwise.cu",
     "matmul_static_scratch.cu",
+    "dwpw_fused_tcgen05.cu",
 ]
 
 NVCC_FLAGS = [

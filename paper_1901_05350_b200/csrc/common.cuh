@@ -161,4 +161,22 @@ cudaError_t launch_pack_filter(const float* f, float* out, int64_t K, int64_t N,
 cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int act, unsigned int* dev_status,
                              cudaStream_t s, int64_t* launches);
 
+// Fused depthwise 3x3 (stride 1) + pointwise block: the depthwise output is produced straight into
+// the tensor-core operand layout in shared memory and never written to global memory.
+// `bt` is the pointwise filter stored [Cout, Cin] (K-contiguous).
+struct DwPwPlan {
+    CUtensorMap map_x, map_b, map_y;
+    ConvGeom g{};   // geometry of the depthwise layer
+    int Co = 0;
+    int block_n = 0, acc_stages = 0, patch_stages = 0, a_stages = 0, b_stages = 0;
+    int tiles_x = 0, tiles_y = 0, num_tiles = 0, grid = 0;
+    size_t smem_bytes = 0;
+};
+bool dwpw_fused_supported(const ConvGeom& dw, int64_t Cout);
+tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, float* y, const ConvGeom& dw,
+                             int64_t Cout, DwPwPlan* plan);
+cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, const float* dw_bias, int dw_act,
+                              const float* pw_bias, int pw_act, unsigned int* dev_status, cudaStream_t s,
+                              int64_t* launches);
+
 }  // namespace tfjsb

@@ -1,0 +1,464 @@
+// Fused depthwise-separable block for sm_100a:
+//
+//     y = act2( pointwise( act1( depthwise3x3(x) + b1 ) ) + b2 )      stride 1, NHWC fp32
+//
+// The depthwise output never goes to global memory.  A persistent CTA walks tiles of 8 x 16 output
+// pixels (= the 128 rows of one tensor-core tile) and, per block of 32 channels (= one k-block):
+//   warp 0       producer: bulk tensor copies (TMA) of the input patch (10 x 18 pixels x 32 channels,
+//                zero-filled outside the image = the 'same' padding) and of the matching 32-column
+//                slice of the pointwise weights Bt[Cout, Cin], each into its own ring of stages;
+//   warps 10-25  depthwise: compute the 128 x 32 block on CUDA cores from the patch (the same
+//                sliding-row scheme and FMA order as the stand-alone kernel), add bias, apply the
+//                activation and write it as the A operand in the 128-byte-swizzled K-major layout;
+//   warp 1       issues tcgen05.mma (TF32, M 128, N = block_n, K 8, four per k-block) on A and Bt,
+//                accumulating over the channel blocks in tensor memory;
+//   warps 2-9    epilogue: tcgen05.ld, pointwise bias + activation, swizzled staging slab, 4-D bulk
+//                tensor store of 2 image rows x 16 pixels x 32 channels (clipped at the image edge).
+// Every wait is bounded (see ptx_sm100.cuh); a timeout raises the abort flag all roles poll and is
+// reported through the context's device status word.
+#include "common.cuh"
+#include "ptx_sm100.cuh"
+#include "umma_tile.cuh"
+
+namespace tfjsb {
+
+using namespace ptx;
+using namespace tile;
+
+namespace {
+
+constexpr int F_THREADS = 832;        // 26 warps
+constexpr int F_DW_WARPS = 16;
+constexpr int F_TH = 8, F_TW = 16;    // output pixels per tile (8 rows x 16 columns = 128 GEMM rows)
+constexpr int F_PH = F_TH + 2, F_PW = F_TW + 2;
+constexpr int F_PATCH_FLOATS = F_PH * F_PW * BLOCK_K;
+constexpr int F_PATCH_BYTES = F_PATCH_FLOATS * 4;              // 23040
+constexpr int F_PATCH_STRIDE = 23 * 1024;                      // stage pitch, keeps stages 1024-aligned
+constexpr int F_MAX_RING = 4;
+
+struct FusedArgs {
+    int C, Co;                // depthwise channels (= K of the GEMM), pointwise output channels (= N)
+    int Ho, Wo;               // = input H, W (stride 1, 'same') or the 'valid' output size
+    int pt, pl;               // padding before
+    int tiles_x, tiles_y;
+    int num_tiles;
+    int block_n;
+    int acc_stages;
+    int patch_stages, a_stages, b_stages;
+    const float* dw_filter;   // [3,3,C,1]
+    const float* dw_bias;     // [C] or null
+    int dw_act;
+    const float* pw_bias;     // [Co] or null
+    int pw_act;
+    unsigned int* dev_status;
+};
+
+__device__ __forceinline__ float4 ld4s(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ void fma4s(float4& acc, const float4& a, const float4& b) {
+    acc.x = fmaf(a.x, b.x, acc.x); acc.y = fmaf(a.y, b.y, acc.y);
+    acc.z = fmaf(a.z, b.z, acc.z); acc.w = fmaf(a.w, b.w, acc.w);
+}
+
+__global__ void __launch_bounds__(F_THREADS, 1)
+dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_b,
+                  const __grid_constant__ CUtensorMap map_y, const FusedArgs args) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_patch_full[F_MAX_RING], bar_patch_empty[F_MAX_RING];
+    __shared__ __align__(8) uint64_t bar_a_full[F_MAX_RING], bar_a_empty[F_MAX_RING];
+    __shared__ __align__(8) uint64_t bar_b_full[F_MAX_RING], bar_b_empty[F_MAX_RING];
+    __shared__ __align__(8) uint64_t bar_acc_full[MAX_ACC_STAGES], bar_acc_empty[MAX_ACC_STAGES];
+    __shared__ __align__(8) uint64_t bar_drain;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag_s;
+
+    volatile int* abort_flag = &abort_flag_s;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int block_n = args.block_n;
+    const int num_k_blocks = args.C / BLOCK_K;
+    const int b_stage_bytes = block_n * BLOCK_K * 4;
+
+    // dynamic shared memory (1024-aligned): [epilogue slabs][patch ring][A ring][B ring]
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t epi_base = smem_base;
+    const uint32_t patch_base = epi_base + EPI_BYTES;
+    const uint32_t a_base = patch_base + (uint32_t)args.patch_stages * F_PATCH_STRIDE;
+    const uint32_t b_base = a_base + (uint32_t)args.a_stages * A_STAGE_BYTES;
+    const float* patch_ptr = reinterpret_cast<const float*>(smem_raw + (patch_base - smem_u32(smem_raw)));
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < F_MAX_RING; ++s) {
+            mbar_init(smem_u32(&bar_patch_full[s]), 1);
+            mbar_init(smem_u32(&bar_patch_empty[s]), F_DW_WARPS);
+            mbar_init(smem_u32(&bar_a_full[s]), F_DW_WARPS);
+            mbar_init(smem_u32(&bar_a_empty[s]), 1);
+            mbar_init(smem_u32(&bar_b_full[s]), 1);
+            mbar_init(smem_u32(&bar_b_empty[s]), 1);
+        }
+        for (int s = 0; s < MAX_ACC_STAGES; ++s) {
+            mbar_init(smem_u32(&bar_acc_full[s]), 1);
+            mbar_init(smem_u32(&bar_acc_empty[s]), 8);
+        }
+        mbar_init(smem_u32(&bar_drain), 1);
+        abort_flag_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_y) : "memory");
+    }
+    const uint32_t tmem_cols = (uint32_t)(args.acc_stages * block_n);
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         smem_u32(&tmem_base_slot)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    const int tiles_per_image = args.tiles_x * args.tiles_y;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- producer
+        if (lane == 0) {
+            int ps = 0, bs = 0;
+            uint32_t pphase = 0, bphase = 0;
+            int issued = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
+                const int n = tile / tiles_per_image;
+                const int rem = tile - n * tiles_per_image;
+                const int ty = rem / args.tiles_x, tx = rem - ty * args.tiles_x;
+                for (int kb = 0; kb < num_k_blocks; ++kb) {
+                    if (!bounded_wait(smem_u32(&bar_patch_empty[ps]), pphase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t pf = smem_u32(&bar_patch_full[ps]);
+                    mbar_arrive_expect_tx(pf, (uint32_t)F_PATCH_BYTES);
+                    tma_load_4d(patch_base + (uint32_t)ps * F_PATCH_STRIDE, &map_x, pf, kb * BLOCK_K,
+                                tx * F_TW - args.pl, ty * F_TH - args.pt, n);
+                    if (++ps == args.patch_stages) { ps = 0; pphase ^= 1u; }
+                    if (!bounded_wait(smem_u32(&bar_b_empty[bs]), bphase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t bf = smem_u32(&bar_b_full[bs]);
+                    mbar_arrive_expect_tx(bf, (uint32_t)b_stage_bytes);
+                    tma_load_2d(b_base + (uint32_t)bs * (uint32_t)b_stage_bytes, &map_b, bf, kb * BLOCK_K, 0);
+                    if (++bs == args.b_stages) { bs = 0; bphase ^= 1u; }
+                    ++issued;
+                }
+            }
+            if (!ok || *abort_flag) {
+                if (!*abort_flag) {
+                    *abort_flag = 1;
+                    atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_PRODUCER);
+                }
+                // give the copies in flight time to land before the CTA's shared memory is released:
+                // every armed phase completes within the copy latency unless the device is wedged
+                const unsigned long long t0 = global_ns();
+                bool all = false;
+                while (!all && global_ns() - t0 < WAIT_LIMIT_NS) {
+                    all = true;
+                    for (int k = (issued > F_MAX_RING ? issued - F_MAX_RING : 0); k < issued; ++k) {
+                        if (!mbar_try_wait(smem_u32(&bar_patch_full[k % args.patch_stages]),
+                                           (uint32_t)((k / args.patch_stages) & 1)) &&
+                            k >= issued - args.patch_stages)
+                            all = false;
+                        if (!mbar_try_wait(smem_u32(&bar_b_full[k % args.b_stages]), (uint32_t)((k / args.b_stages) & 1)) &&
+                            k >= issued - args.b_stages)
+                            all = false;
+                    }
+                }
+                if (!all) atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_DRAIN);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_tf32(BLOCK_M, block_n);
+            int as = 0, bs = 0, acc = 0;
+            uint32_t aphase = 0, bphase = 0, acc_phase = 0;
+            bool ok = true, issued_any = false;
+            for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
+                if (!bounded_wait(smem_u32(&bar_acc_empty[acc]), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * block_n);
+                for (int kb = 0; kb < num_k_blocks; ++kb) {
+                    if (!bounded_wait(smem_u32(&bar_b_full[bs]), bphase, abort_flag)) { ok = false; break; }
+                    if (!bounded_wait(smem_u32(&bar_a_full[as]), aphase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t a_desc = make_kmajor_sw128_desc(a_base + (uint32_t)as * A_STAGE_BYTES);
+                    const uint64_t b_desc = make_kmajor_sw128_desc(b_base + (uint32_t)bs * (uint32_t)b_stage_bytes);
+#pragma unroll
+                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                        tc_mma_tf32(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                    (kb | k) != 0 ? 1u : 0u);
+                    issued_any = true;
+                    tc_commit(smem_u32(&bar_a_empty[as]));
+                    tc_commit(smem_u32(&bar_b_empty[bs]));
+                    if (++as == args.a_stages) { as = 0; aphase ^= 1u; }
+                    if (++bs == args.b_stages) { bs = 0; bphase ^= 1u; }
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(&bar_acc_full[acc]));
+                if (++acc == args.acc_stages) { acc = 0; acc_phase ^= 1u; }
+            }
+            if (!ok) {
+                if (!*abort_flag) {
+                    *abort_flag = 1;
+                    atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_MMA);
+                }
+                if (issued_any) {
+                    tc_commit(smem_u32(&bar_drain));
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(smem_u32(&bar_drain), 0u)) {
+                        if (global_ns() - t0 > WAIT_LIMIT_NS) {
+                            atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_DRAIN);
+                            break;
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp < 10) {
+        // ---------------------------------------------------------------- epilogue (warps 2..9)
+        const int ew = warp - 2;
+        const int quad = warp & 3;   // TMEM lanes 32*quad.. = image rows 2*quad, 2*quad+1 of the tile
+        const int half = ew >> 2;
+        const uint32_t slab = epi_base + (uint32_t)ew * EPI_SLAB_BYTES;
+        const int chunks_per_tile = block_n / EPI_COLS;
+        int n_chunks = (args.Co + EPI_COLS - 1) / EPI_COLS;
+        if (n_chunks > chunks_per_tile) n_chunks = chunks_per_tile;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        int first_chunk = half;
+        for (int tile = blockIdx.x; tile < args.num_tiles; tile += gridDim.x) {
+            const int n = tile / tiles_per_image;
+            const int rem = tile - n * tiles_per_image;
+            const int ty = rem / args.tiles_x, tx = rem - ty * args.tiles_x;
+            const bool got = bounded_wait(smem_u32(&bar_acc_full[acc]), acc_phase, abort_flag);
+            if (!__all_sync(0xffffffffu, got)) {
+                if (lane == 0 && !*abort_flag) {
+                    *abort_flag = 1;
+                    atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_EPILOGUE);
+                }
+                break;
+            }
+            tc_fence_after();
+            const int oy = ty * F_TH + quad * 2;
+            const bool rows_live = oy < args.Ho;
+            bool released = false;
+            for (int ch = first_chunk; ch < n_chunks; ch += 2) {
+                uint32_t r[32];
+                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * block_n + ch * EPI_COLS);
+                tc_ld_32x32(taddr, r);
+                tc_ld_wait();
+                if (ch + 2 >= n_chunks) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
+                    released = true;
+                }
+                if (!rows_live) continue;
+                const int col0 = ch * EPI_COLS;
+                if (lane == 0) tma_store_wait_read<0>();
+                __syncwarp();
+                const uint32_t row_addr = slab + (uint32_t)lane * 128u;
+                const float* bias = (args.pw_bias != nullptr) ? args.pw_bias + col0 : nullptr;
+                const int cols_left = args.Co - col0;
+                if (args.pw_act == TFJSB_ACT_RELU6) stage_chunk<TFJSB_ACT_RELU6>(r, bias, cols_left, row_addr, lane);
+                else if (args.pw_act == TFJSB_ACT_RELU) stage_chunk<TFJSB_ACT_RELU>(r, bias, cols_left, row_addr, lane);
+                else stage_chunk<TFJSB_ACT_NONE>(r, bias, cols_left, row_addr, lane);
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_4d(&map_y, slab, col0, tx * F_TW, oy, n);
+                    tma_store_commit();
+                }
+            }
+            if (!released) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
+            }
+            if (chunks_per_tile & 1) first_chunk ^= 1;
+            if (++acc == args.acc_stages) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (lane == 0) tma_store_wait_all();
+        __syncwarp();
+    } else {
+        // ---------------------------------------------------------------- depthwise (warps 10..25)
+        // thread = (2 channels, tile column, group of 4 tile rows); GEMM row of a pixel = row*16 + column.
+        // Two channels per thread (not four) so that sixteen warps share a k-block: eight were bound by
+        // their own instruction latency, not by any pipe.
+        const int t = threadIdx.x - 320;
+        const int c2 = t & 15;
+        const int col = (t >> 4) & (F_TW - 1);
+        const int rg = t >> 8;
+        constexpr int R = F_TH / 2;
+        int ps = 0, as = 0;
+        uint32_t pphase = 0, aphase = 0;
+        float2 w[9];
+        float2 b = make_float2(0.f, 0.f);
+        int loaded_kb = -1;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
+            for (int kb = 0; kb < num_k_blocks; ++kb) {
+                if (kb != loaded_kb) {
+                    const int c = kb * BLOCK_K + c2 * 2;
+#pragma unroll
+                    for (int k = 0; k < 9; ++k) w[k] = __ldg(reinterpret_cast<const float2*>(args.dw_filter + (int64_t)k * args.C + c));
+                    if (args.dw_bias) b = __ldg(reinterpret_cast<const float2*>(args.dw_bias + c));
+                    loaded_kb = kb;
+                }
+                bool got = bounded_wait(smem_u32(&bar_patch_full[ps]), pphase, abort_flag);
+                got = got && bounded_wait(smem_u32(&bar_a_empty[as]), aphase ^ 1u, abort_flag);
+                if (!__all_sync(0xffffffffu, got)) {
+                    if (lane == 0 && !*abort_flag) {
+                        *abort_flag = 1;
+                        atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_DEPTHWISE);
+                    }
+                    ok = false;
+                    break;
+                }
+                float2 acc[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) acc[r] = make_float2(0.f, 0.f);
+                const float* patch = patch_ptr + (size_t)ps * (F_PATCH_STRIDE / 4) + ((rg * R) * F_PW + col) * BLOCK_K + c2 * 2;
+#pragma unroll
+                for (int j = 0; j < R + 2; ++j) {
+                    const float* row = patch + j * F_PW * BLOCK_K;
+                    const float2 v0 = *reinterpret_cast<const float2*>(row);
+                    const float2 v1 = *reinterpret_cast<const float2*>(row + BLOCK_K);
+                    const float2 v2 = *reinterpret_cast<const float2*>(row + 2 * BLOCK_K);
+#pragma unroll
+                    for (int ky = 0; ky < 3; ++ky) {
+                        const int d = j - ky;
+                        if (d >= 0 && d < R) {
+                            acc[d].x = fmaf(v0.x, w[ky * 3 + 0].x, acc[d].x); acc[d].y = fmaf(v0.y, w[ky * 3 + 0].y, acc[d].y);
+                            acc[d].x = fmaf(v1.x, w[ky * 3 + 1].x, acc[d].x); acc[d].y = fmaf(v1.y, w[ky * 3 + 1].y, acc[d].y);
+                            acc[d].x = fmaf(v2.x, w[ky * 3 + 2].x, acc[d].x); acc[d].y = fmaf(v2.y, w[ky * 3 + 2].y, acc[d].y);
+                        }
+                    }
+                }
+                const uint32_t a_stage = a_base + (uint32_t)as * A_STAGE_BYTES;
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const float vx = apply_act(acc[r].x + b.x, args.dw_act);
+                    const float vy = apply_act(acc[r].y + b.y, args.dw_act);
+                    const int p = (rg * R + r) * F_TW + col;
+                    const uint32_t dst = a_stage + (uint32_t)p * 128u + (uint32_t)(((c2 >> 1) ^ (p & 7)) << 4) + (uint32_t)((c2 & 1) << 3);
+                    asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(dst), "f"(vx), "f"(vy) : "memory");
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&bar_a_full[as]));
+                    mbar_arrive(smem_u32(&bar_patch_empty[ps]));
+                }
+                if (++ps == args.patch_stages) { ps = 0; pphase ^= 1u; }
+                if (++as == args.a_stages) { as = 0; aphase ^= 1u; }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols)
+                     : "memory");
+    }
+}
+
+}  // namespace
+
+bool dwpw_fused_supported(const ConvGeom& dw, int64_t Cout) {
+    const int64_t tiles = dw.N * ((dw.Ho + F_TH - 1) / F_TH) * ((dw.Wo + F_TW - 1) / F_TW);
+    return dw.fh == 3 && dw.fw == 3 && dw.sh == 1 && dw.sw == 1 && dw.dh == 1 && dw.dw == 1 && dw.mult == 1 &&
+           dw.C >= BLOCK_K && dw.C % BLOCK_K == 0 && Cout >= 4 && Cout <= 256 && Cout % 4 == 0 && tiles >= 1 &&
+           tiles < (1LL << 31) && dw.N < (1LL << 31);
+}
+
+tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, float* y, const ConvGeom& dw,
+                             int64_t Cout, DwPwPlan* plan) {
+    if (!dwpw_fused_supported(dw, Cout)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the fused block kernel");
+    if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+    plan->g = dw;
+    plan->Co = (int)Cout;
+    int bn = 32;
+    while (bn < Cout) bn <<= 1;
+    plan->block_n = bn;
+    plan->acc_stages = bn == 256 ? 2 : MAX_ACC_STAGES;
+    plan->a_stages = 3;
+    plan->b_stages = bn == 256 ? 2 : 3;
+    const int fixed = EPI_BYTES + plan->a_stages * A_STAGE_BYTES + plan->b_stages * bn * BLOCK_K * 4;
+    int ps = (SMEM_LIMIT - 2048 - fixed) / F_PATCH_STRIDE;
+    if (ps > F_MAX_RING) ps = F_MAX_RING;
+    if (ps < 2) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "no room for the input patch ring");
+    plan->patch_stages = ps;
+    plan->smem_bytes = (size_t)1024 + fixed + (size_t)ps * F_PATCH_STRIDE;
+    plan->tiles_x = (dw.Wo + F_TW - 1) / F_TW;
+    plan->tiles_y = (dw.Ho + F_TH - 1) / F_TH;
+    const int64_t tiles = dw.N * plan->tiles_x * plan->tiles_y;
+    plan->num_tiles = (int)tiles;
+    plan->grid = (int)(tiles < ctx->sm_count ? tiles : ctx->sm_count);
+
+    auto encode = [&](CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides,
+                      const cuuint32_t* box, CUtensorMapSwizzle swz, const char* what) -> tfjsb_status {
+        cuuint32_t elem[4] = {1u, 1u, 1u, 1u};
+        CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<void*>(base), dims,
+                                       strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS)
+            return fail(ctx, TFJSB_ERR_CUDA, std::string("cuTensorMapEncodeTiled failed for ") + what + " (CUresult " +
+                                                 std::to_string((int)r) + ")");
+        return TFJSB_OK;
+    };
+    tfjsb_status st;
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)dw.C, (cuuint64_t)dw.W, (cuuint64_t)dw.H, (cuuint64_t)dw.N};
+        cuuint64_t strides[3] = {(cuuint64_t)dw.C * 4u, (cuuint64_t)dw.W * dw.C * 4u, (cuuint64_t)dw.H * dw.W * dw.C * 4u};
+        cuuint32_t box[4] = {(cuuint32_t)BLOCK_K, (cuuint32_t)F_PW, (cuuint32_t)F_PH, 1u};
+        if ((st = encode(&plan->map_x, x, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE, "the block input")) != TFJSB_OK) return st;
+    }
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)dw.C, (cuuint64_t)Cout};
+        cuuint64_t strides[1] = {(cuuint64_t)dw.C * 4u};
+        cuuint32_t box[2] = {(cuuint32_t)BLOCK_K, (cuuint32_t)bn};
+        if ((st = encode(&plan->map_b, bt, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, "the pointwise weights")) != TFJSB_OK) return st;
+    }
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)Cout, (cuuint64_t)dw.Wo, (cuuint64_t)dw.Ho, (cuuint64_t)dw.N};
+        cuuint64_t strides[3] = {(cuuint64_t)Cout * 4u, (cuuint64_t)dw.Wo * Cout * 4u, (cuuint64_t)dw.Ho * dw.Wo * Cout * 4u};
+        cuuint32_t box[4] = {(cuuint32_t)EPI_COLS, (cuuint32_t)F_TW, 2u, 1u};
+        if ((st = encode(&plan->map_y, y, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, "the block output")) != TFJSB_OK) return st;
+    }
+    return TFJSB_OK;
+}
+
+cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, const float* dw_bias, int dw_act,
+                              const float* pw_bias, int pw_act, unsigned int* dev_status, cudaStream_t s,
+                              int64_t* launches) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(dwpw_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 2048);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    FusedArgs a;
+    a.C = plan.g.C; a.Co = plan.Co;
+    a.Ho = plan.g.Ho; a.Wo = plan.g.Wo;
+    a.pt = plan.g.pt; a.pl = plan.g.pl;
+    a.tiles_x = plan.tiles_x; a.tiles_y = plan.tiles_y;
+    a.num_tiles = plan.num_tiles;
+    a.block_n = plan.block_n;
+    a.acc_stages = plan.acc_stages;
+    a.patch_stages = plan.patch_stages; a.a_stages = plan.a_stages; a.b_stages = plan.b_stages;
+    a.dw_filter = dw_filter; a.dw_bias = dw_bias; a.dw_act = dw_act;
+    a.pw_bias = pw_bias; a.pw_act = pw_act;
+    a.dev_status = dev_status;
+    dwpw_fused_kernel<<<plan.grid, F_THREADS, plan.smem_bytes, s>>>(plan.map_x, plan.map_b, plan.map_y, a);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace tfjsb

@@ -30,6 +30,10 @@ struct Step {
     GemmTf32Plan plan{};
     DepthwisePlan dw_plan{};
     bool plan_built = false;
+    // a depthwise layer followed by a pointwise layer can run as one fused kernel (the pointwise step
+    // is then skipped); the separate plans are kept for the keep-all debug mode
+    bool fuse_next = false;
+    DwPwPlan fused_plan{};
     int32_t out_rank = 4;
     int64_t out_dims[4] = {0, 0, 0, 0};
     int64_t out_elems = 0;
@@ -128,6 +132,7 @@ tfjsb_status bind_all(tfjsb_model* m, const float* input, float* output) {
     const int n = (int)m->steps.size();
     const float* cur = input;
     size_t keep_off = 0;
+    int region = 0;  // arena region the next launched kernel writes
     for (int i = 0; i < n; ++i) {
         Step& st = m->steps[i];
         float* dst;
@@ -135,10 +140,25 @@ tfjsb_status bind_all(tfjsb_model* m, const float* input, float* output) {
         else if (m->keep_all) {
             dst = m->keep_all_arena + keep_off;
             keep_off += (size_t)((st.out_elems + 63) / 64 * 64);
-        } else dst = m->arena + (size_t)(i & 1) * m->region_elems;
+        } else {
+            dst = m->arena + (size_t)region * m->region_elems;
+            // A fused pair is one kernel: it reads the first layer's input and writes the second
+            // layer's output, so the pair takes one region (the first layer's own output buffer is
+            // never written) and the region flips once per kernel, not once per layer.
+            if (!st.fuse_next) region ^= 1;
+        }
         tfjsb_status rc = bind_step(m, st, cur, dst);
         if (rc != TFJSB_OK) return rc;
         cur = dst;
+    }
+    if (!m->keep_all) {
+        for (int i = 0; i + 1 < n; ++i) {
+            Step& st = m->steps[i];
+            if (!st.fuse_next) continue;
+            Step& pw = m->steps[i + 1];
+            tfjsb_status rc = dwpw_fused_plan(m->ctx, st.in, pw.filter_km, pw.out, st.g, pw.N, &st.fused_plan);
+            if (rc != TFJSB_OK) return rc;
+        }
     }
     m->bound_in = input;
     m->bound_out = output;
@@ -192,6 +212,9 @@ tfjsb_model* make_batch_view(tfjsb_model* parent, int64_t n) {
     return v;
 }
 
+cudaError_t launch_layers(tfjsb_model* m, int i, cudaStream_t s, int* consumed);
+int launches_per_run(const tfjsb_model* m);
+
 void drop_graph(tfjsb_model* m) {
     if (m->graph_exec) {
         cudaGraphExecDestroy(m->graph_exec);
@@ -211,8 +234,8 @@ tfjsb_status capture_graph(tfjsb_model* m) {
         return cuda_fail(ctx, e, "cudaStreamBeginCapture");
     const int64_t before = ctx->launches;
     cudaError_t launch_err = cudaSuccess;
-    for (const Step& step : m->steps)
-        if ((launch_err = launch_step(m, step, m->capture_stream)) != cudaSuccess) break;
+    for (int i = 0, used = 1; i < (int)m->steps.size(); i += used)
+        if ((launch_err = launch_layers(m, i, m->capture_stream, &used)) != cudaSuccess) break;
     ctx->launches = before;  // recorded, not run
     cudaGraph_t graph = nullptr;
     e = cudaStreamEndCapture(m->capture_stream, &graph);
@@ -225,6 +248,26 @@ tfjsb_status capture_graph(tfjsb_model* m) {
     cudaGraphDestroy(graph);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaGraphInstantiate");
     return TFJSB_OK;
+}
+
+// Launches layer i (and, when it is fused with its successor, that one too); returns how many layers ran.
+cudaError_t launch_layers(tfjsb_model* m, int i, cudaStream_t s, int* consumed) {
+    const Step& st = m->steps[i];
+    if (st.fuse_next && !m->keep_all) {
+        const Step& pw = m->steps[i + 1];
+        *consumed = 2;
+        return launch_dwpw_fused(st.fused_plan, st.filter, st.bias, st.act, pw.bias, pw.act, m->ctx->dev_status, s,
+                                 &m->ctx->launches);
+    }
+    *consumed = 1;
+    return launch_step(m, st, s);
+}
+
+int launches_per_run(const tfjsb_model* m) {
+    int n = (int)m->steps.size();
+    if (!m->keep_all)
+        for (const Step& st : m->steps) n -= st.fuse_next ? 1 : 0;
+    return n;
 }
 
 tfjsb_status check_io(tfjsb_model* m, const tfjsb_tensor* input, const tfjsb_tensor* output) {
@@ -393,6 +436,15 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
     for (size_t i = 0; i + 1 < m->steps.size(); ++i)
         if (m->steps[i].out_elems > largest) largest = m->steps[i].out_elems;
     m->region_elems = (size_t)((largest + 63) / 64 * 64);
+    if (m->use_tf32 && !getenv("TFJSB_NO_FUSION")) {
+        for (size_t i = 0; i + 1 < m->steps.size(); ++i) {
+            Step& dw = m->steps[i];
+            const Step& pw = m->steps[i + 1];
+            if (dw.kind == STEP_DEPTHWISE && pw.kind == STEP_GEMM_TF32 && pw.K == dw.g.Co &&
+                pw.M == dw.g.N * dw.g.Ho * dw.g.Wo && dwpw_fused_supported(dw.g, pw.N))
+                dw.fuse_next = true;
+        }
+    }
     if ((st = dev_alloc(m, 2 * m->region_elems, &m->arena)) != TFJSB_OK) return bail(st, ctx->last_error);
     cudaError_t e = cudaDeviceSynchronize();  // weight transposes done
     if (e != cudaSuccess) return bail(TFJSB_ERR_CUDA, std::string("model set-up: ") + cudaGetErrorString(e));
@@ -428,7 +480,7 @@ tfjsb_status tfjsb_model_output_shape(tfjsb_model* m, int32_t* rank, int64_t dim
     return TFJSB_OK;
 }
 
-int32_t tfjsb_model_launches_per_run(tfjsb_model* m) { return m ? (int32_t)m->steps.size() : -1; }
+int32_t tfjsb_model_launches_per_run(tfjsb_model* m) { return m ? (int32_t)launches_per_run(m) : -1; }
 
 tfjsb_status tfjsb_run_model(tfjsb_model* m, const tfjsb_tensor* input, tfjsb_tensor* output, void* stream) {
     if (!m) return TFJSB_ERR_INVALID_ARG;
@@ -443,11 +495,11 @@ tfjsb_status tfjsb_run_model(tfjsb_model* m, const tfjsb_tensor* input, tfjsb_te
         if (!m->graph_exec && (st = capture_graph(m)) != TFJSB_OK) return st;
         cudaError_t e = cudaGraphLaunch(m->graph_exec, s);
         if (e != cudaSuccess) return cuda_fail(m->ctx, e, "cudaGraphLaunch");
-        m->ctx->launches += (int64_t)m->steps.size();
+        m->ctx->launches += launches_per_run(m);
         return TFJSB_OK;
     }
-    for (const Step& step : m->steps) {
-        cudaError_t e = launch_step(m, step, s);
+    for (int i = 0, used = 1; i < (int)m->steps.size(); i += used) {
+        cudaError_t e = launch_layers(m, i, s, &used);
         if (e != cudaSuccess) return cuda_fail(m->ctx, e, "layer launch");
     }
     return TFJSB_OK;
@@ -572,10 +624,11 @@ tfjsb_status tfjsb_model_profile(tfjsb_model* m, const tfjsb_tensor* input, tfjs
     tfjsb_status rc = TFJSB_OK;
     for (int r = 0; r < reps && rc == TFJSB_OK; ++r) {
         cudaEventRecord(ev[0], s);
-        for (int i = 0; i < n; ++i) {
-            cudaError_t e = launch_step(m, m->steps[i], s);
+        for (int i = 0, used = 1; i < n; i += used) {
+            cudaError_t e = launch_layers(m, i, s, &used);
             if (e != cudaSuccess) { rc = cuda_fail(ctx, e, "layer launch"); break; }
-            cudaEventRecord(ev[i + 1], s);
+            // a fused pair reports its whole time under the first layer and zero under the second
+            for (int k = 1; k <= used; ++k) cudaEventRecord(ev[i + k], s);
         }
         cudaError_t e = cudaStreamSynchronize(s);
         if (e != cudaSuccess) { rc = cuda_fail(ctx, e, "cudaStreamSynchronize"); break; }

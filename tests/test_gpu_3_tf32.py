@@ -160,3 +160,47 @@ def test_tf32_result_is_deterministic(ctx):
     for _ in range(3):
         assert same_bits(host(ctx.matmul(a, b)), first)
     ctx.check_device_status()
+
+
+FUSED_BLOCK_CASES = [
+    # N, H, W, C, Cout, pad: depthwise 3x3 stride 1 + pointwise, run by the executor as one fused kernel
+    (1, 112, 112, 32, 64, "same"),     # config 2
+    (2, 20, 37, 32, 8, "same"),        # ragged tiles in both directions, Cout below one chunk
+    (3, 14, 14, 128, 128, "same"),     # four k-blocks, image smaller than the 16-wide tile
+    (2, 7, 7, 256, 256, "same"),       # eight k-blocks, 256-wide accumulator (two stages)
+    (1, 30, 33, 64, 100, "valid"),     # 'valid': no padding offset, Cout not a multiple of 32
+    (5, 56, 56, 96, 36, "same"),       # more tiles than SMs, three k-blocks
+]
+
+
+@pytest.mark.parametrize("case", FUSED_BLOCK_CASES)
+def test_fused_depthwise_pointwise_block(ctx, oracle, case):
+    from seeded_inputs.workloads import Layer
+
+    N, H, W, C, Cout, pad = case
+    x = si.uniform(311, 0, (N, H, W, C), 0, 6)
+    layers = [Layer("depthwise_conv2d", (3, 3), (1, 1), (1, 1), pad, "relu6", 1, "dw"),
+              Layer("conv2d", (1, 1), (1, 1), (1, 1), "same", "relu6", Cout, "pw")]
+    si.make_model_weights(layers, C, 311)
+    model = ctx.model(layers, x.shape)
+    assert model.launches_per_run == 1          # the two layers run as one kernel
+    got = host(model.run(dev(x)))
+    ctx.check_device_status()
+    want = oracle.run_model(layers, x)
+    assert got.shape == want.shape
+    assert rel_fro(got, want) <= TF32_TOL
+    model.set_keep_all(True)                    # debug mode: the two stand-alone kernels
+    assert model.launches_per_run == 2
+    unfused = host(model.run(dev(x)))
+    assert same_bits(got, unfused)              # same arithmetic in the same order
+    model.close()
+    # small integers: exact in TF32 and fp32, so bit-identical to the oracle
+    xi = si.small_integers(312, 0, x.shape, 0, 3)
+    for layer in layers:
+        layer.filter = si.small_integers(312, 1, layer.filter.shape, -2, 2)
+        layer.bias = si.small_integers(312, 2, layer.bias.shape, -2, 2)
+        layer.act = "none"
+    model = ctx.model(layers, x.shape)
+    assert same_bits(host(model.run(dev(xi))), oracle.run_model(layers, xi))
+    ctx.check_device_status()
+    model.close()
