@@ -211,6 +211,14 @@ tfjsb_status tfjsb_run_model(tfjsb_model* model, const tfjsb_tensor* input, tfjs
  * run). */
 tfjsb_status tfjsb_run_model_host(tfjsb_model* model, const float* host_input, float* host_output, void* stream);
 
+/* A stride-1 3x3 depthwise layer followed by a pointwise layer (<= 512 output channels, depthwise
+ * channels a multiple of 32) can run as ONE kernel that keeps the depthwise output in shared
+ * memory as the tensor-core operand, so the intermediate tensor is neither written nor read back.
+ * mode 0: never; 1 (default): where the pair has enough 8x16-pixel tiles for the fused kernel to be
+ * the faster choice; 2: wherever the shapes allow.  Results are bit-identical in every mode.  The
+ * keep-all debug mode always runs the layers separately. */
+tfjsb_status tfjsb_model_set_fusion(tfjsb_model* model, int mode);
+
 /* Replays one run as a CUDA graph instead of enqueueing the layers one by one (the enqueue cost per
  * program is what the paper's async design hides, Sec. 4.1.1; a graph removes it from the host).
  * The graph is captured on a private stream at the next tfjsb_run_model, for the input / output

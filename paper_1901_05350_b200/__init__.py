@@ -31,7 +31,7 @@ EXPORTS = [
     "tfjsb_launch_count", "tfjsb_window_out_shape", "tfjsb_matmul", "tfjsb_matmul_static_scratch", "tfjsb_conv2d", "tfjsb_depthwise_conv2d",
     "tfjsb_avg_pool", "tfjsb_softmax", "tfjsb_bias_act", "tfjsb_model_create", "tfjsb_model_destroy",
     "tfjsb_model_output_shape", "tfjsb_model_launches_per_run", "tfjsb_run_model", "tfjsb_run_model_host",
-    "tfjsb_model_set_keep_all", "tfjsb_model_set_graph", "tfjsb_model_layer_output", "tfjsb_model_profile",
+    "tfjsb_model_set_keep_all", "tfjsb_model_set_graph", "tfjsb_model_set_fusion", "tfjsb_model_layer_output", "tfjsb_model_profile",
 ]
 
 
@@ -93,6 +93,7 @@ def _load_library() -> ctypes.CDLL:
     lib.tfjsb_run_model_host.argtypes = [vp, vp, vp, vp]
     lib.tfjsb_model_set_keep_all.argtypes = [vp, i32]
     lib.tfjsb_model_set_graph.argtypes = [vp, i32]
+    lib.tfjsb_model_set_fusion.argtypes = [vp, i32]
     lib.tfjsb_model_layer_output.argtypes = [vp, i32, tp]
     lib.tfjsb_model_profile.argtypes = [vp, tp, tp, i32, ctypes.POINTER(ctypes.c_float), vp]
     return lib
@@ -306,6 +307,10 @@ class Model:
 
     def set_keep_all(self, keep_all: bool):
         self.ctx._check(lib.tfjsb_model_set_keep_all(self._h, int(keep_all)))
+
+    def set_fusion(self, mode: str):
+        """'off', 'auto' (default) or 'always': run depthwise + pointwise pairs as one fused kernel."""
+        self.ctx._check(lib.tfjsb_model_set_fusion(self._h, {"off": 0, "auto": 1, "always": 2}[mode]))
 
     def set_graph(self, use_graph: bool):
         """Replay runs as a CUDA graph captured inside the library (run once without it first)."""

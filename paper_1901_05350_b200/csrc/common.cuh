@@ -168,7 +168,7 @@ struct DwPwPlan {
     CUtensorMap map_x, map_b, map_y;
     ConvGeom g{};   // geometry of the depthwise layer
     int Co = 0;
-    int block_n = 0, acc_stages = 0, patch_stages = 0, a_stages = 0, b_stages = 0;
+    int block_n = 0, n_sub = 1, acc_stages = 0, patch_stages = 0, a_stages = 0, b_stages = 0;
     int tiles_x = 0, tiles_y = 0, num_tiles = 0, grid = 0;
     size_t smem_bytes = 0;
 };

@@ -42,7 +42,8 @@ struct FusedArgs {
     int pt, pl;               // padding before
     int tiles_x, tiles_y;
     int num_tiles;
-    int block_n;
+    int block_n;              // accumulator columns per MMA group (<= 256)
+    int n_sub;                // MMA groups per k-block: 1, or 2 when 256 < Cout <= 512 (they share the A tile)
     int acc_stages;
     int patch_stages, a_stages, b_stages;
     const float* dw_filter;   // [3,3,C,1]
@@ -105,7 +106,8 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_y) : "memory");
     }
-    const uint32_t tmem_cols = (uint32_t)(args.acc_stages * block_n);
+    const int acc_cols = block_n * args.n_sub;  // accumulator columns per tile
+    const uint32_t tmem_cols = (uint32_t)(args.acc_stages * acc_cols);
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                          smem_u32(&tmem_base_slot)),
@@ -137,11 +139,14 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     tma_load_4d(patch_base + (uint32_t)ps * F_PATCH_STRIDE, &map_x, pf, kb * BLOCK_K,
                                 tx * F_TW - args.pl, ty * F_TH - args.pt, n);
                     if (++ps == args.patch_stages) { ps = 0; pphase ^= 1u; }
-                    if (!bounded_wait(smem_u32(&bar_b_empty[bs]), bphase ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t bf = smem_u32(&bar_b_full[bs]);
-                    mbar_arrive_expect_tx(bf, (uint32_t)b_stage_bytes);
-                    tma_load_2d(b_base + (uint32_t)bs * (uint32_t)b_stage_bytes, &map_b, bf, kb * BLOCK_K, 0);
-                    if (++bs == args.b_stages) { bs = 0; bphase ^= 1u; }
+                    for (int h = 0; ok && h < args.n_sub; ++h) {
+                        if (!bounded_wait(smem_u32(&bar_b_empty[bs]), bphase ^ 1u, abort_flag)) { ok = false; break; }
+                        const uint32_t bf = smem_u32(&bar_b_full[bs]);
+                        mbar_arrive_expect_tx(bf, (uint32_t)b_stage_bytes);
+                        tma_load_2d(b_base + (uint32_t)bs * (uint32_t)b_stage_bytes, &map_b, bf, kb * BLOCK_K, h * block_n);
+                        if (++bs == args.b_stages) { bs = 0; bphase ^= 1u; }
+                    }
+                    if (!ok) break;
                     ++issued;
                 }
             }
@@ -161,9 +166,12 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                                            (uint32_t)((k / args.patch_stages) & 1)) &&
                             k >= issued - args.patch_stages)
                             all = false;
-                        if (!mbar_try_wait(smem_u32(&bar_b_full[k % args.b_stages]), (uint32_t)((k / args.b_stages) & 1)) &&
-                            k >= issued - args.b_stages)
-                            all = false;
+                        for (int h = 0; h < args.n_sub; ++h) {
+                            const int kk = k * args.n_sub + h;  // index of the B copy in its own ring
+                            if (kk >= issued * args.n_sub - args.b_stages &&
+                                !mbar_try_wait(smem_u32(&bar_b_full[kk % args.b_stages]), (uint32_t)((kk / args.b_stages) & 1)))
+                                all = false;
+                        }
                     }
                 }
                 if (!all) atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_DRAIN);
@@ -179,22 +187,25 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
                 if (!bounded_wait(smem_u32(&bar_acc_empty[acc]), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * block_n);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * acc_cols);
                 for (int kb = 0; kb < num_k_blocks; ++kb) {
-                    if (!bounded_wait(smem_u32(&bar_b_full[bs]), bphase, abort_flag)) { ok = false; break; }
                     if (!bounded_wait(smem_u32(&bar_a_full[as]), aphase, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
                     const uint64_t a_desc = make_kmajor_sw128_desc(a_base + (uint32_t)as * A_STAGE_BYTES);
-                    const uint64_t b_desc = make_kmajor_sw128_desc(b_base + (uint32_t)bs * (uint32_t)b_stage_bytes);
+                    for (int h = 0; h < args.n_sub; ++h) {
+                        if (!bounded_wait(smem_u32(&bar_b_full[bs]), bphase, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint64_t b_desc = make_kmajor_sw128_desc(b_base + (uint32_t)bs * (uint32_t)b_stage_bytes);
 #pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                        tc_mma_tf32(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                    (kb | k) != 0 ? 1u : 0u);
-                    issued_any = true;
+                        for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                            tc_mma_tf32(d_tmem + (uint32_t)(h * block_n), a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k),
+                                        idesc, (kb | k) != 0 ? 1u : 0u);
+                        issued_any = true;
+                        tc_commit(smem_u32(&bar_b_empty[bs]));
+                        if (++bs == args.b_stages) { bs = 0; bphase ^= 1u; }
+                    }
+                    if (!ok) break;
                     tc_commit(smem_u32(&bar_a_empty[as]));
-                    tc_commit(smem_u32(&bar_b_empty[bs]));
                     if (++as == args.a_stages) { as = 0; aphase ^= 1u; }
-                    if (++bs == args.b_stages) { bs = 0; bphase ^= 1u; }
                 }
                 if (!ok) break;
                 tc_commit(smem_u32(&bar_acc_full[acc]));
@@ -223,7 +234,7 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         const int quad = warp & 3;   // TMEM lanes 32*quad.. = image rows 2*quad, 2*quad+1 of the tile
         const int half = ew >> 2;
         const uint32_t slab = epi_base + (uint32_t)ew * EPI_SLAB_BYTES;
-        const int chunks_per_tile = block_n / EPI_COLS;
+        const int chunks_per_tile = acc_cols / EPI_COLS;
         int n_chunks = (args.Co + EPI_COLS - 1) / EPI_COLS;
         if (n_chunks > chunks_per_tile) n_chunks = chunks_per_tile;
         int acc = 0;
@@ -247,7 +258,7 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             bool released = false;
             for (int ch = first_chunk; ch < n_chunks; ch += 2) {
                 uint32_t r[32];
-                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * block_n + ch * EPI_COLS);
+                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * acc_cols + ch * EPI_COLS);
                 tc_ld_32x32(taddr, r);
                 tc_ld_wait();
                 if (ch + 2 >= n_chunks) {
@@ -374,7 +385,7 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 bool dwpw_fused_supported(const ConvGeom& dw, int64_t Cout) {
     const int64_t tiles = dw.N * ((dw.Ho + F_TH - 1) / F_TH) * ((dw.Wo + F_TW - 1) / F_TW);
     return dw.fh == 3 && dw.fw == 3 && dw.sh == 1 && dw.sw == 1 && dw.dh == 1 && dw.dw == 1 && dw.mult == 1 &&
-           dw.C >= BLOCK_K && dw.C % BLOCK_K == 0 && Cout >= 4 && Cout <= 256 && Cout % 4 == 0 && tiles >= 1 &&
+           dw.C >= BLOCK_K && dw.C % BLOCK_K == 0 && Cout >= 4 && Cout <= 512 && Cout % 4 == 0 && tiles >= 1 &&
            tiles < (1LL << 31) && dw.N < (1LL << 31);
 }
 
@@ -385,11 +396,13 @@ tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
     plan->g = dw;
     plan->Co = (int)Cout;
     int bn = 32;
-    while (bn < Cout) bn <<= 1;
+    while (bn < Cout && bn < 256) bn <<= 1;
     plan->block_n = bn;
-    plan->acc_stages = bn == 256 ? 2 : MAX_ACC_STAGES;
-    plan->a_stages = 3;
-    plan->b_stages = bn == 256 ? 2 : 3;
+    plan->n_sub = Cout > 256 ? 2 : 1;
+    // tensor memory has 512 columns: two 256-wide halves leave room for one accumulator stage only
+    plan->acc_stages = plan->n_sub == 2 ? 1 : (bn == 256 ? 2 : MAX_ACC_STAGES);
+    plan->a_stages = plan->n_sub == 2 ? 2 : 3;
+    plan->b_stages = plan->n_sub == 2 ? 3 : (bn == 256 ? 2 : 3);
     const int fixed = EPI_BYTES + plan->a_stages * A_STAGE_BYTES + plan->b_stages * bn * BLOCK_K * 4;
     int ps = (SMEM_LIMIT - 2048 - fixed) / F_PATCH_STRIDE;
     if (ps > F_MAX_RING) ps = F_MAX_RING;
@@ -451,6 +464,7 @@ cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, cons
     a.tiles_x = plan.tiles_x; a.tiles_y = plan.tiles_y;
     a.num_tiles = plan.num_tiles;
     a.block_n = plan.block_n;
+    a.n_sub = plan.n_sub;
     a.acc_stages = plan.acc_stages;
     a.patch_stages = plan.patch_stages; a.a_stages = plan.a_stages; a.b_stages = plan.b_stages;
     a.dw_filter = dw_filter; a.dw_bias = dw_bias; a.dw_act = dw_act;

@@ -33,6 +33,8 @@ struct Step {
     // a depthwise layer followed by a pointwise layer can run as one fused kernel (the pointwise step
     // is then skipped); the separate plans are kept for the keep-all debug mode
     bool fuse_next = false;
+    bool fusable = false;     // the pair's shapes fit the fused kernel
+    bool fuse_pays = false;   // and there are enough tiles for it to be the faster choice
     DwPwPlan fused_plan{};
     int32_t out_rank = 4;
     int64_t out_dims[4] = {0, 0, 0, 0};
@@ -441,8 +443,15 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
             Step& dw = m->steps[i];
             const Step& pw = m->steps[i + 1];
             if (dw.kind == STEP_DEPTHWISE && pw.kind == STEP_GEMM_TF32 && pw.K == dw.g.Co &&
-                pw.M == dw.g.N * dw.g.Ho * dw.g.Wo && dwpw_fused_supported(dw.g, pw.N))
-                dw.fuse_next = true;
+                pw.M == dw.g.N * dw.g.Ho * dw.g.Wo && dwpw_fused_supported(dw.g, pw.N)) {
+                // The fused kernel has one unit of parallelism per 8 x 16 pixel tile: it pays off when
+                // there are several waves of tiles; with few tiles (small batches, 14 x 14 images) the
+                // stand-alone kernels spread channel blocks and column tiles over more SMs.
+                const int64_t tiles = dw.g.N * ((dw.g.Ho + 7) / 8) * ((dw.g.Wo + 15) / 16);
+                dw.fusable = true;
+                dw.fuse_pays = tiles >= 4 * (int64_t)ctx->sm_count;
+                dw.fuse_next = dw.fuse_pays;
+            }
         }
     }
     if ((st = dev_alloc(m, 2 * m->region_elems, &m->arena)) != TFJSB_OK) return bail(st, ctx->last_error);
@@ -502,6 +511,21 @@ tfjsb_status tfjsb_run_model(tfjsb_model* m, const tfjsb_tensor* input, tfjsb_te
         cudaError_t e = launch_layers(m, i, s, &used);
         if (e != cudaSuccess) return cuda_fail(m->ctx, e, "layer launch");
     }
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_model_set_fusion(tfjsb_model* m, int mode) {
+    if (!m) return TFJSB_ERR_INVALID_ARG;
+    if (mode < 0 || mode > 2) return fail(m->ctx, TFJSB_ERR_INVALID_ARG, "fusion mode must be 0 (off), 1 (auto) or 2 (always)");
+    for (Step& st : m->steps) st.fuse_next = st.fusable && (mode == 2 || (mode == 1 && st.fuse_pays));
+    for (tfjsb_model* v : m->slices) {
+        for (Step& st : v->steps) st.fuse_next = st.fusable && (mode == 2 || (mode == 1 && st.fuse_pays));
+        v->bound_in = nullptr; v->bound_out = nullptr;
+        drop_graph(v);
+    }
+    m->bound_in = nullptr;  // buffers and plans are re-assigned on the next run
+    m->bound_out = nullptr;
+    drop_graph(m);
     return TFJSB_OK;
 }
 

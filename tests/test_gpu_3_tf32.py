@@ -170,6 +170,8 @@ FUSED_BLOCK_CASES = [
     (2, 7, 7, 256, 256, "same"),       # eight k-blocks, 256-wide accumulator (two stages)
     (1, 30, 33, 64, 100, "valid"),     # 'valid': no padding offset, Cout not a multiple of 32
     (5, 56, 56, 96, 36, "same"),       # more tiles than SMs, three k-blocks
+    (2, 14, 14, 512, 512, "same"),     # two 256-wide accumulator halves sharing each A tile, 16 k-blocks
+    (1, 9, 20, 64, 320, "same"),       # second half partly empty (320 = 256 + 64)
 ]
 
 
@@ -183,6 +185,7 @@ def test_fused_depthwise_pointwise_block(ctx, oracle, case):
               Layer("conv2d", (1, 1), (1, 1), (1, 1), "same", "relu6", Cout, "pw")]
     si.make_model_weights(layers, C, 311)
     model = ctx.model(layers, x.shape)
+    model.set_fusion("always")                  # small cases: 'auto' would keep the layers apart
     assert model.launches_per_run == 1          # the two layers run as one kernel
     got = host(model.run(dev(x)))
     ctx.check_device_status()
@@ -201,6 +204,7 @@ def test_fused_depthwise_pointwise_block(ctx, oracle, case):
         layer.bias = si.small_integers(312, 2, layer.bias.shape, -2, 2)
         layer.act = "none"
     model = ctx.model(layers, x.shape)
+    model.set_fusion("always")
     assert same_bits(host(model.run(dev(xi))), oracle.run_model(layers, xi))
     ctx.check_device_status()
     model.close()
