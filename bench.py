@@ -143,11 +143,35 @@ def layer_work(layers, in_shape, window_out_shape):
     return rows
 
 
+def merge_fused(rows, ms):
+    """The executor may run a depthwise layer and the pointwise layer after it as one kernel; the
+    profile then reports the pair's time under the depthwise layer and ~0 under the pointwise one.
+    Such pairs become one row: the fused kernel reads the depthwise input and writes the pointwise
+    output, the intermediate tensor is never in HBM."""
+    out_rows, out_ms = [], []
+    i = 0
+    while i < len(rows):
+        r = rows[i]
+        if (r["kernel"] == "depthwise3x3" and i + 1 < len(rows) and rows[i + 1]["kernel"] == "gemm_tf32"
+                and ms[i + 1] < 0.02 * ms[i]):
+            pw = rows[i + 1]
+            inter = 4 * r["units"]  # the depthwise output = the pointwise input, counted once in each row
+            out_rows.append(dict(name=r["name"] + "+" + pw["name"], kernel="dwpw_fused", flops=r["flops"] + pw["flops"],
+                                 bytes=r["bytes"] + pw["bytes"] - 2 * inter, units=pw["units"]))
+            out_ms.append(ms[i] + ms[i + 1])
+            i += 2
+        else:
+            out_rows.append(r)
+            out_ms.append(ms[i])
+            i += 1
+    return out_rows, out_ms
+
+
 def roofline_rows(rows, ms, peaks, fp32_tflops):
     tf32_peak = peaks["bf16_tflops_sustained"] / 2.0  # dense TF32 is nominally half of dense bf16
     out = []
     for row, t_ms in zip(rows, ms):
-        on_tensor_cores = row["kernel"] in ("gemm_tf32", "conv2d_igemm_tf32")
+        on_tensor_cores = row["kernel"] in ("gemm_tf32", "conv2d_igemm_tf32", "dwpw_fused")
         compute_peak = tf32_peak if on_tensor_cores else fp32_tflops
         t_compute = row["flops"] / (compute_peak * 1e12)
         t_hbm = row["bytes"] / (peaks["hbm_gbs"] * 1e9)
@@ -314,7 +338,8 @@ def run_ours(args):
         reps = max(5, min(50, args.steps))
         ms = model.profile(x, out=out, reps=reps)
         fp32_tflops = props.multi_processor_count * 128 * 2 * (clocks["sm_max_mhz"] or 1965) * 1e6 / 1e12
-        rows = roofline_rows(layer_work(layers, x_host.shape, tfjsb.window_out_shape), ms, peaks, fp32_tflops)
+        work, ms = merge_fused(layer_work(layers, x_host.shape, tfjsb.window_out_shape), ms)
+        rows = roofline_rows(work, ms, peaks, fp32_tflops)
         by_kernel = {}
         for r in rows:
             k = by_kernel.setdefault(r["kernel"], dict(ms=0.0, launches=0))

@@ -44,6 +44,20 @@ __device__ __forceinline__ float apply_act(float v, int act) {
     const float r6 = relu6_nan(v);
     return act == TFJSB_ACT_NONE ? v : (act == TFJSB_ACT_RELU6 ? r6 : r);
 }
+// Two independent fp32 FMAs in one instruction (sm_100 packed fp32): acc.{x,y} += a.{x,y} * b.{x,y},
+// each lane rounded exactly like a scalar fmaf.  Halves the issue slots of the CUDA-core kernels,
+// which are bound by instruction issue.
+__device__ __forceinline__ void fma2(float2& acc, const float2& a, const float2& b) {
+    unsigned long long& d = reinterpret_cast<unsigned long long&>(acc);
+    asm("fma.rn.f32x2 %0, %1, %2, %0;"
+        : "+l"(d)
+        : "l"(reinterpret_cast<const unsigned long long&>(a)), "l"(reinterpret_cast<const unsigned long long&>(b)));
+}
+__device__ __forceinline__ void fma4_packed(float4& acc, const float4& a, const float4& b) {
+    fma2(reinterpret_cast<float2*>(&acc)[0], reinterpret_cast<const float2*>(&a)[0], reinterpret_cast<const float2*>(&b)[0]);
+    fma2(reinterpret_cast<float2*>(&acc)[1], reinterpret_cast<const float2*>(&a)[1], reinterpret_cast<const float2*>(&b)[1]);
+}
+
 template <int ACT>
 __device__ __forceinline__ float apply_act_t(float v) {
     if (ACT == TFJSB_ACT_NONE) return v;

@@ -277,9 +277,9 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
                 for (int ky = 0; ky < 3; ++ky) {
                     const int d = j - ky;
                     if (d >= 0 && d % S == 0 && d / S < R) {
-                        fma4(acc[d / S], v0, w[ky * 3 + 0]);
-                        fma4(acc[d / S], v1, w[ky * 3 + 1]);
-                        fma4(acc[d / S], v2, w[ky * 3 + 2]);
+                        fma4_packed(acc[d / S], v0, w[ky * 3 + 0]);
+                        fma4_packed(acc[d / S], v1, w[ky * 3 + 1]);
+                        fma4_packed(acc[d / S], v2, w[ky * 3 + 2]);
                     }
                 }
             }
