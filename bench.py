@@ -246,6 +246,7 @@ def run_ours(args):
 
     import paper_1901_05350_b200 as tfjsb
     import seeded_inputs as si
+    from paper_1901_05350_b200 import replicas
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -295,11 +296,7 @@ def run_ours(args):
     launches = ctx.launch_count - launches0
     clocks = sampler.stop()
     ctx.check_device_status()
-    elapsed_ms = start.elapsed_time(stop)
-    if distributed:
-        t = torch.tensor([elapsed_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = replicas.max_over_ranks(start.elapsed_time(stop), device="cuda")
     value = world * BATCH * args.steps / (elapsed_ms * 1e-3)
 
     # ---- end to end: pinned host input in, probabilities back to the host, every step
@@ -314,11 +311,7 @@ def run_ours(args):
         model.run_host(hin, hout)
     stop.record(stream)
     barrier()
-    e2e_ms = start.elapsed_time(stop)
-    if distributed:
-        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = replicas.max_over_ranks(start.elapsed_time(stop), device="cuda")
     e2e = {"value": world * BATCH * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
            "h2d_bytes_per_step": int(hin.numel() * 4), "d2h_bytes_per_step": int(hout.numel() * 4), "steps": e2e_steps}
 
