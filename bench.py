@@ -153,7 +153,7 @@ def merge_fused(rows, ms):
     while i < len(rows):
         r = rows[i]
         if (r["kernel"] == "depthwise3x3" and i + 1 < len(rows) and rows[i + 1]["kernel"] == "gemm_tf32"
-                and ms[i + 1] < 0.02 * ms[i]):
+                and ms[i + 1] < 0.1 * ms[i]):
             pw = rows[i + 1]
             inter = 4 * r["units"]  # the depthwise output = the pointwise input, counted once in each row
             out_rows.append(dict(name=r["name"] + "+" + pw["name"], kernel="dwpw_fused", flops=r["flops"] + pw["flops"],
