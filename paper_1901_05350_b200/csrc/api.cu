@@ -9,6 +9,8 @@ using namespace tfjsb;
 
 namespace tfjsb {
 
+thread_local bool g_launch_pdl = false;
+
 tfjsb_status fail(tfjsb_ctx* ctx, tfjsb_status st, const std::string& msg) {
     if (ctx) ctx->last_error = msg;
     return st;

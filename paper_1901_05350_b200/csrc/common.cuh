@@ -7,6 +7,7 @@
 #include <stdint.h>
 
 #include <string>
+#include <utility>
 
 #include "tfjsb.h"
 
@@ -95,6 +96,27 @@ tfjsb_status fail(tfjsb_ctx* ctx, tfjsb_status st, const std::string& msg);
 tfjsb_status cuda_fail(tfjsb_ctx* ctx, cudaError_t err, const char* what);
 // Grows `s` to at least `bytes` (frees and reallocates; callers keep stream order in mind).
 tfjsb_status ensure_scratch(tfjsb_ctx* ctx, Scratch* s, size_t bytes);
+
+// ---- kernel launch with optional programmatic dependent launch --------------------------------------
+// The executor sets this while it enqueues a model: its kernels all call pdl_wait() before reading
+// their inputs, so each may be launched while the previous one drains and only its prologue
+// (barrier set-up, tensor-map prefetch, TMEM allocation) overlaps.  Off for stand-alone op calls.
+extern thread_local bool g_launch_pdl;
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_launch_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // ---- geometry of one convolution / pooling call -----------------------------------------------
 struct ConvGeom {

@@ -182,6 +182,8 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
     }
     __syncthreads();
+    ptx::pdl_launch_dependents();
+    ptx::pdl_wait();  // the input is the previous kernel's output
 
     const int num_tiles = (int)t.num_tiles;
     const int first = blockIdx.x, step = gridDim.x;
@@ -329,8 +331,8 @@ cudaError_t launch_tma_instance(const DepthwisePlan& plan, const float* f, const
         attr_set = true;
     }
     DwTiling t{plan.tiles_x, plan.tiles_y, plan.c_blocks, plan.stages, (long long)plan.num_tiles};
-    kernel<<<plan.grid, DW_TMA_THREADS, plan.smem_bytes, s>>>(plan.map_x, f, bias, act, y, g, t, dev_status);
-    return cudaGetLastError();
+    return launch_k(kernel, dim3(plan.grid), dim3(DW_TMA_THREADS), plan.smem_bytes, s, plan.map_x, f, bias, act, y, g, t,
+                    dev_status);
 }
 
 int pow2_at_most(int v, int cap) {

@@ -120,6 +120,8 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     const int tiles_per_image = args.tiles_x * args.tiles_y;
+    pdl_launch_dependents();
+    pdl_wait();  // the block input is the previous kernel's output
 
     if (warp == 0) {
         // ---------------------------------------------------------------- producer
@@ -470,9 +472,10 @@ cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, cons
     a.dw_filter = dw_filter; a.dw_bias = dw_bias; a.dw_act = dw_act;
     a.pw_bias = pw_bias; a.pw_act = pw_act;
     a.dev_status = dev_status;
-    dwpw_fused_kernel<<<plan.grid, F_THREADS, plan.smem_bytes, s>>>(plan.map_x, plan.map_b, plan.map_y, a);
+    cudaError_t e = launch_k(dwpw_fused_kernel, dim3(plan.grid), dim3(F_THREADS), plan.smem_bytes, s, plan.map_x, plan.map_b,
+                             plan.map_y, a);
     ++*launches;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace tfjsb

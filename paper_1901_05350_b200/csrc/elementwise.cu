@@ -1,6 +1,7 @@
 // Bandwidth-bound helpers: the standalone bias+activation op, avgPool, softmax, and the
 // 2-D transpose used to make matMul operands K-contiguous.
 #include "common.cuh"
+#include "ptx_sm100.cuh"
 
 namespace tfjsb {
 
@@ -77,6 +78,8 @@ __global__ void avg_pool_global_kernel(const float* __restrict__ x, float* __res
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c = blockIdx.x * 32 + lane;
     const int64_t n = blockIdx.y;
+    ptx::pdl_launch_dependents();
+    ptx::pdl_wait();
     float acc = 0.0f;
     if (c < C) {
         const float* base = x + n * (int64_t)HW * C + c;
@@ -111,6 +114,8 @@ __global__ void softmax_rows_kernel(const float* __restrict__ x, float* __restri
     const float* xr = x + (int64_t)blockIdx.x * cols;
     float* yr = y + (int64_t)blockIdx.x * cols;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    ptx::pdl_launch_dependents();
+    ptx::pdl_wait();
 
     float m = -INFINITY;
     for (int64_t j = threadIdx.x; j < cols; j += kThreads) m = fmaxf(m, xr[j]);
@@ -202,7 +207,9 @@ cudaError_t launch_avg_pool(const float* x, float* y, const ConvGeom& g, cudaStr
                         g.N <= 65535;
     if (global) {
         dim3 grid((g.C + 31) / 32, (unsigned)g.N);
-        avg_pool_global_kernel<<<grid, 256, 0, s>>>(x, y, g.H * g.W, g.C);
+        cudaError_t e = launch_k(avg_pool_global_kernel, grid, dim3(256), 0, s, x, y, g.H * g.W, g.C);
+        ++*launches;
+        return e;
     } else {
         avg_pool_window_kernel<<<grid_for(n_out, kThreads, 148 * 16), kThreads, 0, s>>>(x, y, g, n_out);
     }
@@ -214,9 +221,9 @@ cudaError_t launch_softmax(const float* x, float* y, int64_t rows, int64_t cols,
                            int64_t* launches) {
     if (rows == 0) return cudaSuccess;
     // gridDim.x is 2^31-1: enough for any tensor that fits in memory
-    softmax_rows_kernel<<<(unsigned)rows, kThreads, 0, s>>>(x, y, cols);
+    cudaError_t e = launch_k(softmax_rows_kernel, dim3((unsigned)rows), dim3(kThreads), 0, s, x, y, cols);
     ++*launches;
-    return cudaGetLastError();
+    return e;
 }
 
 cudaError_t launch_transpose(const float* in, float* out, int64_t rows, int64_t cols, cudaStream_t s,

@@ -70,6 +70,8 @@ struct tfjsb_model {
     cudaEvent_t compute_done = nullptr;
     bool is_view = false;
     // optional CUDA-graph replay of one run (tfjsb_model_set_graph): captured for the current binding
+    // programmatic dependent launch between the layers' kernels (each waits before reading its input)
+    bool use_pdl = true;
     bool use_graph = false;
     cudaGraphExec_t graph_exec = nullptr;
     cudaStream_t capture_stream = nullptr;
@@ -196,6 +198,7 @@ tfjsb_model* make_batch_view(tfjsb_model* parent, int64_t n) {
     v->ctx = parent->ctx;
     v->is_view = true;
     v->use_tf32 = parent->use_tf32;
+    v->use_pdl = parent->use_pdl;
     v->arena = parent->arena;
     v->region_elems = parent->region_elems;
     v->steps = parent->steps;
@@ -253,8 +256,14 @@ tfjsb_status capture_graph(tfjsb_model* m) {
 }
 
 // Launches layer i (and, when it is fused with its successor, that one too); returns how many layers ran.
+struct PdlScope {
+    explicit PdlScope(bool on) { g_launch_pdl = on; }
+    ~PdlScope() { g_launch_pdl = false; }
+};
+
 cudaError_t launch_layers(tfjsb_model* m, int i, cudaStream_t s, int* consumed) {
     const Step& st = m->steps[i];
+    PdlScope pdl(m->use_pdl);
     if (st.fuse_next && !m->keep_all) {
         const Step& pw = m->steps[i + 1];
         *consumed = 2;
@@ -304,6 +313,7 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
     tfjsb_model* m = new tfjsb_model();
     m->ctx = ctx;
     m->use_tf32 = ctx->math == TFJSB_MATH_TF32 && ctx->encode_tiled != nullptr;
+    m->use_pdl = getenv("TFJSB_NO_PDL") == nullptr;
     for (int i = 0; i < 4; ++i) m->in_dims[i] = input_dims[i];
     m->in_elems = input_dims[0] * input_dims[1] * input_dims[2] * input_dims[3];
 

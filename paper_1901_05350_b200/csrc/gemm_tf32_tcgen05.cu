@@ -195,6 +195,10 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    // everything above touched only this CTA's shared and tensor memory; the inputs come from the
+    // previous kernel in the stream
+    pdl_launch_dependents();
+    pdl_wait();
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
@@ -562,6 +566,7 @@ cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int ac
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
+    cudaError_t e;
     KernelArgs args;
     args.M = (int)plan.M; args.N = (int)plan.N; args.K = (int)plan.K;
     args.block_n = plan.block_n;
@@ -575,11 +580,13 @@ cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int ac
     args.x = plan.x;
     args.g = plan.g;
     if (plan.gather)
-        gemm_tf32_kernel<true><<<plan.grid, CONV_THREADS, plan.smem_bytes, s>>>(plan.map_a, plan.map_b, plan.map_c, args);
+        e = launch_k(gemm_tf32_kernel<true>, dim3(plan.grid), dim3(CONV_THREADS), plan.smem_bytes, s, plan.map_a, plan.map_b,
+                     plan.map_c, args);
     else
-        gemm_tf32_kernel<false><<<plan.grid, GEMM_THREADS, plan.smem_bytes, s>>>(plan.map_a, plan.map_b, plan.map_c, args);
+        e = launch_k(gemm_tf32_kernel<false>, dim3(plan.grid), dim3(GEMM_THREADS), plan.smem_bytes, s, plan.map_a, plan.map_b,
+                     plan.map_c, args);
     ++*launches;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace tfjsb

@@ -125,6 +125,14 @@ __device__ __forceinline__ uint32_t make_idesc_tf32(int m, int n) {
 }
 
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization attribute may
+// start while its predecessor in the stream is still running; it must call pdl_wait() before it
+// touches memory the predecessor writes (the wait returns once the predecessor has completed and its
+// writes are visible; it returns at once for an ordinary launch).  pdl_launch_dependents() tells the
+// scheduler that the successor may begin its own prologue.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // 4-D tiled store (coordinates innermost first); parts of the box outside the tensor are dropped.
 __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
     asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(map),
