@@ -71,8 +71,39 @@ __global__ void avg_pool_window_kernel(const float* __restrict__ x, float* __res
     }
 }
 
-// Global pool: a block owns (image n, 32 consecutive channels).  Lane = channel (coalesced 128-byte
-// rows), the 8 warps stride over the H*W positions, partial sums meet in shared memory.
+// Global pool: a block owns (image n, 128 consecutive channels).  Lane = 4 channels (one float4, so a
+// warp reads 512 contiguous bytes per position), the 8 warps stride over the H*W positions, partial
+// sums meet in shared memory.  C % 4 == 0.
+__global__ void avg_pool_global_vec4_kernel(const float* __restrict__ x, float* __restrict__ y, int HW, int C) {
+    __shared__ float4 partial[8][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int c = (blockIdx.x * 32 + lane) * 4;
+    const int64_t n = blockIdx.y;
+    ptx::pdl_launch_dependents();
+    ptx::pdl_wait();
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c < C) {
+        const float* base = x + n * (int64_t)HW * C + c;
+        for (int p = warp; p < HW; p += 8) {
+            const float4 v = *reinterpret_cast<const float4*>(base + (int64_t)p * C);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+    }
+    partial[warp][lane] = acc;
+    __syncthreads();
+    if (warp == 0 && c < C) {
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+            const float4 v = partial[w][lane];
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        }
+        const float inv = (float)HW;
+        *reinterpret_cast<float4*>(y + n * C + c) = make_float4(s.x / inv, s.y / inv, s.z / inv, s.w / inv);
+    }
+}
+
+// The same with one channel per lane, for channel counts that are not multiples of 4.
 __global__ void avg_pool_global_kernel(const float* __restrict__ x, float* __restrict__ y, int HW, int C) {
     __shared__ float partial[8][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -206,8 +237,14 @@ cudaError_t launch_avg_pool(const float* x, float* y, const ConvGeom& g, cudaStr
     const bool global = g.Ho == 1 && g.Wo == 1 && g.fh == g.H && g.fw == g.W && g.pt == 0 && g.pl == 0 &&
                         g.N <= 65535;
     if (global) {
-        dim3 grid((g.C + 31) / 32, (unsigned)g.N);
-        cudaError_t e = launch_k(avg_pool_global_kernel, grid, dim3(256), 0, s, x, y, g.H * g.W, g.C);
+        cudaError_t e;
+        if (g.C % 4 == 0) {
+            dim3 grid((g.C / 4 + 31) / 32, (unsigned)g.N);
+            e = launch_k(avg_pool_global_vec4_kernel, grid, dim3(256), 0, s, x, y, g.H * g.W, g.C);
+        } else {
+            dim3 grid((g.C + 31) / 32, (unsigned)g.N);
+            e = launch_k(avg_pool_global_kernel, grid, dim3(256), 0, s, x, y, g.H * g.W, g.C);
+        }
         ++*launches;
         return e;
     } else {

@@ -183,7 +183,8 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
     }
-    const uint32_t tmem_cols = (uint32_t)(acc_stages * block_n);  // 128, 256 or 512: a power of two >= 32
+    uint32_t tmem_cols = 32;  // allocations are powers of two >= 32 columns
+    while (tmem_cols < (uint32_t)(acc_stages * block_n)) tmem_cols <<= 1;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                          smem_u32(&tmem_base_slot)),
@@ -464,6 +465,13 @@ int choose_block_n(int64_t M, int64_t N, int sm_count) {
     while (bn < 256 && bn < N) bn <<= 1;
     const int64_t m_tiles = (M + BLOCK_M - 1) / BLOCK_M;
     while (bn > 32 && m_tiles * ((N + bn - 1) / bn) < sm_count) bn >>= 1;
+    if (bn == 256 && N > 256) {
+        // Wave quantisation: every tile of a launch costs the same, so the launch takes
+        // ceil(tiles / SMs) rounds of one tile each.  192-wide tiles (six 32-column chunks) sometimes
+        // fill the last round where 256-wide ones leave most SMs idle (196 tiles on 148 SMs).
+        auto rounds = [&](int w) { return (m_tiles * ((N + w - 1) / w) + sm_count - 1) / sm_count; };
+        if (rounds(192) * 192 < rounds(256) * 256) bn = 192;
+    }
     return bn;
 }
 
@@ -496,7 +504,7 @@ namespace {
 tfjsb_status plan_common(tfjsb_ctx* ctx, const float* bt, int64_t k_pitch, float* c, GemmTf32Plan* plan) {
     const int64_t M = plan->M, N = plan->N;
     plan->block_n = choose_block_n(M, N, ctx->sm_count);
-    plan->acc_stages = plan->block_n == 256 ? 2 : MAX_ACC_STAGES;
+    plan->acc_stages = plan->block_n > 128 ? 2 : MAX_ACC_STAGES;
     const int stage_bytes = A_STAGE_BYTES + plan->block_n * BLOCK_K * 4;
     int stages = (SMEM_LIMIT - 1024 - EPI_BYTES - 512) / stage_bytes;
     if (stages > MAX_STAGES) stages = MAX_STAGES;

@@ -33,6 +33,7 @@ GEMM_SHAPES = [
     (4100, 36, 260),      # N just above one 256 tile
     (49, 1024, 1024),     # many k-blocks: the stage ring wraps several times
     (20000, 256, 512),    # more tiles than SMs: persistent loop, both accumulator stages reused
+    (6272, 512, 1024),    # 196 tiles of 256 columns on 148 SMs: the 192-column tile is chosen instead
 ]
 
 
