@@ -1,6 +1,7 @@
 // C ABI of libtfjsb.so: context, shape inference, argument checks and dispatch of the op calls.
 // All validation happens here, on the host, before anything is launched.
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "common.cuh"
@@ -340,6 +341,14 @@ tfjsb_status tfjsb_conv2d(tfjsb_ctx* ctx, const tfjsb_tensor* x, const tfjsb_ten
         if ((e = launch_pack_filter(pf, ctx->scratch_b.ptr, (int64_t)g.fh * g.fw * g.C, Cout, k_pad, s, &ctx->launches)) !=
             cudaSuccess)
             return cuda_fail(ctx, e, "filter packing");
+        if (conv_patch_supported(g) && !getenv("TFJSB_NO_PATCH_CONV")) {
+            DwPwPlan pplan;
+            if ((st = conv_patch_plan(ctx, px, ctx->scratch_b.ptr, py, g, &pplan)) != TFJSB_OK) return st;
+            if ((e = launch_dwpw_fused(pplan, nullptr, nullptr, TFJSB_ACT_NONE, pbias, act, ctx->dev_status, s,
+                                       &ctx->launches)) != cudaSuccess)
+                return cuda_fail(ctx, e, "patch conv2d launch");
+            return TFJSB_OK;
+        }
         GemmTf32Plan plan;
         if ((st = conv_igemm_plan(ctx, px, ctx->scratch_b.ptr, py, g, &plan)) != TFJSB_OK) return st;
         if ((e = launch_gemm_tf32(plan, pbias, act, ctx->dev_status, s, &ctx->launches)) != cudaSuccess)

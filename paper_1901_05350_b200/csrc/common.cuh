@@ -207,10 +207,19 @@ struct DwPwPlan {
     int block_n = 0, n_sub = 1, acc_stages = 0, patch_stages = 0, a_stages = 0, b_stages = 0;
     int tiles_x = 0, tiles_y = 0, num_tiles = 0, grid = 0;
     size_t smem_bytes = 0;
+    int patch_bytes = 0, patch_stride = 0;
+    // small-window convolution mode of the same kernel
+    bool conv = false;
+    int row_floats = 0, patch_rows = 0;
 };
 bool dwpw_fused_supported(const ConvGeom& dw, int64_t Cout);
 tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, float* y, const ConvGeom& dw,
                              int64_t Cout, DwPwPlan* plan);
+// conv2d with fh*fw*Cin <= 32 on the same kernel (input patch by bulk tensor copy, im2col in shared
+// memory); `bt` is the filter packed [Cout, 32].  Launched with launch_dwpw_fused (pw_bias / pw_act = the
+// convolution's bias and activation; the depthwise arguments are ignored).
+bool conv_patch_supported(const ConvGeom& g);
+tfjsb_status conv_patch_plan(tfjsb_ctx* ctx, const float* x, const float* bt, float* y, const ConvGeom& g, DwPwPlan* plan);
 cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, const float* dw_bias, int dw_act,
                               const float* pw_bias, int pw_act, unsigned int* dev_status, cudaStream_t s,
                               int64_t* launches);

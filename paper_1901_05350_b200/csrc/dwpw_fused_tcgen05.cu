@@ -16,6 +16,13 @@
 //                tensor store of 2 image rows x 16 pixels x 32 channels (clipped at the image edge).
 // Every wait is bounded (see ptx_sm100.cuh); a timeout raises the abort flag all roles poll and is
 // reported through the context's device status word.
+//
+// Small-window convolution mode (template parameter CONV): a conv2d whose whole im2col row fits one
+// k-block (fh*fw*Cin <= 32, e.g. a 3x3 stem on RGB input) runs on the same pipeline.  The producer
+// brings the input patch of a tile in by one 3-D copy over x viewed as [N, H, W*Cin], four warps
+// rearrange it into the A operand (thread = pixel), the packed filter [Cout, 32] stays resident as
+// B, and the block is 14 warps so that two CTAs share an SM: per tile every role costs mostly its
+// own synchronisation, and two CTAs double each of them.
 #include "common.cuh"
 #include "ptx_sm100.cuh"
 #include "umma_tile.cuh"
@@ -27,14 +34,18 @@ using namespace tile;
 
 namespace {
 
-constexpr int F_THREADS = 832;        // 26 warps
+constexpr int F_THREADS = 832;        // 26 warps: producer, MMA, 8 epilogue, 16 depthwise; one CTA per SM
 constexpr int F_DW_WARPS = 16;
+constexpr int F_CONV_THREADS = 448;   // 14 warps: producer, MMA, 8 epilogue, 4 im2col; two CTAs per SM
+constexpr int F_CONV_CMP_WARPS = 4;
+constexpr int F_CONV_SMEM = 112 * 1024;  // per-CTA dynamic budget that lets two CTAs share an SM's 228 KiB
 constexpr int F_TH = 8, F_TW = 16;    // output pixels per tile (8 rows x 16 columns = 128 GEMM rows)
 constexpr int F_PH = F_TH + 2, F_PW = F_TW + 2;
 constexpr int F_PATCH_FLOATS = F_PH * F_PW * BLOCK_K;
 constexpr int F_PATCH_BYTES = F_PATCH_FLOATS * 4;              // 23040
 constexpr int F_PATCH_STRIDE = 23 * 1024;                      // stage pitch, keeps stages 1024-aligned
-constexpr int F_MAX_RING = 4;
+constexpr int F_MAX_RING = 12;
+constexpr int F_MAX_ACC = 8;           // accumulator stages (32-column tiles of the small-window mode use all)
 
 struct FusedArgs {
     int C, Co;                // depthwise channels (= K of the GEMM), pointwise output channels (= N)
@@ -46,6 +57,10 @@ struct FusedArgs {
     int n_sub;                // MMA groups per k-block: 1, or 2 when 256 < Cout <= 512 (they share the A tile)
     int acc_stages;
     int patch_stages, a_stages, b_stages;
+    int patch_bytes, patch_stride;   // bytes of one input patch and pitch of the patch ring
+    // small-window convolution mode (CONV): the patch holds (8-1)*sh+fh rows of row_floats floats
+    int cin, fw_cin, sh, sw, row_floats, k_total;
+    int koff[32];             // patch offset of im2col column k relative to the pixel's window origin
     const float* dw_filter;   // [3,3,C,1]
     const float* dw_bias;     // [C] or null
     int dw_act;
@@ -60,44 +75,59 @@ __device__ __forceinline__ void fma4s(float4& acc, const float4& a, const float4
     acc.z = fmaf(a.z, b.z, acc.z); acc.w = fmaf(a.w, b.w, acc.w);
 }
 
-__global__ void __launch_bounds__(F_THREADS, 1)
+template <bool CONV>
+__global__ void __launch_bounds__(CONV ? F_CONV_THREADS : F_THREADS, CONV ? 2 : 1)
 dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ CUtensorMap map_y, const FusedArgs args) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_patch_full[F_MAX_RING], bar_patch_empty[F_MAX_RING];
-    __shared__ __align__(8) uint64_t bar_a_full[F_MAX_RING], bar_a_empty[F_MAX_RING];
-    __shared__ __align__(8) uint64_t bar_b_full[F_MAX_RING], bar_b_empty[F_MAX_RING];
-    __shared__ __align__(8) uint64_t bar_acc_full[MAX_ACC_STAGES], bar_acc_empty[MAX_ACC_STAGES];
+    constexpr int RING = CONV ? F_MAX_RING : 4;       // deepest ring of this mode (the patch ring)
+    constexpr int ACCS = CONV ? F_MAX_ACC : MAX_ACC_STAGES;
+    __shared__ __align__(8) uint64_t bar_patch_full[RING], bar_patch_empty[RING];
+    __shared__ __align__(8) uint64_t bar_a_full[4], bar_a_empty[4];
+    __shared__ __align__(8) uint64_t bar_b_full[4], bar_b_empty[4];
+    __shared__ __align__(8) uint64_t bar_acc_full[ACCS], bar_acc_empty[ACCS];
     __shared__ __align__(8) uint64_t bar_drain;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
 
+    // Role split of the warps after the producer and the MMA issuer.  The small-window mode has
+    // little arithmetic per tile: what bounds a tile there is the fixed cost of each role's
+    // synchronisation (barrier waits, fences, MMA issue), so it runs as two small CTAs per SM, which
+    // doubles every role, instead of one large CTA.
+    constexpr int EPI_WARPS = 8;
+    constexpr int CMP_WARPS = CONV ? F_CONV_CMP_WARPS : F_DW_WARPS;
+    constexpr int CMP_WARP0 = 2 + EPI_WARPS;
+    constexpr int EPI_GROUPS = EPI_WARPS / 4;
+    static_assert((CMP_WARP0 + CMP_WARPS) * 32 == (CONV ? F_CONV_THREADS : F_THREADS), "role split must cover the block");
+
     volatile int* abort_flag = &abort_flag_s;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int block_n = args.block_n;
-    const int num_k_blocks = args.C / BLOCK_K;
+    const int num_k_blocks = CONV ? 1 : args.C / BLOCK_K;
     const int b_stage_bytes = block_n * BLOCK_K * 4;
 
     // dynamic shared memory (1024-aligned): [epilogue slabs][patch ring][A ring][B ring]
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t epi_base = smem_base;
-    const uint32_t patch_base = epi_base + EPI_BYTES;
-    const uint32_t a_base = patch_base + (uint32_t)args.patch_stages * F_PATCH_STRIDE;
+    const uint32_t patch_base = epi_base + (uint32_t)(EPI_WARPS * EPI_SLAB_BYTES);
+    const uint32_t a_base = patch_base + (uint32_t)(args.patch_stages * args.patch_stride);
     const uint32_t b_base = a_base + (uint32_t)args.a_stages * A_STAGE_BYTES;
     const float* patch_ptr = reinterpret_cast<const float*>(smem_raw + (patch_base - smem_u32(smem_raw)));
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < F_MAX_RING; ++s) {
+        for (int s = 0; s < RING; ++s) {
             mbar_init(smem_u32(&bar_patch_full[s]), 1);
-            mbar_init(smem_u32(&bar_patch_empty[s]), F_DW_WARPS);
-            mbar_init(smem_u32(&bar_a_full[s]), F_DW_WARPS);
+            mbar_init(smem_u32(&bar_patch_empty[s]), CMP_WARPS);
+        }
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(smem_u32(&bar_a_full[s]), CMP_WARPS);
             mbar_init(smem_u32(&bar_a_empty[s]), 1);
             mbar_init(smem_u32(&bar_b_full[s]), 1);
             mbar_init(smem_u32(&bar_b_empty[s]), 1);
         }
-        for (int s = 0; s < MAX_ACC_STAGES; ++s) {
+        for (int s = 0; s < ACCS; ++s) {
             mbar_init(smem_u32(&bar_acc_full[s]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[s]), 8);
+            mbar_init(smem_u32(&bar_acc_empty[s]), EPI_WARPS);
         }
         mbar_init(smem_u32(&bar_drain), 1);
         abort_flag_s = 0;
@@ -137,11 +167,17 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 for (int kb = 0; kb < num_k_blocks; ++kb) {
                     if (!bounded_wait(smem_u32(&bar_patch_empty[ps]), pphase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t pf = smem_u32(&bar_patch_full[ps]);
-                    mbar_arrive_expect_tx(pf, (uint32_t)F_PATCH_BYTES);
-                    tma_load_4d(patch_base + (uint32_t)ps * F_PATCH_STRIDE, &map_x, pf, kb * BLOCK_K,
-                                tx * F_TW - args.pl, ty * F_TH - args.pt, n);
+                    mbar_arrive_expect_tx(pf, (uint32_t)args.patch_bytes);
+                    if (CONV)
+                        tma_load_3d(patch_base + (uint32_t)(ps * args.patch_stride), &map_x, pf,
+                                    (tx * F_TW * args.sw - args.pl) * args.cin, ty * F_TH * args.sh - args.pt, n);
+                    else
+                        tma_load_4d(patch_base + (uint32_t)(ps * args.patch_stride), &map_x, pf, kb * BLOCK_K,
+                                    tx * F_TW - args.pl, ty * F_TH - args.pt, n);
                     if (++ps == args.patch_stages) { ps = 0; pphase ^= 1u; }
-                    for (int h = 0; ok && h < args.n_sub; ++h) {
+                    // the packed filter of the small-window mode is one stage: loaded once, never released
+                    const int b_loads = (CONV && issued > 0) ? 0 : args.n_sub;
+                    for (int h = 0; ok && h < b_loads; ++h) {
                         if (!bounded_wait(smem_u32(&bar_b_empty[bs]), bphase ^ 1u, abort_flag)) { ok = false; break; }
                         const uint32_t bf = smem_u32(&bar_b_full[bs]);
                         mbar_arrive_expect_tx(bf, (uint32_t)b_stage_bytes);
@@ -163,18 +199,21 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 bool all = false;
                 while (!all && global_ns() - t0 < WAIT_LIMIT_NS) {
                     all = true;
-                    for (int k = (issued > F_MAX_RING ? issued - F_MAX_RING : 0); k < issued; ++k) {
+                    for (int k = (issued > RING ? issued - RING : 0); k < issued; ++k) {
                         if (!mbar_try_wait(smem_u32(&bar_patch_full[k % args.patch_stages]),
                                            (uint32_t)((k / args.patch_stages) & 1)) &&
                             k >= issued - args.patch_stages)
                             all = false;
-                        for (int h = 0; h < args.n_sub; ++h) {
+                        for (int h = 0; h < (CONV ? 0 : args.n_sub); ++h) {
                             const int kk = k * args.n_sub + h;  // index of the B copy in its own ring
                             if (kk >= issued * args.n_sub - args.b_stages &&
                                 !mbar_try_wait(smem_u32(&bar_b_full[kk % args.b_stages]), (uint32_t)((kk / args.b_stages) & 1)))
                                 all = false;
                         }
                     }
+                }
+                if (CONV && issued > 0 && all) {
+                    while (!(all = mbar_try_wait(smem_u32(&bar_b_full[0]), 0u)) && global_ns() - t0 < WAIT_LIMIT_NS) {}
                 }
                 if (!all) atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_DRAIN);
             }
@@ -194,7 +233,9 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     if (!bounded_wait(smem_u32(&bar_a_full[as]), aphase, abort_flag)) { ok = false; break; }
                     const uint64_t a_desc = make_kmajor_sw128_desc(a_base + (uint32_t)as * A_STAGE_BYTES);
                     for (int h = 0; h < args.n_sub; ++h) {
-                        if (!bounded_wait(smem_u32(&bar_b_full[bs]), bphase, abort_flag)) { ok = false; break; }
+                        if (!CONV || !issued_any) {
+                            if (!bounded_wait(smem_u32(&bar_b_full[bs]), bphase, abort_flag)) { ok = false; break; }
+                        }
                         tc_fence_after();
                         const uint64_t b_desc = make_kmajor_sw128_desc(b_base + (uint32_t)bs * (uint32_t)b_stage_bytes);
 #pragma unroll
@@ -202,8 +243,10 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                             tc_mma_tf32(d_tmem + (uint32_t)(h * block_n), a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k),
                                         idesc, (kb | k) != 0 ? 1u : 0u);
                         issued_any = true;
-                        tc_commit(smem_u32(&bar_b_empty[bs]));
-                        if (++bs == args.b_stages) { bs = 0; bphase ^= 1u; }
+                        if (!CONV) {
+                            tc_commit(smem_u32(&bar_b_empty[bs]));
+                            if (++bs == args.b_stages) { bs = 0; bphase ^= 1u; }
+                        }
                     }
                     if (!ok) break;
                     tc_commit(smem_u32(&bar_a_empty[as]));
@@ -230,18 +273,22 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 }
             }
         }
-    } else if (warp < 10) {
-        // ---------------------------------------------------------------- epilogue (warps 2..9)
+    } else if (warp < CMP_WARP0) {
+        // ---------------------------------------------------------------- epilogue (warps 2..)
+        // Groups of four warps (one per TMEM lane quarter) take the 32-column chunks round-robin,
+        // across tile boundaries.
         const int ew = warp - 2;
         const int quad = warp & 3;   // TMEM lanes 32*quad.. = image rows 2*quad, 2*quad+1 of the tile
-        const int half = ew >> 2;
+        const int group = ew >> 2;
         const uint32_t slab = epi_base + (uint32_t)ew * EPI_SLAB_BYTES;
         const int chunks_per_tile = acc_cols / EPI_COLS;
         int n_chunks = (args.Co + EPI_COLS - 1) / EPI_COLS;
         if (n_chunks > chunks_per_tile) n_chunks = chunks_per_tile;
         int acc = 0;
         uint32_t acc_phase = 0;
-        int first_chunk = half;
+        int first_chunk = group;
+        // round-robin over tile boundaries: a tile of n_chunks chunks moves every group's first chunk
+        const int chunk_shift = EPI_GROUPS - (n_chunks & (EPI_GROUPS - 1));
         for (int tile = blockIdx.x; tile < args.num_tiles; tile += gridDim.x) {
             const int n = tile / tiles_per_image;
             const int rem = tile - n * tiles_per_image;
@@ -258,12 +305,12 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             const int oy = ty * F_TH + quad * 2;
             const bool rows_live = oy < args.Ho;
             bool released = false;
-            for (int ch = first_chunk; ch < n_chunks; ch += 2) {
+            for (int ch = first_chunk; ch < n_chunks; ch += EPI_GROUPS) {
                 uint32_t r[32];
                 const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * acc_cols + ch * EPI_COLS);
                 tc_ld_32x32(taddr, r);
                 tc_ld_wait();
-                if (ch + 2 >= n_chunks) {
+                if (ch + EPI_GROUPS >= n_chunks) {
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
@@ -291,17 +338,59 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
             }
-            if (chunks_per_tile & 1) first_chunk ^= 1;
+            first_chunk = (first_chunk + chunk_shift) & (EPI_GROUPS - 1);
             if (++acc == args.acc_stages) { acc = 0; acc_phase ^= 1u; }
         }
         if (lane == 0) tma_store_wait_all();
         __syncwarp();
     } else {
+        if (CONV) {
+            // ------------------------------------------------------------ im2col from the patch (warps 10..13)
+            // Small-window convolution (fh*fw*Cin <= 32: one k-block): thread = pixel of the tile;
+            // column k = (ky*fw + kx)*Cin + ci of a pixel's im2col row sits in the patch
+            // at row r*sh + ky, float (c*sw)*Cin + kx*Cin + ci.
+            const int p = threadIdx.x - CMP_WARP0 * 32;  // thread = pixel of the tile = row of A
+            const int r = p >> 4, c = p & 15;
+            static_assert(CMP_WARPS * 32 == BLOCK_M || !CONV, "one thread per A row");
+            const int origin = (r * args.sh) * args.row_floats + (c * args.sw) * args.cin;
+            int ps = 0, as = 0;
+            uint32_t pphase = 0, aphase = 0;
+            for (int tile = blockIdx.x; tile < args.num_tiles; tile += gridDim.x) {
+                bool got = bounded_wait(smem_u32(&bar_patch_full[ps]), pphase, abort_flag);
+                got = got && bounded_wait(smem_u32(&bar_a_empty[as]), aphase ^ 1u, abort_flag);
+                if (!__all_sync(0xffffffffu, got)) {
+                    if (lane == 0 && !*abort_flag) {
+                        *abort_flag = 1;
+                        atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_DEPTHWISE);
+                    }
+                    break;
+                }
+                const float* patch = patch_ptr + (size_t)ps * (args.patch_stride / 4) + origin;
+                const uint32_t row_addr = a_base + (uint32_t)as * A_STAGE_BYTES + (uint32_t)p * 128u;
+#pragma unroll
+                for (int h = 0; h < BLOCK_K / 4; ++h) {
+                    float v[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) v[e] = 4 * h + e < args.k_total ? patch[args.koff[4 * h + e]] : 0.0f;
+                    const uint32_t dst = row_addr + (uint32_t)((h ^ (p & 7)) << 4);
+                    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3])
+                                 : "memory");
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&bar_a_full[as]));
+                    mbar_arrive(smem_u32(&bar_patch_empty[ps]));
+                }
+                if (++ps == args.patch_stages) { ps = 0; pphase ^= 1u; }
+                if (++as == args.a_stages) { as = 0; aphase ^= 1u; }
+            }
+        } else {
         // ---------------------------------------------------------------- depthwise (warps 10..25)
         // thread = (2 channels, tile column, group of 4 tile rows); GEMM row of a pixel = row*16 + column.
         // Two channels per thread (not four) so that sixteen warps share a k-block: eight were bound by
         // their own instruction latency, not by any pipe.
-        const int t = threadIdx.x - 320;
+        const int t = threadIdx.x - CMP_WARP0 * 32;
         const int c2 = t & 15;
         const int col = (t >> 4) & (F_TW - 1);
         const int rg = t >> 8;
@@ -370,6 +459,7 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 if (++as == args.a_stages) { as = 0; aphase ^= 1u; }
             }
         }
+        }
     }
 
     // ---------------------------------------------------------------- teardown
@@ -407,9 +497,12 @@ tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
     plan->b_stages = plan->n_sub == 2 ? 3 : (bn == 256 ? 2 : 3);
     const int fixed = EPI_BYTES + plan->a_stages * A_STAGE_BYTES + plan->b_stages * bn * BLOCK_K * 4;
     int ps = (SMEM_LIMIT - 2048 - fixed) / F_PATCH_STRIDE;
-    if (ps > F_MAX_RING) ps = F_MAX_RING;
+    if (ps > 4) ps = 4;
     if (ps < 2) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "no room for the input patch ring");
+    plan->conv = false;
     plan->patch_stages = ps;
+    plan->patch_bytes = F_PATCH_BYTES;
+    plan->patch_stride = F_PATCH_STRIDE;
     plan->smem_bytes = (size_t)1024 + fixed + (size_t)ps * F_PATCH_STRIDE;
     plan->tiles_x = (dw.Wo + F_TW - 1) / F_TW;
     plan->tiles_y = (dw.Ho + F_TH - 1) / F_TH;
@@ -450,12 +543,95 @@ tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
     return TFJSB_OK;
 }
 
+// ---- small-window convolution on the same kernel ----------------------------------------------------
+// conv2d whose whole im2col row fits one k-block (fh*fw*Cin <= 32, e.g. the 3x3x3 stem): the input
+// patch of an 8 x 16 pixel tile comes in by one 3-D bulk tensor copy over x viewed as
+// [N, H, W*Cin] and the compute warps only rearrange it into the A operand.
+bool conv_patch_supported(const ConvGeom& g) {
+    const int64_t k = (int64_t)g.fh * g.fw * g.C;
+    const int64_t row_floats = (((int64_t)(F_TW - 1) * g.sw + g.fw) * g.C + 3) / 4 * 4;
+    const int64_t rows = (int64_t)(F_TH - 1) * g.sh + g.fh;
+    const int64_t tiles = g.N * ((g.Ho + F_TH - 1) / F_TH) * ((g.Wo + F_TW - 1) / F_TW);
+    return k <= BLOCK_K && g.dh == 1 && g.dw == 1 && g.mult == 1 && g.Co >= 4 && g.Co <= 128 && g.Co % 4 == 0 &&
+           row_floats <= 256 && rows <= 256 && ((int64_t)g.W * g.C) % 4 == 0 && (g.pl * g.C) % 4 == 0 &&
+           ((int64_t)F_TW * g.sw * g.C) % 4 == 0 && rows * row_floats * 4 <= 15 * 1024 && tiles >= 1 && tiles < (1LL << 31) &&
+           g.N < (1LL << 31);
+}
+
+tfjsb_status conv_patch_plan(tfjsb_ctx* ctx, const float* x, const float* bt, float* y, const ConvGeom& g, DwPwPlan* plan) {
+    if (!conv_patch_supported(g)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the patch convolution kernel");
+    if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+    plan->conv = true;
+    plan->g = g;
+    plan->Co = g.Co;
+    int bn = 32;
+    while (bn < g.Co) bn <<= 1;
+    plan->block_n = bn;
+    plan->n_sub = 1;
+    // two CTAs per SM: each takes half of tensor memory (256 columns) and half of shared memory
+    plan->acc_stages = 256 / bn < F_MAX_ACC ? 256 / bn : F_MAX_ACC;
+    plan->a_stages = 2;
+    plan->b_stages = 1;  // the packed filter stays resident
+    const int row_floats = (((F_TW - 1) * g.sw + g.fw) * g.C + 3) / 4 * 4;
+    const int rows = (F_TH - 1) * g.sh + g.fh;
+    plan->row_floats = row_floats;
+    plan->patch_rows = rows;
+    plan->patch_bytes = rows * row_floats * 4;
+    plan->patch_stride = (plan->patch_bytes + 1023) / 1024 * 1024;
+    const int fixed = EPI_BYTES + plan->a_stages * A_STAGE_BYTES + plan->b_stages * bn * BLOCK_K * 4;
+    // small patches: a deep ring keeps enough input bytes in flight to cover the DRAM latency
+    int ring = (F_CONV_SMEM - 1024 - fixed) / plan->patch_stride;
+    if (ring > F_MAX_RING) ring = F_MAX_RING;
+    if (ring < 2) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "no room for the input patch ring");
+    plan->patch_stages = ring;
+    plan->smem_bytes = (size_t)1024 + fixed + (size_t)plan->patch_stages * plan->patch_stride;
+    plan->tiles_x = (g.Wo + F_TW - 1) / F_TW;
+    plan->tiles_y = (g.Ho + F_TH - 1) / F_TH;
+    const int64_t tiles = g.N * plan->tiles_x * plan->tiles_y;
+    plan->num_tiles = (int)tiles;
+    plan->grid = (int)(tiles < 2 * ctx->sm_count ? tiles : 2 * ctx->sm_count);
+    auto encode = [&](CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides,
+                      const cuuint32_t* box, CUtensorMapSwizzle swz, const char* what) -> tfjsb_status {
+        cuuint32_t elem[4] = {1u, 1u, 1u, 1u};
+        CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<void*>(base), dims,
+                                       strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS)
+            return fail(ctx, TFJSB_ERR_CUDA, std::string("cuTensorMapEncodeTiled failed for ") + what + " (CUresult " +
+                                                 std::to_string((int)r) + ")");
+        return TFJSB_OK;
+    };
+    tfjsb_status st;
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)g.W * g.C, (cuuint64_t)g.H, (cuuint64_t)g.N};
+        cuuint64_t strides[2] = {(cuuint64_t)g.W * g.C * 4u, (cuuint64_t)g.H * g.W * g.C * 4u};
+        cuuint32_t box[3] = {(cuuint32_t)row_floats, (cuuint32_t)rows, 1u};
+        if ((st = encode(&plan->map_x, x, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE, "the convolution input")) != TFJSB_OK) return st;
+    }
+    {
+        const int64_t k_pad = BLOCK_K;
+        cuuint64_t dims[2] = {(cuuint64_t)k_pad, (cuuint64_t)g.Co};
+        cuuint64_t strides[1] = {(cuuint64_t)k_pad * 4u};
+        cuuint32_t box[2] = {(cuuint32_t)BLOCK_K, (cuuint32_t)bn};
+        if ((st = encode(&plan->map_b, bt, 2, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, "the packed filter")) != TFJSB_OK) return st;
+    }
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)g.Co, (cuuint64_t)g.Wo, (cuuint64_t)g.Ho, (cuuint64_t)g.N};
+        cuuint64_t strides[3] = {(cuuint64_t)g.Co * 4u, (cuuint64_t)g.Wo * g.Co * 4u, (cuuint64_t)g.Ho * g.Wo * g.Co * 4u};
+        cuuint32_t box[4] = {(cuuint32_t)EPI_COLS, (cuuint32_t)F_TW, 2u, 1u};
+        if ((st = encode(&plan->map_y, y, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, "the convolution output")) != TFJSB_OK) return st;
+    }
+    return TFJSB_OK;
+}
+
 cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, const float* dw_bias, int dw_act,
                               const float* pw_bias, int pw_act, unsigned int* dev_status, cudaStream_t s,
                               int64_t* launches) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(dwpw_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 2048);
+        cudaError_t e = cudaFuncSetAttribute(dwpw_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 2048);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(dwpw_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, F_CONV_SMEM);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -469,11 +645,20 @@ cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, cons
     a.n_sub = plan.n_sub;
     a.acc_stages = plan.acc_stages;
     a.patch_stages = plan.patch_stages; a.a_stages = plan.a_stages; a.b_stages = plan.b_stages;
+    a.patch_bytes = plan.patch_bytes; a.patch_stride = plan.patch_stride;
+    a.cin = plan.g.C; a.fw_cin = plan.g.fw * plan.g.C; a.sh = plan.g.sh; a.sw = plan.g.sw;
+    a.row_floats = plan.row_floats; a.k_total = plan.g.fh * plan.g.fw * plan.g.C;
+    for (int k = 0; k < 32; ++k) {
+        const int ky = a.fw_cin > 0 ? k / a.fw_cin : 0;
+        a.koff[k] = (plan.conv && k < a.k_total) ? ky * plan.row_floats + (k - ky * a.fw_cin) : 0;
+    }
     a.dw_filter = dw_filter; a.dw_bias = dw_bias; a.dw_act = dw_act;
     a.pw_bias = pw_bias; a.pw_act = pw_act;
     a.dev_status = dev_status;
-    cudaError_t e = launch_k(dwpw_fused_kernel, dim3(plan.grid), dim3(F_THREADS), plan.smem_bytes, s, plan.map_x, plan.map_b,
-                             plan.map_y, a);
+    cudaError_t e = plan.conv ? launch_k(dwpw_fused_kernel<true>, dim3(plan.grid), dim3(F_CONV_THREADS), plan.smem_bytes, s,
+                                         plan.map_x, plan.map_b, plan.map_y, a)
+                              : launch_k(dwpw_fused_kernel<false>, dim3(plan.grid), dim3(F_THREADS), plan.smem_bytes, s,
+                                         plan.map_x, plan.map_b, plan.map_y, a);
     ++*launches;
     return e;
 }

@@ -32,6 +32,7 @@ struct Step {
     bool plan_built = false;
     // a depthwise layer followed by a pointwise layer can run as one fused kernel (the pointwise step
     // is then skipped); the separate plans are kept for the keep-all debug mode
+    bool conv_patch = false;  // STEP_CONV_TF32 through the patch kernel (whole im2col row in one k-block)
     bool fuse_next = false;
     bool fusable = false;     // the pair's shapes fit the fused kernel
     bool fuse_pays = false;   // and there are enough tiles for it to be the faster choice
@@ -118,7 +119,8 @@ tfjsb_status bind_step(tfjsb_model* m, Step& st, const float* in, float* out) {
         st.plan_built = true;
     }
     if (st.kind == STEP_CONV_TF32 && (changed || !st.plan_built)) {
-        tfjsb_status rc = conv_igemm_plan(m->ctx, in, st.filter_km, out, st.g, &st.plan);
+        tfjsb_status rc = st.conv_patch ? conv_patch_plan(m->ctx, in, st.filter_km, out, st.g, &st.fused_plan)
+                                        : conv_igemm_plan(m->ctx, in, st.filter_km, out, st.g, &st.plan);
         if (rc != TFJSB_OK) return rc;
         st.plan_built = true;
     }
@@ -172,8 +174,12 @@ tfjsb_status bind_all(tfjsb_model* m, const float* input, float* output) {
 cudaError_t launch_step(tfjsb_model* m, const Step& st, cudaStream_t s) {
     tfjsb_ctx* ctx = m->ctx;
     switch (st.kind) {
-        case STEP_GEMM_TF32:
         case STEP_CONV_TF32:
+            if (st.conv_patch)
+                return launch_dwpw_fused(st.fused_plan, nullptr, nullptr, TFJSB_ACT_NONE, st.bias, st.act, ctx->dev_status, s,
+                                         &ctx->launches);
+            return launch_gemm_tf32(st.plan, st.bias, st.act, ctx->dev_status, s, &ctx->launches);
+        case STEP_GEMM_TF32:
             return launch_gemm_tf32(st.plan, st.bias, st.act, ctx->dev_status, s, &ctx->launches);
         case STEP_GEMM_FP32:
             return launch_gemm_fp32(st.in, st.K, 1, st.filter, st.N, 1, st.bias, st.act, st.out, st.N, st.M, st.N, st.K,
@@ -423,6 +429,7 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
                 return bail(TFJSB_ERR_INVALID_ARG, where + "unknown layer kind");
         }
         if (step.kind == STEP_CONV_TF32) {
+            step.conv_patch = conv_patch_supported(step.g) && !getenv("TFJSB_NO_PATCH_CONV");
             // filter [fh*fw*Cin, Cout] -> [Cout, k_pad] once, on the device
             const int64_t k_pad = conv_igemm_k_pad(step.g);
             if ((st = dev_alloc(m, (size_t)(k_pad * step.g.Co), &step.filter_km)) != TFJSB_OK) return bail(st, ctx->last_error);

@@ -120,6 +120,10 @@ IGEMM_CASES = [
     (3, 9, 9, 30, 1, 1, 52, (2, 2), "same", (1, 1)),      # strided 1x1
     (1, 6, 6, 72, 3, 3, 4, (1, 1), "valid", (1, 1)),      # K = 648: the stage ring wraps
     (5, 40, 40, 8, 3, 3, 260, (1, 1), "same", (1, 1)),    # Cout just above one 256-wide tile, many pixel tiles
+    (3, 37, 50, 3, 3, 3, 16, (2, 2), "valid", (1, 1)),    # patch kernel: ragged tiles, 'valid'
+    (2, 30, 30, 3, 3, 3, 8, (1, 1), "valid", (1, 1)),     # patch kernel: stride 1
+    (1, 19, 23, 4, 2, 2, 12, (1, 1), "same", (1, 1)),     # patch kernel: 2x2 window, Cin 4, pad after only
+    (2, 21, 21, 1, 5, 5, 32, (2, 2), "valid", (1, 1)),    # patch kernel: one input channel, 5x5 (K = 25)
 ]
 
 
