@@ -27,6 +27,7 @@ SOURCES = [
     "elementwise.cu",
     "gemm_fp32_simt.cu",
     "gemm_tf32_tcgen05.cu",
+    "gemm_tf32_pair.cu",
     "conv2d_fp32_simt.cu",
     "depthwise.cu",
     "matmul_static_scratch.cu",

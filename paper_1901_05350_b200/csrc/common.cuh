@@ -177,6 +177,8 @@ struct GemmTf32Plan {
     int num_tiles;
     int grid;
     size_t smem_bytes;
+    // CTA-pair kernel (gemm_tf32_pair.cu): 256 x block_n tiles shared by two CTAs
+    bool pair = false;
     // implicit-GEMM convolution: A is gathered from x by the kernel instead of copied
     bool gather = false;
     const float* x = nullptr;
@@ -185,6 +187,13 @@ struct GemmTf32Plan {
 bool gemm_tf32_supported(int64_t M, int64_t N, int64_t K);
 tfjsb_status gemm_tf32_plan(tfjsb_ctx* ctx, const float* a, const float* bt, float* c, int64_t M, int64_t N,
                             int64_t K, GemmTf32Plan* plan);
+// The same GEMM on CTA pairs; gemm_tf32_plan picks it where it is the faster kernel (environment
+// variable TFJSB_GEMM_PAIR: 0 = never, 1 = wherever the shape allows, unset = by shape).
+bool gemm_tf32_pair_preferred(int64_t M, int64_t N, int64_t K, int sm_count);
+tfjsb_status gemm_tf32_pair_plan(tfjsb_ctx* ctx, const float* a, const float* bt, float* c, int64_t M, int64_t N,
+                                 int64_t K, GemmTf32Plan* plan);
+cudaError_t launch_gemm_tf32_pair(const GemmTf32Plan& plan, const float* bias, int act, unsigned int* dev_status,
+                                  cudaStream_t s, int64_t* launches);
 // Implicit-GEMM convolution on the same kernel: M = N*Ho*Wo output pixels, K = fh*fw*Cin, N = Cout.
 // `bt` is the filter packed as [Cout, k_pad] (K-contiguous, zero padded to a multiple of 32).
 bool conv_igemm_supported(const ConvGeom& g);

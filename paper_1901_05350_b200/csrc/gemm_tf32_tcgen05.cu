@@ -29,6 +29,8 @@
 // Every wait is bounded: a wait that exceeds WAIT_LIMIT_NS raises an abort flag that all roles
 // poll, ORs a code into the context's device status word, and the CTA drains its copies, frees
 // its tensor memory and returns.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "ptx_sm100.cuh"
 #include "umma_tile.cuh"
@@ -526,7 +528,11 @@ tfjsb_status gemm_tf32_plan(tfjsb_ctx* ctx, const float* a, const float* bt, flo
                             int64_t K, GemmTf32Plan* plan) {
     if (!gemm_tf32_supported(M, N, K)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the TF32 GEMM");
     if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+    const char* pair_env = getenv("TFJSB_GEMM_PAIR");
+    const bool use_pair = pair_env ? (pair_env[0] == '1' && N >= 64) : gemm_tf32_pair_preferred(M, N, K, ctx->sm_count);
+    if (use_pair) return gemm_tf32_pair_plan(ctx, a, bt, c, M, N, K, plan);
     plan->M = M; plan->N = N; plan->K = K;
+    plan->pair = false;
     plan->gather = false;
     plan->x = nullptr;
     tfjsb_status st;
@@ -554,6 +560,7 @@ tfjsb_status conv_igemm_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
     plan->N = g.Co;
     plan->K = (int64_t)g.fh * g.fw * g.C;
     plan->gather = true;
+    plan->pair = false;
     plan->x = x;
     plan->g = g;
     tfjsb_status st = plan_common(ctx, bt, conv_igemm_k_pad(g), y, plan);
@@ -564,6 +571,7 @@ tfjsb_status conv_igemm_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
 
 cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int act, unsigned int* dev_status,
                              cudaStream_t s, int64_t* launches) {
+    if (plan.pair) return launch_gemm_tf32_pair(plan, bias, act, dev_status, s, launches);
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(gemm_tf32_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
