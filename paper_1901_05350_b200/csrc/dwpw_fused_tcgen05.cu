@@ -7,13 +7,20 @@
 //   warp 0       producer: bulk tensor copies (TMA) of the input patch (10 x 18 pixels x 32 channels,
 //                zero-filled outside the image = the 'same' padding) and of the matching 32-column
 //                slice of the pointwise weights Bt[Cout, Cin], each into its own ring of stages;
-//   warps 10-25  depthwise: compute the 128 x 32 block on CUDA cores from the patch (the same
-//                sliding-row scheme and FMA order as the stand-alone kernel), add bias, apply the
-//                activation and write it as the A operand in the 128-byte-swizzled K-major layout;
+//   warps 10-25  depthwise: two groups of eight warps take alternate k-blocks (two are in flight, so
+//                one group's load and FMA latency hides behind the other's); a thread computes
+//                2 channels x 2 columns x 4 rows from the patch on CUDA cores (each value it loads
+//                serves up to six outputs; the same FMA order as the stand-alone kernel), adds
+//                bias, applies the activation and writes the result as the A operand in the
+//                128-byte-swizzled K-major layout;
 //   warp 1       issues tcgen05.mma (TF32, M 128, N = block_n, K 8, four per k-block) on A and Bt,
 //                accumulating over the channel blocks in tensor memory;
 //   warps 2-9    epilogue: tcgen05.ld, pointwise bias + activation, swizzled staging slab, 4-D bulk
 //                tensor store of 2 image rows x 16 pixels x 32 channels (clipped at the image edge).
+// The kernel is bound by shared-memory bandwidth (patch written once and read by the depthwise
+// threads, A written and read back by the tensor core, Bt slices, output staging), so the pointwise
+// weights stay resident in shared memory for the whole kernel when all their k-blocks fit (up to
+// four), instead of being fetched again for every tile.
 // Every wait is bounded (see ptx_sm100.cuh); a timeout raises the abort flag all roles poll and is
 // reported through the context's device status word.
 //
@@ -36,6 +43,8 @@ namespace {
 
 constexpr int F_THREADS = 832;        // 26 warps: producer, MMA, 8 epilogue, 16 depthwise; one CTA per SM
 constexpr int F_DW_WARPS = 16;
+constexpr int F_DW_GROUPS = 2;        // groups of depthwise warps that take alternate k-blocks
+constexpr int F_DW_GROUP_WARPS = F_DW_WARPS / F_DW_GROUPS;
 constexpr int F_CONV_THREADS = 448;   // 14 warps: producer, MMA, 8 epilogue, 4 im2col; two CTAs per SM
 constexpr int F_CONV_CMP_WARPS = 4;
 constexpr int F_CONV_SMEM = 112 * 1024;  // per-CTA dynamic budget that lets two CTAs share an SM's 228 KiB
@@ -57,6 +66,7 @@ struct FusedArgs {
     int n_sub;                // MMA groups per k-block: 1, or 2 when 256 < Cout <= 512 (they share the A tile)
     int acc_stages;
     int patch_stages, a_stages, b_stages;
+    int b_resident;           // the B ring holds every k-block's slice: loaded during the first tile, never released
     int patch_bytes, patch_stride;   // bytes of one input patch and pitch of the patch ring
     // small-window convolution mode (CONV): the patch holds (8-1)*sh+fh rows of row_floats floats
     int cin, fw_cin, sh, sw, row_floats, k_total;
@@ -96,6 +106,7 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     // doubles every role, instead of one large CTA.
     constexpr int EPI_WARPS = 8;
     constexpr int CMP_WARPS = CONV ? F_CONV_CMP_WARPS : F_DW_WARPS;
+    constexpr int GROUP_WARPS = CONV ? F_CONV_CMP_WARPS : F_DW_GROUP_WARPS;  // warps that fill one A stage
     constexpr int CMP_WARP0 = 2 + EPI_WARPS;
     constexpr int EPI_GROUPS = EPI_WARPS / 4;
     static_assert((CMP_WARP0 + CMP_WARPS) * 32 == (CONV ? F_CONV_THREADS : F_THREADS), "role split must cover the block");
@@ -117,10 +128,10 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     if (threadIdx.x == 0) {
         for (int s = 0; s < RING; ++s) {
             mbar_init(smem_u32(&bar_patch_full[s]), 1);
-            mbar_init(smem_u32(&bar_patch_empty[s]), CMP_WARPS);
+            mbar_init(smem_u32(&bar_patch_empty[s]), GROUP_WARPS);
         }
         for (int s = 0; s < 4; ++s) {
-            mbar_init(smem_u32(&bar_a_full[s]), CMP_WARPS);
+            mbar_init(smem_u32(&bar_a_full[s]), GROUP_WARPS);
             mbar_init(smem_u32(&bar_a_empty[s]), 1);
             mbar_init(smem_u32(&bar_b_full[s]), 1);
             mbar_init(smem_u32(&bar_b_empty[s]), 1);
@@ -175,8 +186,9 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                         tma_load_4d(patch_base + (uint32_t)(ps * args.patch_stride), &map_x, pf, kb * BLOCK_K,
                                     tx * F_TW - args.pl, ty * F_TH - args.pt, n);
                     if (++ps == args.patch_stages) { ps = 0; pphase ^= 1u; }
-                    // the packed filter of the small-window mode is one stage: loaded once, never released
-                    const int b_loads = (CONV && issued > 0) ? 0 : args.n_sub;
+                    // resident weights (and the packed filter of the small-window mode) are loaded during
+                    // the first tile only and never released
+                    const int b_loads = (args.b_resident && issued >= num_k_blocks) ? 0 : args.n_sub;
                     for (int h = 0; ok && h < b_loads; ++h) {
                         if (!bounded_wait(smem_u32(&bar_b_empty[bs]), bphase ^ 1u, abort_flag)) { ok = false; break; }
                         const uint32_t bf = smem_u32(&bar_b_full[bs]);
@@ -204,7 +216,7 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                                            (uint32_t)((k / args.patch_stages) & 1)) &&
                             k >= issued - args.patch_stages)
                             all = false;
-                        for (int h = 0; h < (CONV ? 0 : args.n_sub); ++h) {
+                        for (int h = 0; h < (args.b_resident ? 0 : args.n_sub); ++h) {
                             const int kk = k * args.n_sub + h;  // index of the B copy in its own ring
                             if (kk >= issued * args.n_sub - args.b_stages &&
                                 !mbar_try_wait(smem_u32(&bar_b_full[kk % args.b_stages]), (uint32_t)((kk / args.b_stages) & 1)))
@@ -212,8 +224,10 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                         }
                     }
                 }
-                if (CONV && issued > 0 && all) {
-                    while (!(all = mbar_try_wait(smem_u32(&bar_b_full[0]), 0u)) && global_ns() - t0 < WAIT_LIMIT_NS) {}
+                if (args.b_resident && all) {
+                    const int loaded = issued < num_k_blocks ? issued : num_k_blocks;
+                    for (int k = 0; all && k < loaded; ++k)
+                        while (!(all = mbar_try_wait(smem_u32(&bar_b_full[k]), 0u)) && global_ns() - t0 < WAIT_LIMIT_NS) {}
                 }
                 if (!all) atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_DRAIN);
             }
@@ -225,6 +239,7 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             int as = 0, bs = 0, acc = 0;
             uint32_t aphase = 0, bphase = 0, acc_phase = 0;
             bool ok = true, issued_any = false;
+            bool first_tile = true;
             for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
                 if (!bounded_wait(smem_u32(&bar_acc_empty[acc]), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -233,7 +248,7 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     if (!bounded_wait(smem_u32(&bar_a_full[as]), aphase, abort_flag)) { ok = false; break; }
                     const uint64_t a_desc = make_kmajor_sw128_desc(a_base + (uint32_t)as * A_STAGE_BYTES);
                     for (int h = 0; h < args.n_sub; ++h) {
-                        if (!CONV || !issued_any) {
+                        if (!args.b_resident || first_tile) {
                             if (!bounded_wait(smem_u32(&bar_b_full[bs]), bphase, abort_flag)) { ok = false; break; }
                         }
                         tc_fence_after();
@@ -243,10 +258,9 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                             tc_mma_tf32(d_tmem + (uint32_t)(h * block_n), a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k),
                                         idesc, (kb | k) != 0 ? 1u : 0u);
                         issued_any = true;
-                        if (!CONV) {
-                            tc_commit(smem_u32(&bar_b_empty[bs]));
-                            if (++bs == args.b_stages) { bs = 0; bphase ^= 1u; }
-                        }
+                        if (!args.b_resident) tc_commit(smem_u32(&bar_b_empty[bs]));
+                        // resident: stage kb again for the next tile, its first phase (parity 0) long complete
+                        if (++bs == args.b_stages) { bs = 0; if (!args.b_resident) bphase ^= 1u; }
                     }
                     if (!ok) break;
                     tc_commit(smem_u32(&bar_a_empty[as]));
@@ -254,6 +268,7 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 }
                 if (!ok) break;
                 tc_commit(smem_u32(&bar_acc_full[acc]));
+                first_tile = false;
                 if (++acc == args.acc_stages) { acc = 0; acc_phase ^= 1u; }
             }
             if (!ok) {
@@ -387,74 +402,87 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             }
         } else {
         // ---------------------------------------------------------------- depthwise (warps 10..25)
-        // thread = (2 channels, tile column, group of 4 tile rows); GEMM row of a pixel = row*16 + column.
-        // Two channels per thread (not four) so that sixteen warps share a k-block: eight were bound by
-        // their own instruction latency, not by any pipe.
+        // Two groups of eight warps take the k-blocks in turn.  Within a group, thread = (2 channels,
+        // 2 tile columns, 4 tile rows): it walks the six patch rows its outputs need once, loading four
+        // pixels per row; GEMM row of a pixel = row*16 + column.
         const int t = threadIdx.x - CMP_WARP0 * 32;
-        const int c2 = t & 15;
-        const int col = (t >> 4) & (F_TW - 1);
-        const int rg = t >> 8;
+        const int group = t / (F_DW_GROUP_WARPS * 32);
+        const int tg = t - group * (F_DW_GROUP_WARPS * 32);
+        const int c2 = tg & 15;
+        const int colg = (tg >> 4) & (F_TW / 2 - 1);
+        const int rg = tg >> 7;
         constexpr int R = F_TH / 2;
+        static_assert(F_DW_GROUP_WARPS * 32 == 16 * (F_TW / 2) * (F_TH / R), "one thread per 2 channels x 2 columns x R rows");
         int ps = 0, as = 0;
         uint32_t pphase = 0, aphase = 0;
+        int turn = 0;  // which group's turn the next k-block is
         float2 w[9];
         float2 b = make_float2(0.f, 0.f);
         int loaded_kb = -1;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
             for (int kb = 0; kb < num_k_blocks; ++kb) {
-                if (kb != loaded_kb) {
-                    const int c = kb * BLOCK_K + c2 * 2;
+                if (turn == group) {
+                    if (kb != loaded_kb) {
+                        const int c = kb * BLOCK_K + c2 * 2;
 #pragma unroll
-                    for (int k = 0; k < 9; ++k) w[k] = __ldg(reinterpret_cast<const float2*>(args.dw_filter + (int64_t)k * args.C + c));
-                    if (args.dw_bias) b = __ldg(reinterpret_cast<const float2*>(args.dw_bias + c));
-                    loaded_kb = kb;
-                }
-                bool got = bounded_wait(smem_u32(&bar_patch_full[ps]), pphase, abort_flag);
-                got = got && bounded_wait(smem_u32(&bar_a_empty[as]), aphase ^ 1u, abort_flag);
-                if (!__all_sync(0xffffffffu, got)) {
-                    if (lane == 0 && !*abort_flag) {
-                        *abort_flag = 1;
-                        atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_DEPTHWISE);
+                        for (int k = 0; k < 9; ++k) w[k] = __ldg(reinterpret_cast<const float2*>(args.dw_filter + (int64_t)k * args.C + c));
+                        if (args.dw_bias) b = __ldg(reinterpret_cast<const float2*>(args.dw_bias + c));
+                        loaded_kb = kb;
                     }
-                    ok = false;
-                    break;
-                }
-                float2 acc[R];
+                    bool got = bounded_wait(smem_u32(&bar_patch_full[ps]), pphase, abort_flag);
+                    got = got && bounded_wait(smem_u32(&bar_a_empty[as]), aphase ^ 1u, abort_flag);
+                    if (!__all_sync(0xffffffffu, got)) {
+                        if (lane == 0 && !*abort_flag) {
+                            *abort_flag = 1;
+                            atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_DEPTHWISE);
+                        }
+                        ok = false;
+                        break;
+                    }
+                    float2 acc[R][2];
 #pragma unroll
-                for (int r = 0; r < R; ++r) acc[r] = make_float2(0.f, 0.f);
-                const float* patch = patch_ptr + (size_t)ps * (F_PATCH_STRIDE / 4) + ((rg * R) * F_PW + col) * BLOCK_K + c2 * 2;
+                    for (int r = 0; r < R; ++r) acc[r][0] = acc[r][1] = make_float2(0.f, 0.f);
+                    const float* patch = patch_ptr + (size_t)ps * (F_PATCH_STRIDE / 4) + ((rg * R) * F_PW + colg * 2) * BLOCK_K + c2 * 2;
 #pragma unroll
-                for (int j = 0; j < R + 2; ++j) {
-                    const float* row = patch + j * F_PW * BLOCK_K;
-                    const float2 v0 = *reinterpret_cast<const float2*>(row);
-                    const float2 v1 = *reinterpret_cast<const float2*>(row + BLOCK_K);
-                    const float2 v2 = *reinterpret_cast<const float2*>(row + 2 * BLOCK_K);
+                    for (int j = 0; j < R + 2; ++j) {
+                        const float* row = patch + j * F_PW * BLOCK_K;
+                        float2 v[4];
 #pragma unroll
-                    for (int ky = 0; ky < 3; ++ky) {
-                        const int d = j - ky;
-                        if (d >= 0 && d < R) {
-                            acc[d].x = fmaf(v0.x, w[ky * 3 + 0].x, acc[d].x); acc[d].y = fmaf(v0.y, w[ky * 3 + 0].y, acc[d].y);
-                            acc[d].x = fmaf(v1.x, w[ky * 3 + 1].x, acc[d].x); acc[d].y = fmaf(v1.y, w[ky * 3 + 1].y, acc[d].y);
-                            acc[d].x = fmaf(v2.x, w[ky * 3 + 2].x, acc[d].x); acc[d].y = fmaf(v2.y, w[ky * 3 + 2].y, acc[d].y);
+                        for (int q = 0; q < 4; ++q) v[q] = *reinterpret_cast<const float2*>(row + q * BLOCK_K);
+#pragma unroll
+                        for (int ky = 0; ky < 3; ++ky) {
+                            const int d = j - ky;
+                            if (d >= 0 && d < R) {
+#pragma unroll
+                                for (int cc = 0; cc < 2; ++cc) {
+                                    fma2(acc[d][cc], v[cc + 0], w[ky * 3 + 0]);
+                                    fma2(acc[d][cc], v[cc + 1], w[ky * 3 + 1]);
+                                    fma2(acc[d][cc], v[cc + 2], w[ky * 3 + 2]);
+                                }
+                            }
                         }
                     }
-                }
-                const uint32_t a_stage = a_base + (uint32_t)as * A_STAGE_BYTES;
+                    const uint32_t a_stage = a_base + (uint32_t)as * A_STAGE_BYTES;
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    const float vx = apply_act(acc[r].x + b.x, args.dw_act);
-                    const float vy = apply_act(acc[r].y + b.y, args.dw_act);
-                    const int p = (rg * R + r) * F_TW + col;
-                    const uint32_t dst = a_stage + (uint32_t)p * 128u + (uint32_t)(((c2 >> 1) ^ (p & 7)) << 4) + (uint32_t)((c2 & 1) << 3);
-                    asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(dst), "f"(vx), "f"(vy) : "memory");
+                    for (int r = 0; r < R; ++r) {
+#pragma unroll
+                        for (int cc = 0; cc < 2; ++cc) {
+                            const float vx = apply_act(acc[r][cc].x + b.x, args.dw_act);
+                            const float vy = apply_act(acc[r][cc].y + b.y, args.dw_act);
+                            const int p = (rg * R + r) * F_TW + colg * 2 + cc;
+                            const uint32_t dst = a_stage + (uint32_t)p * 128u + (uint32_t)(((c2 >> 1) ^ (p & 7)) << 4) + (uint32_t)((c2 & 1) << 3);
+                            asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(dst), "f"(vx), "f"(vy) : "memory");
+                        }
+                    }
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(smem_u32(&bar_a_full[as]));
+                        mbar_arrive(smem_u32(&bar_patch_empty[ps]));
+                    }
                 }
-                fence_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(smem_u32(&bar_a_full[as]));
-                    mbar_arrive(smem_u32(&bar_patch_empty[ps]));
-                }
+                if (++turn == F_DW_GROUPS) turn = 0;
                 if (++ps == args.patch_stages) { ps = 0; pphase ^= 1u; }
                 if (++as == args.a_stages) { as = 0; aphase ^= 1u; }
             }
@@ -495,6 +523,11 @@ tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
     plan->acc_stages = plan->n_sub == 2 ? 1 : (bn == 256 ? 2 : MAX_ACC_STAGES);
     plan->a_stages = plan->n_sub == 2 ? 2 : 3;
     plan->b_stages = plan->n_sub == 2 ? 3 : (bn == 256 ? 2 : 3);
+    // all of Bt resident when its k-blocks fit the B ring's four barriers and leave room for three patches
+    const int k_blocks = dw.C / BLOCK_K;
+    plan->b_resident = plan->n_sub == 1 && k_blocks <= 4 &&
+                       EPI_BYTES + plan->a_stages * A_STAGE_BYTES + k_blocks * bn * BLOCK_K * 4 + 3 * F_PATCH_STRIDE <= SMEM_LIMIT - 2048;
+    if (plan->b_resident) plan->b_stages = k_blocks;
     const int fixed = EPI_BYTES + plan->a_stages * A_STAGE_BYTES + plan->b_stages * bn * BLOCK_K * 4;
     int ps = (SMEM_LIMIT - 2048 - fixed) / F_PATCH_STRIDE;
     if (ps > 4) ps = 4;
@@ -572,6 +605,7 @@ tfjsb_status conv_patch_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
     plan->acc_stages = 256 / bn < F_MAX_ACC ? 256 / bn : F_MAX_ACC;
     plan->a_stages = 2;
     plan->b_stages = 1;  // the packed filter stays resident
+    plan->b_resident = true;
     const int row_floats = (((F_TW - 1) * g.sw + g.fw) * g.C + 3) / 4 * 4;
     const int rows = (F_TH - 1) * g.sh + g.fh;
     plan->row_floats = row_floats;
@@ -645,6 +679,7 @@ cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, cons
     a.n_sub = plan.n_sub;
     a.acc_stages = plan.acc_stages;
     a.patch_stages = plan.patch_stages; a.a_stages = plan.a_stages; a.b_stages = plan.b_stages;
+    a.b_resident = plan.b_resident ? 1 : 0;
     a.patch_bytes = plan.patch_bytes; a.patch_stride = plan.patch_stride;
     a.cin = plan.g.C; a.fw_cin = plan.g.fw * plan.g.C; a.sh = plan.g.sh; a.sw = plan.g.sw;
     a.row_floats = plan.row_floats; a.k_total = plan.g.fh * plan.g.fw * plan.g.C;
