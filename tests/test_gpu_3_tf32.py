@@ -67,6 +67,54 @@ def test_matmul_tf32_parity(ctx, oracle, mkn):
         assert rel_fro(got[rows], want) <= TF32_TOL
 
 
+SPLIT_K_SHAPES = [
+    # M, K, N: few output tiles and a long K loop, so the planner cuts K into slices (work item = tile x slice)
+    (128, 1024, 1000),   # dense layer at batch 128
+    (1, 1024, 1000),     # dense layer at batch 1
+    (49, 1024, 1024),    # pw13 at batch 1
+    (196, 512, 512),     # pw7 at batch 1: two row tiles, the second mostly empty
+    (300, 4100, 72),     # K not a multiple of the slice length: the last slice is short and ragged
+    (512, 512, 512),     # config 1
+]
+
+
+@pytest.mark.parametrize("mkn", SPLIT_K_SHAPES)
+def test_matmul_split_k_agrees_with_unsplit_and_oracle(ctx, oracle, monkeypatch, mkn):
+    M, K, N = mkn
+    a = si.uniform(311, 0, (M, K), -1, 1)
+    b = si.uniform(311, 1, (K, N), -1, 1)
+    monkeypatch.delenv("TFJSB_NO_SPLIT_K", raising=False)
+    launches = ctx.launch_count
+    split = host(ctx.matmul(dev(a), dev(b)))
+    split_launches = ctx.launch_count - launches
+    again = host(ctx.matmul(dev(a), dev(b)))
+    monkeypatch.setenv("TFJSB_NO_SPLIT_K", "1")
+    launches = ctx.launch_count
+    whole = host(ctx.matmul(dev(a), dev(b)))
+    whole_launches = ctx.launch_count - launches
+    ctx.check_device_status()
+    assert split_launches == whole_launches + 1          # the reduction kernel: K really was cut
+    assert same_bits(split, again)                        # slices are added in a fixed order
+    want = oracle.matmul(a, b)
+    assert rel_fro(split, want) <= TF32_TOL and rel_fro(whole, want) <= TF32_TOL
+    assert rel_fro(split, oracle.matmul(a, b, operand="tf32_rz")) <= MATCHED_TOL
+    ai = si.small_integers(312, 0, (M, K), -8, 8)
+    bi = si.small_integers(312, 1, (K, N), -8, 8)
+    monkeypatch.delenv("TFJSB_NO_SPLIT_K", raising=False)
+    assert same_bits(host(ctx.matmul(dev(ai), dev(bi))), (ai.astype(np.int64) @ bi.astype(np.int64)).astype(np.float32))
+
+
+def test_dense_split_k_fused_bias_and_activation(ctx, oracle):
+    # the reduction kernel applies bias and activation: [128,1,1,1024] x [1,1,1024,1000] + bias, relu6
+    x = si.uniform(313, 0, (128, 1, 1, 1024), 0, 1)
+    f = si.normal(313, 1, (1, 1, 1024, 1000), 0, float(np.sqrt(2.0 / 1024)))
+    b = si.normal(313, 2, (1000,), 0, 0.5)
+    for act in ("none", "relu6"):
+        got = host(ctx.conv2d(dev(x), dev(f), bias=dev(b), act=act))
+        assert rel_fro(got, oracle.conv2d(x, f, bias=b, act=act)) <= TF32_TOL
+    ctx.check_device_status()
+
+
 @pytest.mark.parametrize("ta,tb", [(False, True), (True, False), (True, True)])
 def test_matmul_tf32_transposes(ctx, oracle, ta, tb):
     M, K, N = 260, 96, 132
@@ -181,7 +229,7 @@ FUSED_BLOCK_CASES = [
 
 
 @pytest.mark.parametrize("case", FUSED_BLOCK_CASES)
-def test_fused_depthwise_pointwise_block(ctx, oracle, case):
+def test_fused_depthwise_pointwise_block(ctx, oracle, monkeypatch, case):
     from seeded_inputs.workloads import Layer
 
     N, H, W, C, Cout, pad = case
@@ -197,10 +245,12 @@ def test_fused_depthwise_pointwise_block(ctx, oracle, case):
     want = oracle.run_model(layers, x)
     assert got.shape == want.shape
     assert rel_fro(got, want) <= TF32_TOL
+    monkeypatch.setenv("TFJSB_NO_SPLIT_K", "1")  # (a pointwise GEMM cut along K adds in another order)
     model.set_keep_all(True)                    # debug mode: the two stand-alone kernels
-    assert model.launches_per_run == 2
     unfused = host(model.run(dev(x)))
+    assert model.launches_per_run == 2
     assert same_bits(got, unfused)              # same arithmetic in the same order
+    monkeypatch.delenv("TFJSB_NO_SPLIT_K")
     model.close()
     # small integers: exact in TF32 and fp32, so bit-identical to the oracle
     xi = si.small_integers(312, 0, x.shape, 0, 3)
