@@ -299,21 +299,36 @@ def run_ours(args):
     elapsed_ms = replicas.max_over_ranks(start.elapsed_time(stop), device="cuda")
     value = world * BATCH * args.steps / (elapsed_ms * 1e-3)
 
-    # ---- end to end: pinned host input in, probabilities back to the host, every step
-    hin = torch.from_numpy(x_host).pin_memory()
-    hout = torch.empty(model.output_shape).pin_memory()
+    # ---- end to end: pinned host input in, probabilities back to the host, every step.  The library's
+    # asynchronous host call keeps two steps in flight (two sets of device staging buffers), so the
+    # 77 MB input copy of step i+1 overlaps the computation of step i; every step still copies its own
+    # input in and its own result out, and the last result is waited for inside the timed region.
+    hins = [torch.from_numpy(x_host).pin_memory() for _ in range(2)]
+    houts = [torch.empty(model.output_shape).pin_memory() for _ in range(2)]
     e2e_steps = max(3, min(args.steps, 50))
-    for _ in range(3):
-        model.run_host(hin, hout)
+    for i in range(4):
+        model.run_host_async(hins[i % 2], houts[i % 2])
+    model.host_wait()
     barrier()
     start.record(stream)
-    for _ in range(e2e_steps):
-        model.run_host(hin, hout)
+    for i in range(e2e_steps):
+        model.run_host_async(hins[i % 2], houts[i % 2])
+    model.host_wait()
     stop.record(stream)
     barrier()
     e2e_ms = replicas.max_over_ranks(start.elapsed_time(stop), device="cuda")
+    # the same with one step at a time (the blocking call): the latency-oriented figure
+    start.record(stream)
+    for i in range(e2e_steps):
+        model.run_host(hins[i % 2], houts[i % 2])
+    stop.record(stream)
+    barrier()
+    e2e_blocking_ms = replicas.max_over_ranks(start.elapsed_time(stop), device="cuda")
+    assert torch.equal(houts[0], houts[1])
     e2e = {"value": world * BATCH * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
-           "h2d_bytes_per_step": int(hin.numel() * 4), "d2h_bytes_per_step": int(hout.numel() * 4), "steps": e2e_steps}
+           "h2d_bytes_per_step": int(hins[0].numel() * 4), "d2h_bytes_per_step": int(houts[0].numel() * 4), "steps": e2e_steps,
+           "api": "tfjsb_run_model_host_async + tfjsb_model_host_wait, two steps in flight",
+           "blocking_api_value": world * BATCH * e2e_steps / (e2e_blocking_ms * 1e-3)}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),

@@ -211,6 +211,18 @@ tfjsb_status tfjsb_run_model(tfjsb_model* model, const tfjsb_tensor* input, tfjs
  * run). */
 tfjsb_status tfjsb_run_model_host(tfjsb_model* model, const float* host_input, float* host_output, void* stream);
 
+/* The asynchronous form of the same run (the data() promise of Sec. 3.6 beside the blocking
+ * dataSync()): enqueues the copy of `host_input` to the device, the run and the copy of the result to
+ * `host_output`, and returns without waiting.  The model keeps two sets of device staging buffers and
+ * alternates between them, so the input copy of one run overlaps the computation of the run before
+ * it; a third call first waits for the first to finish.  `host_input` must be ready when the call is
+ * made (the copy does not wait for work queued on `stream`), and neither buffer may be touched until
+ * tfjsb_model_host_wait has returned (or a later call has had to wait for that run).  Runs complete in
+ * the order of the calls; use one `stream` for all of them. */
+tfjsb_status tfjsb_run_model_host_async(tfjsb_model* model, const float* host_input, float* host_output, void* stream);
+/* Blocks until every run enqueued by tfjsb_run_model_host_async has delivered its output. */
+tfjsb_status tfjsb_model_host_wait(tfjsb_model* model);
+
 /* A stride-1 3x3 depthwise layer followed by a pointwise layer (<= 512 output channels, depthwise
  * channels a multiple of 32) can run as ONE kernel that keeps the depthwise output in shared
  * memory as the tensor-core operand, so the intermediate tensor is neither written nor read back.

@@ -31,6 +31,7 @@ EXPORTS = [
     "tfjsb_launch_count", "tfjsb_window_out_shape", "tfjsb_matmul", "tfjsb_matmul_static_scratch", "tfjsb_conv2d", "tfjsb_depthwise_conv2d",
     "tfjsb_avg_pool", "tfjsb_softmax", "tfjsb_bias_act", "tfjsb_model_create", "tfjsb_model_destroy",
     "tfjsb_model_output_shape", "tfjsb_model_launches_per_run", "tfjsb_run_model", "tfjsb_run_model_host",
+    "tfjsb_run_model_host_async", "tfjsb_model_host_wait",
     "tfjsb_model_set_keep_all", "tfjsb_model_set_graph", "tfjsb_model_set_fusion", "tfjsb_model_layer_output", "tfjsb_model_profile",
 ]
 
@@ -91,6 +92,8 @@ def _load_library() -> ctypes.CDLL:
     lib.tfjsb_model_launches_per_run.restype = ctypes.c_int32
     lib.tfjsb_run_model.argtypes = [vp, tp, tp, vp]
     lib.tfjsb_run_model_host.argtypes = [vp, vp, vp, vp]
+    lib.tfjsb_run_model_host_async.argtypes = [vp, vp, vp, vp]
+    lib.tfjsb_model_host_wait.argtypes = [vp]
     lib.tfjsb_model_set_keep_all.argtypes = [vp, i32]
     lib.tfjsb_model_set_graph.argtypes = [vp, i32]
     lib.tfjsb_model_set_fusion.argtypes = [vp, i32]
@@ -304,6 +307,20 @@ class Model:
             raise ValueError("host tensors must have the model's input / output shapes")
         self.ctx._check(lib.tfjsb_run_model_host(self._h, host_in.data_ptr(), host_out.data_ptr(), _stream()))
         return host_out
+
+    def run_host_async(self, host_in, host_out):
+        """Enqueue a forward pass from/to host memory and return at once; up to two may be outstanding
+        (the copy of one overlaps the computation of the one before).  Keep both tensors alive and
+        untouched until host_wait() returns."""
+        if host_in.is_cuda or host_out.is_cuda or not host_in.is_contiguous() or not host_out.is_contiguous():
+            raise TypeError("run_host_async takes contiguous CPU tensors")
+        if tuple(host_in.shape) != self.input_shape or tuple(host_out.shape) != self.output_shape:
+            raise ValueError("host tensors must have the model's input / output shapes")
+        self.ctx._check(lib.tfjsb_run_model_host_async(self._h, host_in.data_ptr(), host_out.data_ptr(), _stream()))
+
+    def host_wait(self):
+        """Block until every run_host_async() call has delivered its output."""
+        self.ctx._check(lib.tfjsb_model_host_wait(self._h))
 
     def set_keep_all(self, keep_all: bool):
         self.ctx._check(lib.tfjsb_model_set_keep_all(self._h, int(keep_all)))

@@ -58,19 +58,25 @@ struct tfjsb_model {
     bool keep_all = false;
     float* gemm_ws = nullptr;    // split-K workspace shared by the GEMM layers (they run one after the other)
     size_t gemm_ws_bytes = 0;
-    float* staged_in = nullptr;  // device copies used by tfjsb_run_model_host
-    float* staged_out = nullptr;
+    // Host-buffer runs (tfjsb_run_model_host / _async) alternate between two sets of device staging
+    // buffers, so that the input copy of one run can overlap the computation of the run before it.
+    float* staged_in[2] = {nullptr, nullptr};
+    float* staged_out[2] = {nullptr, nullptr};
+    cudaEvent_t host_run_done[2] = {nullptr, nullptr};  // recorded after a run's output copy
+    bool host_run_pending[2] = {false, false};
+    int next_staging = 0;
     bool use_tf32 = true;
     // caller buffers the first/last tensor maps were last encoded for
     const void* bound_in = nullptr;
     void* bound_out = nullptr;
-    // tfjsb_run_model_host pipelines the batch in slices: slice c+1 is copied to the device on a
-    // stream of its own while slice c is computed.  Each slice has a view of this model with a
-    // smaller batch: the same weights and arena, its own shapes, plans and fixed staging addresses.
+    // Host-buffer runs pipeline the batch in slices: slice c+1 is copied to the device on a stream
+    // of its own while slice c is computed.  Each slice has a view of this model with a smaller
+    // batch: the same weights and arena, its own shapes, plans and fixed staging addresses.  There is
+    // one set of views and events per staging buffer: entry b * n_slices + c.
     std::vector<tfjsb_model*> slices;
     std::vector<cudaEvent_t> slice_copied;
+    int n_slices = 0;
     cudaStream_t copy_stream = nullptr;
-    cudaEvent_t compute_done = nullptr;
     bool is_view = false;
     // optional CUDA-graph replay of one run (tfjsb_model_set_graph): captured for the current binding
     // programmatic dependent launch between the layers' kernels (each waits before reading its input)
@@ -508,7 +514,8 @@ tfjsb_status tfjsb_model_destroy(tfjsb_model* m) {
         delete v;
     }
     for (cudaEvent_t e : m->slice_copied) cudaEventDestroy(e);
-    if (m->compute_done) cudaEventDestroy(m->compute_done);
+    for (cudaEvent_t e : m->host_run_done)
+        if (e) cudaEventDestroy(e);
     if (m->copy_stream) cudaStreamDestroy(m->copy_stream);
     for (float* p : m->owned) cudaFree(p);
     --m->ctx->live_models;
@@ -571,70 +578,114 @@ tfjsb_status tfjsb_model_set_graph(tfjsb_model* m, int use_graph) {
     return TFJSB_OK;
 }
 
-tfjsb_status tfjsb_run_model_host(tfjsb_model* m, const float* host_input, float* host_output, void* stream) {
-    if (!m) return TFJSB_ERR_INVALID_ARG;
+}  // extern "C"
+
+namespace {
+
+// Enqueues one run from / to host memory on staging set `b` and records host_run_done[b]; no waiting
+// except for the run that last used the same staging set.
+tfjsb_status enqueue_host_run(tfjsb_model* m, const float* host_input, float* host_output, cudaStream_t s, int b) {
     tfjsb_ctx* ctx = m->ctx;
-    if (!host_input || !host_output) return fail(ctx, TFJSB_ERR_INVALID_ARG, "host_input / host_output is null");
     tfjsb_status st;
-    const Step& last = m->steps.back();
-    if (!m->staged_in) {
-        if ((st = dev_alloc(m, (size_t)m->in_elems, &m->staged_in)) != TFJSB_OK) return st;
-        if ((st = dev_alloc(m, (size_t)last.out_elems, &m->staged_out)) != TFJSB_OK) return st;
-    }
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e;
-    const int64_t n = m->in_dims[0];
-    // four slices: more of them lose more to per-launch fixed costs than the extra overlap returns
-    int n_slices = (n % 4 == 0 && n >= 32) ? 4 : 1;
-    if (const char* env = getenv("TFJSB_HOST_SLICES")) {  // tuning knob: 1 disables the pipelining
-        const int v = atoi(env);
-        if (v >= 1 && n % v == 0 && m->slices.empty()) n_slices = v;
-        else if (!m->slices.empty()) n_slices = (int)m->slices.size();
+    const Step& last = m->steps.back();
+    if (m->host_run_pending[b]) {  // its output has been delivered and its staging buffers are free after this
+        if ((e = cudaEventSynchronize(m->host_run_done[b])) != cudaSuccess) return cuda_fail(ctx, e, "cudaEventSynchronize");
+        m->host_run_pending[b] = false;
     }
-    if (n_slices > 1 && !m->keep_all) {
+    if (!m->staged_in[b]) {
+        if ((st = dev_alloc(m, (size_t)m->in_elems, &m->staged_in[b])) != TFJSB_OK) return st;
+        if ((st = dev_alloc(m, (size_t)last.out_elems, &m->staged_out[b])) != TFJSB_OK) return st;
+        if ((e = cudaEventCreateWithFlags(&m->host_run_done[b], cudaEventDisableTiming)) != cudaSuccess)
+            return cuda_fail(ctx, e, "cudaEventCreate");
+    }
+    if (m->keep_all) {
+        // debug mode: the whole batch through the model itself, so that every layer's output stays readable
+        e = cudaMemcpyAsync(m->staged_in[b], host_input, (size_t)m->in_elems * 4, cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "host-to-device copy of the input");
+        tfjsb_tensor in{m->staged_in[b], 4, {m->in_dims[0], m->in_dims[1], m->in_dims[2], m->in_dims[3]}};
+        tfjsb_tensor out{m->staged_out[b], last.out_rank, {last.out_dims[0], last.out_dims[1], last.out_dims[2], last.out_dims[3]}};
+        if ((st = tfjsb_run_model(m, &in, &out, s)) != TFJSB_OK) return st;
+    } else {
         if (m->slices.empty()) {
+            const int64_t n = m->in_dims[0];
+            // four slices: more of them lose more to per-launch fixed costs than the extra overlap returns
+            int n_slices = (n % 4 == 0 && n >= 32) ? 4 : 1;
+            if (const char* env = getenv("TFJSB_HOST_SLICES")) {  // tuning knob: 1 disables the slicing
+                const int v = atoi(env);
+                if (v >= 1 && n % v == 0) n_slices = v;
+            }
             if ((e = cudaStreamCreateWithFlags(&m->copy_stream, cudaStreamNonBlocking)) != cudaSuccess)
                 return cuda_fail(ctx, e, "cudaStreamCreate");
-            if ((e = cudaEventCreateWithFlags(&m->compute_done, cudaEventDisableTiming)) != cudaSuccess)
-                return cuda_fail(ctx, e, "cudaEventCreate");
-            for (int c = 0; c < n_slices; ++c) {
+            for (int i = 0; i < 2 * n_slices; ++i) {
                 cudaEvent_t ev;
                 if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess)
                     return cuda_fail(ctx, e, "cudaEventCreate");
                 m->slice_copied.push_back(ev);
                 m->slices.push_back(make_batch_view(m, n / n_slices));
             }
+            m->n_slices = n_slices;
         }
+        const int n_slices = m->n_slices;
         const int64_t in_slice = m->in_elems / n_slices, out_slice = last.out_elems / n_slices;
-        // the copy stream starts after whatever the caller queued on `stream` before this call
-        if ((e = cudaEventRecord(m->compute_done, s)) != cudaSuccess) return cuda_fail(ctx, e, "cudaEventRecord");
-        if ((e = cudaStreamWaitEvent(m->copy_stream, m->compute_done, 0)) != cudaSuccess) return cuda_fail(ctx, e, "cudaStreamWaitEvent");
+        // The copies wait for nothing on `stream`: the staging set is free (checked above), so they may
+        // run while an earlier run is still computing.
         for (int c = 0; c < n_slices; ++c) {
-            e = cudaMemcpyAsync(m->staged_in + c * in_slice, host_input + c * in_slice, (size_t)in_slice * 4,
+            e = cudaMemcpyAsync(m->staged_in[b] + c * in_slice, host_input + c * in_slice, (size_t)in_slice * 4,
                                 cudaMemcpyHostToDevice, m->copy_stream);
             if (e != cudaSuccess) return cuda_fail(ctx, e, "host-to-device copy of the input");
-            if ((e = cudaEventRecord(m->slice_copied[c], m->copy_stream)) != cudaSuccess) return cuda_fail(ctx, e, "cudaEventRecord");
+            if ((e = cudaEventRecord(m->slice_copied[b * n_slices + c], m->copy_stream)) != cudaSuccess)
+                return cuda_fail(ctx, e, "cudaEventRecord");
         }
         for (int c = 0; c < n_slices; ++c) {
-            tfjsb_model* v = m->slices[c];
-            if ((e = cudaStreamWaitEvent(s, m->slice_copied[c], 0)) != cudaSuccess) return cuda_fail(ctx, e, "cudaStreamWaitEvent");
-            tfjsb_tensor in{m->staged_in + c * in_slice, 4, {v->in_dims[0], v->in_dims[1], v->in_dims[2], v->in_dims[3]}};
+            tfjsb_model* v = m->slices[b * n_slices + c];
+            if ((e = cudaStreamWaitEvent(s, m->slice_copied[b * n_slices + c], 0)) != cudaSuccess)
+                return cuda_fail(ctx, e, "cudaStreamWaitEvent");
+            tfjsb_tensor in{m->staged_in[b] + c * in_slice, 4, {v->in_dims[0], v->in_dims[1], v->in_dims[2], v->in_dims[3]}};
             const Step& vl = v->steps.back();
-            tfjsb_tensor out{m->staged_out + c * out_slice, vl.out_rank, {vl.out_dims[0], vl.out_dims[1], vl.out_dims[2], vl.out_dims[3]}};
-            if ((st = tfjsb_run_model(v, &in, &out, stream)) != TFJSB_OK) return st;
+            tfjsb_tensor out{m->staged_out[b] + c * out_slice, vl.out_rank, {vl.out_dims[0], vl.out_dims[1], vl.out_dims[2], vl.out_dims[3]}};
+            if ((st = tfjsb_run_model(v, &in, &out, s)) != TFJSB_OK) return st;
             v->use_graph = true;  // the first pass ran launch by launch; later passes replay a graph
         }
-    } else {
-        e = cudaMemcpyAsync(m->staged_in, host_input, (size_t)m->in_elems * 4, cudaMemcpyHostToDevice, s);
-        if (e != cudaSuccess) return cuda_fail(ctx, e, "host-to-device copy of the input");
-        tfjsb_tensor in{m->staged_in, 4, {m->in_dims[0], m->in_dims[1], m->in_dims[2], m->in_dims[3]}};
-        tfjsb_tensor out{m->staged_out, last.out_rank, {last.out_dims[0], last.out_dims[1], last.out_dims[2], last.out_dims[3]}};
-        if ((st = tfjsb_run_model(m, &in, &out, stream)) != TFJSB_OK) return st;
     }
-    e = cudaMemcpyAsync(host_output, m->staged_out, (size_t)last.out_elems * 4, cudaMemcpyDeviceToHost, s);
+    e = cudaMemcpyAsync(host_output, m->staged_out[b], (size_t)last.out_elems * 4, cudaMemcpyDeviceToHost, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "device-to-host copy of the output");
-    e = cudaStreamSynchronize(s);
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaStreamSynchronize");
+    if ((e = cudaEventRecord(m->host_run_done[b], s)) != cudaSuccess) return cuda_fail(ctx, e, "cudaEventRecord");
+    m->host_run_pending[b] = true;
+    return TFJSB_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+tfjsb_status tfjsb_run_model_host_async(tfjsb_model* m, const float* host_input, float* host_output, void* stream) {
+    if (!m) return TFJSB_ERR_INVALID_ARG;
+    if (!host_input || !host_output) return fail(m->ctx, TFJSB_ERR_INVALID_ARG, "host_input / host_output is null");
+    const int b = m->next_staging;
+    tfjsb_status st = enqueue_host_run(m, host_input, host_output, static_cast<cudaStream_t>(stream), b);
+    if (st == TFJSB_OK) m->next_staging = b ^ 1;
+    return st;
+}
+
+tfjsb_status tfjsb_model_host_wait(tfjsb_model* m) {
+    if (!m) return TFJSB_ERR_INVALID_ARG;
+    for (int k = 0; k < 2; ++k) {
+        const int b = (m->next_staging + k) & 1;  // older run first
+        if (!m->host_run_pending[b]) continue;
+        cudaError_t e = cudaEventSynchronize(m->host_run_done[b]);
+        if (e != cudaSuccess) return cuda_fail(m->ctx, e, "cudaEventSynchronize");
+        m->host_run_pending[b] = false;
+    }
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_run_model_host(tfjsb_model* m, const float* host_input, float* host_output, void* stream) {
+    tfjsb_status st = tfjsb_run_model_host_async(m, host_input, host_output, stream);
+    if (st != TFJSB_OK) return st;
+    if ((st = tfjsb_model_host_wait(m)) != TFJSB_OK) return st;
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(m->ctx, e, "cudaStreamSynchronize");
     return TFJSB_OK;
 }
 

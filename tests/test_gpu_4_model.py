@@ -120,6 +120,18 @@ def test_config5_mobilenet_100_224_batch128_sampled_images(ctx, oracle):
     assert same_bits(hout.numpy(), probs)
     model.run_host(hin, hout.zero_())  # second call: the slices replay their captured graphs
     assert same_bits(hout.numpy(), probs)
+    # asynchronous host runs: three calls in a row (the third has to wait for the first, whose staging
+    # buffers it reuses), different inputs, outputs checked after one wait
+    hin2 = torch.from_numpy(np.ascontiguousarray(x[::-1])).pin_memory()  # the images in reverse order
+    hout2, hout3 = torch.zeros(128, 1000).pin_memory(), torch.zeros(128, 1000).pin_memory()
+    hout.zero_()
+    model.run_host_async(hin, hout)
+    model.run_host_async(hin2, hout2)
+    model.run_host_async(hin, hout3)
+    model.host_wait()
+    ctx.check_device_status()
+    assert same_bits(hout.numpy(), probs) and same_bits(hout3.numpy(), probs)
+    assert same_bits(hout2.numpy(), probs[::-1])
     # graph replay of the whole-batch run gives the same bits as launch-by-launch
     out2 = torch.empty(128, 1000, device="cuda")
     model.set_graph(True)
