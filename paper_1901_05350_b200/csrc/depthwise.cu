@@ -133,6 +133,21 @@ __global__ void depthwise_generic_kernel(const float* __restrict__ x, const floa
     }
 }
 
+// Bias, activation and store of one thread's R output rows (4 channels each) of the pipelined kernel.
+template <int ACT, int R>
+__device__ __forceinline__ void store_rows(const float4 (&acc)[R], const float4 b, float* yp, int64_t row_pitch, int rows) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        if (r < rows) {
+            float4 v = acc[r];
+            v.x = apply_act_t<ACT>(v.x + b.x); v.y = apply_act_t<ACT>(v.y + b.y);
+            v.z = apply_act_t<ACT>(v.z + b.z); v.w = apply_act_t<ACT>(v.w + b.w);
+            *reinterpret_cast<float4*>(yp) = v;
+        }
+        yp += row_pitch;
+    }
+}
+
 // ---- pipelined kernel ---------------------------------------------------------------------------
 constexpr int DW_CB = 32;          // channels per tile: one 128-byte line per pixel
 constexpr int DW_MAX_STAGES = 4;
@@ -289,16 +304,11 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bar_empty[slot]));
             float* yp = y + (((int64_t)info.w * g.Ho + oy0) * g.Wo + ox) * g.Co + c;
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                if (oy0 + r < g.Ho) {
-                    float4 v = acc[r];
-                    v.x = apply_act(v.x + b.x, act); v.y = apply_act(v.y + b.y, act);
-                    v.z = apply_act(v.z + b.z, act); v.w = apply_act(v.w + b.w, act);
-                    *reinterpret_cast<float4*>(yp) = v;
-                }
-                yp += row_pitch;
-            }
+            const int rows = g.Ho - oy0;
+            // the activation is chosen once per tile, not once per value: the kernel is close to issue bound
+            if (act == TFJSB_ACT_RELU6) store_rows<TFJSB_ACT_RELU6, R>(acc, b, yp, row_pitch, rows);
+            else if (act == TFJSB_ACT_RELU) store_rows<TFJSB_ACT_RELU, R>(acc, b, yp, row_pitch, rows);
+            else store_rows<TFJSB_ACT_NONE, R>(acc, b, yp, row_pitch, rows);
         } else {
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bar_empty[slot]));

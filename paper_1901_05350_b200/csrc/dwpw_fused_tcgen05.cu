@@ -85,6 +85,27 @@ __device__ __forceinline__ void fma4s(float4& acc, const float4& a, const float4
     acc.z = fmaf(a.z, b.z, acc.z); acc.w = fmaf(a.w, b.w, acc.w);
 }
 
+// Bias, activation and the swizzled store of one depthwise thread's 4 rows x 2 columns x 2 channels
+// into the A operand (GEMM row of a pixel = row*16 + column).  The activation is a template parameter:
+// the kernel is close to instruction-issue bound, and a run-time choice costs two extra instructions
+// per value.
+template <int ACT>
+__device__ __forceinline__ void store_depthwise_block(const float2 (&acc)[F_TH / 2][2], const float2 b, uint32_t a_stage,
+                                                      int rg, int colg, int c2) {
+    constexpr int R = F_TH / 2;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
+            const float vx = apply_act_t<ACT>(acc[r][cc].x + b.x);
+            const float vy = apply_act_t<ACT>(acc[r][cc].y + b.y);
+            const int p = (rg * R + r) * F_TW + colg * 2 + cc;
+            const uint32_t dst = a_stage + (uint32_t)p * 128u + (uint32_t)(((c2 >> 1) ^ (p & 7)) << 4) + (uint32_t)((c2 & 1) << 3);
+            asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(dst), "f"(vx), "f"(vy) : "memory");
+        }
+    }
+}
+
 template <bool CONV>
 __global__ void __launch_bounds__(CONV ? F_CONV_THREADS : F_THREADS, CONV ? 2 : 1)
 dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_b,
@@ -464,17 +485,9 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                         }
                     }
                     const uint32_t a_stage = a_base + (uint32_t)as * A_STAGE_BYTES;
-#pragma unroll
-                    for (int r = 0; r < R; ++r) {
-#pragma unroll
-                        for (int cc = 0; cc < 2; ++cc) {
-                            const float vx = apply_act(acc[r][cc].x + b.x, args.dw_act);
-                            const float vy = apply_act(acc[r][cc].y + b.y, args.dw_act);
-                            const int p = (rg * R + r) * F_TW + colg * 2 + cc;
-                            const uint32_t dst = a_stage + (uint32_t)p * 128u + (uint32_t)(((c2 >> 1) ^ (p & 7)) << 4) + (uint32_t)((c2 & 1) << 3);
-                            asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(dst), "f"(vx), "f"(vy) : "memory");
-                        }
-                    }
+                    if (args.dw_act == TFJSB_ACT_RELU6) store_depthwise_block<TFJSB_ACT_RELU6>(acc, b, a_stage, rg, colg, c2);
+                    else if (args.dw_act == TFJSB_ACT_RELU) store_depthwise_block<TFJSB_ACT_RELU>(acc, b, a_stage, rg, colg, c2);
+                    else store_depthwise_block<TFJSB_ACT_NONE>(acc, b, a_stage, rg, colg, c2);
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0) {
