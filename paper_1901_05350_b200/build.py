@@ -28,6 +28,7 @@ SOURCES = [
     "gemm_fp32_simt.cu",
     "gemm_tf32_tcgen05.cu",
     "gemm_tf32_pair.cu",
+    "gemm_tf32_splitk.cu",
     "conv2d_fp32_simt.cu",
     "depthwise.cu",
     "matmul_static_scratch.cu",

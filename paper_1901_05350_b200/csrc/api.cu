@@ -190,7 +190,6 @@ tfjsb_status tfjsb_shutdown(tfjsb_ctx* ctx) {
     if (ctx->dev_status) cudaFree(ctx->dev_status);
     if (ctx->scratch_a.ptr) cudaFree(ctx->scratch_a.ptr);
     if (ctx->scratch_b.ptr) cudaFree(ctx->scratch_b.ptr);
-    if (ctx->scratch_ws.ptr) cudaFree(ctx->scratch_ws.ptr);
     delete ctx;
     return TFJSB_OK;
 }
@@ -276,9 +275,7 @@ tfjsb_status tfjsb_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_ten
             b_km = ctx->scratch_b.ptr;
         }
         GemmTf32Plan plan;
-        const size_t ws_bytes = gemm_tf32_workspace_bytes(M, N, K, ctx->sm_count);
-        if (ws_bytes && (st = ensure_scratch(ctx, &ctx->scratch_ws, ws_bytes)) != TFJSB_OK) return st;
-        if ((st = gemm_tf32_plan(ctx, a_km, b_km, pc, M, N, K, &plan, ws_bytes ? ctx->scratch_ws.ptr : nullptr, ws_bytes)) != TFJSB_OK) return st;
+        if ((st = gemm_tf32_plan(ctx, a_km, b_km, pc, M, N, K, &plan)) != TFJSB_OK) return st;
         if ((e = launch_gemm_tf32(plan, nullptr, TFJSB_ACT_NONE, ctx->dev_status, s, &ctx->launches)) != cudaSuccess)
             return cuda_fail(ctx, e, "tf32 gemm launch");
         return TFJSB_OK;
@@ -328,9 +325,7 @@ tfjsb_status tfjsb_conv2d(tfjsb_ctx* ctx, const tfjsb_tensor* x, const tfjsb_ten
             if ((e = launch_transpose(pf, ctx->scratch_b.ptr, K, N, s, &ctx->launches)) != cudaSuccess)
                 return cuda_fail(ctx, e, "transpose(filter)");
             GemmTf32Plan plan;
-            const size_t ws_bytes = gemm_tf32_workspace_bytes(M, N, K, ctx->sm_count);
-            if (ws_bytes && (st = ensure_scratch(ctx, &ctx->scratch_ws, ws_bytes)) != TFJSB_OK) return st;
-            if ((st = gemm_tf32_plan(ctx, px, ctx->scratch_b.ptr, py, M, N, K, &plan, ws_bytes ? ctx->scratch_ws.ptr : nullptr, ws_bytes)) != TFJSB_OK) return st;
+            if ((st = gemm_tf32_plan(ctx, px, ctx->scratch_b.ptr, py, M, N, K, &plan)) != TFJSB_OK) return st;
             if ((e = launch_gemm_tf32(plan, pbias, act, ctx->dev_status, s, &ctx->launches)) != cudaSuccess)
                 return cuda_fail(ctx, e, "tf32 gemm launch");
             return TFJSB_OK;

@@ -86,7 +86,6 @@ struct tfjsb_ctx {
     unsigned int* dev_status = nullptr;  // device status word
     tfjsb::EncodeTiledFn encode_tiled = nullptr;
     tfjsb::Scratch scratch_a, scratch_b;  // transposed operands of tfjsb_matmul
-    tfjsb::Scratch scratch_ws;            // split-K workspace of the stand-alone GEMM calls
     int64_t launches = 0;
     int live_models = 0;
 };
@@ -180,24 +179,18 @@ struct GemmTf32Plan {
     size_t smem_bytes;
     // CTA-pair kernel (gemm_tf32_pair.cu): 256 x block_n tiles shared by two CTAs
     bool pair = false;
-    // split K: partial sums go to ws [splits, m_pad, N], a second kernel reduces them into c
-    int splits = 1, kb_per_split = 0;
-    int64_t m_pad = 0;
-    float* ws = nullptr;
-    float* c = nullptr;
+    // cluster split-K kernel (gemm_tf32_splitk.cu): `splits` CTAs per tile, reduced through shared memory
+    bool cluster_split = false;
+    int splits = 1, kb_per_split = 0;  // slices of the K loop (= cluster size) and k-blocks per slice
+    float* c = nullptr;                // C, which that kernel stores directly
     // implicit-GEMM convolution: A is gathered from x by the kernel instead of copied
     bool gather = false;
     const float* x = nullptr;
     ConvGeom g{};
 };
 bool gemm_tf32_supported(int64_t M, int64_t N, int64_t K);
-// `ws` (optional) is scratch for split K, at least gemm_tf32_workspace_bytes(...) large for the plan to
-// be allowed to cut the K loop; it must stay valid, and unused by anything else in flight, while
-// the plan is launched.
 tfjsb_status gemm_tf32_plan(tfjsb_ctx* ctx, const float* a, const float* bt, float* c, int64_t M, int64_t N,
-                            int64_t K, GemmTf32Plan* plan, float* ws = nullptr, size_t ws_bytes = 0);
-// Scratch the plan may use (0: this shape is never split).
-size_t gemm_tf32_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count);
+                            int64_t K, GemmTf32Plan* plan);
 // The same GEMM on CTA pairs; gemm_tf32_plan picks it where it is the faster kernel (environment
 // variable TFJSB_GEMM_PAIR: 0 = never, 1 = wherever the shape allows, unset = by shape).
 bool gemm_tf32_pair_preferred(int64_t M, int64_t N, int64_t K, int sm_count);
@@ -205,6 +198,12 @@ tfjsb_status gemm_tf32_pair_plan(tfjsb_ctx* ctx, const float* a, const float* bt
                                  int64_t K, GemmTf32Plan* plan);
 cudaError_t launch_gemm_tf32_pair(const GemmTf32Plan& plan, const float* bias, int act, unsigned int* dev_status,
                                   cudaStream_t s, int64_t* launches);
+// Split K across the CTAs of a cluster, for GEMMs with too few tiles for the SMs (gemm_tf32_splitk.cu).
+bool gemm_tf32_splitk_choice(int64_t M, int64_t N, int64_t K, int sm_count, int* block_n, int* splits);
+tfjsb_status gemm_tf32_splitk_plan(tfjsb_ctx* ctx, const float* a, const float* bt, float* c, int64_t M, int64_t N,
+                                   int64_t K, int block_n, int splits, GemmTf32Plan* plan);
+cudaError_t launch_gemm_tf32_splitk(const GemmTf32Plan& plan, const float* bias, int act, unsigned int* dev_status,
+                                    cudaStream_t s, int64_t* launches);
 // Implicit-GEMM convolution on the same kernel: M = N*Ho*Wo output pixels, K = fh*fw*Cin, N = Cout.
 // `bt` is the filter packed as [Cout, k_pad] (K-contiguous, zero padded to a multiple of 32).
 bool conv_igemm_supported(const ConvGeom& g);

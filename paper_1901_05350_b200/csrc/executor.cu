@@ -56,8 +56,6 @@ struct tfjsb_model {
     size_t region_elems = 0;     // elements per ping-pong region
     float* keep_all_arena = nullptr;
     bool keep_all = false;
-    float* gemm_ws = nullptr;    // split-K workspace shared by the GEMM layers (they run one after the other)
-    size_t gemm_ws_bytes = 0;
     // Host-buffer runs (tfjsb_run_model_host / _async) alternate between two sets of device staging
     // buffers, so that the input copy of one run can overlap the computation of the run before it.
     float* staged_in[2] = {nullptr, nullptr};
@@ -122,7 +120,7 @@ tfjsb_status bind_step(tfjsb_model* m, Step& st, const float* in, float* out) {
     st.in = in;
     st.out = out;
     if (st.kind == STEP_GEMM_TF32 && (changed || !st.plan_built)) {
-        tfjsb_status rc = gemm_tf32_plan(m->ctx, in, st.filter_km, out, st.M, st.N, st.K, &st.plan, m->gemm_ws, m->gemm_ws_bytes);
+        tfjsb_status rc = gemm_tf32_plan(m->ctx, in, st.filter_km, out, st.M, st.N, st.K, &st.plan);
         if (rc != TFJSB_OK) return rc;
         st.plan_built = true;
     }
@@ -214,8 +212,6 @@ tfjsb_model* make_batch_view(tfjsb_model* parent, int64_t n) {
     v->use_tf32 = parent->use_tf32;
     v->use_pdl = parent->use_pdl;
     v->arena = parent->arena;
-    v->gemm_ws = parent->gemm_ws;
-    v->gemm_ws_bytes = parent->gemm_ws_bytes;
     v->region_elems = parent->region_elems;
     v->steps = parent->steps;
     for (int i = 0; i < 4; ++i) v->in_dims[i] = parent->in_dims[i];
@@ -291,17 +287,9 @@ cudaError_t launch_layers(tfjsb_model* m, int i, cudaStream_t s, int* consumed) 
 }
 
 int launches_per_run(const tfjsb_model* m) {
-    int n = 0;
-    for (size_t i = 0; i < m->steps.size(); ++i) {
-        const Step& st = m->steps[i];
-        if (st.fuse_next && !m->keep_all) {  // one kernel for this layer and the next
-            ++n;
-            ++i;
-            continue;
-        }
-        // a GEMM cut along K is two kernels: the partial sums, then their reduction
-        n += (st.kind == STEP_GEMM_TF32 && st.plan_built && st.plan.splits > 1) ? 2 : 1;
-    }
+    int n = (int)m->steps.size();
+    if (!m->keep_all)
+        for (const Step& st : m->steps) n -= st.fuse_next ? 1 : 0;
     return n;
 }
 
@@ -490,12 +478,6 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
         }
     }
     if ((st = dev_alloc(m, 2 * m->region_elems, &m->arena)) != TFJSB_OK) return bail(st, ctx->last_error);
-    for (const Step& sp : m->steps)
-        if (sp.kind == STEP_GEMM_TF32) {
-            const size_t need = gemm_tf32_workspace_bytes(sp.M, sp.N, sp.K, ctx->sm_count);
-            if (need > m->gemm_ws_bytes) m->gemm_ws_bytes = need;
-        }
-    if (m->gemm_ws_bytes && (st = dev_alloc(m, m->gemm_ws_bytes / sizeof(float), &m->gemm_ws)) != TFJSB_OK) return bail(st, ctx->last_error);
     cudaError_t e = cudaDeviceSynchronize();  // weight transposes done
     if (e != cudaSuccess) return bail(TFJSB_ERR_CUDA, std::string("model set-up: ") + cudaGetErrorString(e));
     ++ctx->live_models;

@@ -334,8 +334,8 @@ tfjsb_status gemm_tf32_pair_plan(tfjsb_ctx* ctx, const float* a, const float* bt
     plan->gather = false;
     plan->x = nullptr;
     plan->pair = true;
+    plan->cluster_split = false;
     plan->splits = 1;
-    plan->ws = nullptr;
     plan->c = c;
     int bn = 256;
     while (bn > 64 && bn / 2 >= N) bn >>= 1;

@@ -26,13 +26,6 @@
 // Ragged edges need no special code: rows/columns past M, N or K are zero-filled on load and
 // clipped on store by the tensor maps.
 //
-// Split K.  A GEMM with few output tiles and a long K loop (the dense layer, every pointwise layer at
-// small batch) leaves most SMs idle while a few walk all the k-blocks one after the other.  Such a
-// GEMM is cut along K as well: work item = (tile, slice of the k-blocks); each item stores its partial
-// sums, without bias or activation, into its slice of a workspace [slices, M rounded up to 128, N],
-// and a second kernel adds the slices in a fixed order, adds the bias, applies the activation and
-// writes C.  The result does not depend on which SM ran which item.
-//
 // Every wait is bounded: a wait that exceeds WAIT_LIMIT_NS raises an abort flag that all roles
 // poll, ORs a code into the context's device status word, and the CTA drains its copies, frees
 // its tensor memory and returns.
@@ -141,9 +134,6 @@ struct KernelArgs {
     int n_tiles;    // tiles along N
     int num_tiles;  // total
     int acc_stages;  // accumulator stages in tensor memory: 2 (block_n 256) or 4
-    int splits;        // slices of the K loop (1 = none); a work item is (tile, slice), slice fastest
-    int kb_per_split;  // k-blocks per slice
-    int m_pad;         // rows per slice of the split-K workspace
     const float* bias;
     int act;
     unsigned int* dev_status;
@@ -222,14 +212,11 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 #pragma unroll
             for (int s = 0; s < MAX_STAGES; ++s) armed[s] = -1;
             bool ok = true;
-            for (int item = blockIdx.x; ok && item < args.num_tiles; item += gridDim.x) {
-                const int tile = item / args.splits, slice = item - tile * args.splits;
+            for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
                 const int m0 = (tile / args.n_tiles) * BLOCK_M;
                 const int n0 = (tile % args.n_tiles) * block_n;
                 (void)m0;
-                const int kb_begin = slice * args.kb_per_split;
-                const int kb_end = min(num_k_blocks, kb_begin + args.kb_per_split);
-                for (int kb = kb_begin; kb < kb_end; ++kb) {
+                for (int kb = 0; kb < num_k_blocks; ++kb) {
                     if (!bounded_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_flag)) {
                         if (!*abort_flag) {
                             *abort_flag = 1;
@@ -280,13 +267,11 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             uint32_t acc_phase = 0;
             bool ok = true;
             bool issued_any = false;
-            for (int item = blockIdx.x; ok && item < args.num_tiles; item += gridDim.x) {
+            for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
                 if (!bounded_wait(smem_u32(&bar_acc_empty[acc]), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * block_n);
-                const int kb_first = (item % args.splits) * args.kb_per_split;
-                const int kb_count = min(num_k_blocks - kb_first, args.kb_per_split);
-                for (int kb = 0; kb < kb_count; ++kb) {
+                for (int kb = 0; kb < num_k_blocks; ++kb) {
                     if (!bounded_wait(smem_u32(&bar_full[stage]), phase, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_addr = stage_base + (uint32_t)stage * (uint32_t)stage_bytes;
@@ -338,8 +323,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         bool ok = true;
         const int chunks_per_tile = block_n / EPI_COLS;
         int first_chunk = half;  // parity bookkeeping: chunk `ch` of this tile is ours when (ch - first_chunk) is even
-        for (int item = blockIdx.x; ok && item < args.num_tiles; item += gridDim.x) {
-            const int tile = item / args.splits, slice = item - tile * args.splits;
+        for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
             const int m0 = (tile / args.n_tiles) * BLOCK_M;
             const int n0 = (tile % args.n_tiles) * block_n;
             // every lane polls (each needs the acquire), the vote keeps the warp uniform
@@ -386,8 +370,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    // with split K, map_c is the workspace viewed as [slices * m_pad, N]
-                    tma_store_2d(&map_c, slab, col0, slice * args.m_pad + row0);
+                    tma_store_2d(&map_c, slab, col0, row0);
                     tma_store_commit();
                 }
             }
@@ -479,43 +462,6 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     }
 }
 
-// C[m, n] = act( sum over slices of ws[slice, m, n] + bias[n] ), slices added in index order.
-__global__ void __launch_bounds__(256)
-splitk_reduce_kernel(const float* __restrict__ ws, const float* __restrict__ bias, float* __restrict__ c, int64_t M, int n4,
-                     int splits, int64_t slice_pitch4, int act) {
-    pdl_launch_dependents();
-    pdl_wait();  // the partial sums come from the GEMM kernel launched just before
-    const float4* ws4 = reinterpret_cast<const float4*>(ws);
-    const float4* bias4 = reinterpret_cast<const float4*>(bias);
-    float4* c4 = reinterpret_cast<float4*>(c);
-    const int64_t total = M * n4;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        float4 v = ws4[i];
-        for (int sl = 1; sl < splits; ++sl) {
-            const float4 p = ws4[sl * slice_pitch4 + i];
-            v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
-        }
-        if (bias != nullptr) {
-            const float4 b = __ldg(bias4 + (i % n4));
-            v.x += b.x; v.y += b.y; v.z += b.z; v.w += b.w;
-        }
-        v.x = apply_act(v.x, act); v.y = apply_act(v.y, act); v.z = apply_act(v.z, act); v.w = apply_act(v.w, act);
-        c4[i] = v;
-    }
-}
-
-constexpr int MAX_SPLITS = 8;
-constexpr int MIN_KB_PER_SPLIT = 4;
-
-// Slices of the K loop for a GEMM whose `tiles` output tiles cannot occupy the SMs (1 = do not split).
-int choose_splits(int64_t tiles, int64_t num_k_blocks, int sm_count) {
-    if (tiles >= sm_count) return 1;
-    int64_t want = (sm_count + tiles - 1) / tiles;
-    if (want > MAX_SPLITS) want = MAX_SPLITS;
-    if (want > num_k_blocks / MIN_KB_PER_SPLIT) want = num_k_blocks / MIN_KB_PER_SPLIT;
-    return want < 2 ? 1 : (int)want;
-}
-
 int choose_block_n(int64_t M, int64_t N, int sm_count) {
     int bn = 32;
     while (bn < 256 && bn < N) bn <<= 1;
@@ -559,10 +505,6 @@ namespace {
 // tile choice, pipeline depth and the B / C tensor maps shared by the GEMM and the convolution
 tfjsb_status plan_common(tfjsb_ctx* ctx, const float* bt, int64_t k_pitch, float* c, GemmTf32Plan* plan) {
     const int64_t M = plan->M, N = plan->N;
-    plan->splits = 1;
-    plan->kb_per_split = 0;
-    plan->m_pad = 0;
-    plan->ws = nullptr;
     plan->block_n = choose_block_n(M, N, ctx->sm_count);
     plan->acc_stages = plan->block_n > 128 ? 2 : MAX_ACC_STAGES;
     const int stage_bytes = A_STAGE_BYTES + plan->block_n * BLOCK_K * 4;
@@ -582,60 +524,26 @@ tfjsb_status plan_common(tfjsb_ctx* ctx, const float* bt, int64_t k_pitch, float
 
 }  // namespace
 
-size_t gemm_tf32_workspace_bytes(int64_t M, int64_t N, int64_t K, int sm_count) {
-    if (!gemm_tf32_supported(M, N, K)) return 0;
-    const int64_t m_tiles = (M + BLOCK_M - 1) / BLOCK_M;
-    if (m_tiles * ((N + 31) / 32) >= sm_count) return 0;  // enough tiles without cutting K
-    return (size_t)MAX_SPLITS * m_tiles * BLOCK_M * N * sizeof(float);
-}
-
 tfjsb_status gemm_tf32_plan(tfjsb_ctx* ctx, const float* a, const float* bt, float* c, int64_t M, int64_t N,
-                            int64_t K, GemmTf32Plan* plan, float* ws, size_t ws_bytes) {
+                            int64_t K, GemmTf32Plan* plan) {
     if (!gemm_tf32_supported(M, N, K)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the TF32 GEMM");
     if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
     const char* pair_env = getenv("TFJSB_GEMM_PAIR");
     const bool use_pair = pair_env ? (pair_env[0] == '1' && N >= 64) : gemm_tf32_pair_preferred(M, N, K, ctx->sm_count);
     if (use_pair) return gemm_tf32_pair_plan(ctx, a, bt, c, M, N, K, plan);
+    {
+        // few tiles and a long K loop: the K loop is cut across the CTAs of a cluster (gemm_tf32_splitk.cu)
+        int split_bn = 0, split_s = 0;
+        if (!getenv("TFJSB_NO_SPLIT_K") && gemm_tf32_splitk_choice(M, N, K, ctx->sm_count, &split_bn, &split_s))
+            return gemm_tf32_splitk_plan(ctx, a, bt, c, M, N, K, split_bn, split_s, plan);
+    }
     plan->M = M; plan->N = N; plan->K = K;
     plan->pair = false;
+    plan->cluster_split = false;
     plan->gather = false;
     plan->x = nullptr;
-    plan->c = c;
     tfjsb_status st;
     if ((st = plan_common(ctx, bt, K, c, plan)) != TFJSB_OK) return st;
-    if (ws != nullptr && !getenv("TFJSB_NO_SPLIT_K")) {
-        // Split K: widest tile first (wide MMAs are the efficient ones), the K loop cut into as many
-        // slices as it takes to give every SM an item.
-        const int64_t m_tiles = (M + BLOCK_M - 1) / BLOCK_M;
-        const int64_t nkb = (K + BLOCK_K - 1) / BLOCK_K;
-        int bn = 32;
-        while (bn < 256 && bn < N) bn <<= 1;
-        int splits = 1;
-        for (;; bn >>= 1) {
-            splits = choose_splits(m_tiles * ((N + bn - 1) / bn), nkb, ctx->sm_count);
-            if (bn == 32 || splits * m_tiles * ((N + bn - 1) / bn) >= ctx->sm_count) break;
-        }
-        const int64_t m_pad = m_tiles * BLOCK_M;
-        if (splits > 1 && (size_t)splits * m_pad * N * sizeof(float) <= ws_bytes && splits * m_pad < (1LL << 31) - 256) {
-            int kbs = (int)((nkb + splits - 1) / splits);
-            splits = (int)((nkb + kbs - 1) / kbs);  // no empty slice
-            plan->block_n = bn;
-            plan->acc_stages = bn > 128 ? 2 : MAX_ACC_STAGES;
-            const int stage_bytes = A_STAGE_BYTES + bn * BLOCK_K * 4;
-            int stages = (SMEM_LIMIT - 1024 - EPI_BYTES - 512) / stage_bytes;
-            plan->stages = stages > MAX_STAGES ? MAX_STAGES : stages;
-            plan->smem_bytes = (size_t)1024 + EPI_BYTES + (size_t)plan->stages * stage_bytes;
-            plan->splits = splits;
-            plan->kb_per_split = kbs;
-            plan->m_pad = m_pad;
-            plan->ws = ws;
-            const int64_t items = m_tiles * ((N + bn - 1) / bn) * splits;
-            plan->num_tiles = (int)items;
-            plan->grid = (int)(items < ctx->sm_count ? items : ctx->sm_count);
-            if ((st = encode_2d(ctx, &plan->map_b, bt, K, N, BLOCK_K, bn, "B")) != TFJSB_OK) return st;
-            if ((st = encode_2d(ctx, &plan->map_c, ws, N, splits * m_pad, EPI_COLS, 32, "the split-K workspace")) != TFJSB_OK) return st;
-        }
-    }
     return encode_2d(ctx, &plan->map_a, a, K, M, BLOCK_K, BLOCK_M, "A");
 }
 
@@ -660,6 +568,7 @@ tfjsb_status conv_igemm_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
     plan->K = (int64_t)g.fh * g.fw * g.C;
     plan->gather = true;
     plan->pair = false;
+    plan->cluster_split = false;
     plan->x = x;
     plan->g = g;
     tfjsb_status st = plan_common(ctx, bt, conv_igemm_k_pad(g), y, plan);
@@ -671,6 +580,7 @@ tfjsb_status conv_igemm_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
 cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int act, unsigned int* dev_status,
                              cudaStream_t s, int64_t* launches) {
     if (plan.pair) return launch_gemm_tf32_pair(plan, bias, act, dev_status, s, launches);
+    if (plan.cluster_split) return launch_gemm_tf32_splitk(plan, bias, act, dev_status, s, launches);
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(gemm_tf32_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -689,12 +599,8 @@ cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int ac
     args.n_tiles = (int)((plan.N + plan.block_n - 1) / plan.block_n);
     args.num_tiles = plan.num_tiles;
     args.acc_stages = plan.acc_stages;
-    const bool split = plan.splits > 1;
-    args.splits = plan.splits;
-    args.kb_per_split = split ? plan.kb_per_split : (int)((plan.K + BLOCK_K - 1) / BLOCK_K);
-    args.m_pad = (int)plan.m_pad;
-    args.bias = split ? nullptr : bias;  // the reduction kernel applies them
-    args.act = split ? TFJSB_ACT_NONE : act;
+    args.bias = bias;
+    args.act = act;
     args.dev_status = dev_status;
     args.x = plan.x;
     args.g = plan.g;
@@ -705,14 +611,6 @@ cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int ac
         e = launch_k(gemm_tf32_kernel<false>, dim3(plan.grid), dim3(GEMM_THREADS), plan.smem_bytes, s, plan.map_a, plan.map_b,
                      plan.map_c, args);
     ++*launches;
-    if (e == cudaSuccess && split) {
-        const int n4 = (int)(plan.N / 4);
-        const int64_t total = plan.M * n4;
-        const int blocks = (int)((total + 255) / 256 < 592 ? (total + 255) / 256 : 592);
-        e = launch_k(splitk_reduce_kernel, dim3(blocks), dim3(256), 0, s, (const float*)plan.ws, bias, plan.c, plan.M, n4,
-                     plan.splits, plan.m_pad * n4, act);
-        ++*launches;
-    }
     return e;
 }
 

@@ -84,17 +84,13 @@ def test_matmul_split_k_agrees_with_unsplit_and_oracle(ctx, oracle, monkeypatch,
     a = si.uniform(311, 0, (M, K), -1, 1)
     b = si.uniform(311, 1, (K, N), -1, 1)
     monkeypatch.delenv("TFJSB_NO_SPLIT_K", raising=False)
-    launches = ctx.launch_count
     split = host(ctx.matmul(dev(a), dev(b)))
-    split_launches = ctx.launch_count - launches
     again = host(ctx.matmul(dev(a), dev(b)))
     monkeypatch.setenv("TFJSB_NO_SPLIT_K", "1")
-    launches = ctx.launch_count
     whole = host(ctx.matmul(dev(a), dev(b)))
-    whole_launches = ctx.launch_count - launches
     ctx.check_device_status()
-    assert split_launches == whole_launches + 1          # the reduction kernel: K really was cut
-    assert same_bits(split, again)                        # slices are added in a fixed order
+    assert not same_bits(split, whole)                    # another summation order: K really was cut
+    assert same_bits(split, again)                        # slices are added in a fixed order, whichever finishes first
     want = oracle.matmul(a, b)
     assert rel_fro(split, want) <= TF32_TOL and rel_fro(whole, want) <= TF32_TOL
     assert rel_fro(split, oracle.matmul(a, b, operand="tf32_rz")) <= MATCHED_TOL
@@ -105,7 +101,7 @@ def test_matmul_split_k_agrees_with_unsplit_and_oracle(ctx, oracle, monkeypatch,
 
 
 def test_dense_split_k_fused_bias_and_activation(ctx, oracle):
-    # the reduction kernel applies bias and activation: [128,1,1,1024] x [1,1,1024,1000] + bias, relu6
+    # the reduction applies bias and activation: [128,1,1,1024] x [1,1,1024,1000] + bias, relu6
     x = si.uniform(313, 0, (128, 1, 1, 1024), 0, 1)
     f = si.normal(313, 1, (1, 1, 1024, 1000), 0, float(np.sqrt(2.0 / 1024)))
     b = si.normal(313, 2, (1000,), 0, 0.5)

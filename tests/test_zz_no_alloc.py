@@ -3,12 +3,9 @@
 tfjsb_matmul_static_scratch exists for callers that cannot call cudaMalloc where they call the
 library (a real-time loop that may not block on the allocator, a service with a device-memory
 budget fixed at start-up): it transposes operands into a fixed array inside the library instead
-of allocated scratch.  It runs the same GEMM kernel on the same data as tfjsb_matmul, so its output
+of allocated scratch.  It runs the same kernels on the same data as tfjsb_matmul, so its output
 must be bit-identical, call after call, although the array still holds the previous call's
-operands.  (tfjsb_matmul may also cut the K loop of a small problem into slices, which needs an
-allocated workspace and adds the products in another order; the comparison is made bit for bit with
-that switched off and within the accumulation-order tolerance, 2e-5, with it on.)  This file is
-collected last so that a run that stops at the first failure has already
+operands.  This file is collected last so that a run that stops at the first failure has already
 run every other test.
 """
 import numpy as np
@@ -20,15 +17,8 @@ from helpers import dev, host, rel_fro, same_bits
 pytestmark = pytest.mark.gpu
 
 
-def test_static_scratch_matmul_matches_matmul_on_two_calls_in_a_row(ctx, oracle, monkeypatch):
+def test_static_scratch_matmul_matches_matmul_on_two_calls_in_a_row(ctx, oracle):
     import torch
-
-    def unsplit_matmul(*args):
-        monkeypatch.setenv("TFJSB_NO_SPLIT_K", "1")
-        try:
-            return host(ctx.matmul(*args))
-        finally:
-            monkeypatch.delenv("TFJSB_NO_SPLIT_K")
 
     cases = [
         # M, K, N, transpose_a, transpose_b: the second call is smaller, leaving stale data behind it
@@ -45,8 +35,7 @@ def test_static_scratch_matmul_matches_matmul_on_two_calls_in_a_row(ctx, oracle,
         assert torch.cuda.memory_allocated() == before
         ctx.check_device_status()
         got = host(out)
-        assert same_bits(got, unsplit_matmul(ad, bd, ta, tb))
-        assert rel_fro(got, host(ctx.matmul(ad, bd, ta, tb))) <= 2e-5
+        assert same_bits(got, host(ctx.matmul(ad, bd, ta, tb)))
         assert rel_fro(got, oracle.matmul(a, b, ta, tb)) <= 5e-3
     # the first problem's shape again, with new values, straight after a different problem:
     # whatever the array still holds must not leak into the result
@@ -55,7 +44,7 @@ def test_static_scratch_matmul_matches_matmul_on_two_calls_in_a_row(ctx, oracle,
     b = si.uniform(902, 1, (K, N), -1, 1)
     out = torch.empty(M, N, device="cuda")
     ctx.matmul_static_scratch(dev(a), dev(b), ta, tb, out=out)
-    assert same_bits(host(out), unsplit_matmul(dev(a), dev(b), ta, tb))
+    assert same_bits(host(out), host(ctx.matmul(dev(a), dev(b), ta, tb)))
     ctx.check_device_status()
 
 
