@@ -53,6 +53,8 @@ def _load():
         lib.orc_bias_act.argtypes = [fp, i64, i64, fp, i32, fp]
         lib.orc_avg_pool.argtypes = [fp, i64, i32, i32, i32, i32, i32, i32, i32, i32, fp]
         lib.orc_softmax.argtypes = [fp, i64, i64, fp]
+        lib.orc_max_pool.argtypes = [fp, i64, i32, i32, i32, i32, i32, i32, i32, i32, fp]
+        lib.orc_binary.argtypes = [i32, fp, fp, i64, i64, fp]
         _lib = lib
     return _lib
 
@@ -162,6 +164,42 @@ def avg_pool(x, filter_size, strides, pad="valid") -> np.ndarray:
     if rc:
         raise RuntimeError(f"orc_avg_pool failed ({rc})")
     return y
+
+
+def max_pool(x, filter_size, strides, pad="valid") -> np.ndarray:
+    x = _f32(x)
+    N, H, W, C = x.shape
+    Ho, _, _ = window_geometry(H, filter_size[0], strides[0], 1, pad)
+    Wo, _, _ = window_geometry(W, filter_size[1], strides[1], 1, pad)
+    y = np.empty((N, Ho, Wo, C), dtype=np.float32)
+    rc = _load().orc_max_pool(_ptr(x), N, H, W, C, filter_size[0], filter_size[1], strides[0], strides[1],
+                              PAD[pad], _ptr(y))
+    if rc:
+        raise RuntimeError(f"orc_max_pool failed ({rc})")
+    return y
+
+
+BINARY_OP = {"add": 0, "sub": 1, "mul": 2}
+
+
+def binary(op: str, a, b) -> np.ndarray:
+    """a op b, elementwise; b has a's shape or is a vector of a's last dimension."""
+    a, b = _f32(a), _f32(b)
+    if b.shape != a.shape and b.shape != (a.shape[-1],):
+        raise ValueError("b must have a's shape or be a vector of a's last dimension")
+    out = np.empty_like(a)
+    rc = _load().orc_binary(BINARY_OP[op], _ptr(a), _ptr(b), a.size, b.size, _ptr(out))
+    if rc:
+        raise RuntimeError(f"orc_binary failed ({rc})")
+    return out
+
+
+def batch_matmul(a, b, transpose_a: bool = False, transpose_b: bool = False, operand: str = "fp32") -> np.ndarray:
+    """Rank-3 matMul: one rank-2 product per leading index."""
+    a, b = _f32(a), _f32(b)
+    if a.ndim != 3 or b.ndim != 3 or a.shape[0] != b.shape[0]:
+        raise ValueError("batch_matmul takes rank-3 tensors with equal leading dimensions")
+    return np.stack([matmul(a[i], b[i], transpose_a, transpose_b, operand) for i in range(a.shape[0])])
 
 
 def softmax(x) -> np.ndarray:

@@ -253,6 +253,51 @@ int orc_avg_pool(const float* x, int64_t N, int H, int W, int C, int fh, int fw,
     return 0;
 }
 
+// y[n,oy,ox,c] = largest in-bounds window element (padding never takes part; a NaN in the window gives NaN).
+// tf.maxPool: not defined in the paper; TensorFlow's definition, with the window geometry above.
+int orc_max_pool(const float* x, int64_t N, int H, int W, int C, int fh, int fw, int sh, int sw, int pad_mode,
+                 float* y) {
+    int Ho, Wo, pt, pb, pl, pr;
+    if (!x || !y) return 1;
+    if (!window_geometry(H, fh, sh, 1, pad_mode, &Ho, &pt, &pb)) return 2;
+    if (!window_geometry(W, fw, sw, 1, pad_mode, &Wo, &pl, &pr)) return 2;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t n = 0; n < N; ++n) {
+        for (int oy = 0; oy < Ho; ++oy) {
+            for (int ox = 0; ox < Wo; ++ox) {
+                for (int c = 0; c < C; ++c) {
+                    float m = -std::numeric_limits<float>::infinity();
+                    for (int ky = 0; ky < fh; ++ky) {
+                        const int iy = oy * sh - pt + ky;
+                        if (iy < 0 || iy >= H) continue;
+                        for (int kx = 0; kx < fw; ++kx) {
+                            const int ix = ox * sw - pl + kx;
+                            if (ix < 0 || ix >= W) continue;
+                            const float v = x[((n * H + iy) * (int64_t)W + ix) * C + c];
+                            if (v > m || v != v) m = v;  // once m is NaN no comparison replaces it
+                        }
+                    }
+                    y[((n * Ho + oy) * (int64_t)Wo + ox) * C + c] = m;
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+// Elementwise binary op of Sec. 4.1 (the addition shader of Fig. 3 computes one output value per
+// invocation): out[i] = a[i] op b[i % b_len], one fp32 operation per element.  b_len = n: same
+// shapes; b_len = the last dimension: b is a vector broadcast along every other dimension.
+// op: 0 add, 1 subtract, 2 multiply.
+int orc_binary(int op, const float* a, const float* b, int64_t n, int64_t b_len, float* out) {
+    if (!a || !b || !out || b_len < 1 || op < 0 || op > 2) return 1;
+    for (int64_t i = 0; i < n; ++i) {
+        const float u = a[i], v = b[i % b_len];
+        out[i] = op == 0 ? u + v : (op == 1 ? u - v : u * v);
+    }
+    return 0;
+}
+
 // p[r, j] = exp(x[r,j] - max_r) / sum_k exp(x[r,k] - max_r), over the last dimension.
 int orc_softmax(const float* x, int64_t rows, int64_t cols, float* y) {
     if (!x || !y || cols < 1) return 1;

@@ -415,6 +415,65 @@ def test_avg_pool_asymmetric_same_padding_divisor(oracle):
     assert y[0, 0, 1, 0] == np.float32(x[0, 0:3, 2:4, 0].mean())
 
 
+# ------------------------------------------------------------------ maxPool, elementwise binary ops, rank-3 matMul
+@pytest.mark.parametrize("H,W,k,s,pad", [(7, 7, 7, 1, "valid"), (8, 6, 2, 2, "valid"), (7, 7, 3, 1, "same"),
+                                         (9, 9, 3, 2, "same"), (8, 8, 3, 2, "same"), (6, 5, 3, 1, "valid")])
+def test_max_pool_matches_library_pooling_on_explicitly_padded_input(oracle, H, W, k, s, pad):
+    x = si.uniform(53, 0, (2, H, W, 3), -1, 1)
+    got = oracle.max_pool(x, (k, k), (s, s), pad)
+    xt = torch.from_numpy(x).permute(0, 3, 1, 2)
+    if pad == "same":  # TF padding built by hand (extra element after), filled with -inf so it never wins
+        _, pt, pb = oracle.window_geometry(H, k, s, 1, pad)
+        _, pl, pr = oracle.window_geometry(W, k, s, 1, pad)
+        xt = F.pad(xt, (pl, pr, pt, pb), value=float("-inf"))
+    want = F.max_pool2d(xt, k, s).permute(0, 2, 3, 1).numpy()
+    assert got.shape == want.shape
+    assert np.array_equal(got, want)  # a selection: exact
+
+
+def test_max_pool_hand_values_asymmetric_padding_and_nan(oracle):
+    # in=4, k=3, s=2, 'same': out=2, pad 0 before / 1 after
+    x = np.arange(16, dtype=np.float32).reshape(1, 4, 4, 1)
+    y = oracle.max_pool(x, (3, 3), (2, 2), "same")
+    assert y[0, :, :, 0].tolist() == [[10.0, 11.0], [14.0, 15.0]]
+    neg = -np.abs(si.uniform(54, 0, (1, 5, 5, 2), 1, 2))          # all negative: zero padding would win wrongly
+    assert oracle.max_pool(neg, (3, 3), (1, 1), "same").max() < 0
+    x[0, 3, 3, 0] = np.nan                                         # a NaN wins its windows and no other
+    y = oracle.max_pool(x, (3, 3), (2, 2), "same")
+    assert np.isnan(y[0, 1, 1, 0]) and y[0, 0, 0, 0] == 10.0 and y[0, 0, 1, 0] == 11.0 and y[0, 1, 0, 0] == 14.0
+    assert np.array_equal(oracle.max_pool(x[:, :3, :3], (1, 1), (1, 1), "valid"), x[:, :3, :3])  # 1x1 window: identity
+
+
+@pytest.mark.parametrize("op,fn", [("add", np.add), ("sub", np.subtract), ("mul", np.multiply)])
+def test_binary_ops_are_one_fp32_operation_per_element(oracle, op, fn):
+    a = si.normal(55, 0, (3, 5, 7, 6), 0, 10)
+    b = si.normal(55, 1, (3, 5, 7, 6), 0, 10)
+    assert np.array_equal(oracle.binary(op, a, b), fn(a, b))                    # numpy fp32: the same single rounding
+    v = si.normal(55, 2, (6,), 0, 10)
+    assert np.array_equal(oracle.binary(op, a, v), fn(a, v[None, None, None, :]))  # vector along the last dimension
+    exact = fn(a.astype(np.float64), b.astype(np.float64))
+    assert np.all(np.abs(oracle.binary(op, a, b) - exact) <= np.spacing(np.abs(exact).astype(np.float32)) / 2 + 0)
+    assert np.array_equal(oracle.binary("add", a, np.zeros_like(a)), a)
+    assert np.array_equal(oracle.binary("mul", a, np.ones(6, np.float32)), a)
+    assert np.array_equal(oracle.binary("sub", a, a), np.zeros_like(a))
+
+
+def test_batch_matmul_is_one_product_per_leading_index(oracle):
+    a = si.uniform(56, 0, (4, 9, 13), -1, 1)
+    b = si.uniform(56, 1, (4, 13, 5), -1, 1)
+    got = oracle.batch_matmul(a, b)
+    want = np.einsum("bik,bkj->bij", a.astype(np.float64), b.astype(np.float64))
+    assert got.shape == (4, 9, 5)
+    np.testing.assert_allclose(got, want, rtol=0, atol=2e-7 * 13)
+    ai = si.small_integers(57, 0, (3, 6, 8), -8, 8)
+    bi = si.small_integers(57, 1, (3, 7, 8), -8, 8)
+    want_i = np.einsum("bik,bjk->bij", ai.astype(np.int64), bi.astype(np.int64)).astype(np.float32)
+    assert np.array_equal(oracle.batch_matmul(ai, bi, transpose_b=True), want_i)
+    # a product must not see its neighbours: permuting the leading index permutes the result
+    perm = [2, 0, 3, 1]
+    assert np.array_equal(oracle.batch_matmul(a[perm], b[perm]), got[perm])
+
+
 # ------------------------------------------------------------------ softmax
 def test_softmax_invariants_and_library(oracle):
     from scipy.special import softmax as sp_softmax
