@@ -66,6 +66,7 @@ typedef enum { TFJSB_ACT_NONE = 0, TFJSB_ACT_RELU = 1, TFJSB_ACT_RELU6 = 2 } tfj
  *         wherever the shape allows, CUDA cores otherwise.  Default.
  *   FP32  CUDA-core FFMA everywhere: the variant kept for exactness checks. */
 typedef enum { TFJSB_MATH_TF32 = 0, TFJSB_MATH_FP32 = 1 } tfjsb_math;
+typedef enum { TFJSB_BINARY_ADD = 0, TFJSB_BINARY_SUB = 1, TFJSB_BINARY_MUL = 2 } tfjsb_binary_op;
 
 /* ---- context ------------------------------------------------------------------------ */
 
@@ -150,6 +151,28 @@ tfjsb_status tfjsb_depthwise_conv2d(tfjsb_ctx* ctx, const tfjsb_tensor* x, const
  * window elements divided by their number (padding never counts). */
 tfjsb_status tfjsb_avg_pool(tfjsb_ctx* ctx, const tfjsb_tensor* x, const int filter_size[2], const int strides[2],
                             tfjsb_pad pad, tfjsb_tensor* out, void* stream);
+
+/* tf.maxPool.  x [N,H,W,C] -> out [N,Ho,Wo,C]; each output is the largest in-bounds window element
+ * (padding never takes part; a NaN in the window gives NaN).  Not defined in the paper: TensorFlow's
+ * definition, with the window geometry of tfjsb_window_out_shape. */
+tfjsb_status tfjsb_max_pool(tfjsb_ctx* ctx, const tfjsb_tensor* x, const int filter_size[2], const int strides[2],
+                            tfjsb_pad pad, tfjsb_tensor* out, void* stream);
+
+/* tf.add / tf.sub / tf.mul: out = a op b, elementwise (the addition shader of Fig. 3, Sec. 4.1, computes
+ * one output value per invocation; here one per thread, four per thread when the sizes allow).
+ * a, out: rank 1..4, same shape.  b: a's shape, or a rank-1 vector of a's last dimension, broadcast
+ * along every other dimension.  One fp32 operation per element, rounded to nearest: exact parity with
+ * any IEEE implementation.  `out` may not alias an input. */
+tfjsb_status tfjsb_binary(tfjsb_ctx* ctx, tfjsb_binary_op op, const tfjsb_tensor* a, const tfjsb_tensor* b,
+                          tfjsb_tensor* out, void* stream);
+
+/* tf.matMul on rank-3 tensors (Sec. 3.3 names the op; Listing 2 prints the rank-2 case): one rank-2
+ * product per leading index.  a [B,M,K] (or [B,K,M] if transpose_a), b [B,K,N] (or [B,N,K] if
+ * transpose_b), out [B,M,N].  Each product takes the same kernels, math mode and tolerances as
+ * tfjsb_matmul; products whose slices are not 16-byte aligned (M*K, K*N or M*N not a multiple of 4)
+ * run on the CUDA-core fp32 kernel. */
+tfjsb_status tfjsb_batch_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_tensor* b, int transpose_a,
+                                int transpose_b, tfjsb_tensor* out, void* stream);
 
 /* tf.softmax over the last dimension of a rank 1..4 tensor:
  *   out[..., j] = exp(x[..., j] - max_j x) / sum_k exp(x[..., k] - max_j x). */

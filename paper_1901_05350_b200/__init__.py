@@ -22,13 +22,14 @@ from . import build as _build
 PAD = {"valid": 0, "same": 1}
 ACT = {"none": 0, "relu": 1, "relu6": 2}
 MATH = {"tf32": 0, "fp32": 1}
+BINARY_OP = {"add": 0, "sub": 1, "mul": 2}
 LAYER_KIND = {"conv2d": 0, "depthwise_conv2d": 1, "avg_pool": 2, "global_avg_pool": 2, "dense": 3, "softmax": 4}
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "UNSUPPORTED", 4: "CUDA", 5: "TIMEOUT", 6: "OOM"}
 
 EXPORTS = [
     "tfjsb_init", "tfjsb_shutdown", "tfjsb_set_math", "tfjsb_last_error", "tfjsb_check_device_status",
-    "tfjsb_launch_count", "tfjsb_window_out_shape", "tfjsb_matmul", "tfjsb_matmul_static_scratch", "tfjsb_conv2d", "tfjsb_depthwise_conv2d",
+    "tfjsb_launch_count", "tfjsb_window_out_shape", "tfjsb_matmul", "tfjsb_batch_matmul", "tfjsb_max_pool", "tfjsb_binary", "tfjsb_matmul_static_scratch", "tfjsb_conv2d", "tfjsb_depthwise_conv2d",
     "tfjsb_avg_pool", "tfjsb_softmax", "tfjsb_bias_act", "tfjsb_model_create", "tfjsb_model_destroy",
     "tfjsb_model_output_shape", "tfjsb_model_launches_per_run", "tfjsb_run_model", "tfjsb_run_model_host",
     "tfjsb_run_model_host_async", "tfjsb_model_host_wait",
@@ -80,6 +81,9 @@ def _load_library() -> ctypes.CDLL:
     lib.tfjsb_window_out_shape.argtypes = [i64, i32, i32, i32, i32, ctypes.POINTER(i64), ip, ip]
     lib.tfjsb_matmul.argtypes = [vp, tp, tp, i32, i32, tp, vp]
     lib.tfjsb_matmul_static_scratch.argtypes = [vp, tp, tp, i32, i32, tp, vp]
+    lib.tfjsb_batch_matmul.argtypes = [vp, tp, tp, i32, i32, tp, vp]
+    lib.tfjsb_max_pool.argtypes = [vp, tp, ip, ip, i32, tp, vp]
+    lib.tfjsb_binary.argtypes = [vp, i32, tp, tp, tp, vp]
     lib.tfjsb_conv2d.argtypes = [vp, tp, tp, ip, i32, ip, tp, i32, tp, vp]
     lib.tfjsb_depthwise_conv2d.argtypes = [vp, tp, tp, ip, i32, ip, tp, i32, tp, vp]
     lib.tfjsb_avg_pool.argtypes = [vp, tp, ip, ip, i32, tp, vp]
@@ -230,6 +234,27 @@ class Context:
             out = self._conv_out(x, filter_size[0], filter_size[1], strides, pad, (1, 1), x.shape[3])
         self._check(lib.tfjsb_avg_pool(self._h, _desc(x), _int2(filter_size), _int2(strides), PAD[pad], _desc(out),
                                        _stream()))
+        return out
+
+    def max_pool(self, x, filter_size, strides, pad="valid", out=None):
+        if out is None:
+            out = self._conv_out(x, filter_size[0], filter_size[1], strides, pad, (1, 1), x.shape[3])
+        self._check(lib.tfjsb_max_pool(self._h, _desc(x), _int2(filter_size), _int2(strides), PAD[pad], _desc(out),
+                                       _stream()))
+        return out
+
+    def binary(self, op: str, a, b, out=None):
+        """a op b elementwise, op in 'add' / 'sub' / 'mul'; b has a's shape or is a vector of a's last dimension."""
+        out = self._empty(a.shape) if out is None else out
+        self._check(lib.tfjsb_binary(self._h, BINARY_OP[op], _desc(a), _desc(b), _desc(out), _stream()))
+        return out
+
+    def batch_matmul(self, a, b, transpose_a: bool = False, transpose_b: bool = False, out=None):
+        M = a.shape[2] if transpose_a else a.shape[1]
+        N = b.shape[1] if transpose_b else b.shape[2]
+        out = self._empty((a.shape[0], M, N)) if out is None else out
+        self._check(lib.tfjsb_batch_matmul(self._h, _desc(a), _desc(b), int(transpose_a), int(transpose_b), _desc(out),
+                                           _stream()))
         return out
 
     def softmax(self, logits, out=None):

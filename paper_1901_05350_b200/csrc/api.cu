@@ -235,30 +235,15 @@ tfjsb_status tfjsb_window_out_shape(int64_t in, int k, int stride, int dilation,
     return TFJSB_OK;
 }
 
-tfjsb_status tfjsb_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_tensor* b, int transpose_a,
-                          int transpose_b, tfjsb_tensor* out, void* stream) {
-    TFJSB_REQUIRE_CTX(ctx);
+// One rank-2 product C[M,N] = op(A) op(B) on device pointers (arguments already validated): the tensor
+// cores when the math mode, the shape and the alignment of the pointers allow, else the CUDA-core kernel.
+static tfjsb_status matmul_2d(tfjsb_ctx* ctx, const float* pa, const float* pb, float* pc, int64_t M, int64_t K, int64_t N,
+                              int transpose_a, int transpose_b, cudaStream_t s) {
     tfjsb_status st;
-    if ((st = check_tensor(ctx, a, "a", 2, 2)) != TFJSB_OK) return st;
-    if ((st = check_tensor(ctx, b, "b", 2, 2)) != TFJSB_OK) return st;
-    if ((st = check_tensor(ctx, out, "out", 2, 2)) != TFJSB_OK) return st;
-    const int64_t M = transpose_a ? a->dims[1] : a->dims[0];
-    const int64_t K = transpose_a ? a->dims[0] : a->dims[1];
-    const int64_t Kb = transpose_b ? b->dims[1] : b->dims[0];
-    const int64_t N = transpose_b ? b->dims[0] : b->dims[1];
-    if (K != Kb)
-        return fail(ctx, TFJSB_ERR_SHAPE, "inner dimensions differ: " + std::to_string(K) + " vs " + std::to_string(Kb));
-    if (out->dims[0] != M || out->dims[1] != N)
-        return fail(ctx, TFJSB_ERR_SHAPE, "out must be [" + std::to_string(M) + "," + std::to_string(N) + "]");
-    if (overlaps(out, a) || overlaps(out, b)) return fail(ctx, TFJSB_ERR_INVALID_ARG, "out aliases an input");
-    if (M == 0 || N == 0) return TFJSB_OK;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const float* pa = static_cast<const float*>(a->data);
-    const float* pb = static_cast<const float*>(b->data);
-    float* pc = static_cast<float*>(out->data);
     cudaError_t e;
 
-    if (ctx->math == TFJSB_MATH_TF32 && gemm_tf32_supported(M, N, K) && ctx->encode_tiled) {
+    if (ctx->math == TFJSB_MATH_TF32 && gemm_tf32_supported(M, N, K) && ctx->encode_tiled && aligned16(pa) && aligned16(pb) &&
+        aligned16(pc)) {
         // make both operands K-contiguous: A as [M,K], B as [N,K]
         const float* a_km = pa;
         const float* b_km = pb;
@@ -285,6 +270,58 @@ tfjsb_status tfjsb_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_ten
     if ((e = launch_gemm_fp32(pa, a_rs, a_cs, pb, b_rs, b_cs, nullptr, TFJSB_ACT_NONE, pc, N, M, N, K, s,
                               &ctx->launches)) != cudaSuccess)
         return cuda_fail(ctx, e, "fp32 gemm launch");
+    return TFJSB_OK;
+}
+
+
+tfjsb_status tfjsb_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_tensor* b, int transpose_a,
+                          int transpose_b, tfjsb_tensor* out, void* stream) {
+    TFJSB_REQUIRE_CTX(ctx);
+    tfjsb_status st;
+    if ((st = check_tensor(ctx, a, "a", 2, 2)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, b, "b", 2, 2)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, out, "out", 2, 2)) != TFJSB_OK) return st;
+    const int64_t M = transpose_a ? a->dims[1] : a->dims[0];
+    const int64_t K = transpose_a ? a->dims[0] : a->dims[1];
+    const int64_t Kb = transpose_b ? b->dims[1] : b->dims[0];
+    const int64_t N = transpose_b ? b->dims[0] : b->dims[1];
+    if (K != Kb)
+        return fail(ctx, TFJSB_ERR_SHAPE, "inner dimensions differ: " + std::to_string(K) + " vs " + std::to_string(Kb));
+    if (out->dims[0] != M || out->dims[1] != N)
+        return fail(ctx, TFJSB_ERR_SHAPE, "out must be [" + std::to_string(M) + "," + std::to_string(N) + "]");
+    if (overlaps(out, a) || overlaps(out, b)) return fail(ctx, TFJSB_ERR_INVALID_ARG, "out aliases an input");
+    if (M == 0 || N == 0) return TFJSB_OK;
+    return matmul_2d(ctx, static_cast<const float*>(a->data), static_cast<const float*>(b->data),
+                     static_cast<float*>(out->data), M, K, N, transpose_a, transpose_b, static_cast<cudaStream_t>(stream));
+}
+
+tfjsb_status tfjsb_batch_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_tensor* b, int transpose_a,
+                                int transpose_b, tfjsb_tensor* out, void* stream) {
+    TFJSB_REQUIRE_CTX(ctx);
+    tfjsb_status st;
+    if ((st = check_tensor(ctx, a, "a", 3, 3)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, b, "b", 3, 3)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, out, "out", 3, 3)) != TFJSB_OK) return st;
+    const int64_t B = a->dims[0];
+    if (b->dims[0] != B || out->dims[0] != B) return fail(ctx, TFJSB_ERR_SHAPE, "leading dimensions differ");
+    const int64_t M = transpose_a ? a->dims[2] : a->dims[1];
+    const int64_t K = transpose_a ? a->dims[1] : a->dims[2];
+    const int64_t Kb = transpose_b ? b->dims[2] : b->dims[1];
+    const int64_t N = transpose_b ? b->dims[1] : b->dims[2];
+    if (K != Kb)
+        return fail(ctx, TFJSB_ERR_SHAPE, "inner dimensions differ: " + std::to_string(K) + " vs " + std::to_string(Kb));
+    if (out->dims[1] != M || out->dims[2] != N)
+        return fail(ctx, TFJSB_ERR_SHAPE, "out must be [B," + std::to_string(M) + "," + std::to_string(N) + "]");
+    if (overlaps(out, a) || overlaps(out, b)) return fail(ctx, TFJSB_ERR_INVALID_ARG, "out aliases an input");
+    if (B == 0 || M == 0 || N == 0) return TFJSB_OK;
+    const float* pa = static_cast<const float*>(a->data);
+    const float* pb = static_cast<const float*>(b->data);
+    float* pc = static_cast<float*>(out->data);
+    for (int64_t i = 0; i < B; ++i) {
+        st = matmul_2d(ctx, pa + i * M * K, pb + i * K * N, pc + i * M * N, M, K, N, transpose_a, transpose_b,
+                       static_cast<cudaStream_t>(stream));
+        if (st != TFJSB_OK) return st;
+    }
     return TFJSB_OK;
 }
 
@@ -408,6 +445,50 @@ tfjsb_status tfjsb_avg_pool(tfjsb_ctx* ctx, const tfjsb_tensor* x, const int fil
     cudaError_t e = launch_avg_pool(static_cast<const float*>(x->data), static_cast<float*>(out->data), g,
                                     static_cast<cudaStream_t>(stream), &ctx->launches);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "avg_pool launch");
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_max_pool(tfjsb_ctx* ctx, const tfjsb_tensor* x, const int filter_size[2], const int strides[2],
+                            tfjsb_pad pad, tfjsb_tensor* out, void* stream) {
+    TFJSB_REQUIRE_CTX(ctx);
+    tfjsb_status st;
+    if ((st = check_tensor(ctx, x, "x", 4, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, out, "out", 4, 4)) != TFJSB_OK) return st;
+    if (!filter_size) return fail(ctx, TFJSB_ERR_INVALID_ARG, "filter_size is null");
+    const int ones[2] = {1, 1};
+    ConvGeom g;
+    if ((st = conv_geometry(ctx, x, filter_size[0], filter_size[1], strides, pad, ones, x->dims[3], out, &g)) != TFJSB_OK)
+        return st;
+    if (overlaps(out, x)) return fail(ctx, TFJSB_ERR_INVALID_ARG, "out aliases an input");
+    if (numel(out) == 0) return TFJSB_OK;
+    cudaError_t e = launch_max_pool(static_cast<const float*>(x->data), static_cast<float*>(out->data), g,
+                                    static_cast<cudaStream_t>(stream), &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "max_pool launch");
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_binary(tfjsb_ctx* ctx, tfjsb_binary_op op, const tfjsb_tensor* a, const tfjsb_tensor* b,
+                          tfjsb_tensor* out, void* stream) {
+    TFJSB_REQUIRE_CTX(ctx);
+    tfjsb_status st;
+    if (op != TFJSB_BINARY_ADD && op != TFJSB_BINARY_SUB && op != TFJSB_BINARY_MUL)
+        return fail(ctx, TFJSB_ERR_INVALID_ARG, "unknown binary op");
+    if ((st = check_tensor(ctx, a, "a", 1, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, b, "b", 1, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, out, "out", 1, 4)) != TFJSB_OK) return st;
+    bool out_ok = out->rank == a->rank;
+    for (int i = 0; out_ok && i < a->rank; ++i) out_ok = out->dims[i] == a->dims[i];
+    if (!out_ok) return fail(ctx, TFJSB_ERR_SHAPE, "out must have the shape of a");
+    bool same = b->rank == a->rank;
+    for (int i = 0; same && i < a->rank; ++i) same = b->dims[i] == a->dims[i];
+    const bool vector = b->rank == 1 && b->dims[0] == a->dims[a->rank - 1];
+    if (!same && !vector) return fail(ctx, TFJSB_ERR_SHAPE, "b must have a's shape or be a vector of a's last dimension");
+    if (overlaps(out, a) || overlaps(out, b)) return fail(ctx, TFJSB_ERR_INVALID_ARG, "out aliases an input");
+    if (numel(a) == 0) return TFJSB_OK;
+    cudaError_t e = launch_binary(op, static_cast<const float*>(a->data), static_cast<const float*>(b->data),
+                                  static_cast<float*>(out->data), numel(a), numel(b), static_cast<cudaStream_t>(stream),
+                                  &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "binary op launch");
     return TFJSB_OK;
 }
 

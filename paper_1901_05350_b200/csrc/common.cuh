@@ -135,6 +135,10 @@ cudaError_t launch_bias_act(const float* x, const float* bias, float* y, int64_t
                             cudaStream_t s, int64_t* launches);
 cudaError_t launch_avg_pool(const float* x, float* y, const ConvGeom& g, cudaStream_t s, int64_t* launches);
 cudaError_t launch_softmax(const float* x, float* y, int64_t rows, int64_t cols, cudaStream_t s, int64_t* launches);
+cudaError_t launch_max_pool(const float* x, float* y, const ConvGeom& g, cudaStream_t s, int64_t* launches);
+// out[i] = a[i] op b[i % b_len] (op: tfjsb_binary_op)
+cudaError_t launch_binary(int op, const float* a, const float* b, float* out, int64_t n, int64_t b_len, cudaStream_t s,
+                          int64_t* launches);
 // out[c, r] = in[r, c] for in of shape [rows, cols]
 cudaError_t launch_transpose(const float* in, float* out, int64_t rows, int64_t cols, cudaStream_t s,
                              int64_t* launches);

@@ -71,6 +71,58 @@ __global__ void avg_pool_window_kernel(const float* __restrict__ x, float* __res
     }
 }
 
+// ---- maxPool ----------------------------------------------------------------------------------
+// One thread per output element, channel fastest (coalesced).  Padding never takes part; max.NaN keeps
+// a NaN that is in the window.
+__global__ void max_pool_window_kernel(const float* __restrict__ x, float* __restrict__ y, ConvGeom g,
+                                       int64_t n_out) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_out; i += stride) {
+        const int c = (int)(i % g.C);
+        int64_t t = i / g.C;
+        const int ox = (int)(t % g.Wo); t /= g.Wo;
+        const int oy = (int)(t % g.Ho);
+        const int64_t n = t / g.Ho;
+        float m = __int_as_float(0xff800000);  // -inf
+        for (int ky = 0; ky < g.fh; ++ky) {
+            const int iy = oy * g.sh - g.pt + ky;
+            if (iy < 0 || iy >= g.H) continue;
+            for (int kx = 0; kx < g.fw; ++kx) {
+                const int ix = ox * g.sw - g.pl + kx;
+                if (ix < 0 || ix >= g.W) continue;
+                const float v = x[((n * g.H + iy) * (int64_t)g.W + ix) * g.C + c];
+                asm("max.NaN.f32 %0, %0, %1;" : "+f"(m) : "f"(v));
+            }
+        }
+        y[i] = m;
+    }
+}
+
+// ---- elementwise binary ops (the addition shader of the paper's Fig. 3: one output value per thread) ----
+// out[i] = a[i] op b[i % b_len]; OP 0 add, 1 subtract, 2 multiply: one fp32 operation, so bit-exact.
+template <int OP>
+__device__ __forceinline__ float binary_op(float u, float v) {
+    return OP == 0 ? __fadd_rn(u, v) : (OP == 1 ? __fsub_rn(u, v) : __fmul_rn(u, v));
+}
+// float4 path: n and b_len multiples of 4 (a float4 never straddles a period of b)
+template <int OP>
+__global__ void binary_vec4_kernel(const float4* __restrict__ a, const float4* __restrict__ b, float4* __restrict__ out,
+                                   int64_t n4, int64_t b_len4) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        const float4 u = a[i];
+        const float4 v = b_len4 == n4 ? b[i] : __ldg(b + i % b_len4);
+        out[i] = make_float4(binary_op<OP>(u.x, v.x), binary_op<OP>(u.y, v.y), binary_op<OP>(u.z, v.z), binary_op<OP>(u.w, v.w));
+    }
+}
+template <int OP>
+__global__ void binary_scalar_kernel(const float* __restrict__ a, const float* __restrict__ b, float* __restrict__ out,
+                                     int64_t n, int64_t b_len) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+        out[i] = binary_op<OP>(a[i], b[i % b_len]);
+}
+
 // Global pool: a block owns (image n, 128 consecutive channels).  Lane = 4 channels (one float4, so a
 // warp reads 512 contiguous bytes per position), the 8 warps stride over the H*W positions, partial
 // sums meet in shared memory.  C % 4 == 0.
@@ -84,7 +136,16 @@ __global__ void avg_pool_global_vec4_kernel(const float* __restrict__ x, float* 
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     if (c < C) {
         const float* base = x + n * (int64_t)HW * C + c;
-        for (int p = warp; p < HW; p += 8) {
+        // four loads in flight per thread (the sum order stays p ascending)
+        int p = warp;
+        for (; p + 24 < HW; p += 32) {
+            float4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const float4*>(base + (int64_t)(p + 8 * u) * C);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { acc.x += v[u].x; acc.y += v[u].y; acc.z += v[u].z; acc.w += v[u].w; }
+        }
+        for (; p < HW; p += 8) {
             const float4 v = *reinterpret_cast<const float4*>(base + (int64_t)p * C);
             acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
         }
@@ -252,6 +313,33 @@ cudaError_t launch_avg_pool(const float* x, float* y, const ConvGeom& g, cudaStr
     }
     ++*launches;
     return cudaGetLastError();
+}
+
+cudaError_t launch_max_pool(const float* x, float* y, const ConvGeom& g, cudaStream_t s, int64_t* launches) {
+    const int64_t n_out = g.N * g.Ho * g.Wo * g.C;
+    if (n_out == 0) return cudaSuccess;
+    max_pool_window_kernel<<<grid_for(n_out, kThreads, 148 * 16), kThreads, 0, s>>>(x, y, g, n_out);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+template <int OP>
+static cudaError_t launch_binary_op(const float* a, const float* b, float* out, int64_t n, int64_t b_len, cudaStream_t s) {
+    if (n % 4 == 0 && b_len % 4 == 0)
+        binary_vec4_kernel<OP><<<grid_for(n / 4, kThreads, 148 * 16), kThreads, 0, s>>>(
+            reinterpret_cast<const float4*>(a), reinterpret_cast<const float4*>(b), reinterpret_cast<float4*>(out), n / 4, b_len / 4);
+    else
+        binary_scalar_kernel<OP><<<grid_for(n, kThreads, 148 * 16), kThreads, 0, s>>>(a, b, out, n, b_len);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_binary(int op, const float* a, const float* b, float* out, int64_t n, int64_t b_len, cudaStream_t s,
+                          int64_t* launches) {
+    if (n == 0) return cudaSuccess;
+    ++*launches;
+    if (op == TFJSB_BINARY_ADD) return launch_binary_op<0>(a, b, out, n, b_len, s);
+    if (op == TFJSB_BINARY_SUB) return launch_binary_op<1>(a, b, out, n, b_len, s);
+    return launch_binary_op<2>(a, b, out, n, b_len, s);
 }
 
 cudaError_t launch_softmax(const float* x, float* y, int64_t rows, int64_t cols, cudaStream_t s,

@@ -5,6 +5,9 @@
     python -m paper_1901_05350_b200.run_workload --workload block --batch 32 --steps 3
     python -m paper_1901_05350_b200.run_workload --workload depthwise --batch 128 --hw 14 --channels 512 --stride 1
     python -m paper_1901_05350_b200.run_workload --workload pointwise --batch 128 --hw 14 --channels 512 --cout 512
+    python -m paper_1901_05350_b200.run_workload --workload maxpool --batch 128 --hw 112 --channels 64 --stride 2
+    python -m paper_1901_05350_b200.run_workload --workload add --batch 128 --hw 56 --channels 128
+    python -m paper_1901_05350_b200.run_workload --workload batch_matmul --batch 16 --size 1024
 
 A plain driver for profilers and quick timing: it builds the inputs, runs `--warmup` untimed and
 `--steps` timed passes on one stream, prints the mean device time per pass, and exits.
@@ -20,7 +23,8 @@ sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
 
 def main() -> int:
     ap = argparse.ArgumentParser()
-    ap.add_argument("--workload", choices=["mobilenet224", "mobilenet128_025", "matmul", "block", "depthwise", "pointwise"],
+    ap.add_argument("--workload", choices=["mobilenet224", "mobilenet128_025", "matmul", "block", "depthwise", "pointwise", "maxpool", "add",
+                             "batch_matmul"],
                     default="mobilenet224")
     ap.add_argument("--batch", type=int, default=128)
     ap.add_argument("--size", type=int, default=512, help="matmul: M = K = N")
@@ -55,6 +59,22 @@ def main() -> int:
         def step():
             ctx.depthwise_conv2d(x, wd, dw.strides, dw.pad, dw.dilations, bd, dw.act, out=mid)
             ctx.conv2d(mid, wp, pw.strides, pw.pad, pw.dilations, bp, pw.act, out=out)
+    elif args.workload == "batch_matmul":
+        a = torch.from_numpy(si.uniform(7, 0, (args.batch, args.size, args.size), -1.0, 1.0)).cuda()
+        b = torch.from_numpy(si.uniform(7, 1, (args.batch, args.size, args.size), -1.0, 1.0)).cuda()
+        out = torch.empty(args.batch, args.size, args.size, device="cuda")
+        step = lambda: ctx.batch_matmul(a, b, False, True, out=out)  # b given K-contiguous: no transpose pass
+    elif args.workload in ("maxpool", "add"):
+        x = torch.from_numpy(si.uniform(7, 0, (args.batch, args.hw, args.hw, args.channels), -1.0, 1.0)).cuda()
+        if args.workload == "maxpool":
+            strides = (args.stride, args.stride)
+            out = ctx.max_pool(x, (3, 3), strides, "same")
+            step = lambda: ctx.max_pool(x, (3, 3), strides, "same", out=out)
+        else:
+            y = torch.from_numpy(si.uniform(7, 1, x.shape, -1.0, 1.0)).cuda()
+            out = torch.empty_like(x)
+            step = lambda: ctx.binary("add", x, y, out=out)
+        print(f"{args.workload}: {x.numel() * 4 / 1e6:.1f} MB in per operand, {out.numel() * 4 / 1e6:.1f} MB out")
     elif args.workload in ("depthwise", "pointwise"):
         x = torch.from_numpy(si.uniform(7, 0, (args.batch, args.hw, args.hw, args.channels), 0.0, 6.0)).cuda()
         if args.workload == "depthwise":
