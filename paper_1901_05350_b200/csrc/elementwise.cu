@@ -98,6 +98,36 @@ __global__ void max_pool_window_kernel(const float* __restrict__ x, float* __res
     }
 }
 
+// The same with four channels per thread (C % 4 == 0): one 16-byte load per window element, a warp
+// reads 512 contiguous bytes per tap; neighbouring outputs' windows overlap in L1/L2.
+__device__ __forceinline__ void max4_nan(float4& m, const float4& v) {
+    asm("max.NaN.f32 %0, %0, %1;" : "+f"(m.x) : "f"(v.x));
+    asm("max.NaN.f32 %0, %0, %1;" : "+f"(m.y) : "f"(v.y));
+    asm("max.NaN.f32 %0, %0, %1;" : "+f"(m.z) : "f"(v.z));
+    asm("max.NaN.f32 %0, %0, %1;" : "+f"(m.w) : "f"(v.w));
+}
+__global__ void max_pool_vec4_kernel(const float* __restrict__ x, float* __restrict__ y, ConvGeom g, int64_t n_out4) {
+    const int C4 = g.C >> 2;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_out4; i += stride) {
+        const int c = (int)(i % C4) * 4;
+        int64_t t = i / C4;
+        const int ox = (int)(t % g.Wo); t /= g.Wo;
+        const int oy = (int)(t % g.Ho);
+        const int64_t n = t / g.Ho;
+        const float ninf = __int_as_float(0xff800000);
+        float4 m = make_float4(ninf, ninf, ninf, ninf);
+        const int iy0 = oy * g.sh - g.pt, ix0 = ox * g.sw - g.pl;
+        const int ky0 = iy0 < 0 ? -iy0 : 0, ky1 = min(g.fh, g.H - iy0);
+        const int kx0 = ix0 < 0 ? -ix0 : 0, kx1 = min(g.fw, g.W - ix0);
+        for (int ky = ky0; ky < ky1; ++ky) {
+            const float* row = x + ((n * g.H + iy0 + ky) * (int64_t)g.W + ix0) * g.C + c;
+            for (int kx = kx0; kx < kx1; ++kx) max4_nan(m, __ldg(reinterpret_cast<const float4*>(row + (int64_t)kx * g.C)));
+        }
+        *reinterpret_cast<float4*>(y + i * 4) = m;
+    }
+}
+
 // ---- elementwise binary ops (the addition shader of the paper's Fig. 3: one output value per thread) ----
 // out[i] = a[i] op b[i % b_len]; OP 0 add, 1 subtract, 2 multiply: one fp32 operation, so bit-exact.
 template <int OP>
@@ -318,7 +348,10 @@ cudaError_t launch_avg_pool(const float* x, float* y, const ConvGeom& g, cudaStr
 cudaError_t launch_max_pool(const float* x, float* y, const ConvGeom& g, cudaStream_t s, int64_t* launches) {
     const int64_t n_out = g.N * g.Ho * g.Wo * g.C;
     if (n_out == 0) return cudaSuccess;
-    max_pool_window_kernel<<<grid_for(n_out, kThreads, 148 * 16), kThreads, 0, s>>>(x, y, g, n_out);
+    if (g.C % 4 == 0)
+        max_pool_vec4_kernel<<<grid_for(n_out / 4, kThreads, 148 * 32), kThreads, 0, s>>>(x, y, g, n_out / 4);
+    else
+        max_pool_window_kernel<<<grid_for(n_out, kThreads, 148 * 16), kThreads, 0, s>>>(x, y, g, n_out);
     ++*launches;
     return cudaGetLastError();
 }
