@@ -168,9 +168,10 @@ tfjsb_status tfjsb_binary(tfjsb_ctx* ctx, tfjsb_binary_op op, const tfjsb_tensor
 
 /* tf.matMul on rank-3 tensors (Sec. 3.3 names the op; Listing 2 prints the rank-2 case): one rank-2
  * product per leading index.  a [B,M,K] (or [B,K,M] if transpose_a), b [B,K,N] (or [B,N,K] if
- * transpose_b), out [B,M,N].  Each product takes the same kernels, math mode and tolerances as
- * tfjsb_matmul; products whose slices are not 16-byte aligned (M*K, K*N or M*N not a multiple of 4)
- * run on the CUDA-core fp32 kernel. */
+ * transpose_b), out [B,M,N].  Same math mode and tolerances as tfjsb_matmul.  With K and N multiples
+ * of 4 all B products run as ONE launch of the tensor-core kernel (the batch is a third dimension of
+ * its tensor maps, tile = (product, rows, columns)); otherwise each product runs on its own, on the
+ * CUDA-core fp32 kernel where its slices are not 16-byte aligned. */
 tfjsb_status tfjsb_batch_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_tensor* b, int transpose_a,
                                 int transpose_b, tfjsb_tensor* out, void* stream);
 

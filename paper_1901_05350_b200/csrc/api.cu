@@ -317,6 +317,33 @@ tfjsb_status tfjsb_batch_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfj
     const float* pa = static_cast<const float*>(a->data);
     const float* pb = static_cast<const float*>(b->data);
     float* pc = static_cast<float*>(out->data);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (B > 1 && ctx->math == TFJSB_MATH_TF32 && gemm_tf32_supported(M, N, K) && ctx->encode_tiled) {
+        // All products in one launch of the tensor-core kernel: their tiles share the SMs.  Operands
+        // that are not K-contiguous are transposed into scratch first, one product at a time.
+        cudaError_t e;
+        const float* a_km = pa;
+        const float* b_km = pb;
+        if (transpose_a) {
+            if ((st = ensure_scratch(ctx, &ctx->scratch_a, (size_t)B * M * K * 4)) != TFJSB_OK) return st;
+            for (int64_t i = 0; i < B; ++i)
+                if ((e = launch_transpose(pa + i * M * K, ctx->scratch_a.ptr + i * M * K, K, M, s, &ctx->launches)) != cudaSuccess)
+                    return cuda_fail(ctx, e, "transpose(a)");
+            a_km = ctx->scratch_a.ptr;
+        }
+        if (!transpose_b) {
+            if ((st = ensure_scratch(ctx, &ctx->scratch_b, (size_t)B * N * K * 4)) != TFJSB_OK) return st;
+            for (int64_t i = 0; i < B; ++i)
+                if ((e = launch_transpose(pb + i * N * K, ctx->scratch_b.ptr + i * N * K, K, N, s, &ctx->launches)) != cudaSuccess)
+                    return cuda_fail(ctx, e, "transpose(b)");
+            b_km = ctx->scratch_b.ptr;
+        }
+        GemmTf32Plan plan;
+        if ((st = gemm_tf32_plan(ctx, a_km, b_km, pc, M, N, K, &plan, B)) != TFJSB_OK) return st;
+        if ((e = launch_gemm_tf32(plan, nullptr, TFJSB_ACT_NONE, ctx->dev_status, s, &ctx->launches)) != cudaSuccess)
+            return cuda_fail(ctx, e, "batched tf32 gemm launch");
+        return TFJSB_OK;
+    }
     for (int64_t i = 0; i < B; ++i) {
         st = matmul_2d(ctx, pa + i * M * K, pb + i * K * N, pc + i * M * N, M, K, N, transpose_a, transpose_b,
                        static_cast<cudaStream_t>(stream));

@@ -175,6 +175,7 @@ cudaError_t launch_depthwise(const DepthwisePlan& plan, const float* x, const fl
 struct GemmTf32Plan {
     CUtensorMap map_a, map_b, map_c;
     int64_t M, N, K;
+    int64_t batches = 1;  // independent products of this shape in one launch (single-CTA kernel only)
     int block_n;       // 32..256
     int stages;
     int acc_stages;
@@ -193,8 +194,9 @@ struct GemmTf32Plan {
     ConvGeom g{};
 };
 bool gemm_tf32_supported(int64_t M, int64_t N, int64_t K);
+// `batches` > 1: that many products of the same shape, operands and results stored one after the other.
 tfjsb_status gemm_tf32_plan(tfjsb_ctx* ctx, const float* a, const float* bt, float* c, int64_t M, int64_t N,
-                            int64_t K, GemmTf32Plan* plan);
+                            int64_t K, GemmTf32Plan* plan, int64_t batches = 1);
 // The same GEMM on CTA pairs; gemm_tf32_plan picks it where it is the faster kernel (environment
 // variable TFJSB_GEMM_PAIR: 0 = never, 1 = wherever the shape allows, unset = by shape).
 bool gemm_tf32_pair_preferred(int64_t M, int64_t N, int64_t K, int sm_count);

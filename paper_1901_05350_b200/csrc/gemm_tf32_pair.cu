@@ -337,6 +337,7 @@ tfjsb_status gemm_tf32_pair_plan(tfjsb_ctx* ctx, const float* a, const float* bt
     plan->cluster_split = false;
     plan->splits = 1;
     plan->c = c;
+    plan->batches = 1;
     int bn = 256;
     while (bn > 64 && bn / 2 >= N) bn >>= 1;
     plan->block_n = bn;

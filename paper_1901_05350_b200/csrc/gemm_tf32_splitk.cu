@@ -317,6 +317,7 @@ tfjsb_status gemm_tf32_splitk_plan(tfjsb_ctx* ctx, const float* a, const float* 
     plan->pair = false;
     plan->x = nullptr;
     plan->c = c;
+    plan->batches = 1;
     plan->cluster_split = true;
     const int64_t nkb = (K + BLOCK_K - 1) / BLOCK_K;
     const int kbs = (int)((nkb + splits - 1) / splits);

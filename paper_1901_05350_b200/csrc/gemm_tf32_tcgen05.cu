@@ -24,7 +24,9 @@
 //               its own instruction latency, hence eight.
 //               The two accumulator stages let the epilogue of tile i overlap the MMAs of tile i+1.
 // Ragged edges need no special code: rows/columns past M, N or K are zero-filled on load and
-// clipped on store by the tensor maps.
+// clipped on store by the tensor maps.  A batch of independent products of one shape (rank-3 matMul)
+// is one launch: the tensor maps carry the batch as a third dimension, and a tile is (batch, rows,
+// columns), so the tiles of all products share the SMs.
 //
 // Every wait is bounded: a wait that exceeds WAIT_LIMIT_NS raises an abort flag that all roles
 // poll, ORs a code into the context's device status word, and the CTA drains its copies, frees
@@ -132,7 +134,8 @@ struct KernelArgs {
     int block_n;
     int stages;
     int n_tiles;    // tiles along N
-    int num_tiles;  // total
+    int tiles_per_batch;  // tiles of one product (rows x columns)
+    int num_tiles;  // total, over all products of the batch
     int acc_stages;  // accumulator stages in tensor memory: 2 (block_n 256) or 4
     const float* bias;
     int act;
@@ -213,8 +216,9 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             for (int s = 0; s < MAX_STAGES; ++s) armed[s] = -1;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
-                const int m0 = (tile / args.n_tiles) * BLOCK_M;
-                const int n0 = (tile % args.n_tiles) * block_n;
+                const int batch = tile / args.tiles_per_batch, in_batch = tile - batch * args.tiles_per_batch;
+                const int m0 = (in_batch / args.n_tiles) * BLOCK_M;
+                const int n0 = (in_batch % args.n_tiles) * block_n;
                 (void)m0;
                 for (int kb = 0; kb < num_k_blocks; ++kb) {
                     if (!bounded_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_flag)) {
@@ -231,9 +235,9 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         mbar_arrive_expect_tx(full, (uint32_t)(stage_bytes - A_STAGE_BYTES));
                     } else {
                         mbar_arrive_expect_tx(full, (uint32_t)stage_bytes);
-                        tma_load_2d(a_dst, &map_a, full, kb * BLOCK_K, m0);
+                        tma_load_3d(a_dst, &map_a, full, kb * BLOCK_K, m0, batch);
                     }
-                    tma_load_2d(a_dst + A_STAGE_BYTES, &map_b, full, kb * BLOCK_K, n0);
+                    tma_load_3d(a_dst + A_STAGE_BYTES, &map_b, full, kb * BLOCK_K, n0, batch);
 #pragma unroll
                     for (int s = 0; s < MAX_STAGES; ++s)
                         if (s == stage) armed[s] = (int)phase;
@@ -324,8 +328,9 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         const int chunks_per_tile = block_n / EPI_COLS;
         int first_chunk = half;  // parity bookkeeping: chunk `ch` of this tile is ours when (ch - first_chunk) is even
         for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
-            const int m0 = (tile / args.n_tiles) * BLOCK_M;
-            const int n0 = (tile % args.n_tiles) * block_n;
+            const int batch = tile / args.tiles_per_batch, in_batch = tile - batch * args.tiles_per_batch;
+            const int m0 = (in_batch / args.n_tiles) * BLOCK_M;
+            const int n0 = (in_batch % args.n_tiles) * block_n;
             // every lane polls (each needs the acquire), the vote keeps the warp uniform
             const bool got = bounded_wait(smem_u32(&bar_acc_full[acc]), acc_phase, abort_flag);
             if (!__all_sync(0xffffffffu, got)) {
@@ -370,7 +375,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    tma_store_2d(&map_c, slab, col0, row0);
+                    tma_store_3d(&map_c, slab, col0, row0, batch);
                     tma_store_commit();
                 }
             }
@@ -462,10 +467,10 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     }
 }
 
-int choose_block_n(int64_t M, int64_t N, int sm_count) {
+int choose_block_n(int64_t M, int64_t N, int sm_count, int64_t batches) {
     int bn = 32;
     while (bn < 256 && bn < N) bn <<= 1;
-    const int64_t m_tiles = (M + BLOCK_M - 1) / BLOCK_M;
+    const int64_t m_tiles = batches * ((M + BLOCK_M - 1) / BLOCK_M);  // row tiles of all products
     while (bn > 32 && m_tiles * ((N + bn - 1) / bn) < sm_count) bn >>= 1;
     if (bn == 256 && N > 256) {
         // Wave quantisation: every tile of a launch costs the same, so the launch takes
@@ -477,13 +482,14 @@ int choose_block_n(int64_t M, int64_t N, int sm_count) {
     return bn;
 }
 
+// A batch of `batches` row-major matrices [outer, inner] stored one after the other, box = one tile of one matrix.
 tfjsb_status encode_2d(tfjsb_ctx* ctx, CUtensorMap* map, const void* base, int64_t inner, int64_t outer,
-                       int box_inner, int box_outer, const char* what) {
-    cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
-    cuuint64_t strides[1] = {(cuuint64_t)inner * 4u};
-    cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
-    cuuint32_t elem[2] = {1u, 1u};
-    CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides,
+                       int box_inner, int box_outer, const char* what, int64_t batches = 1) {
+    cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)batches};
+    cuuint64_t strides[2] = {(cuuint64_t)inner * 4u, (cuuint64_t)inner * (cuuint64_t)outer * 4u};
+    cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer, 1u};
+    cuuint32_t elem[3] = {1u, 1u, 1u};
+    CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides,
                                    box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS)
@@ -503,9 +509,10 @@ bool gemm_tf32_supported(int64_t M, int64_t N, int64_t K) {
 namespace {
 
 // tile choice, pipeline depth and the B / C tensor maps shared by the GEMM and the convolution
-tfjsb_status plan_common(tfjsb_ctx* ctx, const float* bt, int64_t k_pitch, float* c, GemmTf32Plan* plan) {
+tfjsb_status plan_common(tfjsb_ctx* ctx, const float* bt, int64_t k_pitch, float* c, GemmTf32Plan* plan, int64_t batches = 1) {
     const int64_t M = plan->M, N = plan->N;
-    plan->block_n = choose_block_n(M, N, ctx->sm_count);
+    plan->batches = batches;
+    plan->block_n = choose_block_n(M, N, ctx->sm_count, batches);
     plan->acc_stages = plan->block_n > 128 ? 2 : MAX_ACC_STAGES;
     const int stage_bytes = A_STAGE_BYTES + plan->block_n * BLOCK_K * 4;
     int stages = (SMEM_LIMIT - 1024 - EPI_BYTES - 512) / stage_bytes;
@@ -513,25 +520,27 @@ tfjsb_status plan_common(tfjsb_ctx* ctx, const float* bt, int64_t k_pitch, float
     plan->stages = stages;
     plan->smem_bytes = (size_t)1024 + EPI_BYTES + (size_t)stages * stage_bytes;
     const int64_t n_tiles = (N + plan->block_n - 1) / plan->block_n;
-    const int64_t tiles = ((M + BLOCK_M - 1) / BLOCK_M) * n_tiles;
+    const int64_t tiles = batches * ((M + BLOCK_M - 1) / BLOCK_M) * n_tiles;
+    if (tiles >= (1LL << 31)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "too many tiles");
     plan->num_tiles = (int)tiles;
     plan->grid = (int)(tiles < ctx->sm_count ? tiles : ctx->sm_count);
     tfjsb_status st;
-    if ((st = encode_2d(ctx, &plan->map_b, bt, k_pitch, N, BLOCK_K, plan->block_n, "B")) != TFJSB_OK) return st;
-    if ((st = encode_2d(ctx, &plan->map_c, c, N, M, EPI_COLS, 32, "C")) != TFJSB_OK) return st;
+    if ((st = encode_2d(ctx, &plan->map_b, bt, k_pitch, N, BLOCK_K, plan->block_n, "B", batches)) != TFJSB_OK) return st;
+    if ((st = encode_2d(ctx, &plan->map_c, c, N, M, EPI_COLS, 32, "C", batches)) != TFJSB_OK) return st;
     return TFJSB_OK;
 }
 
 }  // namespace
 
 tfjsb_status gemm_tf32_plan(tfjsb_ctx* ctx, const float* a, const float* bt, float* c, int64_t M, int64_t N,
-                            int64_t K, GemmTf32Plan* plan) {
-    if (!gemm_tf32_supported(M, N, K)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the TF32 GEMM");
+                            int64_t K, GemmTf32Plan* plan, int64_t batches) {
+    if (!gemm_tf32_supported(M, N, K) || batches < 1 || batches >= (1LL << 31))
+        return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the TF32 GEMM");
     if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
     const char* pair_env = getenv("TFJSB_GEMM_PAIR");
     const bool use_pair = pair_env ? (pair_env[0] == '1' && N >= 64) : gemm_tf32_pair_preferred(M, N, K, ctx->sm_count);
-    if (use_pair) return gemm_tf32_pair_plan(ctx, a, bt, c, M, N, K, plan);
-    {
+    if (batches == 1 && use_pair) return gemm_tf32_pair_plan(ctx, a, bt, c, M, N, K, plan);
+    if (batches == 1) {
         // few tiles and a long K loop: the K loop is cut across the CTAs of a cluster (gemm_tf32_splitk.cu)
         int split_bn = 0, split_s = 0;
         if (!getenv("TFJSB_NO_SPLIT_K") && gemm_tf32_splitk_choice(M, N, K, ctx->sm_count, &split_bn, &split_s))
@@ -543,8 +552,8 @@ tfjsb_status gemm_tf32_plan(tfjsb_ctx* ctx, const float* a, const float* bt, flo
     plan->gather = false;
     plan->x = nullptr;
     tfjsb_status st;
-    if ((st = plan_common(ctx, bt, K, c, plan)) != TFJSB_OK) return st;
-    return encode_2d(ctx, &plan->map_a, a, K, M, BLOCK_K, BLOCK_M, "A");
+    if ((st = plan_common(ctx, bt, K, c, plan, batches)) != TFJSB_OK) return st;
+    return encode_2d(ctx, &plan->map_a, a, K, M, BLOCK_K, BLOCK_M, "A", batches);
 }
 
 int64_t conv_igemm_k_pad(const ConvGeom& g) {
@@ -597,6 +606,7 @@ cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int ac
     args.block_n = plan.block_n;
     args.stages = plan.stages;
     args.n_tiles = (int)((plan.N + plan.block_n - 1) / plan.block_n);
+    args.tiles_per_batch = (int)(plan.num_tiles / (plan.batches > 0 ? plan.batches : 1));
     args.num_tiles = plan.num_tiles;
     args.acc_stages = plan.acc_stages;
     args.bias = bias;
