@@ -5,11 +5,13 @@
 // For GEMMs with few output tiles and a long K loop (the dense layer; every pointwise layer at small
 // batch), where the persistent kernel would leave most SMs idle while a few walk all the k-blocks
 // one after the other.  A cluster of S CTAs (2, 4 or 8) owns one 128 x block_n tile; CTA r
-// accumulates the r-th slice of the k-blocks in its tensor memory, copies the partial tile into its
-// own shared memory, and after a cluster barrier every CTA sums one band of 128/S rows over all S
-// partial tiles, read from the partners' shared memory in slice order, adds the bias, applies the
-// activation and stores its band of C.  No workspace in global memory, no second kernel, and the
-// result does not depend on which slice finishes first.
+// accumulates the r-th slice of the k-blocks in its tensor memory and then sends every band of 128/S
+// rows of its partial tile to the shared memory of the CTA that owns the band (stores into the
+// partner's shared memory); after one cluster barrier every CTA finds the S partial copies of its
+// band in its own shared memory, adds them in slice order, adds the bias, applies the activation and
+// stores its band of C.  No workspace in global memory, no second kernel, no access to a partner's
+// memory after the barrier (so a CTA may leave as soon as it is done), and the result does not
+// depend on which slice finishes first.
 //
 // Per CTA, 6 warps: warp 0 producer (bulk tensor copies into a ring of stages), warp 1 tensor-memory
 // allocation and MMA issue, warps 2-5 one per tensor-memory lane quadrant: accumulator -> shared
@@ -48,9 +50,12 @@ struct SplitArgs {
     unsigned int* dev_status;
 };
 
-__device__ __forceinline__ float4 ld_cluster_v4(uint32_t cluster_addr) {
+__device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ float4 ld_shared_v4(uint32_t addr) {
     float4 v;
-    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr) : "memory");
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
     return v;
 }
 
@@ -80,7 +85,7 @@ gemm_tf32_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     const int n0 = (tile % args.n_tiles) * block_n;
 
     // dynamic shared memory, the same layout in every CTA of the cluster:
-    //   [partial tile: 4 lane quadrants x chunks x (32 rows x 128 B, swizzled)][stage 0: A | B][stage 1] ...
+    //   [this CTA's band of every slice: S x (128/S rows) x chunks x 128 B, 16-byte pieces swizzled by row][stage 0: A | B] ...
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t partial_base = smem_base;
     const uint32_t stage_base = smem_base + (uint32_t)(BLOCK_M * block_n * 4);
@@ -191,17 +196,23 @@ gemm_tf32_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             }
         }
     } else {
-        // ---------------------------------------------------------------- accumulator -> shared memory (warps 2..5)
+        // ---------------------------------------------------------------- accumulator -> the band owners' shared memory (warps 2..5)
         const int quad = warp & 3;  // the tensor-memory lanes this warp may read: 32*quad ..
         const bool got = bounded_wait(smem_u32(&bar_acc_full), 0u, abort_flag);
         if (__all_sync(0xffffffffu, got)) {
             tc_fence_after();
+            const int rows_per = BLOCK_M / splits;
+            const int row = quad * 32 + lane;            // this lane's row of the tile
+            const int owner = row / rows_per, i = row - owner * rows_per;
             for (int ch = 0; ch < chunks; ++ch) {
                 uint32_t r[32];
                 tc_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ch * EPI_COLS), r);
                 tc_ld_wait();
-                const uint32_t slab = partial_base + (uint32_t)((quad * chunks + ch) * EPI_SLAB_BYTES);
-                stage_chunk<TFJSB_ACT_NONE>(r, nullptr, EPI_COLS, slab + (uint32_t)lane * 128u, lane);
+                // slot of (slice = this CTA, band row i, chunk ch) in the owner's shared memory
+                const uint32_t dst = map_to_cta(partial_base + (uint32_t)((((int)rank * rows_per + i) * chunks + ch) * 128), (uint32_t)owner);
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    st_cluster_v4(dst + (uint32_t)((j ^ (i & 7)) << 4), r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
             }
         } else if (lane == 0 && !*abort_flag) {
             *abort_flag = 1;
@@ -209,41 +220,37 @@ gemm_tf32_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         }
     }
 
-    // ---------------------------------------------------------------- reduction across the cluster
+    // ---------------------------------------------------------------- reduction of this CTA's band
     tc_fence_before();
     __syncthreads();
-    cluster_arrive();   // every partial tile is in its CTA's shared memory ...
-    cluster_wait();     // ... and visible to the partners
+    cluster_arrive();   // this CTA's stores into its partners' shared memory are done ...
+    cluster_wait();     // ... and every partner's stores into this one are visible
     if (warp >= 2) {
-        const int rows_per = BLOCK_M / splits;           // this CTA's band of the tile
-        const int total = rows_per * chunks * 8;         // 16-byte pieces in the band
+        const int rows_per = BLOCK_M / splits;
+        const int total = rows_per * chunks * 8;         // 16-byte pieces in the band (a multiple of 128)
         for (int e = (int)threadIdx.x - 64; e < total; e += S_THREADS - 64) {
-            const int j = e & 7;                          // piece of the 128-byte chunk row: consecutive threads, consecutive bytes of C
+            const int j = e & 7;                          // consecutive threads, consecutive bytes of C
             const int ch = (e >> 3) % chunks;
-            const int row = (int)rank * rows_per + (e >> 3) / chunks;
-            const int quad = row >> 5, lr = row & 31;
-            const uint32_t local = partial_base + (uint32_t)((quad * chunks + ch) * EPI_SLAB_BYTES) + (uint32_t)lr * 128u +
-                                   (uint32_t)((j ^ (lr & 7)) << 4);
-            float4 v = ld_cluster_v4(map_to_cta(local, 0u));
-            for (int s = 1; s < splits; ++s) {
-                const float4 p = ld_cluster_v4(map_to_cta(local, (uint32_t)s));
+            const int i = (e >> 3) / chunks;
+            const int grow = m0 + (int)rank * rows_per + i, gcol = n0 + ch * EPI_COLS + 4 * j;
+            const bool live = grow < args.M && gcol < args.N;   // N % 4 == 0: a quad is all in or all out
+            float4 bq = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (args.bias != nullptr && live) bq = __ldg(reinterpret_cast<const float4*>(args.bias + gcol));
+            const uint32_t piece = partial_base + (uint32_t)((i * chunks + ch) * 128) + (uint32_t)((j ^ (i & 7)) << 4);
+            const uint32_t slice_pitch = (uint32_t)(rows_per * chunks * 128);
+            float4 v = ld_shared_v4(piece);
+            for (int sl = 1; sl < splits; ++sl) {
+                const float4 p = ld_shared_v4(piece + (uint32_t)sl * slice_pitch);
                 v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
             }
-            const int grow = m0 + row, gcol = n0 + ch * EPI_COLS + 4 * j;
-            if (grow < args.M && gcol < args.N) {   // N % 4 == 0: a quad is all in or all out
-                if (args.bias != nullptr) {
-                    const float4 b = __ldg(reinterpret_cast<const float4*>(args.bias + gcol));
-                    v.x += b.x; v.y += b.y; v.z += b.z; v.w += b.w;
-                }
-                v.x = apply_act(v.x, args.act); v.y = apply_act(v.y, args.act);
-                v.z = apply_act(v.z, args.act); v.w = apply_act(v.w, args.act);
+            if (live) {
+                v.x = apply_act(v.x + bq.x, args.act); v.y = apply_act(v.y + bq.y, args.act);
+                v.z = apply_act(v.z + bq.z, args.act); v.w = apply_act(v.w + bq.w, args.act);
                 *reinterpret_cast<float4*>(args.c + (int64_t)grow * args.N + gcol) = v;
             }
         }
     }
-    // nobody leaves while a partner may still be reading its shared memory
-    cluster_arrive();
-    cluster_wait();
+    // nothing touches a partner's shared memory after the barrier above: no second barrier before leaving
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
