@@ -39,7 +39,7 @@ __device__ __forceinline__ void fma4(float4& acc, const float4& a, const float4&
     acc.z = fmaf(a.z, b.z, acc.z); acc.w = fmaf(a.w, b.w, acc.w);
 }
 
-template <int S, int ROWS>
+template <int S, int ROWS, int D = 1>
 __global__ void __launch_bounds__(DW_THREADS)
 depthwise3x3_kernel(const float* __restrict__ x, const float* __restrict__ f, const float* __restrict__ bias,
                     int act, float* __restrict__ y, ConvGeom g, int tc, int c4_tiles) {
@@ -64,12 +64,12 @@ depthwise3x3_kernel(const float* __restrict__ x, const float* __restrict__ f, co
     const int iy_base = oy0 * S - g.pt;
     const int ix_base = ox * S - g.pl;
     const bool in_x0 = ix_base >= 0 && ix_base < g.W;
-    const bool in_x1 = ix_base + 1 >= 0 && ix_base + 1 < g.W;
-    const bool in_x2 = ix_base + 2 >= 0 && ix_base + 2 < g.W;
+    const bool in_x1 = ix_base + D >= 0 && ix_base + D < g.W;       // D: dilation (taps D pixels apart)
+    const bool in_x2 = ix_base + 2 * D >= 0 && ix_base + 2 * D < g.W;
     const float* xn = x + n * (int64_t)g.H * g.W * g.C + c;
     const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
 
-    constexpr int IN_ROWS = (ROWS - 1) * S + 3;
+    constexpr int IN_ROWS = (ROWS - 1) * S + 2 * D + 1;
 #pragma unroll
     for (int j = 0; j < IN_ROWS; ++j) {
         const int iy = iy_base + j;
@@ -77,12 +77,12 @@ depthwise3x3_kernel(const float* __restrict__ x, const float* __restrict__ f, co
         if (iy >= 0 && iy < g.H) {
             const float* row = xn + ((int64_t)iy * g.W + ix_base) * g.C;
             if (in_x0) v0 = ld4(row);
-            if (in_x1) v1 = ld4(row + g.C);
-            if (in_x2) v2 = ld4(row + 2 * g.C);
+            if (in_x1) v1 = ld4(row + D * g.C);
+            if (in_x2) v2 = ld4(row + 2 * D * g.C);
         }
 #pragma unroll
         for (int ky = 0; ky < 3; ++ky) {
-            const int t = j - ky;
+            const int t = j - ky * D;
             if (t >= 0 && t % S == 0 && t / S < ROWS) {
                 const int r = t / S;
                 fma4(acc[r], v0, w[ky * 3 + 0]);
@@ -157,24 +157,24 @@ struct DwTiling {
     long long num_tiles;
 };
 
-template <int S, int TW, int R>
+template <int S, int TW, int R, int D = 1>
 struct DwTile {
     static constexpr int RG = 32 / TW;                 // row groups of threads: 256 = 8 quads x TW x RG
     static constexpr int TH = RG * R;                  // output rows per tile
-    static constexpr int TWIN = (TW - 1) * S + 3;      // input patch
-    static constexpr int THIN = (TH - 1) * S + 3;
+    static constexpr int TWIN = (TW - 1) * S + 2 * D + 1;  // input patch (D: dilation, taps D pixels apart)
+    static constexpr int THIN = (TH - 1) * S + 2 * D + 1;
     static constexpr int STAGE_FLOATS = THIN * TWIN * DW_CB;
     static constexpr int STAGE_BYTES = STAGE_FLOATS * 4;
 };
 
 constexpr int DW_TMA_THREADS = DW_THREADS + 32;  // eight compute warps and the warp that issues the copies
 
-template <int S, int TW, int R>
+template <int S, int TW, int R, int D = 1>
 __global__ void __launch_bounds__(DW_TMA_THREADS, 2)
 depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __restrict__ f,
                         const float* __restrict__ bias, int act, float* __restrict__ y, ConvGeom g, DwTiling t,
                         unsigned int* dev_status) {
-    using T = DwTile<S, TW, R>;
+    using T = DwTile<S, TW, R, D>;
     extern __shared__ uint8_t dw_smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[DW_MAX_STAGES];   // copy landed (1 arrival + bytes)
     __shared__ __align__(8) uint64_t bar_empty[DW_MAX_STAGES];  // the eight compute warps are done with the stage
@@ -285,14 +285,14 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
 #pragma unroll
             for (int r = 0; r < R; ++r) acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
             const float* patch = smem_f + (size_t)slot * T::STAGE_FLOATS + ((rg * R * S) * T::TWIN + col * S) * DW_CB + c4 * 4;
-            constexpr int IN_ROWS = (R - 1) * S + 3;
+            constexpr int IN_ROWS = (R - 1) * S + 2 * D + 1;
 #pragma unroll
             for (int j = 0; j < IN_ROWS; ++j) {
                 const float* row = patch + j * T::TWIN * DW_CB;
-                const float4 v0 = ld4(row), v1 = ld4(row + DW_CB), v2 = ld4(row + 2 * DW_CB);
+                const float4 v0 = ld4(row), v1 = ld4(row + D * DW_CB), v2 = ld4(row + 2 * D * DW_CB);
 #pragma unroll
                 for (int ky = 0; ky < 3; ++ky) {
-                    const int d = j - ky;
+                    const int d = j - ky * D;
                     if (d >= 0 && d % S == 0 && d / S < R) {
                         fma4_packed(acc[d / S], v0, w[ky * 3 + 0]);
                         fma4_packed(acc[d / S], v1, w[ky * 3 + 1]);
@@ -327,14 +327,16 @@ constexpr DwVariant kDwVariants[] = {
     {1, 8, DwTile<1, 8, 2>::TH, DwTile<1, 8, 2>::STAGE_BYTES},     // 2: images up to 8 wide
     {2, 16, DwTile<2, 16, 2>::TH, DwTile<2, 16, 2>::STAGE_BYTES},  // 3: stride 2
     {2, 8, DwTile<2, 8, 2>::TH, DwTile<2, 8, 2>::STAGE_BYTES},     // 4: stride 2, outputs up to 8 wide
+    {1, 16, DwTile<1, 16, 4, 2>::TH, DwTile<1, 16, 4, 2>::STAGE_BYTES},  // 5: stride 1, dilation 2
+    {1, 16, DwTile<1, 16, 4, 4>::TH, DwTile<1, 16, 4, 4>::STAGE_BYTES},  // 6: stride 1, dilation 4
 };
 constexpr int DW_SMEM_BUDGET = 113 * 1024;  // two CTAs per SM
 
-template <int S, int TW, int R>
+template <int S, int TW, int R, int D = 1>
 cudaError_t launch_tma_instance(const DepthwisePlan& plan, const float* f, const float* bias, int act, float* y,
                                 const ConvGeom& g, unsigned int* dev_status, cudaStream_t s) {
     static bool attr_set = false;
-    auto kernel = depthwise3x3_tma_kernel<S, TW, R>;
+    auto kernel = depthwise3x3_tma_kernel<S, TW, R, D>;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DW_SMEM_BUDGET);
         if (e != cudaSuccess) return e;
@@ -355,14 +357,16 @@ int pow2_at_most(int v, int cap) {
 
 tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const float* x, const ConvGeom& g, DepthwisePlan* plan) {
     plan->variant = -1;
-    const bool shape_ok = g.fh == 3 && g.fw == 3 && g.mult == 1 && g.dh == 1 && g.dw == 1 && g.sh == g.sw &&
+    const bool dilated = g.dh == g.dw && (g.dh == 2 || g.dh == 4) && g.sh == 1;  // atrous layers
+    const bool shape_ok = g.fh == 3 && g.fw == 3 && g.mult == 1 && ((g.dh == 1 && g.dw == 1) || dilated) && g.sh == g.sw &&
                           (g.sh == 1 || g.sh == 2) && (g.C % 4 == 0) && g.C >= DW_CB;
     if (!shape_ok || !ctx->encode_tiled) return TFJSB_OK;
     int v;
-    if (g.sh == 1) v = g.Wo <= 8 ? 2 : ((g.Ho > 8 && g.Ho <= 14) ? 1 : 0);
+    if (dilated) v = g.dh == 2 ? 5 : 6;
+    else if (g.sh == 1) v = g.Wo <= 8 ? 2 : ((g.Ho > 8 && g.Ho <= 14) ? 1 : 0);
     else v = g.Wo <= 8 ? 4 : 3;
     const DwVariant& d = kDwVariants[v];
-    const int twin = (d.TW - 1) * d.S + 3, thin = (d.TH - 1) * d.S + 3;
+    const int twin = (d.TW - 1) * d.S + 2 * g.dw + 1, thin = (d.TH - 1) * d.S + 2 * g.dh + 1;
     cuuint64_t dims[4] = {(cuuint64_t)g.C, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
     cuuint64_t strides[3] = {(cuuint64_t)g.C * 4u, (cuuint64_t)g.W * g.C * 4u, (cuuint64_t)g.H * g.W * g.C * 4u};
     cuuint32_t box[4] = {(cuuint32_t)DW_CB, (cuuint32_t)twin, (cuuint32_t)thin, 1u};
@@ -401,12 +405,16 @@ cudaError_t launch_depthwise(const DepthwisePlan& plan, const float* x, const fl
             case 1: e = launch_tma_instance<1, 16, 7>(plan, f, bias, act, y, g, dev_status, s); break;
             case 2: e = launch_tma_instance<1, 8, 2>(plan, f, bias, act, y, g, dev_status, s); break;
             case 3: e = launch_tma_instance<2, 16, 2>(plan, f, bias, act, y, g, dev_status, s); break;
-            default: e = launch_tma_instance<2, 8, 2>(plan, f, bias, act, y, g, dev_status, s); break;
+            case 4: e = launch_tma_instance<2, 8, 2>(plan, f, bias, act, y, g, dev_status, s); break;
+            case 5: e = launch_tma_instance<1, 16, 4, 2>(plan, f, bias, act, y, g, dev_status, s); break;
+            default: e = launch_tma_instance<1, 16, 4, 4>(plan, f, bias, act, y, g, dev_status, s); break;
         }
         ++*launches;
         return e;
     }
-    const bool fast = g.fh == 3 && g.fw == 3 && g.mult == 1 && g.dh == 1 && g.dw == 1 && g.sh == g.sw &&
+    // dilated windows (the atrous depthwise layers of output-stride-16 / -8 MobileNet variants): stride 1, dilation 2 or 4
+    const bool dilated = g.dh == g.dw && (g.dh == 2 || g.dh == 4) && g.sh == 1;
+    const bool fast = g.fh == 3 && g.fw == 3 && g.mult == 1 && ((g.dh == 1 && g.dw == 1) || dilated) && g.sh == g.sw &&
                       (g.sh == 1 || g.sh == 2) && (g.C % 4 == 0) && g.N <= 65535;
     if (fast) {
         constexpr int ROWS = 4;
@@ -418,7 +426,11 @@ cudaError_t launch_depthwise(const DepthwisePlan& plan, const float* x, const fl
         const int gy = (g.Ho + ROWS - 1) / ROWS;
         if (gx <= 2147483647LL && gy <= 65535) {
             dim3 grid((unsigned)gx, (unsigned)gy, (unsigned)g.N);
-            if (g.sh == 1)
+            if (g.dh == 2)
+                depthwise3x3_kernel<1, ROWS, 2><<<grid, DW_THREADS, 0, s>>>(x, f, bias, act, y, g, tc, c4_tiles);
+            else if (g.dh == 4)
+                depthwise3x3_kernel<1, ROWS, 4><<<grid, DW_THREADS, 0, s>>>(x, f, bias, act, y, g, tc, c4_tiles);
+            else if (g.sh == 1)
                 depthwise3x3_kernel<1, ROWS><<<grid, DW_THREADS, 0, s>>>(x, f, bias, act, y, g, tc, c4_tiles);
             else
                 depthwise3x3_kernel<2, ROWS><<<grid, DW_THREADS, 0, s>>>(x, f, bias, act, y, g, tc, c4_tiles);

@@ -31,7 +31,8 @@ def main() -> int:
     ap.add_argument("--hw", type=int, default=112, help="depthwise / pointwise: input height = width")
     ap.add_argument("--channels", type=int, default=32, help="depthwise / pointwise: input channels")
     ap.add_argument("--cout", type=int, default=64, help="pointwise: output channels")
-    ap.add_argument("--stride", type=int, default=1, help="depthwise: stride")
+    ap.add_argument("--stride", type=int, default=1, help="depthwise / maxpool: stride")
+    ap.add_argument("--dilation", type=int, default=1, help="depthwise: dilation (with stride 1)")
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
     ap.add_argument("--math", choices=["tf32", "fp32"], default="tf32")
@@ -80,9 +81,9 @@ def main() -> int:
         if args.workload == "depthwise":
             w = torch.from_numpy(si.normal(7, 1, (3, 3, args.channels, 1), 0.0, 0.47)).cuda()
             b = torch.from_numpy(si.normal(7, 2, (args.channels,), 0.0, 0.01)).cuda()
-            strides = (args.stride, args.stride)
-            out = ctx.depthwise_conv2d(x, w, strides, "same", (1, 1), b, "relu6")
-            step = lambda: ctx.depthwise_conv2d(x, w, strides, "same", (1, 1), b, "relu6", out=out)
+            strides, dil = (args.stride, args.stride), (args.dilation, args.dilation)
+            out = ctx.depthwise_conv2d(x, w, strides, "same", dil, b, "relu6")
+            step = lambda: ctx.depthwise_conv2d(x, w, strides, "same", dil, b, "relu6", out=out)
         else:
             from seeded_inputs.workloads import Layer
 

@@ -24,6 +24,7 @@ from .workloads import (
     config_matmul,
     config_separable_block,
     config_mobilenet,
+    config_mobilenet_atrous,
     CONFIG_SEEDS,
 )
 
@@ -39,5 +40,6 @@ __all__ = [
     "config_matmul",
     "config_separable_block",
     "config_mobilenet",
+    "config_mobilenet_atrous",
     "CONFIG_SEEDS",
 ]

@@ -60,14 +60,25 @@ _PW_WIDTHS = (64, 128, 128, 256, 256, 512, 512, 512, 512, 512, 512, 1024, 1024)
 _DW_STRIDES = (1, 2, 1, 2, 1, 2, 1, 1, 1, 1, 1, 2, 1)
 
 
-def mobilenet_v1_layers(alpha: float, classes: int = 1000) -> List[Layer]:
-    """MobileNet-v1-style layer list: stem 3x3/2, 13 x (dw 3x3, pw 1x1), pool, dense, softmax."""
+def mobilenet_v1_layers(alpha: float, classes: int = 1000, output_stride: int = 32) -> List[Layer]:
+    """MobileNet-v1-style layer list: stem 3x3/2, 13 x (dw 3x3, pw 1x1), pool, dense, softmax.
+
+    `output_stride` 16 or 8 gives the atrous variant used by dense-prediction models (PoseNet-style):
+    once the feature map has reached that stride, a depthwise layer that would halve it again keeps
+    stride 1 instead and every later depthwise layer is dilated by the strides left out so far."""
     layers = [
         Layer(CONV2D, (3, 3), (2, 2), (1, 1), "same", "relu6", int(32 * alpha), "stem")
     ]
+    current, rate = 2, 1
     for i, (width, stride) in enumerate(zip(_PW_WIDTHS, _DW_STRIDES), start=1):
+        dilation = rate
+        if stride > 1 and current >= output_stride:
+            rate *= stride
+            stride = 1
+        else:
+            current *= stride
         layers.append(
-            Layer(DEPTHWISE, (3, 3), (stride, stride), (1, 1), "same", "relu6", 1, f"dw{i}")
+            Layer(DEPTHWISE, (3, 3), (stride, stride), (dilation, dilation), "same", "relu6", 1, f"dw{i}")
         )
         layers.append(
             Layer(CONV2D, (1, 1), (1, 1), (1, 1), "same", "relu6", int(width * alpha), f"pw{i}")
@@ -134,6 +145,12 @@ def config_separable_block(hw: int = 112, cin: int = 32, cout: int = 64, batch: 
     ]
     make_model_weights(layers, cin, seed)
     return x, layers
+
+
+def config_mobilenet_atrous(alpha: float, hw: int, batch: int, output_stride: int, seed: int, classes: int = 1000):
+    """The atrous variant of config_mobilenet (see mobilenet_v1_layers): input and seeded weights."""
+    layers = make_model_weights(mobilenet_v1_layers(alpha, classes, output_stride), 3, seed)
+    return uniform(seed, 0, (batch, hw, hw, 3), -1.0, 1.0), layers
 
 
 def config_mobilenet(alpha: float, hw: int, batch: int, seed: int, classes: int = 1000):

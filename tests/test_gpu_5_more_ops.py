@@ -1,4 +1,5 @@
-"""GPU parity of the ops beyond the MobileNet path: maxPool, elementwise add / sub / mul, rank-3 matMul.
+"""GPU parity of the ops beyond the MobileNet path: maxPool, elementwise add / sub / mul, rank-3 matMul,
+dilated depthwise convolution and the atrous (output stride 16 / 8) MobileNet variants built from it.
 
 Tolerances.  maxPool selects an input value and add / sub / mul are one correctly rounded fp32
 operation per element, so both must match the oracle bit for bit (NaNs in the same places).  A
@@ -122,3 +123,51 @@ def test_batch_matmul_rejects_bad_arguments(ctx, tfjsb):
     with pytest.raises(tfjsb.TfjsbError) as err:
         ctx.batch_matmul(torch.zeros(2, 4, 8, device="cuda"), torch.zeros(2, 7, 4, device="cuda"))
     assert err.value.status_name == "SHAPE"
+
+
+DILATED_DW_CASES = [
+    # N, H, W, C, dilation: 3x3 depthwise, stride 1, 'same' (the atrous layers of output-stride-16 / -8 models)
+    (2, 14, 14, 512, 2),
+    (1, 28, 28, 256, 4),
+    (3, 9, 11, 32, 2),     # image barely larger than the dilated window
+    (1, 5, 5, 8, 4),       # dilated window larger than the image: most taps fall outside
+    (2, 14, 14, 6, 2),     # channel count not a multiple of 4: the general kernel
+]
+
+
+@pytest.mark.parametrize("case", DILATED_DW_CASES)
+def test_dilated_depthwise_parity(ctx, oracle, case):
+    N, H, W, C, d = case
+    x = si.uniform(505, 0, (N, H, W, C), 0, 6)
+    f = si.normal(505, 1, (3, 3, C, 1), 0, 0.47)
+    b = si.normal(505, 2, (C,), 0, 0.5)
+    got = host(ctx.depthwise_conv2d(dev(x), dev(f), (1, 1), "same", (d, d), dev(b), "relu6"))
+    want = oracle.depthwise_conv2d(x, f, (1, 1), "same", (d, d), b, "relu6")
+    assert got.shape == want.shape and rel_fro(got, want) <= 1e-6
+    xi = si.small_integers(506, 0, x.shape, -8, 8)
+    fi = si.small_integers(506, 1, f.shape, -8, 8)
+    assert same_bits(host(ctx.depthwise_conv2d(dev(xi), dev(fi), (1, 1), "same", (d, d))),
+                     oracle.depthwise_conv2d(xi, fi, (1, 1), "same", (d, d)))
+
+
+@pytest.mark.parametrize("output_stride", [16, 8])
+def test_atrous_mobilenet_every_layer(ctx, oracle, output_stride):
+    """alpha 0.25, 96x96 input, batch 2, output stride 16 / 8: every layer's output against the oracle."""
+    x, layers = si.config_mobilenet_atrous(0.25, 96, 2, output_stride, seed=4243, classes=100)
+    dilations = sorted({l.dilations[0] for l in layers if l.kind == "depthwise_conv2d"})
+    assert dilations == ([1, 2] if output_stride == 16 else [1, 2, 4])
+    want = oracle.run_model(layers, x, keep_all=True)
+    assert want[-4].shape[1] == 96 // output_stride          # spatial size of the last block's output
+    model = ctx.model(layers, x.shape)
+    model.set_keep_all(True)
+    probs = host(model.run(dev(x)))
+    ctx.check_device_status()
+    for i, layer in enumerate(layers):
+        got = host(model.layer_output(i)) if i < len(layers) - 1 else probs
+        assert got.shape == want[i].shape, layer.name
+        assert rel_fro(got, want[i]) <= 2e-2, f"layer {i} ({layer.name}) diverges: {rel_fro(got, want[i]):.3e}"
+    span = float(want[-2].max() - want[-2].min())
+    assert np.max(np.abs(host(model.layer_output(len(layers) - 2)) - want[-2])) <= 1e-2 * span
+    model.set_keep_all(False)
+    assert same_bits(host(model.run(dev(x))), probs)          # the ping-pong run gives the same bits
+    model.close()
