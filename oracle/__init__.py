@@ -212,34 +212,64 @@ def softmax(x) -> np.ndarray:
     return y
 
 
-def run_model(layers: Sequence, x, operand: str = "fp32", keep_all: bool = False):
+def round_bf16(x) -> np.ndarray:
+    """Each fp32 value rounded to the nearest bfloat16 (8 significand bits, ties to even), returned as
+    fp32.  Infinities stay, finite values beyond the largest bfloat16 become infinite, NaN stays NaN.
+
+    This is the 16-bit storage format of the narrow-storage mode (the paper's 16-bit float textures,
+    Sec. 4.1.3, carried over to the format this hardware's tensor cores read).
+    """
+    x = _f32(x)
+    u = x.view(np.uint32).astype(np.uint64)
+    kept_lsb = (u >> np.uint64(16)) & np.uint64(1)
+    r = (u + np.uint64(0x7FFF) + kept_lsb) & np.uint64(0xFFFF0000)
+    out = r.astype(np.uint32).view(np.float32).reshape(x.shape)
+    return np.where(np.isnan(x), np.float32(np.nan), out).astype(np.float32)
+
+
+def run_model(layers: Sequence, x, operand: str = "fp32", keep_all: bool = False, storage: str = "fp32"):
     """Run a layer list (records with kind / filter_hw / strides / dilations / pad / act /
     out_channels / filter / bias) op by op; every layer's fp32 output feeds the next.
 
     Returns the list of all layer outputs when `keep_all`, else the last one.
     global_avg_pool is a 'valid' avgPool whose window is the remaining H x W, followed by the
     free reshape to [batch, C]; dense is matMul then a bias add with no activation.
+
+    storage="bf16": the narrow-storage mode.  Everything that is stored is a bfloat16: the model
+    input, every filter, and the output of every layer except dense and softmax layers and the
+    model's last layer, which stay fp32.  Biases stay fp32 (they are added to the wide sum).  The
+    arithmetic in between is the exact one of the fp32 mode: exact products of the stored values,
+    a wide sum, one rounding to fp32, and then the rounding to the stored format.
     """
+    if storage not in ("fp32", "bf16"):
+        raise ValueError(f"unknown storage {storage!r}")
+    narrow = storage == "bf16"
+    if narrow and operand != "fp32":
+        raise ValueError("narrow storage has no operand rounding of its own: bfloat16 products are exact")
+    stored = round_bf16 if narrow else (lambda t: t)
     outs: List[np.ndarray] = []
-    cur = _f32(x)
-    for layer in layers:
+    cur = stored(_f32(x))
+    layers = list(layers)
+    for li, layer in enumerate(layers):
         kind = layer.kind
         if kind == "conv2d":
-            cur = conv2d(cur, layer.filter, layer.strides, layer.pad, layer.dilations, layer.bias, layer.act,
+            cur = conv2d(cur, stored(layer.filter), layer.strides, layer.pad, layer.dilations, layer.bias, layer.act,
                          operand)
         elif kind == "depthwise_conv2d":
-            cur = depthwise_conv2d(cur, layer.filter, layer.strides, layer.pad, layer.dilations, layer.bias,
+            cur = depthwise_conv2d(cur, stored(layer.filter), layer.strides, layer.pad, layer.dilations, layer.bias,
                                    layer.act)
         elif kind == "global_avg_pool":
             n, h, w, c = cur.shape
             cur = avg_pool(cur, (h, w), (1, 1), "valid").reshape(n, c)
         elif kind == "dense":
-            cur = bias_act(matmul(cur.reshape(cur.shape[0], -1), layer.filter, operand=operand), layer.bias,
+            cur = bias_act(matmul(cur.reshape(cur.shape[0], -1), stored(layer.filter), operand=operand), layer.bias,
                            layer.act)
         elif kind == "softmax":
             cur = softmax(cur)
         else:
             raise ValueError(f"unknown layer kind {kind!r}")
+        if narrow and kind not in ("dense", "softmax") and li != len(layers) - 1:
+            cur = round_bf16(cur)
         if keep_all:
             outs.append(cur)
     return outs if keep_all else cur

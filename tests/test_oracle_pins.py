@@ -541,6 +541,83 @@ def test_small_model_invariants(oracle):
     assert np.array_equal(again, outs[-1])
 
 
+# ------------------------------------------------------------------ narrow (bfloat16) storage
+def test_round_bf16_hand_values_ties_and_specials(oracle):
+    # bfloat16 keeps 8 significand bits: the spacing in [1, 2) is 2^-7
+    cases = [
+        (1.0, 1.0),
+        (1.0 + 2.0 ** -8, 1.0),                      # exactly halfway between 1 and 1 + 2^-7: to the even one
+        (1.0 + 2.0 ** -8 + 2.0 ** -23, 1.0 + 2.0 ** -7),  # just above halfway
+        (1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -6),      # halfway between 1 + 2^-7 (odd) and 1 + 2^-6 (even)
+        (3.14159265, 3.140625),                      # pi: 0x40490FDB -> 0x4049
+        (-2.71828183, -2.71875),                     # -e: 0xC02DF854 -> 0xC02E
+        (0.1, 0.10009765625),                        # 0x3DCCCCCD -> 0x3DCD
+        (256.0 + 1.0, 256.0),                        # spacing 2 in [256, 512): 257 is halfway, 256 is even
+        (256.0 + 3.0, 260.0),                        # halfway between 258 (odd) and 260 (even)
+        (3.3895313892515355e38, 3.3895313892515355e38),  # the largest bfloat16, 0x7F7F0000
+        (3.4028234663852886e38, np.inf),             # the largest fp32 rounds up past it
+        (1e-40, 9.9e-41),                            # subnormal: 0x000116C2 -> 0x0001 0000 = 9.18e-41
+        (0.0, 0.0),
+    ]
+    x = np.array([c[0] for c in cases], dtype=np.float32)
+    got = oracle.round_bf16(x)
+    for (src, want), g in zip(cases, got):
+        if src == 1e-40:
+            assert g.view(np.uint32) == 0x00010000
+        else:
+            assert g == np.float32(want), (src, g, want)
+    sp = oracle.round_bf16(np.array([np.inf, -np.inf, np.nan, -0.0], dtype=np.float32))
+    assert sp[0] == np.inf and sp[1] == -np.inf and np.isnan(sp[2]) and sp[3] == 0 and np.signbit(sp[3])
+    # a NaN whose payload sits only in the dropped bits must not turn into an infinity
+    sneaky = np.array([0x7F800001], dtype=np.uint32).view(np.float32)
+    assert np.isnan(oracle.round_bf16(sneaky)[0])
+
+
+def test_round_bf16_matches_library_conversion(oracle):
+    x = np.concatenate([
+        si.normal(91, 0, (100000,), 0, 3),
+        si.uniform(91, 1, (50000,), -1e-3, 1e-3),
+        (si.uniform(91, 2, (50000,), -1, 1).astype(np.float64) * 1e30).astype(np.float32),
+        np.arange(0, 70000, dtype=np.uint32).view(np.float32),          # subnormals and their ties
+        (np.arange(0, 70000, dtype=np.uint32) + 0x3F7F0000).view(np.float32),  # around 1.0, every low-bit pattern
+    ])
+    want = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
+    got = oracle.round_bf16(x)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    assert np.array_equal(oracle.round_bf16(got), got)  # idempotent
+    assert np.all((got.view(np.uint32) & 0xFFFF) == 0)
+
+
+def test_narrow_storage_model_is_the_fp32_model_on_stored_values(oracle):
+    x, layers = si.config_mobilenet(0.25, 32, 2, seed=78, classes=10)
+    outs = oracle.run_model(layers, x, keep_all=True, storage="bf16")
+    # what is stored is a bfloat16; dense, softmax and the last layer stay fp32
+    for layer, out in zip(layers[:-2], outs[:-2]):
+        assert np.all((out.view(np.uint32) & 0xFFFF) == 0), layer.kind
+    assert np.any((outs[-2].view(np.uint32) & 0xFFFF) != 0)
+    # layer by layer: the fp32 op on the stored input and the stored filter, then one rounding
+    stored = oracle.round_bf16
+    first = oracle.conv2d(stored(x), stored(layers[0].filter), layers[0].strides, layers[0].pad, layers[0].dilations,
+                          layers[0].bias, layers[0].act)
+    assert np.array_equal(outs[0], stored(first))
+    dw = oracle.depthwise_conv2d(outs[0], stored(layers[1].filter), layers[1].strides, layers[1].pad,
+                                 layers[1].dilations, layers[1].bias, layers[1].act)
+    assert np.array_equal(outs[1], stored(dw))
+    n, h, w, c = outs[-4].shape
+    assert np.array_equal(outs[-3], stored(oracle.avg_pool(outs[-4], (h, w), (1, 1), "valid").reshape(n, c)))
+    # on values every format holds exactly (small integers, sums below 256) both modes agree bit for bit
+    xi = si.small_integers(79, 0, (1, 8, 8, 4), -2, 2)
+    li = [si.Layer(kind="conv2d", filter_hw=(3, 3), strides=(1, 1), pad="same", act="relu", out_channels=4,
+                   filter=si.small_integers(79, 1, (3, 3, 4, 4), -1, 1), bias=si.small_integers(79, 2, (4,), -3, 3)),
+          si.Layer(kind="depthwise_conv2d", filter_hw=(3, 3), strides=(1, 1), pad="same", act="relu6", out_channels=1,
+                   filter=si.small_integers(79, 3, (3, 3, 4, 1), -1, 1), bias=None)]
+    assert np.array_equal(oracle.run_model(li, xi, storage="bf16"), oracle.run_model(li, xi))
+    # and close to the fp32 model overall: storage error is 2^-9 relative per stored value
+    full = oracle.run_model(layers, x, keep_all=True)
+    assert rel_fro(outs[-2], full[-2]) < 3e-2
+    assert rel_fro(outs[0], full[0]) < 2.0 ** -7
+
+
 def test_generator_moments_and_reproducibility():
     u = si.uniform(9, 0, (200000,), -1, 1)
     assert u.min() >= -1 and u.max() < 1 and abs(u.mean()) < 5e-3 and abs(u.var() - 1 / 3) < 5e-3
