@@ -64,8 +64,17 @@ typedef enum { TFJSB_ACT_NONE = 0, TFJSB_ACT_RELU = 1, TFJSB_ACT_RELU6 = 2 } tfj
 /* Which multiplier the GEMM-shaped ops (matMul, conv2d, dense) use.
  *   TF32  tensor cores (tcgen05, operands read as TF32, fp32 accumulation in tensor memory)
  *         wherever the shape allows, CUDA cores otherwise.  Default.
- *   FP32  CUDA-core FFMA everywhere: the variant kept for exactness checks. */
-typedef enum { TFJSB_MATH_TF32 = 0, TFJSB_MATH_FP32 = 1 } tfjsb_math;
+ *   FP32  CUDA-core FFMA everywhere: the variant kept for exactness checks.
+ *   BF16  narrow storage (the counterpart of the paper's 16-bit float textures, Sec. 4.1.3): a model
+ *         created in this mode keeps its filters and every layer output except dense / softmax
+ *         outputs and its final result as bfloat16 in device memory (rounded to nearest even, once,
+ *         when stored); products of stored values are exact, sums are fp32, biases stay fp32, and
+ *         1x1 convolutions and dense layers run on the tensor cores (tcgen05 kind::f16).  The model's
+ *         input and output tensors stay fp32 (the input is rounded as it is read).  Supported layers:
+ *         conv2d (must come first), depthwise 3x3 (stride 1 or 2, no dilation, multiplier 1, channels
+ *         a multiple of 8), global avgPool, dense, softmax after dense.  The op entry points that
+ *         take fp32 tensors run their FP32 path in this mode. */
+typedef enum { TFJSB_MATH_TF32 = 0, TFJSB_MATH_FP32 = 1, TFJSB_MATH_BF16 = 2 } tfjsb_math;
 typedef enum { TFJSB_BINARY_ADD = 0, TFJSB_BINARY_SUB = 1, TFJSB_BINARY_MUL = 2 } tfjsb_binary_op;
 
 /* ---- context ------------------------------------------------------------------------ */
@@ -165,6 +174,18 @@ tfjsb_status tfjsb_max_pool(tfjsb_ctx* ctx, const tfjsb_tensor* x, const int fil
  * any IEEE implementation.  `out` may not alias an input. */
 tfjsb_status tfjsb_binary(tfjsb_ctx* ctx, tfjsb_binary_op op, const tfjsb_tensor* a, const tfjsb_tensor* b,
                           tfjsb_tensor* out, void* stream);
+
+/* matMul on bfloat16 storage with the fused epilogue (the GEMM of the BF16 math mode, exposed for
+ * tensors the caller already holds in that format):
+ *   out[M,N] = act( a[M,K] . bt[N,K]^T + bias[N] )
+ * a and bt are DEVICE pointers to bfloat16 (2 bytes per element, row-major, K contiguous: bt is the
+ * right-hand operand stored transposed); bias is a DEVICE pointer to N fp32 values or NULL; out is a
+ * DEVICE pointer to M*N bfloat16 (out_is_bf16 != 0; the sum is rounded to nearest even once, after
+ * bias and activation) or fp32 values.  Products are exact, sums fp32 in tensor memory.  All pointers
+ * 16-byte aligned, K and N multiples of 8; TFJSB_ERR_UNSUPPORTED otherwise.  Enqueues on `stream`
+ * and returns; the caller keeps ownership of every buffer. */
+tfjsb_status tfjsb_matmul_bf16(tfjsb_ctx* ctx, const void* a, const void* bt, const float* bias, tfjsb_act act,
+                               void* out, int out_is_bf16, int64_t M, int64_t N, int64_t K, void* stream);
 
 /* tf.matMul on rank-3 tensors (Sec. 3.3 names the op; Listing 2 prints the rank-2 case): one rank-2
  * product per leading index.  a [B,M,K] (or [B,K,M] if transpose_a), b [B,K,N] (or [B,N,K] if
@@ -268,6 +289,13 @@ tfjsb_status tfjsb_model_set_graph(tfjsb_model* model, int use_graph);
  * to give every layer its own buffer. */
 tfjsb_status tfjsb_model_set_keep_all(tfjsb_model* model, int keep_all);
 tfjsb_status tfjsb_model_layer_output(tfjsb_model* model, int layer, tfjsb_tensor* view);
+/* The same read as fp32 values whatever the layer's storage format: writes the layer's output
+ * (converted from bfloat16 where the model stores it so) into `dst`, a DEVICE buffer of as many
+ * floats as the layer has outputs, on `stream`.  tfjsb_model_layer_output refuses a layer that is
+ * stored as bfloat16 (its view would mislabel the data) with TFJSB_ERR_UNSUPPORTED. */
+tfjsb_status tfjsb_model_layer_output_f32(tfjsb_model* model, int layer, float* dst, void* stream);
+/* Shape of the output of layer `layer`. */
+tfjsb_status tfjsb_model_layer_shape(tfjsb_model* model, int layer, int32_t* rank, int64_t dims[4]);
 
 /* Per-layer device timing (the paper's per-kernel profile, Sec. 3.8): runs the model `reps`
  * times with a CUDA event pair around every layer, synchronises, and writes the mean

@@ -21,7 +21,7 @@ from . import build as _build
 
 PAD = {"valid": 0, "same": 1}
 ACT = {"none": 0, "relu": 1, "relu6": 2}
-MATH = {"tf32": 0, "fp32": 1}
+MATH = {"tf32": 0, "fp32": 1, "bf16": 2}
 BINARY_OP = {"add": 0, "sub": 1, "mul": 2}
 LAYER_KIND = {"conv2d": 0, "depthwise_conv2d": 1, "avg_pool": 2, "global_avg_pool": 2, "dense": 3, "softmax": 4}
 
@@ -34,6 +34,7 @@ EXPORTS = [
     "tfjsb_model_output_shape", "tfjsb_model_launches_per_run", "tfjsb_run_model", "tfjsb_run_model_host",
     "tfjsb_run_model_host_async", "tfjsb_model_host_wait",
     "tfjsb_model_set_keep_all", "tfjsb_model_set_graph", "tfjsb_model_set_fusion", "tfjsb_model_layer_output", "tfjsb_model_profile",
+    "tfjsb_matmul_bf16", "tfjsb_model_layer_output_f32", "tfjsb_model_layer_shape",
 ]
 
 
@@ -103,6 +104,9 @@ def _load_library() -> ctypes.CDLL:
     lib.tfjsb_model_set_fusion.argtypes = [vp, i32]
     lib.tfjsb_model_layer_output.argtypes = [vp, i32, tp]
     lib.tfjsb_model_profile.argtypes = [vp, tp, tp, i32, ctypes.POINTER(ctypes.c_float), vp]
+    lib.tfjsb_matmul_bf16.argtypes = [vp, vp, vp, vp, i32, vp, i32, i64, i64, i64, vp]
+    lib.tfjsb_model_layer_output_f32.argtypes = [vp, i32, vp, vp]
+    lib.tfjsb_model_layer_shape.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)]
     return lib
 
 
@@ -193,6 +197,27 @@ class Context:
         out = self._empty((M, N)) if out is None else out
         self._check(lib.tfjsb_matmul(self._h, _desc(a), _desc(b), int(transpose_a), int(transpose_b), _desc(out),
                                      _stream()))
+        return out
+
+    def matmul_bf16(self, a, bt, bias=None, act="none", out_dtype=None, out=None):
+        """act(a . bt^T + bias) on bfloat16 storage: a [M,K] and bt [N,K] bfloat16 CUDA tensors, bias fp32 [N]
+        or None, result bfloat16 (default) or fp32; products exact, sums fp32 on the tensor cores."""
+        import torch
+
+        for t in (a, bt):
+            if not t.is_cuda or t.dtype != torch.bfloat16 or not t.is_contiguous() or t.dim() != 2:
+                raise TypeError("expected contiguous rank-2 bfloat16 CUDA tensors")
+        if a.shape[1] != bt.shape[1]:
+            raise ValueError("a [M,K] and bt [N,K] must agree in K")
+        M, K, N = a.shape[0], a.shape[1], bt.shape[0]
+        if out is None:
+            out = torch.empty((M, N), dtype=out_dtype or torch.bfloat16, device=a.device)
+        if out.dtype not in (torch.bfloat16, torch.float32) or tuple(out.shape) != (M, N) or not out.is_contiguous():
+            raise TypeError("out must be a contiguous [M,N] bfloat16 or fp32 tensor")
+        if bias is not None and (bias.dtype != torch.float32 or tuple(bias.shape) != (N,) or not bias.is_contiguous()):
+            raise TypeError("bias must be a contiguous fp32 vector of length N")
+        self._check(lib.tfjsb_matmul_bf16(self._h, a.data_ptr(), bt.data_ptr(), None if bias is None else bias.data_ptr(),
+                                          ACT[act], out.data_ptr(), int(out.dtype == torch.bfloat16), M, N, K, _stream()))
         return out
 
     def matmul_static_scratch(self, a, b, transpose_a: bool = False, transpose_b: bool = False, out=None):
@@ -372,6 +397,16 @@ class Model:
 
         torch.cuda.current_stream().synchronize()
         return torch.as_tensor(_View(), device=f"cuda:{self.ctx.device}").clone()
+
+    def layer_output_f32(self, layer: int):
+        """fp32 copy of the output of layer `layer` whatever its storage format (bfloat16 layers are
+        widened on the device); use set_keep_all(True) before the run."""
+        rank = ctypes.c_int32()
+        dims = (ctypes.c_int64 * 4)()
+        self.ctx._check(lib.tfjsb_model_layer_shape(self._h, layer, ctypes.byref(rank), dims))
+        out = self.ctx._empty(tuple(int(dims[i]) for i in range(rank.value)))
+        self.ctx._check(lib.tfjsb_model_layer_output_f32(self._h, layer, out.data_ptr(), _stream()))
+        return out
 
     def profile(self, x, out=None, reps: int = 10):
         """Mean device milliseconds per layer over `reps` runs (event pair around every layer)."""

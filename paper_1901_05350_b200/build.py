@@ -33,6 +33,8 @@ SOURCES = [
     "depthwise.cu",
     "matmul_static_scratch.cu",
     "dwpw_fused_tcgen05.cu",
+    "gemm_bf16_tcgen05.cu",
+    "bf16_storage.cu",
 ]
 
 NVCC_FLAGS = [

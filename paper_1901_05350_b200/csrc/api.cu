@@ -196,7 +196,7 @@ tfjsb_status tfjsb_shutdown(tfjsb_ctx* ctx) {
 
 tfjsb_status tfjsb_set_math(tfjsb_ctx* ctx, tfjsb_math mode) {
     TFJSB_REQUIRE_CTX(ctx);
-    if (mode != TFJSB_MATH_TF32 && mode != TFJSB_MATH_FP32) return fail(ctx, TFJSB_ERR_INVALID_ARG, "unknown math mode");
+    if (mode != TFJSB_MATH_TF32 && mode != TFJSB_MATH_FP32 && mode != TFJSB_MATH_BF16) return fail(ctx, TFJSB_ERR_INVALID_ARG, "unknown math mode");
     ctx->math = mode;
     return TFJSB_OK;
 }
@@ -293,6 +293,25 @@ tfjsb_status tfjsb_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_ten
     if (M == 0 || N == 0) return TFJSB_OK;
     return matmul_2d(ctx, static_cast<const float*>(a->data), static_cast<const float*>(b->data),
                      static_cast<float*>(out->data), M, K, N, transpose_a, transpose_b, static_cast<cudaStream_t>(stream));
+}
+
+tfjsb_status tfjsb_matmul_bf16(tfjsb_ctx* ctx, const void* a, const void* bt, const float* bias, tfjsb_act act, void* out,
+                               int out_is_bf16, int64_t M, int64_t N, int64_t K, void* stream) {
+    TFJSB_REQUIRE_CTX(ctx);
+    if (!a || !bt || !out) return fail(ctx, TFJSB_ERR_INVALID_ARG, "a / bt / out is null");
+    if (act != TFJSB_ACT_NONE && act != TFJSB_ACT_RELU && act != TFJSB_ACT_RELU6)
+        return fail(ctx, TFJSB_ERR_INVALID_ARG, "unknown activation");
+    if (M < 0 || N < 0 || K < 0) return fail(ctx, TFJSB_ERR_SHAPE, "negative size");
+    if (M == 0 || N == 0) return TFJSB_OK;
+    if (!aligned16(a) || !aligned16(bt) || !aligned16(out) || (bias && !aligned16(bias)))
+        return fail(ctx, TFJSB_ERR_UNSUPPORTED, "pointers must be 16-byte aligned");
+    if (a == out || bt == out) return fail(ctx, TFJSB_ERR_INVALID_ARG, "out aliases an input");
+    GemmBf16Plan plan;
+    tfjsb_status st = gemm_bf16_plan(ctx, a, bt, out, out_is_bf16 != 0, M, N, K, &plan);
+    if (st != TFJSB_OK) return st;
+    cudaError_t e = launch_gemm_bf16(plan, bias, act, ctx->dev_status, static_cast<cudaStream_t>(stream), &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "bf16 gemm launch");
+    return TFJSB_OK;
 }
 
 tfjsb_status tfjsb_batch_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_tensor* b, int transpose_a,

@@ -222,6 +222,32 @@ cudaError_t launch_pack_filter(const float* f, float* out, int64_t K, int64_t N,
 cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int act, unsigned int* dev_status,
                              cudaStream_t s, int64_t* launches);
 
+// ---- narrow storage (bfloat16 in memory, fp32 sums) -------------------------------------------------
+// Tensor-core GEMM on bfloat16 operands: C[M,N] = act(A[M,K] . Bt[N,K]^T + bias), C bfloat16 or fp32.
+struct GemmBf16Plan {
+    CUtensorMap map_a, map_b, map_c;
+    int64_t M = 0, N = 0, K = 0;
+    bool c_is_bf16 = true;
+    int block_n = 0, stages = 0, acc_stages = 0, num_tiles = 0, grid = 0;
+    size_t smem_bytes = 0;
+};
+bool gemm_bf16_supported(int64_t M, int64_t N, int64_t K);
+tfjsb_status gemm_bf16_plan(tfjsb_ctx* ctx, const void* a, const void* bt, void* c, bool c_is_bf16, int64_t M, int64_t N,
+                            int64_t K, GemmBf16Plan* plan);
+cudaError_t launch_gemm_bf16(const GemmBf16Plan& plan, const float* bias, int act, unsigned int* dev_status,
+                             cudaStream_t s, int64_t* launches);
+// CUDA-core layers of the same mode.  Filters are fp32 arrays holding bfloat16 values.
+cudaError_t launch_conv_narrow(const void* x, bool x_is_f32, const float* f, const float* bias, int act, void* y,
+                               bool y_is_bf16, const ConvGeom& g, cudaStream_t s, int64_t* launches);
+bool depthwise_narrow_supported(const ConvGeom& g);
+cudaError_t launch_depthwise_narrow(const void* x, const float* f, const float* bias, int act, void* y, bool y_is_bf16,
+                                    const ConvGeom& g, cudaStream_t s, int64_t* launches);
+cudaError_t launch_avg_pool_global_narrow(const void* x, void* y, bool y_is_bf16, int64_t images, int positions, int C,
+                                          cudaStream_t s, int64_t* launches);
+cudaError_t launch_f32_to_bf16(const float* in, void* out, int64_t n, cudaStream_t s, int64_t* launches);
+cudaError_t launch_bf16_to_f32(const void* in, float* out, int64_t n, cudaStream_t s, int64_t* launches);
+cudaError_t launch_round_to_bf16_in_place(float* v, int64_t n, cudaStream_t s, int64_t* launches);
+
 // Fused depthwise 3x3 (stride 1) + pointwise block: the depthwise output is produced straight into
 // the tensor-core operand layout in shared memory and never written to global memory.
 // `bt` is the pointwise filter stored [Cout, Cin] (K-contiguous).

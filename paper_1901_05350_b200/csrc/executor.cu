@@ -17,7 +17,11 @@ using namespace tfjsb;
 
 namespace {
 
-enum StepKind { STEP_GEMM_TF32, STEP_GEMM_FP32, STEP_CONV_TF32, STEP_CONV_FP32, STEP_DEPTHWISE, STEP_POOL, STEP_SOFTMAX };
+enum StepKind {
+    STEP_GEMM_TF32, STEP_GEMM_FP32, STEP_CONV_TF32, STEP_CONV_FP32, STEP_DEPTHWISE, STEP_POOL, STEP_SOFTMAX,
+    // narrow-storage mode (activations and filters bfloat16 in memory, fp32 sums)
+    STEP_GEMM_NARROW, STEP_CONV_NARROW, STEP_DEPTHWISE_NARROW, STEP_POOL_NARROW
+};
 
 struct Step {
     StepKind kind;
@@ -37,6 +41,12 @@ struct Step {
     bool fusable = false;     // the pair's shapes fit the fused kernel
     bool fuse_pays = false;   // and there are enough tiles for it to be the faster choice
     DwPwPlan fused_plan{};
+    // narrow-storage mode: which of the layer's tensors are bfloat16, and the GEMM's bfloat16 filter [N,K]
+    bool is_dense = false;
+    bool in_f32 = true;
+    bool out_bf16 = false;
+    void* filter16 = nullptr;
+    GemmBf16Plan plan16{};
     int32_t out_rank = 4;
     int64_t out_dims[4] = {0, 0, 0, 0};
     int64_t out_elems = 0;
@@ -64,6 +74,7 @@ struct tfjsb_model {
     bool host_run_pending[2] = {false, false};
     int next_staging = 0;
     bool use_tf32 = true;
+    bool narrow = false;  // bfloat16 storage (TFJSB_MATH_BF16 at creation)
     // caller buffers the first/last tensor maps were last encoded for
     const void* bound_in = nullptr;
     void* bound_out = nullptr;
@@ -127,6 +138,11 @@ tfjsb_status bind_step(tfjsb_model* m, Step& st, const float* in, float* out) {
     if (st.kind == STEP_CONV_TF32 && (changed || !st.plan_built)) {
         tfjsb_status rc = st.conv_patch ? conv_patch_plan(m->ctx, in, st.filter_km, out, st.g, &st.fused_plan)
                                         : conv_igemm_plan(m->ctx, in, st.filter_km, out, st.g, &st.plan);
+        if (rc != TFJSB_OK) return rc;
+        st.plan_built = true;
+    }
+    if (st.kind == STEP_GEMM_NARROW && (changed || !st.plan_built)) {
+        tfjsb_status rc = gemm_bf16_plan(m->ctx, in, st.filter16, out, st.out_bf16, st.M, st.N, st.K, &st.plan16);
         if (rc != TFJSB_OK) return rc;
         st.plan_built = true;
     }
@@ -199,6 +215,16 @@ cudaError_t launch_step(tfjsb_model* m, const Step& st, cudaStream_t s) {
             return launch_avg_pool(st.in, st.out, st.g, s, &ctx->launches);
         case STEP_SOFTMAX:
             return launch_softmax(st.in, st.out, st.M, st.N, s, &ctx->launches);
+        case STEP_GEMM_NARROW:
+            return launch_gemm_bf16(st.plan16, st.bias, st.act, ctx->dev_status, s, &ctx->launches);
+        case STEP_CONV_NARROW:
+            return launch_conv_narrow(st.in, st.in_f32, st.filter, st.bias, st.act, st.out, st.out_bf16, st.g, s,
+                                      &ctx->launches);
+        case STEP_DEPTHWISE_NARROW:
+            return launch_depthwise_narrow(st.in, st.filter, st.bias, st.act, st.out, st.out_bf16, st.g, s, &ctx->launches);
+        case STEP_POOL_NARROW:
+            return launch_avg_pool_global_narrow(st.in, st.out, st.out_bf16, st.g.N, st.g.H * st.g.W, st.g.C, s,
+                                                 &ctx->launches);
     }
     return cudaErrorUnknown;
 }
@@ -210,6 +236,7 @@ tfjsb_model* make_batch_view(tfjsb_model* parent, int64_t n) {
     v->ctx = parent->ctx;
     v->is_view = true;
     v->use_tf32 = parent->use_tf32;
+    v->narrow = parent->narrow;
     v->use_pdl = parent->use_pdl;
     v->arena = parent->arena;
     v->region_elems = parent->region_elems;
@@ -325,6 +352,11 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
     tfjsb_model* m = new tfjsb_model();
     m->ctx = ctx;
     m->use_tf32 = ctx->math == TFJSB_MATH_TF32 && ctx->encode_tiled != nullptr;
+    m->narrow = ctx->math == TFJSB_MATH_BF16;
+    if (m->narrow && !ctx->encode_tiled) {
+        delete m;
+        return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+    }
     m->use_pdl = getenv("TFJSB_NO_PDL") == nullptr;
     for (int i = 0; i < 4; ++i) m->in_dims[i] = input_dims[i];
     m->in_elems = input_dims[0] * input_dims[1] * input_dims[2] * input_dims[3];
@@ -373,7 +405,22 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
                 const size_t f_elems = (size_t)g.fh * g.fw * g.C * (dw ? g.mult : g.Co);
                 if ((st = upload(m, L.filter, f_elems, &step.filter)) != TFJSB_OK) return bail(st, ctx->last_error);
                 if (L.bias && (st = upload(m, L.bias, (size_t)g.Co, &step.bias)) != TFJSB_OK) return bail(st, ctx->last_error);
-                if (dw) step.kind = STEP_DEPTHWISE;
+                if (m->narrow) {
+                    // what is stored is a bfloat16: the filter is rounded once, here
+                    cudaError_t e = launch_round_to_bf16_in_place(step.filter, (int64_t)f_elems, 0, &ctx->launches);
+                    if (e != cudaSuccess) return bail(TFJSB_ERR_CUDA, std::string("rounding weights: ") + cudaGetErrorString(e));
+                    if (dw) {
+                        if (li == 0) return bail(TFJSB_ERR_UNSUPPORTED, where + "in the bfloat16 storage mode the first layer must be a conv2d");
+                        if (!depthwise_narrow_supported(g))
+                            return bail(TFJSB_ERR_UNSUPPORTED, where + "the bfloat16 storage mode has depthwise 3x3, stride 1 or 2, "
+                                                                       "no dilation, multiplier 1, channels a multiple of 8");
+                        step.kind = STEP_DEPTHWISE_NARROW;
+                    } else if (li > 0 && g.fh == 1 && g.fw == 1 && g.sh == 1 && g.sw == 1 &&
+                               gemm_bf16_supported(g.N * g.H * g.W, g.Co, g.C)) {
+                        step.M = g.N * g.H * g.W; step.K = g.C; step.N = g.Co;
+                        step.kind = STEP_GEMM_NARROW;
+                    } else step.kind = STEP_CONV_NARROW;
+                } else if (dw) step.kind = STEP_DEPTHWISE;
                 else if (g.fh == 1 && g.fw == 1 && g.sh == 1 && g.sw == 1) {
                     step.M = g.N * g.H * g.W; step.K = g.C; step.N = g.Co;
                     step.kind = (m->use_tf32 && gemm_tf32_supported(step.M, step.N, step.K)) ? STEP_GEMM_TF32 : STEP_GEMM_FP32;
@@ -399,6 +446,12 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
                         return bail(TFJSB_ERR_SHAPE, where + "the pooling window does not fit the input under 'valid' padding");
                 }
                 step.kind = STEP_POOL;
+                if (m->narrow) {
+                    if (li == 0 || !global || (g.C % 8) != 0)
+                        return bail(TFJSB_ERR_UNSUPPORTED, where + "the bfloat16 storage mode has the global average pool only "
+                                                                   "(channels a multiple of 8, not as the first layer)");
+                    step.kind = STEP_POOL_NARROW;
+                }
                 step.g = g;
                 if (global) {
                     step.out_rank = 2;
@@ -418,12 +471,30 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
                 if ((st = upload(m, L.filter, (size_t)(step.K * step.N), &step.filter)) != TFJSB_OK) return bail(st, ctx->last_error);
                 if (L.bias && (st = upload(m, L.bias, (size_t)step.N, &step.bias)) != TFJSB_OK) return bail(st, ctx->last_error);
                 step.kind = (m->use_tf32 && gemm_tf32_supported(step.M, step.N, step.K)) ? STEP_GEMM_TF32 : STEP_GEMM_FP32;
+                if (m->narrow) {
+                    if (li == 0) return bail(TFJSB_ERR_UNSUPPORTED, where + "in the bfloat16 storage mode the first layer must be a conv2d");
+                    cudaError_t e = launch_round_to_bf16_in_place(step.filter, step.K * step.N, 0, &ctx->launches);
+                    if (e != cudaSuccess) return bail(TFJSB_ERR_CUDA, std::string("rounding weights: ") + cudaGetErrorString(e));
+                    step.is_dense = true;
+                    if (gemm_bf16_supported(step.M, step.N, step.K)) step.kind = STEP_GEMM_NARROW;
+                    else {
+                        // a 1x1 convolution over [M,1,1,K]: the filter [K,N] already has that layout
+                        if (step.K > 0x3fffffff || step.N > 0x3fffffff) return bail(TFJSB_ERR_UNSUPPORTED, where + "too wide");
+                        ConvGeom g{};
+                        g.N = step.M; g.H = g.W = 1; g.C = (int)step.K; g.fh = g.fw = 1; g.Co = (int)step.N; g.mult = 1;
+                        g.sh = g.sw = g.dh = g.dw = 1; g.pt = g.pl = 0; g.Ho = g.Wo = 1;
+                        step.g = g;
+                        step.kind = STEP_CONV_NARROW;
+                    }
+                }
                 step.out_rank = 2;
                 step.out_dims[0] = step.M; step.out_dims[1] = step.N;
                 break;
             }
             case TFJSB_LAYER_SOFTMAX: {
                 step.kind = STEP_SOFTMAX;
+                if (m->narrow && (li == 0 || !(m->steps.back().is_dense || m->steps.back().kind == STEP_SOFTMAX)))
+                    return bail(TFJSB_ERR_UNSUPPORTED, where + "in the bfloat16 storage mode softmax follows a dense layer");
                 step.N = d[rank - 1];
                 step.M = 1;
                 for (int i = 0; i < rank - 1; ++i) step.M *= d[i];
@@ -443,6 +514,17 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
                                                step.g.Co, k_pad, 0, &ctx->launches);
             if (e != cudaSuccess) return bail(TFJSB_ERR_CUDA, std::string("packing weights: ") + cudaGetErrorString(e));
         }
+        if (step.kind == STEP_GEMM_NARROW) {
+            // weights [K,N] fp32 -> [N,K] bfloat16 once, on the device
+            float* km32 = nullptr;
+            if ((st = dev_alloc(m, (size_t)(step.K * step.N), &km32)) != TFJSB_OK) return bail(st, ctx->last_error);
+            float* km16 = nullptr;
+            if ((st = dev_alloc(m, (size_t)((step.K * step.N + 1) / 2), &km16)) != TFJSB_OK) return bail(st, ctx->last_error);
+            cudaError_t e = launch_transpose(step.filter, km32, step.K, step.N, 0, &ctx->launches);
+            if (e == cudaSuccess) e = launch_f32_to_bf16(km32, km16, step.K * step.N, 0, &ctx->launches);
+            if (e != cudaSuccess) return bail(TFJSB_ERR_CUDA, std::string("converting weights: ") + cudaGetErrorString(e));
+            step.filter16 = km16;
+        }
         if (step.kind == STEP_GEMM_TF32) {
             // weights [K,N] -> [N,K] once, on the device
             if ((st = dev_alloc(m, (size_t)(step.K * step.N), &step.filter_km)) != TFJSB_OK) return bail(st, ctx->last_error);
@@ -456,6 +538,18 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
         m->steps.push_back(step);
     }
 
+    if (m->narrow) {
+        // every layer output is stored narrow except dense and softmax outputs and the model's result
+        const size_t n = m->steps.size();
+        for (size_t i = 0; i < n; ++i) {
+            Step& sp = m->steps[i];
+            sp.out_bf16 = !sp.is_dense && sp.kind != STEP_SOFTMAX && i + 1 != n;
+            sp.in_f32 = i == 0 || !m->steps[i - 1].out_bf16;
+            if (sp.in_f32 && (sp.kind == STEP_GEMM_NARROW || sp.kind == STEP_DEPTHWISE_NARROW || sp.kind == STEP_POOL_NARROW))
+                return bail(TFJSB_ERR_UNSUPPORTED, "layer " + std::to_string(i) + ": in the bfloat16 storage mode only conv2d and "
+                                                   "softmax layers read an fp32 tensor");
+        }
+    }
     // arena: two regions, each large enough for the largest intermediate
     int64_t largest = 0;
     for (size_t i = 0; i + 1 < m->steps.size(); ++i)
@@ -691,9 +785,33 @@ tfjsb_status tfjsb_model_layer_output(tfjsb_model* m, int layer, tfjsb_tensor* v
     if (layer < 0 || layer >= (int)m->steps.size()) return fail(m->ctx, TFJSB_ERR_INVALID_ARG, "no such layer");
     const Step& st = m->steps[layer];
     if (!st.out) return fail(m->ctx, TFJSB_ERR_INVALID_ARG, "the model has not run yet");
+    if (st.out_bf16)
+        return fail(m->ctx, TFJSB_ERR_UNSUPPORTED, "this layer's output is stored as bfloat16: read it with tfjsb_model_layer_output_f32");
     view->data = st.out;
     view->rank = st.out_rank;
     for (int i = 0; i < 4; ++i) view->dims[i] = i < st.out_rank ? st.out_dims[i] : 0;
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_model_layer_shape(tfjsb_model* m, int layer, int32_t* rank, int64_t dims[4]) {
+    if (!m || !rank || !dims) return TFJSB_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= (int)m->steps.size()) return fail(m->ctx, TFJSB_ERR_INVALID_ARG, "no such layer");
+    const Step& st = m->steps[layer];
+    *rank = st.out_rank;
+    for (int i = 0; i < 4; ++i) dims[i] = i < st.out_rank ? st.out_dims[i] : 0;
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_model_layer_output_f32(tfjsb_model* m, int layer, float* dst, void* stream) {
+    if (!m) return TFJSB_ERR_INVALID_ARG;
+    if (!dst) return fail(m->ctx, TFJSB_ERR_INVALID_ARG, "dst is null");
+    if (layer < 0 || layer >= (int)m->steps.size()) return fail(m->ctx, TFJSB_ERR_INVALID_ARG, "no such layer");
+    const Step& st = m->steps[layer];
+    if (!st.out) return fail(m->ctx, TFJSB_ERR_INVALID_ARG, "the model has not run yet");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = st.out_bf16 ? launch_bf16_to_f32(st.out, dst, st.out_elems, s, &m->ctx->launches)
+                                : cudaMemcpyAsync(dst, st.out, (size_t)st.out_elems * 4, cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(m->ctx, e, "reading a layer's output");
     return TFJSB_OK;
 }
 

@@ -8,6 +8,8 @@
     python -m paper_1901_05350_b200.run_workload --workload maxpool --batch 128 --hw 112 --channels 64 --stride 2
     python -m paper_1901_05350_b200.run_workload --workload add --batch 128 --hw 56 --channels 128
     python -m paper_1901_05350_b200.run_workload --workload batch_matmul --batch 16 --size 1024
+    python -m paper_1901_05350_b200.run_workload --workload mobilenet224 --batch 128 --math bf16 --per-layer
+    python -m paper_1901_05350_b200.run_workload --workload matmul_bf16 --m 25088 --k 512 --n 512
 
 A plain driver for profilers and quick timing: it builds the inputs, runs `--warmup` untimed and
 `--steps` timed passes on one stream, prints the mean device time per pass, and exits.
@@ -24,7 +26,7 @@ sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
 def main() -> int:
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", choices=["mobilenet224", "mobilenet128_025", "matmul", "block", "depthwise", "pointwise", "maxpool", "add",
-                             "batch_matmul"],
+                             "batch_matmul", "matmul_bf16"],
                     default="mobilenet224")
     ap.add_argument("--batch", type=int, default=128)
     ap.add_argument("--size", type=int, default=512, help="matmul: M = K = N")
@@ -35,7 +37,12 @@ def main() -> int:
     ap.add_argument("--dilation", type=int, default=1, help="depthwise: dilation (with stride 1)")
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
-    ap.add_argument("--math", choices=["tf32", "fp32"], default="tf32")
+    ap.add_argument("--math", choices=["tf32", "fp32", "bf16"], default="tf32",
+                    help="bf16: the narrow-storage mode (models only)")
+    ap.add_argument("--m", type=int, default=25088, help="matmul_bf16: rows of A")
+    ap.add_argument("--k", type=int, default=512, help="matmul_bf16: inner dimension")
+    ap.add_argument("--n", type=int, default=512, help="matmul_bf16: rows of Bt")
+    ap.add_argument("--per-layer", action="store_true", help="model workloads: print every layer's mean device time")
     args = ap.parse_args()
 
     import torch
@@ -49,6 +56,11 @@ def main() -> int:
         a, b = torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()
         out = torch.empty(args.size, args.size, device="cuda")
         step = lambda: ctx.matmul(a, b, out=out)
+    elif args.workload == "matmul_bf16":
+        a = torch.from_numpy(si.uniform(7, 0, (args.m, args.k), -1.0, 1.0)).cuda().to(torch.bfloat16)
+        bt = torch.from_numpy(si.uniform(7, 1, (args.n, args.k), -1.0, 1.0)).cuda().to(torch.bfloat16)
+        out = torch.empty(args.m, args.n, dtype=torch.bfloat16, device="cuda")
+        step = lambda: ctx.matmul_bf16(a, bt, out=out)
     elif args.workload == "block":
         x, (dw, pw) = si.config_separable_block(batch=args.batch)
         x = torch.from_numpy(x).cuda()
@@ -99,6 +111,10 @@ def main() -> int:
         x = torch.from_numpy(x).cuda()
         out = torch.empty(model.output_shape, device="cuda")
         step = lambda: model.run(x, out=out)
+        if args.per_layer:
+            model.run(x, out=out)
+            for name, ms in zip(model.layer_names, model.profile(x, out=out, reps=max(args.steps, 1))):
+                print(f"  {name:12s} {ms * 1e3:8.2f} us")
 
     for _ in range(args.warmup):
         step()
