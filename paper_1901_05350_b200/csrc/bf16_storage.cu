@@ -5,7 +5,7 @@
 //
 //   conv_direct_narrow_kernel       conv2d, any window / stride / dilation; reads fp32 (the model input,
 //                                   rounded to bfloat16 as it is read) or bfloat16
-//   depthwise3x3_narrow_kernel      3x3 depthwise, stride 1 or 2, 8 channels x 4 output rows per thread
+//   depthwise3x3_narrow_kernel      3x3 depthwise, stride 1 or 2, 8 channels x 2 output rows per thread
 //   avg_pool_global_narrow_kernel   mean over H x W
 //   convert kernels                 fp32 <-> bfloat16 (weights at set-up, debug read-back)
 #include <cuda_bf16.h>
@@ -121,11 +121,76 @@ conv_direct_narrow_kernel(const IN_T* __restrict__ x, const float* __restrict__ 
     }
 }
 
+// ---- 3x3 conv2d over a 3-channel fp32 image (the usual first layer) ---------------------------------
+// One thread: one output pixel, all COUT (<= 32) output channels.  The 27 input samples are requested
+// up front and rounded to bfloat16; the filter sits in shared memory as [27][COUT] and is read as
+// 16-byte broadcasts; the 27 x COUT multiply-adds are issued two per instruction.
+template <int COUT, bool OUT_NARROW>
+__global__ void __launch_bounds__(128)
+conv3x3_rgb_narrow_kernel(const float* __restrict__ x, const float* __restrict__ f, const float* __restrict__ bias, int act,
+                          void* __restrict__ y, const ConvGeom g, int64_t total) {
+    __shared__ __align__(16) float w_s[27 * COUT];
+    __shared__ __align__(16) float b_s[COUT];
+    for (int i = threadIdx.x; i < 27 * COUT; i += blockDim.x) w_s[i] = __ldg(f + i);  // set-up data, not the predecessor's
+    for (int i = threadIdx.x; i < COUT; i += blockDim.x) b_s[i] = bias ? __ldg(bias + i) : 0.0f;
+    __syncthreads();
+    pdl_launch_dependents();
+    pdl_wait();
+    for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < total; p += (int64_t)gridDim.x * blockDim.x) {
+        const int ox = (int)(p % g.Wo);
+        const int oy = (int)((p / g.Wo) % g.Ho);
+        const int64_t n = p / ((int64_t)g.Wo * g.Ho);
+        const float* xn = x + n * (int64_t)g.H * g.W * 3;
+        const int iy0 = oy * g.sh - g.pt, ix0 = ox * g.sw - g.pl;
+        float xv[27];
+#pragma unroll
+        for (int ky = 0; ky < 3; ++ky) {
+            const int iy = iy0 + ky;
+            const bool row_ok = iy >= 0 && iy < g.H;
+#pragma unroll
+            for (int kx = 0; kx < 3; ++kx) {
+                const int ix = ix0 + kx;
+                const bool ok = row_ok && ix >= 0 && ix < g.W;
+                const float* xp = xn + ((int64_t)iy * g.W + ix) * 3;
+#pragma unroll
+                for (int ci = 0; ci < 3; ++ci) xv[(ky * 3 + kx) * 3 + ci] = ok ? __ldg(xp + ci) : 0.0f;
+            }
+        }
+        float2 acc[COUT / 2];
+#pragma unroll
+        for (int c = 0; c < COUT / 2; ++c) acc[c] = make_float2(0.0f, 0.0f);
+#pragma unroll
+        for (int k = 0; k < 27; ++k) {
+            const float v = round_bf16(xv[k]);
+            const float2 vv = make_float2(v, v);
+#pragma unroll
+            for (int c = 0; c < COUT / 4; ++c) {
+                const float4 w = *reinterpret_cast<const float4*>(&w_s[k * COUT + 4 * c]);
+                fma2(acc[2 * c], vv, make_float2(w.x, w.y));
+                fma2(acc[2 * c + 1], vv, make_float2(w.z, w.w));
+            }
+        }
+#pragma unroll
+        for (int c8 = 0; c8 < COUT / 8; ++c8) {
+            float v[8];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                v[2 * e] = acc[c8 * 4 + e].x + b_s[c8 * 8 + 2 * e];
+                v[2 * e + 1] = acc[c8 * 4 + e].y + b_s[c8 * 8 + 2 * e + 1];
+            }
+            store8<OUT_NARROW>(y, p * COUT + c8 * 8, v, nullptr, act);
+        }
+    }
+}
+
 // ---- depthwise 3x3 ------------------------------------------------------------------------------
 // One thread: eight channels (one 16-byte load per input sample) of DW_ROWS consecutive output rows at
-// one output column.  Input rows are walked once; each contributes to the (up to three) output rows
-// whose windows contain it.  The nine taps of the eight channels stay in registers.
-constexpr int DW_ROWS = 4;
+// one output column.  All of the thread's input samples are requested before the first is used: a
+// thread is one round trip to memory long, not one per input row, and with a dozen 16-byte loads in
+// flight per thread a dozen warps per SM keep enough bytes in flight to cover the memory latency.
+// Each input row contributes to the (up to three) output rows whose windows contain it; the taps come
+// from L1 (every thread of a channel group reads the same 72 values).
+constexpr int DW_ROWS = 2;
 
 template <int S, bool OUT_NARROW>
 __global__ void __launch_bounds__(128)
@@ -134,6 +199,7 @@ depthwise3x3_narrow_kernel(const __nv_bfloat16* __restrict__ x, const float* __r
     pdl_launch_dependents();
     pdl_wait();
     const int c8n = g.C >> 3;
+    constexpr int IN_ROWS = (DW_ROWS - 1) * S + 3;
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
         const int c0 = (int)(t % c8n) * 8;
         int64_t r = t / c8n;
@@ -142,44 +208,42 @@ depthwise3x3_narrow_kernel(const __nv_bfloat16* __restrict__ x, const float* __r
         const int oy0 = (int)(r % row_blocks) * DW_ROWS;
         const int64_t n = r / row_blocks;
 
-        float w[9][8];
+        const __nv_bfloat16* xn = x + n * (int64_t)g.H * g.W * g.C + c0;
+        const int iy_first = oy0 * S - g.pt;
+        const int ix0 = ox * S - g.pl;
+        uint4 raw[IN_ROWS][3];
 #pragma unroll
-        for (int k = 0; k < 9; ++k) {
-            const float4 a = __ldg(reinterpret_cast<const float4*>(f + (int64_t)k * g.C + c0));
-            const float4 b = __ldg(reinterpret_cast<const float4*>(f + (int64_t)k * g.C + c0 + 4));
-            w[k][0] = a.x; w[k][1] = a.y; w[k][2] = a.z; w[k][3] = a.w;
-            w[k][4] = b.x; w[k][5] = b.y; w[k][6] = b.z; w[k][7] = b.w;
+        for (int ir = 0; ir < IN_ROWS; ++ir) {
+            const int iy = iy_first + ir;
+            const bool row_ok = iy >= 0 && iy < g.H;
+#pragma unroll
+            for (int kx = 0; kx < 3; ++kx) {
+                const int ix = ix0 + kx;
+                raw[ir][kx] = make_uint4(0u, 0u, 0u, 0u);
+                if (row_ok && ix >= 0 && ix < g.W)
+                    raw[ir][kx] = __ldg(reinterpret_cast<const uint4*>(xn + ((int64_t)iy * g.W + ix) * g.C));
+            }
         }
         float acc[DW_ROWS][8];
 #pragma unroll
         for (int o = 0; o < DW_ROWS; ++o)
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[o][e] = 0.0f;
-
-        const __nv_bfloat16* xn = x + n * (int64_t)g.H * g.W * g.C + c0;
-        const int iy_first = oy0 * S - g.pt;
-        const int ix0 = ox * S - g.pl;
-        constexpr int IN_ROWS = (DW_ROWS - 1) * S + 3;
 #pragma unroll
-        for (int ir = 0; ir < IN_ROWS; ++ir) {
-            const int iy = iy_first + ir;
-            if (iy < 0 || iy >= g.H) continue;
-            float v[3][8];
+        for (int kx = 0; kx < 3; ++kx) {
 #pragma unroll
-            for (int kx = 0; kx < 3; ++kx) {
-                const int ix = ix0 + kx;
-                uint4 q = make_uint4(0u, 0u, 0u, 0u);
-                if (ix >= 0 && ix < g.W) q = __ldg(reinterpret_cast<const uint4*>(xn + ((int64_t)iy * g.W + ix) * g.C));
-                unpack8(q, v[kx]);
-            }
+            for (int ky = 0; ky < 3; ++ky) {
+                float w[8];
+                const float4 wa = __ldg(reinterpret_cast<const float4*>(f + (int64_t)(ky * 3 + kx) * g.C + c0));
+                const float4 wb = __ldg(reinterpret_cast<const float4*>(f + (int64_t)(ky * 3 + kx) * g.C + c0 + 4));
+                w[0] = wa.x; w[1] = wa.y; w[2] = wa.z; w[3] = wa.w; w[4] = wb.x; w[5] = wb.y; w[6] = wb.z; w[7] = wb.w;
 #pragma unroll
-            for (int o = 0; o < DW_ROWS; ++o) {
-                const int ky = ir - o * S;  // compile-time after unrolling
-                if (ky < 0 || ky > 2) continue;
+                for (int o = 0; o < DW_ROWS; ++o) {
+                    float v[8];
+                    unpack8(raw[o * S + ky][kx], v);
 #pragma unroll
-                for (int kx = 0; kx < 3; ++kx)
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) acc[o][e] = fmaf(v[kx][e], w[ky * 3 + kx][e], acc[o][e]);
+                    for (int e = 0; e < 8; ++e) acc[o][e] = fmaf(v[e], w[e], acc[o][e]);
+                }
             }
         }
 #pragma unroll
@@ -236,16 +300,44 @@ __global__ void round_to_bf16_in_place_kernel(float* __restrict__ v, int64_t n) 
         v[i] = round_bf16(v[i]);
 }
 
+// out [r*N, r*K]: r copies of km [N, K] down the diagonal, zeros elsewhere
+__global__ void block_diagonal_kernel(const float* __restrict__ km, float* __restrict__ out, int64_t N, int64_t K, int r) {
+    const int64_t cols = (int64_t)r * K, total = (int64_t)r * N * cols;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = i / cols, col = i - row * cols;
+        const int64_t j = row / N, n = row - j * N;
+        out[i] = (col / K == j) ? km[n * K + (col - j * K)] : 0.0f;
+    }
+}
+
 int grid_for(int64_t threads, int block) {
     const int64_t blocks = (threads + block - 1) / block;
     const int64_t cap = 148LL * 64;
     return (int)(blocks < 1 ? 1 : (blocks > cap ? cap : blocks));
 }
 
+template <int COUT>
+cudaError_t launch_rgb(const float* x, const float* f, const float* bias, int act, void* y, bool y_is_bf16, const ConvGeom& g,
+                       cudaStream_t s) {
+    const int64_t total = g.N * g.Ho * g.Wo;
+    const dim3 grid(grid_for(total, 128)), block(128);
+    return y_is_bf16 ? launch_k(conv3x3_rgb_narrow_kernel<COUT, true>, grid, block, 0, s, x, f, bias, act, y, g, total)
+                     : launch_k(conv3x3_rgb_narrow_kernel<COUT, false>, grid, block, 0, s, x, f, bias, act, y, g, total);
+}
+
 }  // namespace
 
 cudaError_t launch_conv_narrow(const void* x, bool x_is_f32, const float* f, const float* bias, int act, void* y,
                                bool y_is_bf16, const ConvGeom& g, cudaStream_t s, int64_t* launches) {
+    if (x_is_f32 && g.fh == 3 && g.fw == 3 && g.C == 3 && g.dh == 1 && g.dw == 1 && g.Co <= 32 && (g.Co % 8) == 0) {
+        const float* xf = static_cast<const float*>(x);
+        cudaError_t e = g.Co == 32 ? launch_rgb<32>(xf, f, bias, act, y, y_is_bf16, g, s)
+                        : g.Co == 24 ? launch_rgb<24>(xf, f, bias, act, y, y_is_bf16, g, s)
+                        : g.Co == 16 ? launch_rgb<16>(xf, f, bias, act, y, y_is_bf16, g, s)
+                                     : launch_rgb<8>(xf, f, bias, act, y, y_is_bf16, g, s);
+        ++*launches;
+        return e;
+    }
     const int groups = (g.Co + 7) / 8;
     const int64_t total = g.N * g.Ho * g.Wo * groups;
     const dim3 grid(grid_for(total, 256)), block(256);
@@ -303,6 +395,11 @@ cudaError_t launch_f32_to_bf16(const float* in, void* out, int64_t n, cudaStream
 }
 cudaError_t launch_bf16_to_f32(const void* in, float* out, int64_t n, cudaStream_t s, int64_t* launches) {
     bf16_to_f32_kernel<<<grid_for(n, 256), 256, 0, s>>>(static_cast<const __nv_bfloat16*>(in), out, n);
+    ++*launches;
+    return cudaGetLastError();
+}
+cudaError_t launch_block_diagonal(const float* km, float* out, int64_t N, int64_t K, int r, cudaStream_t s, int64_t* launches) {
+    block_diagonal_kernel<<<grid_for((int64_t)r * N * r * K, 256), 256, 0, s>>>(km, out, N, K, r);
     ++*launches;
     return cudaGetLastError();
 }

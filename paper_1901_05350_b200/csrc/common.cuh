@@ -247,6 +247,8 @@ cudaError_t launch_avg_pool_global_narrow(const void* x, void* y, bool y_is_bf16
 cudaError_t launch_f32_to_bf16(const float* in, void* out, int64_t n, cudaStream_t s, int64_t* launches);
 cudaError_t launch_bf16_to_f32(const void* in, float* out, int64_t n, cudaStream_t s, int64_t* launches);
 cudaError_t launch_round_to_bf16_in_place(float* v, int64_t n, cudaStream_t s, int64_t* launches);
+// out [r*N, r*K] = r copies of km [N, K] down the diagonal, zeros elsewhere
+cudaError_t launch_block_diagonal(const float* km, float* out, int64_t N, int64_t K, int r, cudaStream_t s, int64_t* launches);
 
 // Fused depthwise 3x3 (stride 1) + pointwise block: the depthwise output is produced straight into
 // the tensor-core operand layout in shared memory and never written to global memory.

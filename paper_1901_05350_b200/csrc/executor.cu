@@ -47,6 +47,13 @@ struct Step {
     bool out_bf16 = false;
     void* filter16 = nullptr;
     GemmBf16Plan plan16{};
+    // A pointwise layer with fewer than 64 input channels (K = 8, 16, 32) runs as the GEMM of r = 64 / K
+    // pixels at a time: A [M, K] read as [M / r, 64] (r pixels fill one 128-byte row), the filter laid r
+    // times down the diagonal of a [r N, 64] matrix, and C [M / r, r N] is C [M, N] as it lies in memory.
+    // The tensor core multiplies the zeros too, which such a layer (bound by its memory traffic) can
+    // afford; a k-block of which the copy engine has to zero-fill half is several times slower.
+    int pack_r = 1;
+    float* bias_packed = nullptr;
     int32_t out_rank = 4;
     int64_t out_dims[4] = {0, 0, 0, 0};
     int64_t out_elems = 0;
@@ -142,7 +149,8 @@ tfjsb_status bind_step(tfjsb_model* m, Step& st, const float* in, float* out) {
         st.plan_built = true;
     }
     if (st.kind == STEP_GEMM_NARROW && (changed || !st.plan_built)) {
-        tfjsb_status rc = gemm_bf16_plan(m->ctx, in, st.filter16, out, st.out_bf16, st.M, st.N, st.K, &st.plan16);
+        tfjsb_status rc = gemm_bf16_plan(m->ctx, in, st.filter16, out, st.out_bf16, st.M / st.pack_r, st.N * st.pack_r,
+                                         st.K * st.pack_r, &st.plan16);
         if (rc != TFJSB_OK) return rc;
         st.plan_built = true;
     }
@@ -216,7 +224,8 @@ cudaError_t launch_step(tfjsb_model* m, const Step& st, cudaStream_t s) {
         case STEP_SOFTMAX:
             return launch_softmax(st.in, st.out, st.M, st.N, s, &ctx->launches);
         case STEP_GEMM_NARROW:
-            return launch_gemm_bf16(st.plan16, st.bias, st.act, ctx->dev_status, s, &ctx->launches);
+            return launch_gemm_bf16(st.plan16, st.pack_r > 1 ? st.bias_packed : st.bias, st.act, ctx->dev_status, s,
+                                    &ctx->launches);
         case STEP_CONV_NARROW:
             return launch_conv_narrow(st.in, st.in_f32, st.filter, st.bias, st.act, st.out, st.out_bf16, st.g, s,
                                       &ctx->launches);
@@ -516,12 +525,27 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
         }
         if (step.kind == STEP_GEMM_NARROW) {
             // weights [K,N] fp32 -> [N,K] bfloat16 once, on the device
+            int r = (!step.is_dense && step.K < 64 && 64 % step.K == 0) ? (int)(64 / step.K) : 1;
+            if (r > 1 && (((int64_t)step.g.H * step.g.W) % r != 0 || !gemm_bf16_supported(step.M / r, step.N * r, 64))) r = 1;
+            step.pack_r = r;
+            const size_t w_elems = (size_t)(step.K * step.N) * r * r;
             float* km32 = nullptr;
             if ((st = dev_alloc(m, (size_t)(step.K * step.N), &km32)) != TFJSB_OK) return bail(st, ctx->last_error);
             float* km16 = nullptr;
-            if ((st = dev_alloc(m, (size_t)((step.K * step.N + 1) / 2), &km16)) != TFJSB_OK) return bail(st, ctx->last_error);
+            if ((st = dev_alloc(m, (w_elems + 1) / 2, &km16)) != TFJSB_OK) return bail(st, ctx->last_error);
             cudaError_t e = launch_transpose(step.filter, km32, step.K, step.N, 0, &ctx->launches);
-            if (e == cudaSuccess) e = launch_f32_to_bf16(km32, km16, step.K * step.N, 0, &ctx->launches);
+            if (r > 1) {
+                float* diag = nullptr;
+                if ((st = dev_alloc(m, w_elems, &diag)) != TFJSB_OK) return bail(st, ctx->last_error);
+                if (e == cudaSuccess) e = launch_block_diagonal(km32, diag, step.N, step.K, r, 0, &ctx->launches);
+                km32 = diag;
+                if (step.bias) {
+                    if ((st = dev_alloc(m, (size_t)step.N * r, &step.bias_packed)) != TFJSB_OK) return bail(st, ctx->last_error);
+                    for (int j = 0; j < r && e == cudaSuccess; ++j)
+                        e = cudaMemcpy(step.bias_packed + (size_t)j * step.N, step.bias, (size_t)step.N * 4, cudaMemcpyDeviceToDevice);
+                }
+            }
+            if (e == cudaSuccess) e = launch_f32_to_bf16(km32, km16, (int64_t)w_elems, 0, &ctx->launches);
             if (e != cudaSuccess) return bail(TFJSB_ERR_CUDA, std::string("converting weights: ") + cudaGetErrorString(e));
             step.filter16 = km16;
         }
