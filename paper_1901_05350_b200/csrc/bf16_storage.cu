@@ -5,7 +5,7 @@
 //
 //   conv_direct_narrow_kernel       conv2d, any window / stride / dilation; reads fp32 (the model input,
 //                                   rounded to bfloat16 as it is read) or bfloat16
-//   depthwise3x3_narrow_kernel      3x3 depthwise, stride 1 or 2, 8 channels x 2 output rows per thread
+//   depthwise3x3_narrow_kernel      3x3 depthwise, stride 1 or 2, 8 channels x a 2x2 / 1x2 block of pixels per thread
 //   avg_pool_global_narrow_kernel   mean over H x W
 //   convert kernels                 fp32 <-> bfloat16 (weights at set-up, debug read-back)
 #include <cuda_bf16.h>
@@ -184,74 +184,128 @@ conv3x3_rgb_narrow_kernel(const float* __restrict__ x, const float* __restrict__
 }
 
 // ---- depthwise 3x3 ------------------------------------------------------------------------------
-// One thread: eight channels (one 16-byte load per input sample) of DW_ROWS consecutive output rows at
-// one output column.  All of the thread's input samples are requested before the first is used: a
-// thread is one round trip to memory long, not one per input row, and with a dozen 16-byte loads in
-// flight per thread a dozen warps per SM keep enough bytes in flight to cover the memory latency.
-// Each input row contributes to the (up to three) output rows whose windows contain it; the taps come
-// from L1 (every thread of a channel group reads the same 72 values).
-constexpr int DW_ROWS = 2;
-
-template <int S, bool OUT_NARROW>
+// One thread: eight channels (one 16-byte load per input sample) of a TR x TC block of output pixels.
+// The kernel is bound by instruction issue, not by memory, so the design minimises instructions per
+// output: the block's input samples ((TR-1)S+3 rows x (TC-1)S+3 columns) are each loaded and widened to
+// fp32 once and used by every output whose window contains them; multiply-adds go two per instruction;
+// indices are 32-bit.  All loads are requested before the first is used, so a thread is one round
+// trip to memory long.  Taps come from L1 (every thread of a channel group reads the same 72 values).
+template <int S, int TR, int TC, int ACT, bool OUT_NARROW>
 __global__ void __launch_bounds__(128)
 depthwise3x3_narrow_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ f, const float* __restrict__ bias,
-                           int act, void* __restrict__ y, const ConvGeom g, int row_blocks, int64_t total) {
+                           void* __restrict__ y, const ConvGeom g, int row_blocks, int col_blocks, uint32_t total) {
     pdl_launch_dependents();
     pdl_wait();
-    const int c8n = g.C >> 3;
-    constexpr int IN_ROWS = (DW_ROWS - 1) * S + 3;
-    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
-        const int c0 = (int)(t % c8n) * 8;
-        int64_t r = t / c8n;
-        const int ox = (int)(r % g.Wo);
-        r /= g.Wo;
-        const int oy0 = (int)(r % row_blocks) * DW_ROWS;
-        const int64_t n = r / row_blocks;
+    const uint32_t c8n = (uint32_t)g.C >> 3;  // 16-byte pieces per pixel
+    constexpr int IN_ROWS = (TR - 1) * S + 3, IN_COLS = (TC - 1) * S + 3;
+    for (uint32_t t = blockIdx.x * blockDim.x + threadIdx.x; t < total; t += gridDim.x * blockDim.x) {
+        uint32_t r = t / c8n;
+        const uint32_t cg = t - r * c8n;
+        uint32_t q = r / (uint32_t)col_blocks;
+        const int ox0 = (int)(r - q * (uint32_t)col_blocks) * TC;
+        const uint32_t n = q / (uint32_t)row_blocks;
+        const int oy0 = (int)(q - n * (uint32_t)row_blocks) * TR;
 
-        const __nv_bfloat16* xn = x + n * (int64_t)g.H * g.W * g.C + c0;
+        // 16-byte pieces of this image, this channel group: piece (iy * W + ix) * c8n
+        const uint4* xn = reinterpret_cast<const uint4*>(x) + ((int64_t)n * g.H * g.W * c8n + cg);
         const int iy_first = oy0 * S - g.pt;
-        const int ix0 = ox * S - g.pl;
-        uint4 raw[IN_ROWS][3];
+        const int ix_first = ox0 * S - g.pl;
+        int col_off[IN_COLS];
+        bool col_ok[IN_COLS];
+#pragma unroll
+        for (int ic = 0; ic < IN_COLS; ++ic) {
+            const int ix = ix_first + ic;
+            col_ok[ic] = ix >= 0 && ix < g.W;
+            col_off[ic] = ix * (int)c8n;
+        }
+        uint4 raw[IN_ROWS][IN_COLS];
 #pragma unroll
         for (int ir = 0; ir < IN_ROWS; ++ir) {
             const int iy = iy_first + ir;
             const bool row_ok = iy >= 0 && iy < g.H;
+            const uint4* xr = xn + iy * g.W * (int)c8n;
 #pragma unroll
-            for (int kx = 0; kx < 3; ++kx) {
-                const int ix = ix0 + kx;
-                raw[ir][kx] = make_uint4(0u, 0u, 0u, 0u);
-                if (row_ok && ix >= 0 && ix < g.W)
-                    raw[ir][kx] = __ldg(reinterpret_cast<const uint4*>(xn + ((int64_t)iy * g.W + ix) * g.C));
+            for (int ic = 0; ic < IN_COLS; ++ic) {
+                raw[ir][ic] = make_uint4(0u, 0u, 0u, 0u);
+                if (row_ok && col_ok[ic]) raw[ir][ic] = __ldg(xr + col_off[ic]);
             }
         }
-        float acc[DW_ROWS][8];
+        const float4* fq = reinterpret_cast<const float4*>(f) + 2 * cg;  // tap k: pieces k * (C / 4) + {0, 1}
+        float2 w[9][4];
 #pragma unroll
-        for (int o = 0; o < DW_ROWS; ++o)
+        for (int k = 0; k < 9; ++k) {
+            const float4 wa = __ldg(fq + k * 2 * (int)c8n);
+            const float4 wb = __ldg(fq + k * 2 * (int)c8n + 1);
+            w[k][0] = make_float2(wa.x, wa.y); w[k][1] = make_float2(wa.z, wa.w);
+            w[k][2] = make_float2(wb.x, wb.y); w[k][3] = make_float2(wb.z, wb.w);
+        }
+        // the accumulators start from the bias
+        float2 b2[4];
+        if (bias != nullptr) {
+            const float4 ba = __ldg(reinterpret_cast<const float4*>(bias) + 2 * cg);
+            const float4 bb = __ldg(reinterpret_cast<const float4*>(bias) + 2 * cg + 1);
+            b2[0] = make_float2(ba.x, ba.y); b2[1] = make_float2(ba.z, ba.w);
+            b2[2] = make_float2(bb.x, bb.y); b2[3] = make_float2(bb.z, bb.w);
+        } else {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[o][e] = 0.0f;
+            for (int e = 0; e < 4; ++e) b2[e] = make_float2(0.0f, 0.0f);
+        }
+        float2 acc[TR][TC][4];
 #pragma unroll
-        for (int kx = 0; kx < 3; ++kx) {
+        for (int a = 0; a < TR; ++a)
 #pragma unroll
-            for (int ky = 0; ky < 3; ++ky) {
-                float w[8];
-                const float4 wa = __ldg(reinterpret_cast<const float4*>(f + (int64_t)(ky * 3 + kx) * g.C + c0));
-                const float4 wb = __ldg(reinterpret_cast<const float4*>(f + (int64_t)(ky * 3 + kx) * g.C + c0 + 4));
-                w[0] = wa.x; w[1] = wa.y; w[2] = wa.z; w[3] = wa.w; w[4] = wb.x; w[5] = wb.y; w[6] = wb.z; w[7] = wb.w;
+            for (int b = 0; b < TC; ++b)
 #pragma unroll
-                for (int o = 0; o < DW_ROWS; ++o) {
-                    float v[8];
-                    unpack8(raw[o * S + ky][kx], v);
+                for (int e = 0; e < 4; ++e) acc[a][b][e] = make_float2(0.0f, 0.0f);
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) acc[o][e] = fmaf(v[e], w[e], acc[o][e]);
+        for (int ir = 0; ir < IN_ROWS; ++ir) {
+#pragma unroll
+            for (int ic = 0; ic < IN_COLS; ++ic) {
+                float2 v[4];
+                v[0] = make_float2(bf16_lo(raw[ir][ic].x), bf16_hi(raw[ir][ic].x));
+                v[1] = make_float2(bf16_lo(raw[ir][ic].y), bf16_hi(raw[ir][ic].y));
+                v[2] = make_float2(bf16_lo(raw[ir][ic].z), bf16_hi(raw[ir][ic].z));
+                v[3] = make_float2(bf16_lo(raw[ir][ic].w), bf16_hi(raw[ir][ic].w));
+#pragma unroll
+                for (int a = 0; a < TR; ++a) {
+                    const int ky = ir - a * S;  // all compile-time after unrolling
+                    if (ky < 0 || ky > 2) continue;
+#pragma unroll
+                    for (int b = 0; b < TC; ++b) {
+                        const int kx = ic - b * S;
+                        if (kx < 0 || kx > 2) continue;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) fma2(acc[a][b][e], v[e], w[ky * 3 + kx][e]);
+                    }
                 }
             }
         }
 #pragma unroll
-        for (int o = 0; o < DW_ROWS; ++o) {
-            const int oy = oy0 + o;
+        for (int a = 0; a < TR; ++a) {
+            const int oy = oy0 + a;
             if (oy >= g.Ho) break;
-            const int64_t elem = ((n * g.Ho + oy) * (int64_t)g.Wo + ox) * g.C + c0;
-            store8<OUT_NARROW>(y, elem, acc[o], bias ? bias + c0 : nullptr, act);
+#pragma unroll
+            for (int b = 0; b < TC; ++b) {
+                const int ox = ox0 + b;
+                if (ox >= g.Wo) break;
+                float v[8];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    // the sum of the products first, then one addition of the bias, as everywhere
+                    v[2 * e] = apply_act_t<ACT>(acc[a][b][e].x + b2[e].x);
+                    v[2 * e + 1] = apply_act_t<ACT>(acc[a][b][e].y + b2[e].y);
+                }
+                const int64_t piece = (((int64_t)n * g.Ho + oy) * g.Wo + ox) * c8n + cg;
+                if (OUT_NARROW) {
+                    uint4 o;
+                    o.x = pack_bf16(v[0], v[1]); o.y = pack_bf16(v[2], v[3]); o.z = pack_bf16(v[4], v[5]); o.w = pack_bf16(v[6], v[7]);
+                    static_cast<uint4*>(y)[piece] = o;
+                } else {
+                    float4* dst = static_cast<float4*>(y) + 2 * piece;
+                    dst[0] = make_float4(v[0], v[1], v[2], v[3]);
+                    dst[1] = make_float4(v[4], v[5], v[6], v[7]);
+                }
+            }
         }
     }
 }
@@ -357,22 +411,36 @@ cudaError_t launch_conv_narrow(const void* x, bool x_is_f32, const float* f, con
 
 bool depthwise_narrow_supported(const ConvGeom& g) {
     return g.fh == 3 && g.fw == 3 && g.mult == 1 && g.dh == 1 && g.dw == 1 && g.sh == g.sw && (g.sh == 1 || g.sh == 2) &&
-           (g.C % 8) == 0;
+           (g.C % 8) == 0 && g.N * g.Ho * g.Wo * (g.C / 8) < (1LL << 31) && (int64_t)g.H * g.W * g.C < (1LL << 31);
 }
+
+namespace {
+template <int S, int TR, int TC, int ACT>
+cudaError_t launch_dw_act(const __nv_bfloat16* x, const float* f, const float* bias, void* y, bool y_is_bf16,
+                          const ConvGeom& g, cudaStream_t s) {
+    const int row_blocks = (g.Ho + TR - 1) / TR, col_blocks = (g.Wo + TC - 1) / TC;
+    const uint32_t total = (uint32_t)(g.N * row_blocks * col_blocks * (g.C / 8));
+    const dim3 grid(grid_for(total, 128)), block(128);
+    return y_is_bf16 ? launch_k(depthwise3x3_narrow_kernel<S, TR, TC, ACT, true>, grid, block, 0, s, x, f, bias, y, g,
+                                row_blocks, col_blocks, total)
+                     : launch_k(depthwise3x3_narrow_kernel<S, TR, TC, ACT, false>, grid, block, 0, s, x, f, bias, y, g,
+                                row_blocks, col_blocks, total);
+}
+template <int S, int TR, int TC>
+cudaError_t launch_dw(const __nv_bfloat16* x, const float* f, const float* bias, int act, void* y, bool y_is_bf16,
+                      const ConvGeom& g, cudaStream_t s) {
+    if (act == TFJSB_ACT_RELU6) return launch_dw_act<S, TR, TC, TFJSB_ACT_RELU6>(x, f, bias, y, y_is_bf16, g, s);
+    if (act == TFJSB_ACT_RELU) return launch_dw_act<S, TR, TC, TFJSB_ACT_RELU>(x, f, bias, y, y_is_bf16, g, s);
+    return launch_dw_act<S, TR, TC, TFJSB_ACT_NONE>(x, f, bias, y, y_is_bf16, g, s);
+}
+}  // namespace
 
 cudaError_t launch_depthwise_narrow(const void* x, const float* f, const float* bias, int act, void* y, bool y_is_bf16,
                                     const ConvGeom& g, cudaStream_t s, int64_t* launches) {
-    const int row_blocks = (g.Ho + DW_ROWS - 1) / DW_ROWS;
-    const int64_t total = g.N * row_blocks * g.Wo * (g.C / 8);
-    const dim3 grid(grid_for(total, 128)), block(128);
     const __nv_bfloat16* xh = static_cast<const __nv_bfloat16*>(x);
-    cudaError_t e;
-    if (g.sh == 1)
-        e = y_is_bf16 ? launch_k(depthwise3x3_narrow_kernel<1, true>, grid, block, 0, s, xh, f, bias, act, y, g, row_blocks, total)
-                      : launch_k(depthwise3x3_narrow_kernel<1, false>, grid, block, 0, s, xh, f, bias, act, y, g, row_blocks, total);
-    else
-        e = y_is_bf16 ? launch_k(depthwise3x3_narrow_kernel<2, true>, grid, block, 0, s, xh, f, bias, act, y, g, row_blocks, total)
-                      : launch_k(depthwise3x3_narrow_kernel<2, false>, grid, block, 0, s, xh, f, bias, act, y, g, row_blocks, total);
+    // stride 1: 2 x 2 outputs from 4 x 4 samples; stride 2: 1 x 2 outputs from 3 x 5 samples
+    cudaError_t e = g.sh == 1 ? launch_dw<1, 2, 2>(xh, f, bias, act, y, y_is_bf16, g, s)
+                              : launch_dw<2, 1, 2>(xh, f, bias, act, y, y_is_bf16, g, s);
     ++*launches;
     return e;
 }
