@@ -425,6 +425,35 @@ def run_ours(args):
                               "ms_per_inference_stream": plain_ms, "ms_per_inference_graph_replay": graph_ms,
                               "note": "all weights and activations are L2-resident at batch 1; launch-latency bound"}
             m1.close()
+            # ---- the same model and batch in the narrow-storage mode (bfloat16 in memory, fp32 sums): a second
+            # number beside the headline, never in place of it (the headline's storage format is fp32)
+            ctx.set_math("bf16")
+            try:
+                mn = ctx.model(layers, x_host.shape)
+            finally:
+                ctx.set_math("tf32")
+            on = torch.empty(mn.output_shape, device="cuda")
+            for _ in range(5):
+                mn.run(x, out=on)
+            torch.cuda.synchronize()
+            n_steps = max(20, min(200, args.steps))
+            start.record(stream)
+            for _ in range(n_steps):
+                mn.run(x, out=on)
+            stop.record(stream)
+            torch.cuda.synchronize()
+            ctx.check_device_status()
+            narrow_ms = start.elapsed_time(stop) / n_steps
+            layer_us = [round(v * 1e3, 2) for v in mn.profile(x, out=on, reps=10)]
+            agree = float((on.argmax(-1) == out.argmax(-1)).float().mean())
+            line["narrow_storage"] = {
+                "metric": METRIC + ", bfloat16 storage", "value": BATCH / (narrow_ms * 1e-3), "unit": UNIT,
+                "ms_per_step": narrow_ms, "steps": n_steps,
+                "dtype": "bf16 storage of filters and activations, exact products, f32 sums; model input and output f32",
+                "top1_agreement_with_f32_storage": agree,
+                "per_layer_us": dict(zip(mn.layer_names, layer_us)),
+            }
+            mn.close()
         if cpu_baseline is not None:
             line["cpu_baseline"] = cpu_baseline
         print(json.dumps(line), flush=True)

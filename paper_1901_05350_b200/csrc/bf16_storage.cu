@@ -210,24 +210,34 @@ depthwise3x3_narrow_kernel(const __nv_bfloat16* __restrict__ x, const float* __r
         const uint4* xn = reinterpret_cast<const uint4*>(x) + ((int64_t)n * g.H * g.W * c8n + cg);
         const int iy_first = oy0 * S - g.pt;
         const int ix_first = ox0 * S - g.pl;
-        int col_off[IN_COLS];
-        bool col_ok[IN_COLS];
-#pragma unroll
-        for (int ic = 0; ic < IN_COLS; ++ic) {
-            const int ix = ix_first + ic;
-            col_ok[ic] = ix >= 0 && ix < g.W;
-            col_off[ic] = ix * (int)c8n;
-        }
         uint4 raw[IN_ROWS][IN_COLS];
+        if (iy_first >= 0 && iy_first + IN_ROWS <= g.H && ix_first >= 0 && ix_first + IN_COLS <= g.W) {
+            // the whole window lies inside the image (most blocks): one base address, constant strides
+            const uint4* x0 = xn + (iy_first * g.W + ix_first) * (int)c8n;
+            const int row_pitch = g.W * (int)c8n;
 #pragma unroll
-        for (int ir = 0; ir < IN_ROWS; ++ir) {
-            const int iy = iy_first + ir;
-            const bool row_ok = iy >= 0 && iy < g.H;
-            const uint4* xr = xn + iy * g.W * (int)c8n;
+            for (int ir = 0; ir < IN_ROWS; ++ir)
+#pragma unroll
+                for (int ic = 0; ic < IN_COLS; ++ic) raw[ir][ic] = __ldg(x0 + ir * row_pitch + ic * (int)c8n);
+        } else {
+            int col_off[IN_COLS];
+            bool col_ok[IN_COLS];
 #pragma unroll
             for (int ic = 0; ic < IN_COLS; ++ic) {
-                raw[ir][ic] = make_uint4(0u, 0u, 0u, 0u);
-                if (row_ok && col_ok[ic]) raw[ir][ic] = __ldg(xr + col_off[ic]);
+                const int ix = ix_first + ic;
+                col_ok[ic] = ix >= 0 && ix < g.W;
+                col_off[ic] = ix * (int)c8n;
+            }
+#pragma unroll
+            for (int ir = 0; ir < IN_ROWS; ++ir) {
+                const int iy = iy_first + ir;
+                const bool row_ok = iy >= 0 && iy < g.H;
+                const uint4* xr = xn + iy * g.W * (int)c8n;
+#pragma unroll
+                for (int ic = 0; ic < IN_COLS; ++ic) {
+                    raw[ir][ic] = make_uint4(0u, 0u, 0u, 0u);
+                    if (row_ok && col_ok[ic]) raw[ir][ic] = __ldg(xr + col_off[ic]);
+                }
             }
         }
         const float4* fq = reinterpret_cast<const float4*>(f) + 2 * cg;  // tap k: pieces k * (C / 4) + {0, 1}
