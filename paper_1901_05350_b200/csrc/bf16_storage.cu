@@ -122,9 +122,49 @@ conv_direct_narrow_kernel(const IN_T* __restrict__ x, const float* __restrict__ 
 }
 
 // ---- 3x3 conv2d over a 3-channel fp32 image (the usual first layer) ---------------------------------
-// One thread: one output pixel, all COUT (<= 32) output channels.  The 27 input samples are requested
-// up front and rounded to bfloat16; the filter sits in shared memory as [27][COUT] and is read as
-// 16-byte broadcasts; the 27 x COUT multiply-adds are issued two per instruction.
+// One thread: two output pixels (128 pixels apart, so that a warp's loads and stores stay dense), all
+// COUT (<= 32) output channels of each.  The kernel is bound by the L1 / shared-memory pipe, so it
+// spends as few of that pipe's cycles as it can: the filter sits in shared memory as [27][COUT] and
+// each 16-byte broadcast read of it feeds both pixels; the 27 input samples of a pixel (three runs of
+// nine consecutive floats) are fetched as 8-byte loads where the run is aligned and inside the image.
+// Samples are rounded to bfloat16 as they are used; multiply-adds go two per instruction.
+__device__ __forceinline__ void load_rgb_window(const float* __restrict__ x, const ConvGeom& g, int64_t p, bool live,
+                                                float (&xv)[27]) {
+#pragma unroll
+    for (int k = 0; k < 27; ++k) xv[k] = 0.0f;
+    if (!live) return;
+    const int ox = (int)(p % g.Wo);
+    const int oy = (int)((p / g.Wo) % g.Ho);
+    const int64_t n = p / ((int64_t)g.Wo * g.Ho);
+    const float* xn = x + n * (int64_t)g.H * g.W * 3;
+    const int iy0 = oy * g.sh - g.pt, ix0 = ox * g.sw - g.pl;
+    // a run starts on an 8-byte boundary when (iy * W + ix0) * 3 is even
+    const bool fast = ix0 >= 0 && ix0 + 2 < g.W && (g.W & 1) == 0 && (ix0 & 1) == 0;
+#pragma unroll
+    for (int ky = 0; ky < 3; ++ky) {
+        const int iy = iy0 + ky;
+        if (iy < 0 || iy >= g.H) continue;
+        const float* rp = xn + ((int64_t)iy * g.W + ix0) * 3;
+        if (fast) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float2 v = __ldg(reinterpret_cast<const float2*>(rp) + q);
+                xv[ky * 9 + 2 * q] = v.x;
+                xv[ky * 9 + 2 * q + 1] = v.y;
+            }
+            xv[ky * 9 + 8] = __ldg(rp + 8);
+        } else {
+#pragma unroll
+            for (int kx = 0; kx < 3; ++kx) {
+                const int ix = ix0 + kx;
+                if (ix < 0 || ix >= g.W) continue;
+#pragma unroll
+                for (int ci = 0; ci < 3; ++ci) xv[ky * 9 + kx * 3 + ci] = __ldg(rp + kx * 3 + ci);
+            }
+        }
+    }
+}
+
 template <int COUT, bool OUT_NARROW>
 __global__ void __launch_bounds__(128)
 conv3x3_rgb_narrow_kernel(const float* __restrict__ x, const float* __restrict__ f, const float* __restrict__ bias, int act,
@@ -136,49 +176,43 @@ conv3x3_rgb_narrow_kernel(const float* __restrict__ x, const float* __restrict__
     __syncthreads();
     pdl_launch_dependents();
     pdl_wait();
-    for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < total; p += (int64_t)gridDim.x * blockDim.x) {
-        const int ox = (int)(p % g.Wo);
-        const int oy = (int)((p / g.Wo) % g.Ho);
-        const int64_t n = p / ((int64_t)g.Wo * g.Ho);
-        const float* xn = x + n * (int64_t)g.H * g.W * 3;
-        const int iy0 = oy * g.sh - g.pt, ix0 = ox * g.sw - g.pl;
-        float xv[27];
+    for (int64_t base = (int64_t)blockIdx.x * 256; base < total; base += (int64_t)gridDim.x * 256) {
+        const int64_t p0 = base + threadIdx.x, p1 = p0 + 128;
+        float xa[27], xb[27];
+        load_rgb_window(x, g, p0, p0 < total, xa);
+        load_rgb_window(x, g, p1, p1 < total, xb);
+        float2 acc0[COUT / 2], acc1[COUT / 2];
 #pragma unroll
-        for (int ky = 0; ky < 3; ++ky) {
-            const int iy = iy0 + ky;
-            const bool row_ok = iy >= 0 && iy < g.H;
-#pragma unroll
-            for (int kx = 0; kx < 3; ++kx) {
-                const int ix = ix0 + kx;
-                const bool ok = row_ok && ix >= 0 && ix < g.W;
-                const float* xp = xn + ((int64_t)iy * g.W + ix) * 3;
-#pragma unroll
-                for (int ci = 0; ci < 3; ++ci) xv[(ky * 3 + kx) * 3 + ci] = ok ? __ldg(xp + ci) : 0.0f;
-            }
-        }
-        float2 acc[COUT / 2];
-#pragma unroll
-        for (int c = 0; c < COUT / 2; ++c) acc[c] = make_float2(0.0f, 0.0f);
+        for (int c = 0; c < COUT / 2; ++c) acc0[c] = acc1[c] = make_float2(0.0f, 0.0f);
 #pragma unroll
         for (int k = 0; k < 27; ++k) {
-            const float v = round_bf16(xv[k]);
-            const float2 vv = make_float2(v, v);
+            const float va = round_bf16(xa[k]), vb = round_bf16(xb[k]);
+            const float2 a2 = make_float2(va, va), b2 = make_float2(vb, vb);
 #pragma unroll
             for (int c = 0; c < COUT / 4; ++c) {
                 const float4 w = *reinterpret_cast<const float4*>(&w_s[k * COUT + 4 * c]);
-                fma2(acc[2 * c], vv, make_float2(w.x, w.y));
-                fma2(acc[2 * c + 1], vv, make_float2(w.z, w.w));
+                const float2 wl = make_float2(w.x, w.y), wh = make_float2(w.z, w.w);
+                fma2(acc0[2 * c], a2, wl);
+                fma2(acc0[2 * c + 1], a2, wh);
+                fma2(acc1[2 * c], b2, wl);
+                fma2(acc1[2 * c + 1], b2, wh);
             }
         }
 #pragma unroll
-        for (int c8 = 0; c8 < COUT / 8; ++c8) {
-            float v[8];
+        for (int half = 0; half < 2; ++half) {
+            const int64_t p = half ? p1 : p0;
+            if (p >= total) continue;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                v[2 * e] = acc[c8 * 4 + e].x + b_s[c8 * 8 + 2 * e];
-                v[2 * e + 1] = acc[c8 * 4 + e].y + b_s[c8 * 8 + 2 * e + 1];
+            for (int c8 = 0; c8 < COUT / 8; ++c8) {
+                float v[8];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 a = half ? acc1[c8 * 4 + e] : acc0[c8 * 4 + e];
+                    v[2 * e] = a.x + b_s[c8 * 8 + 2 * e];
+                    v[2 * e + 1] = a.y + b_s[c8 * 8 + 2 * e + 1];
+                }
+                store8<OUT_NARROW>(y, p * COUT + c8 * 8, v, nullptr, act);
             }
-            store8<OUT_NARROW>(y, p * COUT + c8 * 8, v, nullptr, act);
         }
     }
 }
@@ -384,7 +418,7 @@ template <int COUT>
 cudaError_t launch_rgb(const float* x, const float* f, const float* bias, int act, void* y, bool y_is_bf16, const ConvGeom& g,
                        cudaStream_t s) {
     const int64_t total = g.N * g.Ho * g.Wo;
-    const dim3 grid(grid_for(total, 128)), block(128);
+    const dim3 grid(grid_for(total, 256)), block(128);  // 256 pixels per block and pass
     return y_is_bf16 ? launch_k(conv3x3_rgb_narrow_kernel<COUT, true>, grid, block, 0, s, x, f, bias, act, y, g, total)
                      : launch_k(conv3x3_rgb_narrow_kernel<COUT, false>, grid, block, 0, s, x, f, bias, act, y, g, total);
 }
