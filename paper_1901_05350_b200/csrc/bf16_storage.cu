@@ -165,9 +165,9 @@ __device__ __forceinline__ void load_rgb_window(const float* __restrict__ x, con
     }
 }
 
-template <int COUT, bool OUT_NARROW>
+template <int COUT, int ACT, bool OUT_NARROW>
 __global__ void __launch_bounds__(128)
-conv3x3_rgb_narrow_kernel(const float* __restrict__ x, const float* __restrict__ f, const float* __restrict__ bias, int act,
+conv3x3_rgb_narrow_kernel(const float* __restrict__ x, const float* __restrict__ f, const float* __restrict__ bias,
                           void* __restrict__ y, const ConvGeom g, int64_t total) {
     __shared__ __align__(16) float w_s[27 * COUT];
     __shared__ __align__(16) float b_s[COUT];
@@ -199,19 +199,31 @@ conv3x3_rgb_narrow_kernel(const float* __restrict__ x, const float* __restrict__
             }
         }
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const int64_t p = half ? p1 : p0;
-            if (p >= total) continue;
+        for (int c8 = 0; c8 < COUT / 8; ++c8) {
+            const float4 ba = *reinterpret_cast<const float4*>(&b_s[c8 * 8]);
+            const float4 bb = *reinterpret_cast<const float4*>(&b_s[c8 * 8 + 4]);
+            const float b8[8] = {ba.x, ba.y, ba.z, ba.w, bb.x, bb.y, bb.z, bb.w};
 #pragma unroll
-            for (int c8 = 0; c8 < COUT / 8; ++c8) {
+            for (int half = 0; half < 2; ++half) {
+                const int64_t p = half ? p1 : p0;
+                if (p >= total) continue;
                 float v[8];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const float2 a = half ? acc1[c8 * 4 + e] : acc0[c8 * 4 + e];
-                    v[2 * e] = a.x + b_s[c8 * 8 + 2 * e];
-                    v[2 * e + 1] = a.y + b_s[c8 * 8 + 2 * e + 1];
+                    v[2 * e] = apply_act_t<ACT>(a.x + b8[2 * e]);
+                    v[2 * e + 1] = apply_act_t<ACT>(a.y + b8[2 * e + 1]);
                 }
-                store8<OUT_NARROW>(y, p * COUT + c8 * 8, v, nullptr, act);
+                const int64_t elem = p * COUT + c8 * 8;
+                if (OUT_NARROW) {
+                    uint4 o;
+                    o.x = pack_bf16(v[0], v[1]); o.y = pack_bf16(v[2], v[3]); o.z = pack_bf16(v[4], v[5]); o.w = pack_bf16(v[6], v[7]);
+                    *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(y) + elem) = o;
+                } else {
+                    float4* dst = reinterpret_cast<float4*>(static_cast<float*>(y) + elem);
+                    dst[0] = make_float4(v[0], v[1], v[2], v[3]);
+                    dst[1] = make_float4(v[4], v[5], v[6], v[7]);
+                }
             }
         }
     }
@@ -414,13 +426,20 @@ int grid_for(int64_t threads, int block) {
     return (int)(blocks < 1 ? 1 : (blocks > cap ? cap : blocks));
 }
 
+template <int COUT, int ACT>
+cudaError_t launch_rgb_act(const float* x, const float* f, const float* bias, void* y, bool y_is_bf16, const ConvGeom& g,
+                           cudaStream_t s) {
+    const int64_t total = g.N * g.Ho * g.Wo;
+    const dim3 grid(grid_for(total, 256)), block(128);  // 256 pixels per block and pass
+    return y_is_bf16 ? launch_k(conv3x3_rgb_narrow_kernel<COUT, ACT, true>, grid, block, 0, s, x, f, bias, y, g, total)
+                     : launch_k(conv3x3_rgb_narrow_kernel<COUT, ACT, false>, grid, block, 0, s, x, f, bias, y, g, total);
+}
 template <int COUT>
 cudaError_t launch_rgb(const float* x, const float* f, const float* bias, int act, void* y, bool y_is_bf16, const ConvGeom& g,
                        cudaStream_t s) {
-    const int64_t total = g.N * g.Ho * g.Wo;
-    const dim3 grid(grid_for(total, 256)), block(128);  // 256 pixels per block and pass
-    return y_is_bf16 ? launch_k(conv3x3_rgb_narrow_kernel<COUT, true>, grid, block, 0, s, x, f, bias, act, y, g, total)
-                     : launch_k(conv3x3_rgb_narrow_kernel<COUT, false>, grid, block, 0, s, x, f, bias, act, y, g, total);
+    if (act == TFJSB_ACT_RELU6) return launch_rgb_act<COUT, TFJSB_ACT_RELU6>(x, f, bias, y, y_is_bf16, g, s);
+    if (act == TFJSB_ACT_RELU) return launch_rgb_act<COUT, TFJSB_ACT_RELU>(x, f, bias, y, y_is_bf16, g, s);
+    return launch_rgb_act<COUT, TFJSB_ACT_NONE>(x, f, bias, y, y_is_bf16, g, s);
 }
 
 }  // namespace

@@ -9,10 +9,14 @@
 // rounding (to nearest even) to bfloat16 when it is stored narrow.
 //
 // Same structure as the TF32 kernel (one persistent CTA per SM; a producer warp issuing bulk tensor
-// copies into a ring of 128-byte-swizzled stages, an MMA warp, eight epilogue warps; two or four
+// copies into a ring of 128-byte-swizzled stages, an MMA warp, epilogue warps; two or four
 // accumulator stages), and the same bytes per stage: a k-block is 64 bfloat16 = one 128-byte swizzle
 // row, consumed by four `tcgen05.mma.kind::f16` of K = 16.  Half the bytes per element means half the
 // k-blocks for the same K, and half the bytes of A and C to move.
+//
+// With half the bytes per tile the layers with one or two k-blocks per tile are bound by the epilogue's
+// latency per 32 x 32 block (tcgen05.ld, bias, activation, rounding, staging, store), so there are
+// sixteen epilogue warps, four per lane quadrant, taking every fourth block.
 //
 // Every wait is bounded, as in the TF32 kernel.
 #include <cuda_bf16.h>
@@ -29,7 +33,8 @@ using namespace tile;
 namespace {
 
 constexpr int MAX_STAGES = 8;
-constexpr int GEMM_THREADS = 320;  // producer warp, MMA warp, 8 epilogue warps
+constexpr int EPI_WARPS = 16;      // four per tensor-memory lane quadrant
+constexpr int GEMM_THREADS = 64 + EPI_WARPS * 32;  // producer warp, MMA warp, the epilogue warps
 constexpr int BK16 = 64;           // bfloat16 elements per k-block (128 bytes)
 constexpr int UMMA_K16 = 16;       // elements per tcgen05.mma of kind::f16
 
@@ -111,7 +116,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     // dynamic shared memory, aligned to the 1024-byte swizzle pattern: [epilogue slabs][stage 0: A | B]...
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t epi_base = smem_base;
-    const uint32_t stage_base = smem_base + EPI_BYTES;
+    constexpr uint32_t SLAB_BYTES = OUT_BF16 ? 2048u : 4096u;  // 32 rows x 32 columns of the output type
+    const uint32_t stage_base = smem_base + EPI_WARPS * SLAB_BYTES;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -120,7 +126,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         }
         for (int s = 0; s < acc_stages; ++s) {
             mbar_init(smem_u32(&bar_acc_full[s]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[s]), 8);
+            mbar_init(smem_u32(&bar_acc_empty[s]), EPI_WARPS);
         }
         mbar_init(smem_u32(&bar_drain), 1);
         abort_flag_s = 0;
@@ -246,18 +252,19 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             }
         }
     } else {
-        // ---------------------------------------------------------------- epilogue (warps 2..9)
-        // Two warps share each TMEM lane quadrant and take alternate 32-column chunks, counted across
-        // tiles so that with one chunk per tile they alternate tiles.
+        // ---------------------------------------------------------------- epilogue (warps 2..17)
+        // Four warps share each TMEM lane quadrant (a warp may only read lanes 32*(warp%4)..+31) and take
+        // every fourth 32-column block, counted across tiles so that with one block per tile they take
+        // tiles in turn.
         const int ew = warp - 2;
         const int quad = warp & 3;
-        const int half = ew >> 2;
-        const uint32_t slab = epi_base + (uint32_t)ew * EPI_SLAB_BYTES;
+        const int sub = ew >> 2;  // 0..3: which of the quadrant's four warps
+        const uint32_t slab = epi_base + (uint32_t)ew * SLAB_BYTES;
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
         const int chunks_per_tile = block_n / EPI_COLS;
-        int first_chunk = half;
+        int chunk_base = 0;  // blocks of earlier tiles, modulo 4
         for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
             const int m0 = (tile / args.n_tiles) * BLOCK_M;
             const int n0 = (tile % args.n_tiles) * block_n;
@@ -277,12 +284,12 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             if (live_cols < block_n) n_chunks = (live_cols + EPI_COLS - 1) / EPI_COLS;
             const bool rows_live = row0 < args.M;
             bool released = false;
-            for (int ch = first_chunk; ch < n_chunks; ch += 2) {
+            for (int ch = (sub - chunk_base) & 3; ch < n_chunks; ch += 4) {
                 uint32_t r[32];
                 const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * block_n + ch * EPI_COLS);
                 tc_ld_32x32(taddr, r);
                 tc_ld_wait();
-                if (ch + 2 >= n_chunks) {
+                if (ch + 4 >= n_chunks) {
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
@@ -316,7 +323,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
             }
-            if (chunks_per_tile & 1) first_chunk ^= 1;
+            chunk_base = (chunk_base + chunks_per_tile) & 3;
             if (++acc == acc_stages) { acc = 0; acc_phase ^= 1u; }
         }
         if (lane == 0) tma_store_wait_all();
@@ -380,10 +387,11 @@ tfjsb_status gemm_bf16_plan(tfjsb_ctx* ctx, const void* a, const void* bt, void*
     plan->block_n = choose_block_n(M, N, ctx->sm_count);
     plan->acc_stages = plan->block_n > 128 ? 2 : MAX_ACC_STAGES;
     const int stage_bytes = A_STAGE_BYTES + plan->block_n * 128;
-    int stages = (SMEM_LIMIT - 1024 - EPI_BYTES - 512) / stage_bytes;
+    const int epi_bytes = EPI_WARPS * (c_is_bf16 ? 2048 : 4096);
+    int stages = (SMEM_LIMIT - 1024 - epi_bytes - 512) / stage_bytes;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
     plan->stages = stages;
-    plan->smem_bytes = (size_t)1024 + EPI_BYTES + (size_t)stages * stage_bytes;
+    plan->smem_bytes = (size_t)1024 + epi_bytes + (size_t)stages * stage_bytes;
     const int64_t n_tiles = (N + plan->block_n - 1) / plan->block_n;
     const int64_t tiles = ((M + BLOCK_M - 1) / BLOCK_M) * n_tiles;
     if (tiles >= (1LL << 31)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "too many tiles");
