@@ -367,32 +367,46 @@ depthwise3x3_narrow_kernel(const __nv_bfloat16* __restrict__ x, const float* __r
 }
 
 // ---- global average pool ------------------------------------------------------------------------
-// One thread: eight channels of one image; the positions are summed in order in fp32 and divided by
-// their number.
+// Eight lanes share eight channels of one image: lane j sums positions j, j + 8, ... in fp32, the
+// partial sums meet in a butterfly over the eight lanes, and lane 0 divides by the number of positions
+// and stores.  (One thread per channel group left most of the chip idle: 128 images x 128 groups.)
 template <bool OUT_NARROW>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(256)
 avg_pool_global_narrow_kernel(const __nv_bfloat16* __restrict__ x, void* __restrict__ y, int64_t images, int positions, int C) {
     pdl_launch_dependents();
     pdl_wait();
     const int c8n = C >> 3;
-    const int64_t total = images * c8n;
-    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
-        const int c0 = (int)(t % c8n) * 8;
-        const int64_t n = t / c8n;
+    const int64_t total = images * c8n * 8;  // a multiple of 8: the eight lanes of a group stay together
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int lane = threadIdx.x & 31;
+    // whole warps enter the loop body together (the butterfly needs all 32 lanes); lanes past the end idle
+    for (int64_t base = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x - lane); base < total; base += stride) {
+        const int64_t t = base + lane;
+        const bool live = t < total;
+        const int part = (int)(t & 7);
+        const int64_t grp = live ? (t >> 3) : 0;
+        const int c0 = (int)(grp % c8n) * 8;
+        const int64_t n = grp / c8n;
         const __nv_bfloat16* xp = x + n * (int64_t)positions * C + c0;
         float acc[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[e] = 0.0f;
-        for (int p = 0; p < positions; ++p) {
+        for (int p = part; live && p < positions; p += 8) {
             float v[8];
             unpack8(__ldg(reinterpret_cast<const uint4*>(xp + (int64_t)p * C)), v);
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] += v[e];
         }
-        const float count = (float)positions;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e] = __fdiv_rn(acc[e], count);
-        store8<OUT_NARROW>(y, n * C + c0, acc, nullptr, TFJSB_ACT_NONE);
+        for (int m = 1; m < 8; m <<= 1)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], m);
+        if (live && part == 0) {
+            const float count = (float)positions;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = __fdiv_rn(acc[e], count);
+            store8<OUT_NARROW>(y, n * C + c0, acc, nullptr, TFJSB_ACT_NONE);
+        }
     }
 }
 
@@ -510,8 +524,8 @@ cudaError_t launch_depthwise_narrow(const void* x, const float* f, const float* 
 
 cudaError_t launch_avg_pool_global_narrow(const void* x, void* y, bool y_is_bf16, int64_t images, int positions, int C,
                                           cudaStream_t s, int64_t* launches) {
-    const int64_t total = images * (C / 8);
-    const dim3 grid(grid_for(total, 128)), block(128);
+    const int64_t total = images * (C / 8) * 8;
+    const dim3 grid(grid_for(total, 256)), block(256);
     const __nv_bfloat16* xh = static_cast<const __nv_bfloat16*>(x);
     cudaError_t e = y_is_bf16 ? launch_k(avg_pool_global_narrow_kernel<true>, grid, block, 0, s, xh, y, images, positions, C)
                               : launch_k(avg_pool_global_narrow_kernel<false>, grid, block, 0, s, xh, y, images, positions, C);
