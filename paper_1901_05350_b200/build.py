@@ -34,6 +34,7 @@ SOURCES = [
     "matmul_static_scratch.cu",
     "dwpw_fused_tcgen05.cu",
     "gemm_bf16_tcgen05.cu",
+    "gemm_bf16_pair.cu",
     "bf16_storage.cu",
 ]
 

@@ -228,6 +228,7 @@ struct GemmBf16Plan {
     CUtensorMap map_a, map_b, map_c;
     int64_t M = 0, N = 0, K = 0;
     bool c_is_bf16 = true;
+    bool pair = false;  // CTA-pair kernel (gemm_bf16_pair.cu): 256 x block_n tiles shared by two CTAs
     int block_n = 0, stages = 0, acc_stages = 0, num_tiles = 0, grid = 0;
     size_t smem_bytes = 0;
 };
@@ -236,6 +237,13 @@ tfjsb_status gemm_bf16_plan(tfjsb_ctx* ctx, const void* a, const void* bt, void*
                             int64_t K, GemmBf16Plan* plan);
 cudaError_t launch_gemm_bf16(const GemmBf16Plan& plan, const float* bias, int act, unsigned int* dev_status,
                              cudaStream_t s, int64_t* launches);
+// The same GEMM (bfloat16 output only) on CTA pairs; gemm_bf16_plan picks it where it is the faster
+// kernel (TFJSB_GEMM_PAIR: 0 = never, 1 = wherever the shape allows, unset = by shape).
+bool gemm_bf16_pair_preferred(int64_t M, int64_t N, int64_t K, int sm_count);
+tfjsb_status gemm_bf16_pair_plan(tfjsb_ctx* ctx, const void* a, const void* bt, void* c, int64_t M, int64_t N, int64_t K,
+                                 GemmBf16Plan* plan);
+cudaError_t launch_gemm_bf16_pair(const GemmBf16Plan& plan, const float* bias, int act, unsigned int* dev_status,
+                                  cudaStream_t s, int64_t* launches);
 // CUDA-core layers of the same mode.  Filters are fp32 arrays holding bfloat16 values.
 cudaError_t launch_conv_narrow(const void* x, bool x_is_f32, const float* f, const float* bias, int act, void* y,
                                bool y_is_bf16, const ConvGeom& g, cudaStream_t s, int64_t* launches);

@@ -21,6 +21,8 @@
 // Every wait is bounded, as in the TF32 kernel.
 #include <cuda_bf16.h>
 
+#include <cstdlib>
+
 #include "common.cuh"
 #include "ptx_sm100.cuh"
 #include "umma_tile.cuh"
@@ -48,40 +50,6 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, ui
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// Instruction descriptor: fp32 accumulator, bfloat16 A and B (format 1), both K-major.
-__device__ __forceinline__ uint32_t make_idesc_bf16(int m, int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
-}
-
-// One 32-row x 32-column accumulator block, one row per lane: bias, activation, rounding to bfloat16,
-// and the store into the staging slab in the 64-byte swizzle the bulk tensor store expects (rows of
-// 64 bytes; 16-byte piece j of row r lives at piece j ^ ((r / 2) % 4)).
-template <int ACT>
-__device__ __forceinline__ void stage_chunk_bf16(const uint32_t (&r)[32], const float* __restrict__ bias, int cols_left,
-                                                 uint32_t slab, int lane) {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        float v[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[8 * j + e]);
-        if (bias != nullptr && 8 * j < cols_left) {  // N % 8 == 0: a group of eight is all in or all out
-            const float4 b0 = __ldg(reinterpret_cast<const float4*>(bias + 8 * j));
-            const float4 b1 = __ldg(reinterpret_cast<const float4*>(bias + 8 * j + 4));
-            v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
-            v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
-        }
-        uint32_t p[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const __nv_bfloat162 h = __floats2bfloat162_rn(apply_act_t<ACT>(v[2 * e]), apply_act_t<ACT>(v[2 * e + 1]));
-            p[e] = *reinterpret_cast<const uint32_t*>(&h);
-        }
-        const uint32_t dst = slab + (uint32_t)lane * 64u + (uint32_t)((j ^ ((lane >> 1) & 3)) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(p[0]), "r"(p[1]), "r"(p[2]), "r"(p[3])
-                     : "memory");
-    }
-}
-
 struct KernelArgs {
     int M, N, K;
     int block_n;
@@ -382,8 +350,14 @@ tfjsb_status gemm_bf16_plan(tfjsb_ctx* ctx, const void* a, const void* bt, void*
                             int64_t K, GemmBf16Plan* plan) {
     if (!gemm_bf16_supported(M, N, K)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the bfloat16 GEMM");
     if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+    if (c_is_bf16) {
+        const char* pair_env = getenv("TFJSB_GEMM_PAIR");
+        const bool use_pair = pair_env ? (pair_env[0] == '1' && N >= 64) : gemm_bf16_pair_preferred(M, N, K, ctx->sm_count);
+        if (use_pair) return gemm_bf16_pair_plan(ctx, a, bt, c, M, N, K, plan);
+    }
     plan->M = M; plan->N = N; plan->K = K;
     plan->c_is_bf16 = c_is_bf16;
+    plan->pair = false;
     plan->block_n = choose_block_n(M, N, ctx->sm_count);
     plan->acc_stages = plan->block_n > 128 ? 2 : MAX_ACC_STAGES;
     const int stage_bytes = A_STAGE_BYTES + plan->block_n * 128;
@@ -411,6 +385,7 @@ tfjsb_status gemm_bf16_plan(tfjsb_ctx* ctx, const void* a, const void* bt, void*
 
 cudaError_t launch_gemm_bf16(const GemmBf16Plan& plan, const float* bias, int act, unsigned int* dev_status,
                              cudaStream_t s, int64_t* launches) {
+    if (plan.pair) return launch_gemm_bf16_pair(plan, bias, act, dev_status, s, launches);
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(gemm_bf16_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -2,6 +2,8 @@
 // implicit-GEMM convolution, fused depthwise + pointwise block).
 #pragma once
 
+#include <cuda_bf16.h>
+
 #include "common.cuh"
 #include "ptx_sm100.cuh"
 
@@ -37,6 +39,41 @@ __device__ __forceinline__ void stage_chunk(const uint32_t (&r)[32], const float
         v.z = apply_act_t<ACT>(v.z); v.w = apply_act_t<ACT>(v.w);
         const uint32_t dst = row_addr + (uint32_t)((j ^ (lane & 7)) << 4);
         asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+                     : "memory");
+    }
+}
+
+// ---- bfloat16 storage ------------------------------------------------------------------------------
+// Instruction descriptor: fp32 accumulator, bfloat16 A and B (format 1), both K-major.
+__device__ __forceinline__ uint32_t make_idesc_bf16(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+// One 32-row x 32-column accumulator block, one row per lane: bias, activation, rounding to bfloat16,
+// and the store into the staging slab in the 64-byte swizzle the bulk tensor store expects (rows of
+// 64 bytes; 16-byte piece j of row r lives at piece j ^ ((r / 2) % 4)).
+template <int ACT>
+__device__ __forceinline__ void stage_chunk_bf16(const uint32_t (&r)[32], const float* __restrict__ bias, int cols_left,
+                                                 uint32_t slab, int lane) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        float v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[8 * j + e]);
+        if (bias != nullptr && 8 * j < cols_left) {  // N % 8 == 0: a group of eight is all in or all out
+            const float4 b0 = __ldg(reinterpret_cast<const float4*>(bias + 8 * j));
+            const float4 b1 = __ldg(reinterpret_cast<const float4*>(bias + 8 * j + 4));
+            v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
+            v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+        }
+        uint32_t p[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(apply_act_t<ACT>(v[2 * e]), apply_act_t<ACT>(v[2 * e + 1]));
+            p[e] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        const uint32_t dst = slab + (uint32_t)lane * 64u + (uint32_t)((j ^ ((lane >> 1) & 3)) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(p[0]), "r"(p[1]), "r"(p[2]), "r"(p[3])
                      : "memory");
     }
 }

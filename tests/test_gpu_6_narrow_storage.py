@@ -117,6 +117,44 @@ def test_matmul_bf16_parity_with_fused_epilogue(ctx, oracle, mkn):
     check_stored(widen(ctx.matmul_bf16(ad, bd))[rows], oracle.matmul(a[rows], bt, transpose_b=True))
 
 
+PAIR_SHAPES = [
+    (256, 64, 64),       # one pair tile, one k-block, 32 Bt rows per CTA
+    (128, 128, 256),     # the odd CTA's rows are all outside the matrix
+    (300, 104, 72),      # ragged in M, K and N
+    (4100, 40, 264),     # a second tile along N with 8 live columns
+    (520, 1024, 512),    # sixteen k-blocks: the stage ring wraps
+    (20000, 256, 512),   # more tiles than SM pairs: persistent loop, accumulator stages reused
+    (25088, 512, 512),   # pw7-pw11 of the 224 model at batch 128: the shape the planner gives to this kernel
+]
+
+
+@pytest.mark.parametrize("mkn", PAIR_SHAPES)
+def test_matmul_bf16_pair_kernel(ctx, oracle, monkeypatch, mkn):
+    """The CTA-pair kernel (forced on with TFJSB_GEMM_PAIR=1): exact on small integers, within the
+    stored-result bound on random values, and bit-identical to the single-CTA kernel, which adds the
+    same k-blocks in the same order."""
+    M, K, N = mkn
+    ai = bf16_dev(si.small_integers(603, 0, (M, K), -8, 8))
+    bi = bf16_dev(si.small_integers(603, 1, (N, K), -8, 8))
+    a = oracle.round_bf16(si.uniform(604, 0, (M, K), -1, 1))
+    bt = oracle.round_bf16(si.uniform(604, 1, (N, K), -1, 1))
+    bias = si.normal(604, 2, (N,), 0, 2.0)
+    ad, bd, biasd = bf16_dev(a), bf16_dev(bt), dev(bias)
+    monkeypatch.setenv("TFJSB_GEMM_PAIR", "1")
+    exact = widen(ctx.matmul_bf16(ai, bi))
+    pair = widen(ctx.matmul_bf16(ad, bd, bias=biasd, act="relu6"))
+    monkeypatch.setenv("TFJSB_GEMM_PAIR", "0")
+    single = widen(ctx.matmul_bf16(ad, bd, bias=biasd, act="relu6"))
+    ctx.check_device_status()
+    want_int = (widen(ai).astype(np.int64) @ widen(bi).astype(np.int64).T).astype(np.float32)
+    assert same_bits(exact, oracle.round_bf16(want_int))
+    assert same_bits(pair, single)
+    rows = np.arange(M) if M * K * N <= 600_000_000 else np.unique(np.linspace(0, M - 1, 257).astype(np.int64))
+    want = oracle.round_bf16(oracle.bias_act(oracle.matmul(a[rows], bt, transpose_b=True), bias, "relu6"))
+    assert np.all(np.abs(pair[rows] - want) <= 2.0 ** -7 * np.abs(want) + 4e-6 * np.sqrt(K))
+    assert np.count_nonzero(pair[rows] != want) <= 0.02 * want.size
+
+
 def test_matmul_bf16_rejects_what_it_cannot_run(ctx, tfjsb):
     import torch
 
