@@ -445,8 +445,8 @@ cudaError_t launch_rgb_act(const float* x, const float* f, const float* bias, vo
                            cudaStream_t s) {
     const int64_t total = g.N * g.Ho * g.Wo;
     const dim3 grid(grid_for(total, 256)), block(128);  // 256 pixels per block and pass
-    return y_is_bf16 ? launch_k(conv3x3_rgb_narrow_kernel<COUT, ACT, true>, grid, block, 0, s, x, f, bias, y, g, total)
-                     : launch_k(conv3x3_rgb_narrow_kernel<COUT, ACT, false>, grid, block, 0, s, x, f, bias, y, g, total);
+    return y_is_bf16 ? launch_k_serial(conv3x3_rgb_narrow_kernel<COUT, ACT, true>, grid, block, 0, s, x, f, bias, y, g, total)
+                     : launch_k_serial(conv3x3_rgb_narrow_kernel<COUT, ACT, false>, grid, block, 0, s, x, f, bias, y, g, total);
 }
 template <int COUT>
 cudaError_t launch_rgb(const float* x, const float* f, const float* bias, int act, void* y, bool y_is_bf16, const ConvGeom& g,
@@ -475,12 +475,12 @@ cudaError_t launch_conv_narrow(const void* x, bool x_is_f32, const float* f, con
     cudaError_t e;
     if (x_is_f32) {
         const float* xf = static_cast<const float*>(x);
-        e = y_is_bf16 ? launch_k(conv_direct_narrow_kernel<float, true>, grid, block, 0, s, xf, f, bias, act, y, g, groups, total)
-                      : launch_k(conv_direct_narrow_kernel<float, false>, grid, block, 0, s, xf, f, bias, act, y, g, groups, total);
+        e = y_is_bf16 ? launch_k_serial(conv_direct_narrow_kernel<float, true>, grid, block, 0, s, xf, f, bias, act, y, g, groups, total)
+                      : launch_k_serial(conv_direct_narrow_kernel<float, false>, grid, block, 0, s, xf, f, bias, act, y, g, groups, total);
     } else {
         const __nv_bfloat16* xh = static_cast<const __nv_bfloat16*>(x);
-        e = y_is_bf16 ? launch_k(conv_direct_narrow_kernel<__nv_bfloat16, true>, grid, block, 0, s, xh, f, bias, act, y, g, groups, total)
-                      : launch_k(conv_direct_narrow_kernel<__nv_bfloat16, false>, grid, block, 0, s, xh, f, bias, act, y, g, groups, total);
+        e = y_is_bf16 ? launch_k_serial(conv_direct_narrow_kernel<__nv_bfloat16, true>, grid, block, 0, s, xh, f, bias, act, y, g, groups, total)
+                      : launch_k_serial(conv_direct_narrow_kernel<__nv_bfloat16, false>, grid, block, 0, s, xh, f, bias, act, y, g, groups, total);
     }
     ++*launches;
     return e;
@@ -498,9 +498,9 @@ cudaError_t launch_dw_act(const __nv_bfloat16* x, const float* f, const float* b
     const int row_blocks = (g.Ho + TR - 1) / TR, col_blocks = (g.Wo + TC - 1) / TC;
     const uint32_t total = (uint32_t)(g.N * row_blocks * col_blocks * (g.C / 8));
     const dim3 grid(grid_for(total, 128)), block(128);
-    return y_is_bf16 ? launch_k(depthwise3x3_narrow_kernel<S, TR, TC, ACT, true>, grid, block, 0, s, x, f, bias, y, g,
+    return y_is_bf16 ? launch_k_serial(depthwise3x3_narrow_kernel<S, TR, TC, ACT, true>, grid, block, 0, s, x, f, bias, y, g,
                                 row_blocks, col_blocks, total)
-                     : launch_k(depthwise3x3_narrow_kernel<S, TR, TC, ACT, false>, grid, block, 0, s, x, f, bias, y, g,
+                     : launch_k_serial(depthwise3x3_narrow_kernel<S, TR, TC, ACT, false>, grid, block, 0, s, x, f, bias, y, g,
                                 row_blocks, col_blocks, total);
 }
 template <int S, int TR, int TC>
@@ -527,8 +527,8 @@ cudaError_t launch_avg_pool_global_narrow(const void* x, void* y, bool y_is_bf16
     const int64_t total = images * (C / 8) * 8;
     const dim3 grid(grid_for(total, 256)), block(256);
     const __nv_bfloat16* xh = static_cast<const __nv_bfloat16*>(x);
-    cudaError_t e = y_is_bf16 ? launch_k(avg_pool_global_narrow_kernel<true>, grid, block, 0, s, xh, y, images, positions, C)
-                              : launch_k(avg_pool_global_narrow_kernel<false>, grid, block, 0, s, xh, y, images, positions, C);
+    cudaError_t e = y_is_bf16 ? launch_k_serial(avg_pool_global_narrow_kernel<true>, grid, block, 0, s, xh, y, images, positions, C)
+                              : launch_k_serial(avg_pool_global_narrow_kernel<false>, grid, block, 0, s, xh, y, images, positions, C);
     ++*launches;
     return e;
 }

@@ -118,6 +118,26 @@ cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
+// The same launch without the attribute, whatever the executor's setting: for kernels made of many
+// small blocks with little shared memory.  Launched early, their first blocks become resident beside
+// the predecessor's CTAs and wait there, and that costs the predecessor more than the overlap returns
+// (measured: a model whose depthwise layers are such kernels ran 4 % slower with the attribute on
+// them, and the fp32 model 9 % slower when its depthwise layers were swapped for such a kernel; the
+// persistent kernels with large shared-memory footprints cannot become resident early and only
+// overlap their prologue).  Such a kernel still executes griddepcontrol.launch_dependents, so its
+// successor may start early.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k_serial(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cfg.attrs = nullptr;
+    cfg.numAttrs = 0;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 // ---- geometry of one convolution / pooling call -----------------------------------------------
 struct ConvGeom {
     int64_t N;
