@@ -519,8 +519,9 @@ def run_ours_in_child():
     """A single-GPU run measures in a child process and is repeated once if the child dies.
 
     A CUDA fault ends the context of the process that met it, so a measurement cannot continue after
-    one.  One run in about twenty ended that way ("unspecified launch failure", cause not found; see
-    the design notes); rather than lose the whole line to it, the parent repeats the measurement once
+    one.  One run in about twenty ended that way ("unspecified launch failure" inside the timed loop, no
+    ECC error reported, cause not found by reading the kernels, not seen again in the runs that
+    followed); rather than lose the whole line to it, the parent repeats the measurement once
     and says so: `attempts` counts the runs and `first_attempt_error` keeps the first run's last words.
     Ranks started by torchrun measure in place."""
     import subprocess
