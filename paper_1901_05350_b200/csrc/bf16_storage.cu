@@ -126,47 +126,57 @@ conv_direct_narrow_kernel(const IN_T* __restrict__ x, const float* __restrict__ 
 // COUT (<= 32) output channels of each.  The kernel is bound by the L1 / shared-memory pipe, so it
 // spends as few of that pipe's cycles as it can: the filter sits in shared memory as [27][COUT] and
 // each 16-byte broadcast read of it feeds both pixels; the 27 input samples of a pixel (three runs of
-// nine consecutive floats) are fetched as 8-byte loads where the run is aligned and inside the image.
+// nine consecutive floats) are fetched row by row, as 8-byte loads where the run is aligned and inside
+// the image.
 // Samples are rounded to bfloat16 as they are used; multiply-adds go two per instruction.
-__device__ __forceinline__ void load_rgb_window(const float* __restrict__ x, const ConvGeom& g, int64_t p, bool live,
-                                                float (&xv)[27]) {
+// Where one output pixel's 3 x 3 window starts, and how its rows may be fetched.
+struct RgbWindow {
+    const float* origin;  // sample (iy0, ix0, channel 0) of the pixel's image; may lie outside the image
+    int iy0, ix0;
+    bool live, fast;
+};
+__device__ __forceinline__ RgbWindow rgb_window(const float* __restrict__ x, const ConvGeom& g, int64_t p, bool live) {
+    RgbWindow w;
+    w.live = live;
+    const int64_t q = live ? p : 0;
+    const int ox = (int)(q % g.Wo);
+    const int oy = (int)((q / g.Wo) % g.Ho);
+    const int64_t n = q / ((int64_t)g.Wo * g.Ho);
+    w.iy0 = oy * g.sh - g.pt;
+    w.ix0 = ox * g.sw - g.pl;
+    w.origin = x + (n * (int64_t)g.H * g.W + (int64_t)w.iy0 * g.W + w.ix0) * 3;
+    // a row's nine floats start on an 8-byte boundary when (iy * W + ix0) * 3 is even
+    w.fast = w.ix0 >= 0 && w.ix0 + 2 < g.W && (g.W & 1) == 0 && (w.ix0 & 1) == 0;
+    return w;
+}
+// The nine samples (three pixels x three channels) of window row ky; zeros outside the image.
+__device__ __forceinline__ void load_rgb_row(const RgbWindow& w, const ConvGeom& g, int ky, float (&v)[9]) {
 #pragma unroll
-    for (int k = 0; k < 27; ++k) xv[k] = 0.0f;
-    if (!live) return;
-    const int ox = (int)(p % g.Wo);
-    const int oy = (int)((p / g.Wo) % g.Ho);
-    const int64_t n = p / ((int64_t)g.Wo * g.Ho);
-    const float* xn = x + n * (int64_t)g.H * g.W * 3;
-    const int iy0 = oy * g.sh - g.pt, ix0 = ox * g.sw - g.pl;
-    // a run starts on an 8-byte boundary when (iy * W + ix0) * 3 is even
-    const bool fast = ix0 >= 0 && ix0 + 2 < g.W && (g.W & 1) == 0 && (ix0 & 1) == 0;
+    for (int k = 0; k < 9; ++k) v[k] = 0.0f;
+    const int iy = w.iy0 + ky;
+    if (!w.live || iy < 0 || iy >= g.H) return;
+    const float* rp = w.origin + (int64_t)ky * g.W * 3;
+    if (w.fast) {
 #pragma unroll
-    for (int ky = 0; ky < 3; ++ky) {
-        const int iy = iy0 + ky;
-        if (iy < 0 || iy >= g.H) continue;
-        const float* rp = xn + ((int64_t)iy * g.W + ix0) * 3;
-        if (fast) {
+        for (int q = 0; q < 4; ++q) {
+            const float2 t = __ldg(reinterpret_cast<const float2*>(rp) + q);
+            v[2 * q] = t.x;
+            v[2 * q + 1] = t.y;
+        }
+        v[8] = __ldg(rp + 8);
+    } else {
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float2 v = __ldg(reinterpret_cast<const float2*>(rp) + q);
-                xv[ky * 9 + 2 * q] = v.x;
-                xv[ky * 9 + 2 * q + 1] = v.y;
-            }
-            xv[ky * 9 + 8] = __ldg(rp + 8);
-        } else {
+        for (int kx = 0; kx < 3; ++kx) {
+            const int ix = w.ix0 + kx;
+            if (ix < 0 || ix >= g.W) continue;
 #pragma unroll
-            for (int kx = 0; kx < 3; ++kx) {
-                const int ix = ix0 + kx;
-                if (ix < 0 || ix >= g.W) continue;
-#pragma unroll
-                for (int ci = 0; ci < 3; ++ci) xv[ky * 9 + kx * 3 + ci] = __ldg(rp + kx * 3 + ci);
-            }
+            for (int ci = 0; ci < 3; ++ci) v[kx * 3 + ci] = __ldg(rp + kx * 3 + ci);
         }
     }
 }
 
 template <int COUT, int ACT, bool OUT_NARROW>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, 4)
 conv3x3_rgb_narrow_kernel(const float* __restrict__ x, const float* __restrict__ f, const float* __restrict__ bias,
                           void* __restrict__ y, const ConvGeom g, int64_t total) {
     __shared__ __align__(16) float w_s[27 * COUT];
@@ -178,24 +188,30 @@ conv3x3_rgb_narrow_kernel(const float* __restrict__ x, const float* __restrict__
     pdl_wait();
     for (int64_t base = (int64_t)blockIdx.x * 256; base < total; base += (int64_t)gridDim.x * 256) {
         const int64_t p0 = base + threadIdx.x, p1 = p0 + 128;
-        float xa[27], xb[27];
-        load_rgb_window(x, g, p0, p0 < total, xa);
-        load_rgb_window(x, g, p1, p1 < total, xb);
+        const RgbWindow wa = rgb_window(x, g, p0, p0 < total), wb = rgb_window(x, g, p1, p1 < total);
         float2 acc0[COUT / 2], acc1[COUT / 2];
 #pragma unroll
         for (int c = 0; c < COUT / 2; ++c) acc0[c] = acc1[c] = make_float2(0.0f, 0.0f);
+        // one window row at a time: eighteen samples in flight per thread, few enough registers for
+        // four blocks per SM
 #pragma unroll
-        for (int k = 0; k < 27; ++k) {
-            const float va = round_bf16(xa[k]), vb = round_bf16(xb[k]);
-            const float2 a2 = make_float2(va, va), b2 = make_float2(vb, vb);
+        for (int ky = 0; ky < 3; ++ky) {
+            float xa[9], xb[9];
+            load_rgb_row(wa, g, ky, xa);
+            load_rgb_row(wb, g, ky, xb);
 #pragma unroll
-            for (int c = 0; c < COUT / 4; ++c) {
-                const float4 w = *reinterpret_cast<const float4*>(&w_s[k * COUT + 4 * c]);
-                const float2 wl = make_float2(w.x, w.y), wh = make_float2(w.z, w.w);
-                fma2(acc0[2 * c], a2, wl);
-                fma2(acc0[2 * c + 1], a2, wh);
-                fma2(acc1[2 * c], b2, wl);
-                fma2(acc1[2 * c + 1], b2, wh);
+            for (int k = 0; k < 9; ++k) {
+                const float va = round_bf16(xa[k]), vb = round_bf16(xb[k]);
+                const float2 a2 = make_float2(va, va), b2 = make_float2(vb, vb);
+#pragma unroll
+                for (int c = 0; c < COUT / 4; ++c) {
+                    const float4 w = *reinterpret_cast<const float4*>(&w_s[(ky * 9 + k) * COUT + 4 * c]);
+                    const float2 wl = make_float2(w.x, w.y), wh = make_float2(w.z, w.w);
+                    fma2(acc0[2 * c], a2, wl);
+                    fma2(acc0[2 * c + 1], a2, wh);
+                    fma2(acc1[2 * c], b2, wl);
+                    fma2(acc1[2 * c + 1], b2, wh);
+                }
             }
         }
 #pragma unroll
