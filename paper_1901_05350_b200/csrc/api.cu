@@ -298,11 +298,11 @@ tfjsb_status tfjsb_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_ten
 tfjsb_status tfjsb_matmul_bf16(tfjsb_ctx* ctx, const void* a, const void* bt, const float* bias, tfjsb_act act, void* out,
                                int out_is_bf16, int64_t M, int64_t N, int64_t K, void* stream) {
     TFJSB_REQUIRE_CTX(ctx);
-    if (!a || !bt || !out) return fail(ctx, TFJSB_ERR_INVALID_ARG, "a / bt / out is null");
     if (act != TFJSB_ACT_NONE && act != TFJSB_ACT_RELU && act != TFJSB_ACT_RELU6)
         return fail(ctx, TFJSB_ERR_INVALID_ARG, "unknown activation");
     if (M < 0 || N < 0 || K < 0) return fail(ctx, TFJSB_ERR_SHAPE, "negative size");
-    if (M == 0 || N == 0) return TFJSB_OK;
+    if (M == 0 || N == 0) return TFJSB_OK;  // nothing to compute (empty tensors may have null pointers)
+    if (!a || !bt || !out) return fail(ctx, TFJSB_ERR_INVALID_ARG, "a / bt / out is null");
     if (!aligned16(a) || !aligned16(bt) || !aligned16(out) || (bias && !aligned16(bias)))
         return fail(ctx, TFJSB_ERR_UNSUPPORTED, "pointers must be 16-byte aligned");
     if (a == out || bt == out) return fail(ctx, TFJSB_ERR_INVALID_ARG, "out aliases an input");

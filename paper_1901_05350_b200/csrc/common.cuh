@@ -250,6 +250,7 @@ struct GemmBf16Plan {
     bool c_is_bf16 = true;
     bool pair = false;  // CTA-pair kernel (gemm_bf16_pair.cu): 256 x block_n tiles shared by two CTAs
     int block_n = 0, stages = 0, acc_stages = 0, num_tiles = 0, grid = 0;
+    int epi_warps = 16;  // epilogue warps of the single-CTA kernel: 16 for short K loops, 8 otherwise
     size_t smem_bytes = 0;
 };
 bool gemm_bf16_supported(int64_t M, int64_t N, int64_t K);

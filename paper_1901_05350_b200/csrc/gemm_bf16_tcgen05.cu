@@ -15,8 +15,9 @@
 // k-blocks for the same K, and half the bytes of A and C to move.
 //
 // With half the bytes per tile the layers with one or two k-blocks per tile are bound by the epilogue's
-// latency per 32 x 32 block (tcgen05.ld, bias, activation, rounding, staging, store), so there are
-// sixteen epilogue warps, four per lane quadrant, taking every fourth block.
+// latency per 32 x 32 block (tcgen05.ld, bias, activation, rounding, staging, store), so those run with
+// sixteen epilogue warps, four per lane quadrant, taking every fourth block; the layers with long K
+// loops keep eight (the extra warps' polling costs them about 4 %).
 //
 // Every wait is bounded, as in the TF32 kernel.
 #include <cuda_bf16.h>
@@ -35,8 +36,8 @@ using namespace tile;
 namespace {
 
 constexpr int MAX_STAGES = 8;
-constexpr int EPI_WARPS = 16;      // four per tensor-memory lane quadrant
-constexpr int GEMM_THREADS = 64 + EPI_WARPS * 32;  // producer warp, MMA warp, the epilogue warps
+constexpr int MAX_EPI_WARPS = 16;  // eight or sixteen epilogue warps: two or four per tensor-memory lane quadrant
+constexpr int GEMM_THREADS = 64 + MAX_EPI_WARPS * 32;  // producer warp, MMA warp, the epilogue warps
 constexpr int BK16 = 64;           // bfloat16 elements per k-block (128 bytes)
 constexpr int UMMA_K16 = 16;       // elements per tcgen05.mma of kind::f16
 
@@ -57,6 +58,7 @@ struct KernelArgs {
     int n_tiles;
     int num_tiles;
     int acc_stages;
+    int epi_warps;  // 8 or 16
     const float* bias;
     int act;
     unsigned int* dev_status;
@@ -85,7 +87,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t epi_base = smem_base;
     constexpr uint32_t SLAB_BYTES = OUT_BF16 ? 2048u : 4096u;  // 32 rows x 32 columns of the output type
-    const uint32_t stage_base = smem_base + EPI_WARPS * SLAB_BYTES;
+    const uint32_t stage_base = smem_base + (uint32_t)args.epi_warps * SLAB_BYTES;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -94,7 +96,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         }
         for (int s = 0; s < acc_stages; ++s) {
             mbar_init(smem_u32(&bar_acc_full[s]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[s]), EPI_WARPS);
+            mbar_init(smem_u32(&bar_acc_empty[s]), (uint32_t)args.epi_warps);
         }
         mbar_init(smem_u32(&bar_drain), 1);
         abort_flag_s = 0;
@@ -220,19 +222,20 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             }
         }
     } else {
-        // ---------------------------------------------------------------- epilogue (warps 2..17)
-        // Four warps share each TMEM lane quadrant (a warp may only read lanes 32*(warp%4)..+31) and take
-        // every fourth 32-column block, counted across tiles so that with one block per tile they take
-        // tiles in turn.
+        // ---------------------------------------------------------------- epilogue (warps 2..)
+        // Two or four warps share each TMEM lane quadrant (a warp may only read lanes 32*(warp%4)..+31)
+        // and take every second or fourth 32-column block, counted across tiles so that with one block
+        // per tile they take tiles in turn.
         const int ew = warp - 2;
         const int quad = warp & 3;
-        const int sub = ew >> 2;  // 0..3: which of the quadrant's four warps
+        const int sub = ew >> 2;  // which of the quadrant's warps
+        const int per_quad_mask = (args.epi_warps >> 2) - 1;  // 1 or 3
         const uint32_t slab = epi_base + (uint32_t)ew * SLAB_BYTES;
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
         const int chunks_per_tile = block_n / EPI_COLS;
-        int chunk_base = 0;  // blocks of earlier tiles, modulo 4
+        int chunk_base = 0;  // blocks of earlier tiles, modulo the quadrant's warps
         for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
             const int m0 = (tile / args.n_tiles) * BLOCK_M;
             const int n0 = (tile % args.n_tiles) * block_n;
@@ -252,12 +255,12 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             if (live_cols < block_n) n_chunks = (live_cols + EPI_COLS - 1) / EPI_COLS;
             const bool rows_live = row0 < args.M;
             bool released = false;
-            for (int ch = (sub - chunk_base) & 3; ch < n_chunks; ch += 4) {
+            for (int ch = (sub - chunk_base) & per_quad_mask; ch < n_chunks; ch += per_quad_mask + 1) {
                 uint32_t r[32];
                 const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * block_n + ch * EPI_COLS);
                 tc_ld_32x32(taddr, r);
                 tc_ld_wait();
-                if (ch + 4 >= n_chunks) {
+                if (ch + per_quad_mask + 1 >= n_chunks) {
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
@@ -291,7 +294,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
             }
-            chunk_base = (chunk_base + chunks_per_tile) & 3;
+            chunk_base = (chunk_base + chunks_per_tile) & per_quad_mask;
             if (++acc == acc_stages) { acc = 0; acc_phase ^= 1u; }
         }
         if (lane == 0) tma_store_wait_all();
@@ -361,7 +364,8 @@ tfjsb_status gemm_bf16_plan(tfjsb_ctx* ctx, const void* a, const void* bt, void*
     plan->block_n = choose_block_n(M, N, ctx->sm_count);
     plan->acc_stages = plan->block_n > 128 ? 2 : MAX_ACC_STAGES;
     const int stage_bytes = A_STAGE_BYTES + plan->block_n * 128;
-    const int epi_bytes = EPI_WARPS * (c_is_bf16 ? 2048 : 4096);
+    plan->epi_warps = (K + BK16 - 1) / BK16 <= 4 ? 16 : 8;
+    const int epi_bytes = plan->epi_warps * (c_is_bf16 ? 2048 : 4096);
     int stages = (SMEM_LIMIT - 1024 - epi_bytes - 512) / stage_bytes;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
     plan->stages = stages;
@@ -403,15 +407,16 @@ cudaError_t launch_gemm_bf16(const GemmBf16Plan& plan, const float* bias, int ac
     args.n_tiles = (int)((plan.N + plan.block_n - 1) / plan.block_n);
     args.num_tiles = plan.num_tiles;
     args.acc_stages = plan.acc_stages;
+    args.epi_warps = plan.epi_warps;
     args.bias = bias;
     args.act = act;
     args.dev_status = dev_status;
     cudaError_t e;
     if (plan.c_is_bf16)
-        e = launch_k(gemm_bf16_kernel<true>, dim3(plan.grid), dim3(GEMM_THREADS), plan.smem_bytes, s, plan.map_a, plan.map_b,
+        e = launch_k(gemm_bf16_kernel<true>, dim3(plan.grid), dim3(64 + 32 * plan.epi_warps), plan.smem_bytes, s, plan.map_a, plan.map_b,
                      plan.map_c, args);
     else
-        e = launch_k(gemm_bf16_kernel<false>, dim3(plan.grid), dim3(GEMM_THREADS), plan.smem_bytes, s, plan.map_a, plan.map_b,
+        e = launch_k(gemm_bf16_kernel<false>, dim3(plan.grid), dim3(64 + 32 * plan.epi_warps), plan.smem_bytes, s, plan.map_a, plan.map_b,
                      plan.map_c, args);
     ++*launches;
     return e;

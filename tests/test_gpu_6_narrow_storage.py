@@ -170,6 +170,10 @@ def test_matmul_bf16_rejects_what_it_cannot_run(ctx, tfjsb):
     assert e.value.status_name == "UNSUPPORTED"
     with pytest.raises(TypeError):
         ctx.matmul_bf16(a.to(torch.float32), bt)
+    # nothing to compute: no launch, no error
+    before = ctx.launch_count
+    empty = ctx.matmul_bf16(torch.zeros(0, 64, dtype=torch.bfloat16, device="cuda"), bt[:32].contiguous())
+    assert tuple(empty.shape) == (0, 32) and ctx.launch_count == before
 
 
 def narrow_model(ctx, layers, shape):
