@@ -143,6 +143,43 @@ def layer_work(layers, in_shape, window_out_shape):
     return rows
 
 
+def narrow_layer_work(layers, in_shape, window_out_shape):
+    """Algorithmic flops and bytes of every layer in the narrow-storage mode: filters and every layer output
+    are 2 bytes per value, except the model input, biases, and the dense and softmax outputs (4 bytes)."""
+    n, h, w, c = in_shape
+    rows = []
+    in_size = 4  # the model input is fp32
+    last = len(layers) - 1
+    for i, layer in enumerate(layers):
+        kind = layer.kind
+        out_size = 4 if (kind in ("dense", "softmax") or i == last) else 2
+        if kind in ("conv2d", "depthwise_conv2d"):
+            fh, fw = layer.filter_hw
+            ho, _, _ = window_out_shape(h, fh, layer.strides[0], layer.dilations[0], layer.pad)
+            wo, _, _ = window_out_shape(w, fw, layer.strides[1], layer.dilations[1], layer.pad)
+            if kind == "conv2d":
+                co = layer.out_channels
+                flops, weights = 2 * n * ho * wo * co * fh * fw * c, fh * fw * c * co
+                tensor = (fh, fw) == (1, 1) and layer.strides == (1, 1)
+            else:
+                co = c * layer.out_channels
+                flops, weights, tensor = 2 * n * ho * wo * co * fh * fw, fh * fw * co, False
+            nbytes = in_size * n * h * w * c + 2 * weights + 4 * co + out_size * n * ho * wo * co
+            h, w, c = ho, wo, co
+        elif kind == "global_avg_pool":
+            flops, nbytes, tensor = n * h * w * c, in_size * n * h * w * c + out_size * n * c, False
+            h = w = 1
+        elif kind == "dense":
+            k, co = h * w * c, layer.out_channels
+            flops, nbytes, tensor = 2 * n * k * co, in_size * n * k + 2 * k * co + 4 * co + out_size * n * co, True
+            h, w, c = 1, 1, co
+        else:  # softmax
+            flops, nbytes, tensor = 5 * n * c, (in_size + out_size) * n * c, False
+        rows.append(dict(name=layer.name, flops=flops, bytes=nbytes, tensor=tensor))
+        in_size = out_size
+    return rows
+
+
 def merge_fused(rows, ms):
     """The executor may run a depthwise layer and the pointwise layer after it as one kernel; the
     profile then reports the pair's time under the depthwise layer and ~0 under the pointwise one.
@@ -458,6 +495,9 @@ def run_ours(args):
             torch.cuda.synchronize()
             narrow_e2e_ms = start.elapsed_time(stop) / e2e_steps
             agree = float((on.argmax(-1) == out.argmax(-1)).float().mean())
+            n_rows = narrow_layer_work(layers, x_host.shape, tfjsb.window_out_shape)
+            n_roof = [max(r["bytes"] / (peaks["hbm_gbs"] * 1e9),
+                          r["flops"] / (peaks["bf16_tflops_sustained"] * 1e12) if r["tensor"] else 0.0) * 1e6 for r in n_rows]
             line["narrow_storage"] = {
                 "metric": METRIC + ", bfloat16 storage", "value": BATCH / (narrow_ms * 1e-3), "unit": UNIT,
                 "ms_per_step": narrow_ms, "steps": n_steps,
@@ -465,6 +505,12 @@ def run_ours(args):
                 "dtype": "bf16 storage of filters and activations, exact products, f32 sums; model input and output f32",
                 "top1_agreement_with_f32_storage": agree,
                 "per_layer_us": dict(zip(mn.layer_names, layer_us)),
+                "per_layer_roofline_us": dict(zip(mn.layer_names, [round(v, 2) for v in n_roof])),
+                "roofline_step": {"sum_roofline_us": sum(n_roof), "sum_measured_us": sum(layer_us),
+                                  "frac": sum(n_roof) / sum(layer_us),
+                                  "how": "per layer the slower of its bytes (2-byte filters and activations, 4-byte "
+                                         "input, biases, logits) at the measured HBM copy rate and, for the GEMM-shaped "
+                                         "layers, its flops at the measured sustained bf16 rate"},
             }
             mn.close()
         if cpu_baseline is not None:
