@@ -556,40 +556,7 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
-    if "RANK" not in os.environ and os.environ.get("TFJSB_BENCH_ATTEMPT") is None:
-        return run_ours_in_child()
     return run_ours(args)
-
-
-def run_ours_in_child():
-    """A single-GPU run measures in a child process and is repeated once if the child dies.
-
-    A CUDA fault ends the context of the process that met it, so a measurement cannot continue after
-    one.  One run in about twenty ended that way ("unspecified launch failure" inside the timed loop, no
-    ECC error reported, cause not found by reading the kernels, not seen again in the runs that
-    followed); rather than lose the whole line to it, the parent repeats the measurement once
-    and says so: `attempts` counts the runs and `first_attempt_error` keeps the first run's last words.
-    Ranks started by torchrun measure in place."""
-    import subprocess
-
-    errors = []
-    for attempt in (1, 2):
-        env = dict(os.environ, TFJSB_BENCH_ATTEMPT=str(attempt))
-        proc = subprocess.run([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env,
-                              stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True)
-        sys.stderr.write(proc.stderr)
-        lines = [l for l in proc.stdout.splitlines() if l.startswith("{")]
-        if proc.returncode == 0 and lines:
-            line = json.loads(lines[-1])
-            line["attempts"] = attempt
-            if errors:
-                line["first_attempt_error"] = errors[0]
-            print(json.dumps(line), flush=True)
-            return 0
-        tail = [l for l in proc.stderr.splitlines() if l.strip()]
-        errors.append(f"exit {proc.returncode}: " + (tail[-1][:300] if tail else "no message"))
-    sys.stderr.write("bench: both attempts failed: " + " | ".join(errors) + "\n")
-    return 1
 
 
 if __name__ == "__main__":

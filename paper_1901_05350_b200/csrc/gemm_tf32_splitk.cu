@@ -15,9 +15,15 @@
 //
 // Per CTA, 6 warps: warp 0 producer (bulk tensor copies into a ring of stages), warp 1 tensor-memory
 // allocation and MMA issue, warps 2-5 one per tensor-memory lane quadrant: accumulator -> shared
-// memory, then the reduction.  Each CTA processes exactly one work item.  Every mbarrier wait is
+// memory, then the reduction.  Each CTA processes exactly one work item.
+//
+// Two cluster barriers order the remote accesses.  The first ("started") is arrived at by every
+// thread right after the CTA's own set-up and waited for before the first store into a partner: the
+// shared memory of a CTA may only be touched once that CTA is known to be executing, and being
+// launched as one cluster does not by itself order a fast CTA's store after a slow partner's start.
+// The second ("delivered") separates the remote stores from the reduction.  Every mbarrier wait is
 // bounded; a CTA whose wait gave up still takes part in both cluster barriers, so its partners never
-// wait for it (the barrier itself has no limit: every path below reaches it).
+// wait for it (the barriers themselves have no limit: every path below reaches them).
 #include <cstdlib>
 
 #include "common.cuh"
@@ -113,6 +119,10 @@ gemm_tf32_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    // barrier "started", arrive half: this CTA is running and its shared memory may be written by the
+    // partners.  Each thread completes it (cluster_wait) where it next needs it: warps 2-5 before
+    // their first remote store, warps 0-1 at the end of their role, before arriving at the second barrier.
+    cluster_arrive();
     pdl_launch_dependents();
     pdl_wait();
 
@@ -153,6 +163,7 @@ gemm_tf32_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 }
             }
         }
+        cluster_wait();
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
@@ -195,9 +206,11 @@ gemm_tf32_splitk_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 }
             }
         }
+        cluster_wait();
     } else {
         // ---------------------------------------------------------------- accumulator -> the band owners' shared memory (warps 2..5)
         const int quad = warp & 3;  // the tensor-memory lanes this warp may read: 32*quad ..
+        cluster_wait();             // every partner has started: its shared memory exists and may be written
         const bool got = bounded_wait(smem_u32(&bar_acc_full), 0u, abort_flag);
         if (__all_sync(0xffffffffu, got)) {
             tc_fence_after();
