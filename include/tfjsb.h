@@ -297,6 +297,13 @@ tfjsb_status tfjsb_model_layer_output_f32(tfjsb_model* model, int layer, float* 
 /* Shape of the output of layer `layer`. */
 tfjsb_status tfjsb_model_layer_shape(tfjsb_model* model, int layer, int32_t* rank, int64_t dims[4]);
 
+/* Name of the kernel that runs layer `layer` in the model's current mode, as planned for the buffers
+ * of the last run (the per-kernel view of the paper's profiler, Sec. 3.8): written to `name` (a HOST
+ * buffer of `name_len` bytes, NUL-terminated, truncated if too short).  The second layer of a fused
+ * depthwise + pointwise pair reports "(in the previous layer's kernel)".  TFJSB_ERR_INVALID_ARG before
+ * the first run. */
+tfjsb_status tfjsb_model_layer_kernel(tfjsb_model* model, int layer, char* name, int32_t name_len);
+
 /* Per-layer device timing (the paper's per-kernel profile, Sec. 3.8): runs the model `reps`
  * times with a CUDA event pair around every layer, synchronises, and writes the mean
  * milliseconds per layer into ms_per_layer[0..n_layers-1] (host). */

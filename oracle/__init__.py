@@ -55,6 +55,13 @@ def _load():
         lib.orc_softmax.argtypes = [fp, i64, i64, fp]
         lib.orc_max_pool.argtypes = [fp, i64, i32, i32, i32, i32, i32, i32, i32, i32, fp]
         lib.orc_binary.argtypes = [i32, fp, fp, i64, i64, fp]
+        conv_grad = [fp, i64, i32, i32, i32, fp, i32, i32, i32, i32, i32, i32, i32, i32, fp]
+        lib.orc_conv2d_backprop_input.argtypes = conv_grad + [i32]
+        lib.orc_conv2d_backprop_filter.argtypes = conv_grad + [i32]
+        lib.orc_depthwise_backprop_input.argtypes = conv_grad
+        lib.orc_depthwise_backprop_filter.argtypes = conv_grad
+        lib.orc_act_backprop.argtypes = [fp, fp, i64, i32, fp]
+        lib.orc_bias_backprop.argtypes = [fp, i64, i64, fp]
         _lib = lib
     return _lib
 
@@ -200,6 +207,99 @@ def batch_matmul(a, b, transpose_a: bool = False, transpose_b: bool = False, ope
     if a.ndim != 3 or b.ndim != 3 or a.shape[0] != b.shape[0]:
         raise ValueError("batch_matmul takes rank-3 tensors with equal leading dimensions")
     return np.stack([matmul(a[i], b[i], transpose_a, transpose_b, operand) for i in range(a.shape[0])])
+
+
+def _grad_geometry(x_shape, fh, fw, strides, pad, dilations, dy_shape, out_channels):
+    N, H, W, _ = x_shape
+    Ho, _, _ = window_geometry(H, fh, strides[0], dilations[0], pad)
+    Wo, _, _ = window_geometry(W, fw, strides[1], dilations[1], pad)
+    if tuple(dy_shape) != (N, Ho, Wo, out_channels):
+        raise ValueError(f"dy has shape {tuple(dy_shape)}, the forward output has {(N, Ho, Wo, out_channels)}")
+
+
+def conv2d_backprop_input(x_shape, f, dy, strides=(1, 1), pad="same", dilations=(1, 1), operand: str = "fp32") -> np.ndarray:
+    """Gradient of conv2d with respect to its input: the adjoint of x -> conv2d(x, f) applied to dy."""
+    f, dy = _f32(f), _f32(dy)
+    N, H, W, Cin = (int(v) for v in x_shape)
+    fh, fw, fc, Cout = f.shape
+    if fc != Cin:
+        raise ValueError(f"filter has {fc} input channels, x has {Cin}")
+    _grad_geometry(x_shape, fh, fw, strides, pad, dilations, dy.shape, Cout)
+    dx = np.empty((N, H, W, Cin), dtype=np.float32)
+    rc = _load().orc_conv2d_backprop_input(_ptr(dy), N, H, W, Cin, _ptr(f), fh, fw, Cout, strides[0], strides[1], PAD[pad],
+                                           dilations[0], dilations[1], _ptr(dx), OPERAND[operand])
+    if rc:
+        raise RuntimeError(f"orc_conv2d_backprop_input failed ({rc})")
+    return dx
+
+
+def conv2d_backprop_filter(x, filter_shape, dy, strides=(1, 1), pad="same", dilations=(1, 1), operand: str = "fp32") -> np.ndarray:
+    """Gradient of conv2d with respect to its filter [fh, fw, Cin, Cout]."""
+    x, dy = _f32(x), _f32(dy)
+    N, H, W, Cin = x.shape
+    fh, fw, fc, Cout = (int(v) for v in filter_shape)
+    if fc != Cin:
+        raise ValueError(f"filter has {fc} input channels, x has {Cin}")
+    _grad_geometry(x.shape, fh, fw, strides, pad, dilations, dy.shape, Cout)
+    df = np.empty((fh, fw, Cin, Cout), dtype=np.float32)
+    rc = _load().orc_conv2d_backprop_filter(_ptr(x), N, H, W, Cin, _ptr(dy), fh, fw, Cout, strides[0], strides[1], PAD[pad],
+                                            dilations[0], dilations[1], _ptr(df), OPERAND[operand])
+    if rc:
+        raise RuntimeError(f"orc_conv2d_backprop_filter failed ({rc})")
+    return df
+
+
+def depthwise_conv2d_backprop_input(x_shape, f, dy, strides=(1, 1), pad="same", dilations=(1, 1)) -> np.ndarray:
+    f, dy = _f32(f), _f32(dy)
+    N, H, W, C = (int(v) for v in x_shape)
+    fh, fw, fc, mult = f.shape
+    if fc != C:
+        raise ValueError(f"filter has {fc} channels, x has {C}")
+    _grad_geometry(x_shape, fh, fw, strides, pad, dilations, dy.shape, C * mult)
+    dx = np.empty((N, H, W, C), dtype=np.float32)
+    rc = _load().orc_depthwise_backprop_input(_ptr(dy), N, H, W, C, _ptr(f), fh, fw, mult, strides[0], strides[1], PAD[pad],
+                                              dilations[0], dilations[1], _ptr(dx))
+    if rc:
+        raise RuntimeError(f"orc_depthwise_backprop_input failed ({rc})")
+    return dx
+
+
+def depthwise_conv2d_backprop_filter(x, filter_shape, dy, strides=(1, 1), pad="same", dilations=(1, 1)) -> np.ndarray:
+    x, dy = _f32(x), _f32(dy)
+    N, H, W, C = x.shape
+    fh, fw, fc, mult = (int(v) for v in filter_shape)
+    if fc != C:
+        raise ValueError(f"filter has {fc} channels, x has {C}")
+    _grad_geometry(x.shape, fh, fw, strides, pad, dilations, dy.shape, C * mult)
+    df = np.empty((fh, fw, C, mult), dtype=np.float32)
+    rc = _load().orc_depthwise_backprop_filter(_ptr(x), N, H, W, C, _ptr(dy), fh, fw, mult, strides[0], strides[1], PAD[pad],
+                                               dilations[0], dilations[1], _ptr(df))
+    if rc:
+        raise RuntimeError(f"orc_depthwise_backprop_filter failed ({rc})")
+    return df
+
+
+def act_backprop(y, dy, act="none") -> np.ndarray:
+    """Gradient through y = act(z): dy where the activation passed z through (relu: y > 0; relu6: 0 < y < 6), else 0."""
+    y, dy = _f32(y), _f32(dy)
+    if y.shape != dy.shape:
+        raise ValueError("y and dy must have one shape")
+    dz = np.empty_like(y)
+    rc = _load().orc_act_backprop(_ptr(y), _ptr(dy), y.size, ACT[act], _ptr(dz))
+    if rc:
+        raise RuntimeError(f"orc_act_backprop failed ({rc})")
+    return dz
+
+
+def bias_backprop(dz) -> np.ndarray:
+    """Gradient of a bias added along the last dimension: the sum of dz over every other dimension."""
+    dz = _f32(dz)
+    C = dz.shape[-1]
+    db = np.empty((C,), dtype=np.float32)
+    rc = _load().orc_bias_backprop(_ptr(dz), dz.size // C, C, _ptr(db))
+    if rc:
+        raise RuntimeError(f"orc_bias_backprop failed ({rc})")
+    return db
 
 
 def softmax(x) -> np.ndarray:

@@ -24,11 +24,17 @@
 // independent index only spreads output elements over threads; each element's arithmetic
 // is unchanged.
 //
+// Gradients (Sec. 3.5: eager differentiation calls a gradient function per kernel).  The paper names no
+// gradient op; each one here is the adjoint of the forward definition above, written as a gather over
+// the forward op's index relation: every (output, tap) pair that read an input sample in the forward
+// pass sends its gradient back to it, nothing else does.
+//
 // Parity pins (tests/test_oracle_*.py): integer-exact inputs against exact integer
 // arithmetic; torch/scipy library routines on the special cases that reduce to them;
 // an independently written scatter-form evaluator on tiny shapes; identity/delta filters;
 // hand-derived padding tables; algebraic identities; softmax/relu6 invariants; the
-// Listing 2 arithmetic restated in fp32.
+// Listing 2 arithmetic restated in fp32.  Gradients: the adjoint identity <op(x), g> = <x, op^T(g)>
+// on integers (exact), central finite differences of the forward oracle, torch fp64 autograd.
 // Parity unpinned: nothing in this file.  (The seeded number generator is not part of the
 // oracle; both sides consume the same bytes.)
 
@@ -309,6 +315,173 @@ int orc_softmax(const float* x, int64_t rows, int64_t cols, float* y) {
         double sum = 0.0;
         for (int64_t j = 0; j < cols; ++j) sum += std::exp((double)xr[j] - (double)m);
         for (int64_t j = 0; j < cols; ++j) y[r * cols + j] = (float)(std::exp((double)xr[j] - (double)m) / sum);
+    }
+    return 0;
+}
+
+// ---- gradients ------------------------------------------------------------------------------------
+
+// dx[n,iy,ix,ci] = fl32( sum over (oy,ky), (ox,kx), co with oy*sh - pt + ky*dh = iy and ox*sw - pl + kx*dw = ix
+//                        of dy[n,oy,ox,co] * f[ky,kx,ci,co] )
+// The gradient of conv2d with respect to its input (x has shape [N,H,W,Cin]; dy the forward output's shape).
+int orc_conv2d_backprop_input(const float* dy, int64_t N, int H, int W, int Cin, const float* f, int fh, int fw, int Cout,
+                              int sh, int sw, int pad_mode, int dh, int dw, float* dx, int operand_mode) {
+    int Ho, Wo, pt, pb, pl, pr;
+    if (!dy || !f || !dx) return 1;
+    if (!window_geometry(H, fh, sh, dh, pad_mode, &Ho, &pt, &pb)) return 2;
+    if (!window_geometry(W, fw, sw, dw, pad_mode, &Wo, &pl, &pr)) return 2;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t n = 0; n < N; ++n) {
+        for (int iy = 0; iy < H; ++iy) {
+            for (int ix = 0; ix < W; ++ix) {
+                for (int ci = 0; ci < Cin; ++ci) {
+                    double acc = 0.0;
+                    for (int ky = 0; ky < fh; ++ky) {
+                        const int ty = iy + pt - ky * dh;  // = oy*sh
+                        if (ty < 0 || ty % sh != 0 || ty / sh >= Ho) continue;
+                        const int oy = ty / sh;
+                        for (int kx = 0; kx < fw; ++kx) {
+                            const int tx = ix + pl - kx * dw;
+                            if (tx < 0 || tx % sw != 0 || tx / sw >= Wo) continue;
+                            const int ox = tx / sw;
+                            const float* gp = dy + ((n * Ho + oy) * (int64_t)Wo + ox) * Cout;
+                            const float* fp = f + ((int64_t)(ky * fw + kx) * Cin + ci) * Cout;
+                            for (int co = 0; co < Cout; ++co)
+                                acc += operand(gp[co], operand_mode) * operand(fp[co], operand_mode);
+                        }
+                    }
+                    dx[((n * H + iy) * (int64_t)W + ix) * Cin + ci] = (float)acc;
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+// df[ky,kx,ci,co] = fl32( sum_{n,oy,ox} x[n, oy*sh - pt + ky*dh, ox*sw - pl + kx*dw, ci] * dy[n,oy,ox,co] )
+// (samples outside the image are zero and add nothing).  The gradient of conv2d with respect to its filter.
+int orc_conv2d_backprop_filter(const float* x, int64_t N, int H, int W, int Cin, const float* dy, int fh, int fw, int Cout,
+                               int sh, int sw, int pad_mode, int dh, int dw, float* df, int operand_mode) {
+    int Ho, Wo, pt, pb, pl, pr;
+    if (!x || !dy || !df) return 1;
+    if (!window_geometry(H, fh, sh, dh, pad_mode, &Ho, &pt, &pb)) return 2;
+    if (!window_geometry(W, fw, sw, dw, pad_mode, &Wo, &pl, &pr)) return 2;
+#pragma omp parallel for collapse(3) schedule(static)
+    for (int ky = 0; ky < fh; ++ky) {
+        for (int kx = 0; kx < fw; ++kx) {
+            for (int ci = 0; ci < Cin; ++ci) {
+                for (int co = 0; co < Cout; ++co) {
+                    double acc = 0.0;
+                    for (int64_t n = 0; n < N; ++n) {
+                        for (int oy = 0; oy < Ho; ++oy) {
+                            const int iy = oy * sh - pt + ky * dh;
+                            if (iy < 0 || iy >= H) continue;
+                            for (int ox = 0; ox < Wo; ++ox) {
+                                const int ix = ox * sw - pl + kx * dw;
+                                if (ix < 0 || ix >= W) continue;
+                                acc += operand(x[((n * H + iy) * (int64_t)W + ix) * Cin + ci], operand_mode) *
+                                       operand(dy[((n * Ho + oy) * (int64_t)Wo + ox) * Cout + co], operand_mode);
+                            }
+                        }
+                    }
+                    df[((int64_t)(ky * fw + kx) * Cin + ci) * Cout + co] = (float)acc;
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+// dx[n,iy,ix,c] = fl32( sum over (oy,ky), (ox,kx) meeting (iy,ix) as above, and q, of dy[n,oy,ox,c*mult+q] * f[ky,kx,c,q] )
+int orc_depthwise_backprop_input(const float* dy, int64_t N, int H, int W, int C, const float* f, int fh, int fw, int mult,
+                                 int sh, int sw, int pad_mode, int dh, int dw, float* dx) {
+    int Ho, Wo, pt, pb, pl, pr;
+    if (!dy || !f || !dx || mult < 1) return 1;
+    if (!window_geometry(H, fh, sh, dh, pad_mode, &Ho, &pt, &pb)) return 2;
+    if (!window_geometry(W, fw, sw, dw, pad_mode, &Wo, &pl, &pr)) return 2;
+    const int64_t Co = (int64_t)C * mult;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t n = 0; n < N; ++n) {
+        for (int iy = 0; iy < H; ++iy) {
+            for (int ix = 0; ix < W; ++ix) {
+                for (int c = 0; c < C; ++c) {
+                    double acc = 0.0;
+                    for (int ky = 0; ky < fh; ++ky) {
+                        const int ty = iy + pt - ky * dh;
+                        if (ty < 0 || ty % sh != 0 || ty / sh >= Ho) continue;
+                        const int oy = ty / sh;
+                        for (int kx = 0; kx < fw; ++kx) {
+                            const int tx = ix + pl - kx * dw;
+                            if (tx < 0 || tx % sw != 0 || tx / sw >= Wo) continue;
+                            const int ox = tx / sw;
+                            for (int q = 0; q < mult; ++q)
+                                acc += (double)dy[((n * Ho + oy) * (int64_t)Wo + ox) * Co + (int64_t)c * mult + q] *
+                                       (double)f[((int64_t)(ky * fw + kx) * C + c) * mult + q];
+                        }
+                    }
+                    dx[((n * H + iy) * (int64_t)W + ix) * C + c] = (float)acc;
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+// df[ky,kx,c,q] = fl32( sum_{n,oy,ox} x[n, oy*sh - pt + ky*dh, ox*sw - pl + kx*dw, c] * dy[n,oy,ox,c*mult+q] )
+int orc_depthwise_backprop_filter(const float* x, int64_t N, int H, int W, int C, const float* dy, int fh, int fw, int mult,
+                                  int sh, int sw, int pad_mode, int dh, int dw, float* df) {
+    int Ho, Wo, pt, pb, pl, pr;
+    if (!x || !dy || !df || mult < 1) return 1;
+    if (!window_geometry(H, fh, sh, dh, pad_mode, &Ho, &pt, &pb)) return 2;
+    if (!window_geometry(W, fw, sw, dw, pad_mode, &Wo, &pl, &pr)) return 2;
+    const int64_t Co = (int64_t)C * mult;
+#pragma omp parallel for collapse(3) schedule(static)
+    for (int ky = 0; ky < fh; ++ky) {
+        for (int kx = 0; kx < fw; ++kx) {
+            for (int c = 0; c < C; ++c) {
+                for (int q = 0; q < mult; ++q) {
+                    double acc = 0.0;
+                    for (int64_t n = 0; n < N; ++n) {
+                        for (int oy = 0; oy < Ho; ++oy) {
+                            const int iy = oy * sh - pt + ky * dh;
+                            if (iy < 0 || iy >= H) continue;
+                            for (int ox = 0; ox < Wo; ++ox) {
+                                const int ix = ox * sw - pl + kx * dw;
+                                if (ix < 0 || ix >= W) continue;
+                                acc += (double)x[((n * H + iy) * (int64_t)W + ix) * C + c] *
+                                       (double)dy[((n * Ho + oy) * (int64_t)Wo + ox) * Co + (int64_t)c * mult + q];
+                            }
+                        }
+                    }
+                    df[((int64_t)(ky * fw + kx) * C + c) * mult + q] = (float)acc;
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+// Gradient through the fused epilogue y = act(z + bias):  dz[r,c] = dy[r,c] where the activation passed its
+// input through, +0 elsewhere (relu: y > 0; relu6: 0 < y < 6, the clamp's flat parts have zero slope;
+// none: everywhere), written in terms of the forward OUTPUT y, which is what a caller keeps.
+int orc_act_backprop(const float* y, const float* dy, int64_t n, int act, float* dz) {
+    if (!y || !dy || !dz) return 1;
+    for (int64_t i = 0; i < n; ++i) {
+        bool pass = true;
+        if (act == ACT_RELU) pass = y[i] > 0.0f;
+        if (act == ACT_RELU6) pass = y[i] > 0.0f && y[i] < 6.0f;
+        dz[i] = pass ? dy[i] : 0.0f;
+    }
+    return 0;
+}
+
+// db[c] = fl32( sum_r dz[r,c] ): the bias is added to every row, so its gradient is the column sum.
+int orc_bias_backprop(const float* dz, int64_t rows, int64_t C, float* db) {
+    if (!dz || !db) return 1;
+    for (int64_t c = 0; c < C; ++c) {
+        double acc = 0.0;
+        for (int64_t r = 0; r < rows; ++r) acc += (double)dz[r * C + c];
+        db[c] = (float)acc;
     }
     return 0;
 }

@@ -34,7 +34,7 @@ EXPORTS = [
     "tfjsb_model_output_shape", "tfjsb_model_launches_per_run", "tfjsb_run_model", "tfjsb_run_model_host",
     "tfjsb_run_model_host_async", "tfjsb_model_host_wait",
     "tfjsb_model_set_keep_all", "tfjsb_model_set_graph", "tfjsb_model_set_fusion", "tfjsb_model_layer_output", "tfjsb_model_profile",
-    "tfjsb_matmul_bf16", "tfjsb_model_layer_output_f32", "tfjsb_model_layer_shape",
+    "tfjsb_matmul_bf16", "tfjsb_model_layer_output_f32", "tfjsb_model_layer_shape", "tfjsb_model_layer_kernel",
 ]
 
 
@@ -107,6 +107,7 @@ def _load_library() -> ctypes.CDLL:
     lib.tfjsb_matmul_bf16.argtypes = [vp, vp, vp, vp, i32, vp, i32, i64, i64, i64, vp]
     lib.tfjsb_model_layer_output_f32.argtypes = [vp, i32, vp, vp]
     lib.tfjsb_model_layer_shape.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)]
+    lib.tfjsb_model_layer_kernel.argtypes = [vp, i32, ctypes.c_char_p, ctypes.c_int32]
     return lib
 
 
@@ -407,6 +408,15 @@ class Model:
         out = self.ctx._empty(tuple(int(dims[i]) for i in range(rank.value)))
         self.ctx._check(lib.tfjsb_model_layer_output_f32(self._h, layer, out.data_ptr(), _stream()))
         return out
+
+    def layer_kernels(self):
+        """Name of the kernel that runs each layer in the current mode (after at least one run)."""
+        names = []
+        buf = ctypes.create_string_buffer(96)
+        for i in range(self.n_layers):
+            self.ctx._check(lib.tfjsb_model_layer_kernel(self._h, i, buf, len(buf)))
+            names.append(buf.value.decode())
+        return names
 
     def profile(self, x, out=None, reps: int = 10):
         """Mean device milliseconds per layer over `reps` runs (event pair around every layer)."""

@@ -8,6 +8,7 @@
 // the paper's texture recycler, Sec. 4.1.2), tensor maps encoded once against those fixed
 // addresses.  Running (tfjsb_run_model) therefore does no allocation, no shape arithmetic and
 // no synchronisation: it enqueues the kernels and returns (Sec. 4.1.1).
+#include <cstdio>
 #include <cstdlib>
 #include <vector>
 
@@ -814,6 +815,34 @@ tfjsb_status tfjsb_model_layer_output(tfjsb_model* m, int layer, tfjsb_tensor* v
     view->data = st.out;
     view->rank = st.out_rank;
     for (int i = 0; i < 4; ++i) view->dims[i] = i < st.out_rank ? st.out_dims[i] : 0;
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_model_layer_kernel(tfjsb_model* m, int layer, char* name, int32_t name_len) {
+    if (!m || !name || name_len < 1) return TFJSB_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= (int)m->steps.size()) return fail(m->ctx, TFJSB_ERR_INVALID_ARG, "no such layer");
+    const Step& st = m->steps[layer];
+    if (!st.out) return fail(m->ctx, TFJSB_ERR_INVALID_ARG, "the model has not run yet");
+    const bool fused_mode = !m->keep_all;
+    const char* k = "?";
+    if (fused_mode && layer > 0 && m->steps[layer - 1].fuse_next) k = "(in the previous layer's kernel)";
+    else if (fused_mode && st.fuse_next) k = "dwpw_fused_kernel<false>";
+    else switch (st.kind) {
+        case STEP_GEMM_TF32:
+            k = st.plan.pair ? "gemm_tf32_pair_kernel" : st.plan.cluster_split ? "gemm_tf32_splitk_kernel" : "gemm_tf32_kernel<false>";
+            break;
+        case STEP_CONV_TF32: k = st.conv_patch ? "dwpw_fused_kernel<true>" : "gemm_tf32_kernel<true>"; break;
+        case STEP_GEMM_FP32: k = "gemm_fp32_kernel"; break;
+        case STEP_CONV_FP32: k = "conv2d_fp32_kernel"; break;
+        case STEP_DEPTHWISE: k = st.dw_plan.variant >= 0 ? "depthwise3x3_tma_kernel" : "depthwise3x3_kernel"; break;
+        case STEP_POOL: k = (st.g.Ho == 1 && st.g.Wo == 1 && st.g.fh == st.g.H && st.g.fw == st.g.W) ? "avg_pool_global_kernel" : "avg_pool_window_kernel"; break;
+        case STEP_SOFTMAX: k = "softmax_rows_kernel"; break;
+        case STEP_GEMM_NARROW: k = st.plan16.pair ? "gemm_bf16_pair_kernel" : "gemm_bf16_kernel"; break;
+        case STEP_CONV_NARROW: k = "conv_narrow_kernel"; break;
+        case STEP_DEPTHWISE_NARROW: k = "depthwise3x3_narrow_kernel"; break;
+        case STEP_POOL_NARROW: k = "avg_pool_global_narrow_kernel"; break;
+    }
+    snprintf(name, (size_t)name_len, "%s", k);
     return TFJSB_OK;
 }
 

@@ -184,7 +184,7 @@ def narrow_model(ctx, layers, shape):
         ctx.set_math("tf32")
 
 
-def check_logits(got_logits, got_probs, want_logits, want_probs, rel=1e-2):
+def check_logits(got_logits, got_probs, want_logits, want_probs, rel=1e-2, min_decided=1):
     decided = 0
     for i in range(want_logits.shape[0]):
         span = float(want_logits[i].max() - want_logits[i].min())
@@ -197,7 +197,7 @@ def check_logits(got_logits, got_probs, want_logits, want_probs, rel=1e-2):
             assert int(got_logits[i].argmax()) == int(want_logits[i].argmax())
             assert int(got_probs[i].argmax()) == int(want_probs[i].argmax())
         assert abs(float(got_probs[i].astype(np.float64).sum()) - 1) <= 1e-5
-    assert decided >= 1, "no image with a clear top-1 in the oracle; pick another seed"
+    assert decided >= min_decided, f"only {decided} images with a clear top-1 in the oracle; pick another seed"
 
 
 def test_small_model_every_layer(ctx, oracle):
@@ -271,9 +271,62 @@ def test_config3_mobilenet_025_128_narrow(ctx, oracle):
     model.close()
 
 
-def test_config5_mobilenet_100_224_batch128_narrow_sampled_images(ctx, oracle, tfjsb):
-    """The benchmark's model and batch in the narrow-storage mode; the oracle recomputes a sample of the
-    (independent) images one by one."""
+def test_config4_mobilenet_100_224_narrow_every_layer(ctx, oracle):
+    """Config 4 (batch 1, 224 x 224, alpha 1.0) layer by layer: the full-size kernel instances the narrow mode's
+    throughput rests on (the 32-channel first layer, the 2 x 2-tile depthwise at 112 x 112 and 56 x 56)."""
+    x, layers = si.config_mobilenet(1.0, 224, 1, seed=si.CONFIG_SEEDS["mobilenet_100_224"])
+    want = oracle.run_model(layers, x, keep_all=True, storage="bf16")
+    model = narrow_model(ctx, layers, x.shape)
+    model.set_keep_all(True)
+    probs = host(model.run(dev(x)))
+    ctx.check_device_status()
+    for i, layer in enumerate(layers[:-1]):
+        got = host(model.layer_output_f32(i))
+        assert got.shape == want[i].shape, layer.name
+        assert rel_fro(got, want[i]) <= 1e-2, f"layer {i} ({layer.name}) diverges: {rel_fro(got, want[i]):.3e}"
+        if i < len(layers) - 2:
+            assert np.all((got.view(np.uint32) & 0xFFFF) == 0), layer.name
+    for i in (0, 1, 2):  # no accumulated noise yet: at most one bfloat16 step, on few elements
+        steps = bf16_steps(host(model.layer_output_f32(i)), want[i])
+        assert steps.max() <= 1 and np.count_nonzero(steps) <= 0.01 * steps.size, i
+    check_logits(host(model.layer_output_f32(28)), probs, want[28], want[29])
+    model.close()
+
+
+def test_integer_model_full_width_first_layer_and_wide_depthwise(ctx, oracle):
+    """Bit for bit on small integers through the kernel instances of the full-size model: a first layer with
+    32 output channels on an odd-sized image, depthwise layers 57 and 61 pixels wide (stride 1 and 2: the
+    2 x 2 and 1 x 2 register tiles meet a ragged right and bottom edge) and the pixel-packed 32-channel
+    pointwise layer."""
+    x = si.small_integers(611, 0, (2, 115, 121, 3), -2, 2)
+    layers = [
+        si.Layer(kind="conv2d", filter_hw=(3, 3), strides=(2, 2), pad="same", act="relu6", out_channels=32,
+                 filter=si.small_integers(611, 1, (3, 3, 3, 32), -1, 1), bias=si.small_integers(611, 2, (32,), -2, 2)),
+        si.Layer(kind="depthwise_conv2d", filter_hw=(3, 3), strides=(1, 1), pad="same", act="relu6", out_channels=1,
+                 filter=si.small_integers(611, 3, (3, 3, 32, 1), -1, 1), bias=si.small_integers(611, 4, (32,), -2, 2)),
+        si.Layer(kind="conv2d", filter_hw=(1, 1), strides=(1, 1), pad="same", act="relu6", out_channels=64,
+                 filter=si.small_integers(611, 5, (1, 1, 32, 64), -1, 1), bias=si.small_integers(611, 6, (64,), -2, 2)),
+        si.Layer(kind="depthwise_conv2d", filter_hw=(3, 3), strides=(2, 2), pad="same", act="relu6", out_channels=1,
+                 filter=si.small_integers(611, 7, (3, 3, 64, 1), -1, 1), bias=None),
+        si.Layer(kind="conv2d", filter_hw=(1, 1), strides=(1, 1), pad="same", act="none", out_channels=16,
+                 filter=si.small_integers(611, 8, (1, 1, 64, 16), -1, 1), bias=None),
+    ]
+    want = oracle.run_model(layers, x, keep_all=True, storage="bf16")
+    assert all(np.array_equal(a, b) for a, b in zip(want, oracle.run_model(layers, x, keep_all=True)))
+    model = narrow_model(ctx, layers, x.shape)
+    model.set_keep_all(True)
+    out = host(model.run(dev(x)))
+    ctx.check_device_status()
+    assert want[0].shape == (2, 58, 61, 32) and want[3].shape == (2, 29, 31, 64)
+    for i in range(len(layers) - 1):
+        assert same_bits(host(model.layer_output_f32(i)), want[i]), i
+    assert same_bits(out, want[-1])
+    model.close()
+
+
+def test_config5_mobilenet_100_224_batch128_narrow_all_images(ctx, oracle, tfjsb):
+    """The benchmark's model and batch in the narrow-storage mode, every image against the oracle; top-1 is
+    compared on every image whose oracle margin allows, which holds for all 128 with this seed."""
     import torch
 
     x, layers = si.config_mobilenet(1.0, 224, 128, seed=si.CONFIG_SEEDS["mobilenet_100_224_b128"])
@@ -284,9 +337,8 @@ def test_config5_mobilenet_100_224_batch128_narrow_sampled_images(ctx, oracle, t
     ctx.check_device_status()
     probs = host(probs)
     assert probs.shape == (128, 1000)
-    sample = [0, 37, 127]
-    want = oracle.run_model(layers, x[sample], keep_all=True, storage="bf16")
-    check_logits(logits[sample], probs[sample], want[-2], want[-1])
+    want = oracle.run_model(layers, x, keep_all=True, storage="bf16")
+    check_logits(logits, probs, want[-2], want[-1], min_decided=128)
     # a bfloat16 layer cannot be viewed as fp32
     with pytest.raises(tfjsb.TfjsbError) as e:
         model.layer_output(3)
