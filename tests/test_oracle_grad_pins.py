@@ -126,6 +126,7 @@ def test_gradients_against_torch_fp64_autograd(oracle, case):
         ft = torch.from_numpy(fn.astype(np.float64)).requires_grad_(True)
         # HWIO -> OIHW; for a depthwise filter [fh,fw,C,m] the output channel c*m+q has one input channel
         w = ft.permute(3, 2, 0, 1) if groups == 1 else ft.reshape(fn.shape[0], fn.shape[1], -1).permute(2, 0, 1).unsqueeze(1)
+        w = w.contiguous()  # one of torch's CPU convolution paths insists on it
         xp = torch.nn.functional.pad(xt, (pl, pr, pt, pb))
         y = torch.nn.functional.conv2d(xp, w, stride=s, dilation=d, groups=groups)
         y.backward(torch.from_numpy(gn.astype(np.float64)).permute(0, 3, 1, 2))
