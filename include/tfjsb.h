@@ -91,6 +91,11 @@ const char* tfjsb_last_error(tfjsb_ctx* ctx);
  * write.  Returns TFJSB_ERR_TIMEOUT (and clears the word) if any wait gave up since the last
  * check, TFJSB_OK otherwise. */
 tfjsb_status tfjsb_check_device_status(tfjsb_ctx* ctx, void* stream);
+/* Sizes the context's three scratch blocks (transposed matMul operands, partial sums of the filter and
+ * bias gradients) to at least `bytes` each, so that later op calls find them large enough.  An op that
+ * needs more grows its block by allocating a larger one (cudaMalloc, no synchronisation; the old block is
+ * kept until tfjsb_shutdown because kernels in flight may still read it). */
+tfjsb_status tfjsb_reserve_scratch(tfjsb_ctx* ctx, int64_t bytes);
 /* Number of kernels this context (and its models) has launched since creation. */
 int64_t tfjsb_launch_count(tfjsb_ctx* ctx);
 
@@ -112,7 +117,8 @@ tfjsb_status tfjsb_window_out_shape(int64_t in, int k, int stride, int dilation,
  *   when transpose_b.  Rank 2 only.  Inner-dimension or `out` mismatch: TFJSB_ERR_SHAPE.
  * TF32 mode uses the tensor-core kernel when K % 4 == 0 and N % 4 == 0 (row pitches must be
  * multiples of 16 bytes for the bulk tensor copies); operands that are not already K-contiguous
- * are transposed into context-owned scratch first.  Other shapes, and FP32 mode, run on CUDA cores. */
+ * are transposed into context-owned scratch first (grown on demand without synchronising, see
+ * tfjsb_reserve_scratch).  Other shapes, and FP32 mode, run on CUDA cores. */
 tfjsb_status tfjsb_matmul(tfjsb_ctx* ctx, const tfjsb_tensor* a, const tfjsb_tensor* b, int transpose_a,
                           int transpose_b, tfjsb_tensor* out, void* stream);
 
@@ -206,6 +212,45 @@ tfjsb_status tfjsb_softmax(tfjsb_ctx* ctx, const tfjsb_tensor* logits, tfjsb_ten
  * One fp32 add and one clamp per element: results are bit-identical to the definition. */
 tfjsb_status tfjsb_bias_act(tfjsb_ctx* ctx, const tfjsb_tensor* x, const tfjsb_tensor* bias, tfjsb_act act,
                             tfjsb_tensor* out, void* stream);
+
+/* ---- gradients ---------------------------------------------------------------------- */
+
+/* The paper differentiates eagerly: each kernel has a gradient function that the backward pass calls
+ * (Sec. 3.5; model.fit of Sec. 3.2 rests on it).  It names no gradient op and gives none of their
+ * arithmetic; the calls below are the adjoints of the forward definitions above, with TensorFlow's
+ * names.  Geometry arguments (strides, pad, dilations) are those of the FORWARD call; `dy` has the
+ * forward output's shape, which is checked.  Sums over pixels are taken in a fixed order: results do
+ * not depend on scheduling.  1x1 / stride-1 convolutions run their two gradients as matrix products on
+ * the tensor cores in TF32 mode (channel counts multiples of 4; for the filter gradient the pixel count
+ * a multiple of 4); every other case runs on CUDA cores in fp32.  All enqueue on `stream` and return;
+ * the filter and bias gradients use context-owned scratch (see tfjsb_reserve_scratch). */
+
+/* dx[n,iy,ix,ci] = sum over (oy,ky), (ox,kx) with oy*sh - pt + ky*dh = iy and ox*sw - pl + kx*dw = ix, and co,
+ *                  of dy[n,oy,ox,co] * filter[ky,kx,ci,co].
+ * dy [N,Ho,Wo,Cout], filter [fh,fw,Cin,Cout], dx [N,H,W,Cin] (dx's shape names the forward input's). */
+tfjsb_status tfjsb_conv2d_backprop_input(tfjsb_ctx* ctx, const tfjsb_tensor* dy, const tfjsb_tensor* filter,
+                                         const int strides[2], tfjsb_pad pad, const int dilations[2], tfjsb_tensor* dx,
+                                         void* stream);
+/* dfilter[ky,kx,ci,co] = sum_{n,oy,ox} x[n, oy*sh - pt + ky*dh, ox*sw - pl + kx*dw, ci] * dy[n,oy,ox,co]
+ * (samples outside the image are zero).  dfilter's shape names the filter's. */
+tfjsb_status tfjsb_conv2d_backprop_filter(tfjsb_ctx* ctx, const tfjsb_tensor* x, const tfjsb_tensor* dy,
+                                          const int strides[2], tfjsb_pad pad, const int dilations[2],
+                                          tfjsb_tensor* dfilter, void* stream);
+/* The same two gradients of tf.depthwiseConv2d: filter [fh,fw,C,mult], dy [N,Ho,Wo,C*mult], output
+ * channel c*mult+q pairs with input channel c. */
+tfjsb_status tfjsb_depthwise_conv2d_backprop_input(tfjsb_ctx* ctx, const tfjsb_tensor* dy, const tfjsb_tensor* filter,
+                                                   const int strides[2], tfjsb_pad pad, const int dilations[2],
+                                                   tfjsb_tensor* dx, void* stream);
+tfjsb_status tfjsb_depthwise_conv2d_backprop_filter(tfjsb_ctx* ctx, const tfjsb_tensor* x, const tfjsb_tensor* dy,
+                                                    const int strides[2], tfjsb_pad pad, const int dilations[2],
+                                                    tfjsb_tensor* dfilter, void* stream);
+/* Gradient through the fused epilogue y = act(z + bias), given the forward OUTPUT y:
+ *   dz = dy where the activation passed its input through (none: everywhere; relu: y > 0;
+ *   relu6: 0 < y < 6), +0 elsewhere.  Bit-exact.  y, dy, dz: one shape, rank 1..4. */
+tfjsb_status tfjsb_act_backprop(tfjsb_ctx* ctx, const tfjsb_tensor* y, const tfjsb_tensor* dy, tfjsb_act act,
+                                tfjsb_tensor* dz, void* stream);
+/* dbias[c] = sum of dz[..., c] over every other dimension.  dz rank 1..4, dbias [last dim of dz]. */
+tfjsb_status tfjsb_bias_backprop(tfjsb_ctx* ctx, const tfjsb_tensor* dz, tfjsb_tensor* dbias, void* stream);
 
 /* ---- models ------------------------------------------------------------------------- */
 

@@ -35,6 +35,9 @@ EXPORTS = [
     "tfjsb_run_model_host_async", "tfjsb_model_host_wait",
     "tfjsb_model_set_keep_all", "tfjsb_model_set_graph", "tfjsb_model_set_fusion", "tfjsb_model_layer_output", "tfjsb_model_profile",
     "tfjsb_matmul_bf16", "tfjsb_model_layer_output_f32", "tfjsb_model_layer_shape", "tfjsb_model_layer_kernel",
+    "tfjsb_reserve_scratch", "tfjsb_conv2d_backprop_input", "tfjsb_conv2d_backprop_filter",
+    "tfjsb_depthwise_conv2d_backprop_input", "tfjsb_depthwise_conv2d_backprop_filter", "tfjsb_act_backprop",
+    "tfjsb_bias_backprop",
 ]
 
 
@@ -108,6 +111,12 @@ def _load_library() -> ctypes.CDLL:
     lib.tfjsb_model_layer_output_f32.argtypes = [vp, i32, vp, vp]
     lib.tfjsb_model_layer_shape.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)]
     lib.tfjsb_model_layer_kernel.argtypes = [vp, i32, ctypes.c_char_p, ctypes.c_int32]
+    lib.tfjsb_reserve_scratch.argtypes = [vp, i64]
+    for name in ("tfjsb_conv2d_backprop_input", "tfjsb_conv2d_backprop_filter", "tfjsb_depthwise_conv2d_backprop_input",
+                 "tfjsb_depthwise_conv2d_backprop_filter"):
+        getattr(lib, name).argtypes = [vp, tp, tp, ip, i32, ip, tp, vp]
+    lib.tfjsb_act_backprop.argtypes = [vp, tp, tp, i32, tp, vp]
+    lib.tfjsb_bias_backprop.argtypes = [vp, tp, tp, vp]
     return lib
 
 
@@ -292,6 +301,44 @@ class Context:
         out = self._empty(x.shape) if out is None else out
         self._check(lib.tfjsb_bias_act(self._h, _desc(x), None if bias is None else _desc(bias), ACT[act],
                                        _desc(out), _stream()))
+        return out
+
+    def reserve_scratch(self, nbytes: int):
+        self._check(lib.tfjsb_reserve_scratch(self._h, int(nbytes)))
+
+    # -- gradients (geometry arguments are the forward call's)
+    def conv2d_backprop_input(self, x_shape, filter, dy, strides=(1, 1), pad="same", dilations=(1, 1), out=None):
+        out = self._empty(x_shape) if out is None else out
+        self._check(lib.tfjsb_conv2d_backprop_input(self._h, _desc(dy), _desc(filter), _int2(strides), PAD[pad],
+                                                    _int2(dilations), _desc(out), _stream()))
+        return out
+
+    def conv2d_backprop_filter(self, x, filter_shape, dy, strides=(1, 1), pad="same", dilations=(1, 1), out=None):
+        out = self._empty(filter_shape) if out is None else out
+        self._check(lib.tfjsb_conv2d_backprop_filter(self._h, _desc(x), _desc(dy), _int2(strides), PAD[pad],
+                                                     _int2(dilations), _desc(out), _stream()))
+        return out
+
+    def depthwise_conv2d_backprop_input(self, x_shape, filter, dy, strides=(1, 1), pad="same", dilations=(1, 1), out=None):
+        out = self._empty(x_shape) if out is None else out
+        self._check(lib.tfjsb_depthwise_conv2d_backprop_input(self._h, _desc(dy), _desc(filter), _int2(strides), PAD[pad],
+                                                              _int2(dilations), _desc(out), _stream()))
+        return out
+
+    def depthwise_conv2d_backprop_filter(self, x, filter_shape, dy, strides=(1, 1), pad="same", dilations=(1, 1), out=None):
+        out = self._empty(filter_shape) if out is None else out
+        self._check(lib.tfjsb_depthwise_conv2d_backprop_filter(self._h, _desc(x), _desc(dy), _int2(strides), PAD[pad],
+                                                               _int2(dilations), _desc(out), _stream()))
+        return out
+
+    def act_backprop(self, y, dy, act="none", out=None):
+        out = self._empty(y.shape) if out is None else out
+        self._check(lib.tfjsb_act_backprop(self._h, _desc(y), _desc(dy), ACT[act], _desc(out), _stream()))
+        return out
+
+    def bias_backprop(self, dz, out=None):
+        out = self._empty((dz.shape[-1],)) if out is None else out
+        self._check(lib.tfjsb_bias_backprop(self._h, _desc(dz), _desc(out), _stream()))
         return out
 
     def model(self, layers: Sequence, input_shape) -> "Model":

@@ -36,6 +36,7 @@ SOURCES = [
     "gemm_bf16_tcgen05.cu",
     "gemm_bf16_pair.cu",
     "bf16_storage.cu",
+    "backprop.cu",
 ]
 
 NVCC_FLAGS = [

@@ -25,13 +25,13 @@ tfjsb_status cuda_fail(tfjsb_ctx* ctx, cudaError_t err, const char* what) {
 tfjsb_status ensure_scratch(tfjsb_ctx* ctx, Scratch* s, size_t bytes) {
     if (s->bytes >= bytes) return TFJSB_OK;
     if (s->ptr) {
-        // earlier launches may still be reading the old block
-        cudaError_t e = cudaDeviceSynchronize();
-        if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaDeviceSynchronize");
-        cudaFree(s->ptr);
+        // earlier launches may still be reading the old block: keep it until the device is known to be idle
+        ctx->retired.push_back(s->ptr);
         s->ptr = nullptr;
+        if (bytes < 2 * s->bytes) bytes = 2 * s->bytes;
         s->bytes = 0;
     }
+    bytes = (bytes + 255) / 256 * 256;
     cudaError_t e = cudaMalloc(&s->ptr, bytes);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
@@ -190,6 +190,8 @@ tfjsb_status tfjsb_shutdown(tfjsb_ctx* ctx) {
     if (ctx->dev_status) cudaFree(ctx->dev_status);
     if (ctx->scratch_a.ptr) cudaFree(ctx->scratch_a.ptr);
     if (ctx->scratch_b.ptr) cudaFree(ctx->scratch_b.ptr);
+    if (ctx->scratch_c.ptr) cudaFree(ctx->scratch_c.ptr);
+    for (void* p : ctx->retired) cudaFree(p);
     delete ctx;
     return TFJSB_OK;
 }
@@ -575,6 +577,217 @@ tfjsb_status tfjsb_bias_act(tfjsb_ctx* ctx, const tfjsb_tensor* x, const tfjsb_t
                                     static_cast<float*>(out->data), numel(x) / C, C, act,
                                     static_cast<cudaStream_t>(stream), &ctx->launches);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "bias_act launch");
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_reserve_scratch(tfjsb_ctx* ctx, int64_t bytes) {
+    TFJSB_REQUIRE_CTX(ctx);
+    if (bytes < 0) return fail(ctx, TFJSB_ERR_INVALID_ARG, "negative size");
+    tfjsb_status st;
+    if ((st = ensure_scratch(ctx, &ctx->scratch_a, (size_t)bytes)) != TFJSB_OK) return st;
+    if ((st = ensure_scratch(ctx, &ctx->scratch_b, (size_t)bytes)) != TFJSB_OK) return st;
+    return ensure_scratch(ctx, &ctx->scratch_c, (size_t)bytes);
+}
+
+// ---- gradients --------------------------------------------------------------------------------------
+
+namespace {
+
+// Checks shared by the four convolution gradients: `xs` has the forward input's shape, `fs` the filter's,
+// `dy` the forward output's; fills the forward geometry.
+tfjsb_status grad_geometry(tfjsb_ctx* ctx, const tfjsb_tensor* xs, const tfjsb_tensor* fs, const tfjsb_tensor* dy,
+                           const int strides[2], int pad, const int dilations[2], bool depthwise, ConvGeom* g) {
+    if (fs->dims[2] != xs->dims[3])
+        return fail(ctx, TFJSB_ERR_SHAPE, "filter has " + std::to_string(fs->dims[2]) + " input channels, x has " +
+                                              std::to_string(xs->dims[3]));
+    if (fs->dims[0] > 0x7fff || fs->dims[1] > 0x7fff) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "filter window too large");
+    if (depthwise && fs->dims[3] < 1) return fail(ctx, TFJSB_ERR_SHAPE, "channel multiplier must be >= 1");
+    const int64_t co = depthwise ? xs->dims[3] * fs->dims[3] : fs->dims[3];
+    tfjsb_status st = conv_geometry(ctx, xs, (int)fs->dims[0], (int)fs->dims[1], strides, pad, dilations, co, dy, g);
+    if (st != TFJSB_OK) return st;
+    if (depthwise) g->mult = (int)fs->dims[3];
+    return TFJSB_OK;
+}
+
+}  // namespace
+
+tfjsb_status tfjsb_conv2d_backprop_input(tfjsb_ctx* ctx, const tfjsb_tensor* dy, const tfjsb_tensor* filter, const int strides[2],
+                                         tfjsb_pad pad, const int dilations[2], tfjsb_tensor* dx, void* stream) {
+    TFJSB_REQUIRE_CTX(ctx);
+    tfjsb_status st;
+    if ((st = check_tensor(ctx, dy, "dy", 4, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, filter, "filter", 4, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, dx, "dx", 4, 4)) != TFJSB_OK) return st;
+    ConvGeom g;
+    if ((st = grad_geometry(ctx, dx, filter, dy, strides, pad, dilations, false, &g)) != TFJSB_OK) return st;
+    if (overlaps(dx, dy) || overlaps(dx, filter)) return fail(ctx, TFJSB_ERR_INVALID_ARG, "dx aliases an input");
+    if (numel(dx) == 0) return TFJSB_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const float* pg = static_cast<const float*>(dy->data);
+    const float* pf = static_cast<const float*>(filter->data);
+    float* pdx = static_cast<float*>(dx->data);
+    if (numel(dy) == 0 || g.Co == 0) {
+        cudaError_t e = cudaMemsetAsync(pdx, 0, (size_t)numel(dx) * 4, s);
+        return e == cudaSuccess ? TFJSB_OK : cuda_fail(ctx, e, "cudaMemsetAsync");
+    }
+    if (g.fh == 1 && g.fw == 1 && g.sh == 1 && g.sw == 1)
+        // dx [M, Cin] = dy [M, Cout] . f [Cin, Cout]^T: both operands already have the summed index contiguous
+        return matmul_2d(ctx, pg, pf, pdx, g.N * g.H * g.W, g.Co, g.C, 0, 1, s);
+    cudaError_t e = launch_conv2d_backprop_input(pg, pf, pdx, g, ctx->sm_count, s, &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "conv2d_backprop_input launch");
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_conv2d_backprop_filter(tfjsb_ctx* ctx, const tfjsb_tensor* x, const tfjsb_tensor* dy, const int strides[2],
+                                          tfjsb_pad pad, const int dilations[2], tfjsb_tensor* dfilter, void* stream) {
+    TFJSB_REQUIRE_CTX(ctx);
+    tfjsb_status st;
+    if ((st = check_tensor(ctx, x, "x", 4, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, dy, "dy", 4, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, dfilter, "dfilter", 4, 4)) != TFJSB_OK) return st;
+    ConvGeom g;
+    if ((st = grad_geometry(ctx, x, dfilter, dy, strides, pad, dilations, false, &g)) != TFJSB_OK) return st;
+    if (overlaps(dfilter, dy) || overlaps(dfilter, x)) return fail(ctx, TFJSB_ERR_INVALID_ARG, "dfilter aliases an input");
+    if (numel(dfilter) == 0) return TFJSB_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const float* px = static_cast<const float*>(x->data);
+    const float* pg = static_cast<const float*>(dy->data);
+    float* pdf = static_cast<float*>(dfilter->data);
+    cudaError_t e;
+    const int64_t pixels = g.N * g.Ho * g.Wo;
+    if (pixels == 0) {
+        e = cudaMemsetAsync(pdf, 0, (size_t)numel(dfilter) * 4, s);
+        return e == cudaSuccess ? TFJSB_OK : cuda_fail(ctx, e, "cudaMemsetAsync");
+    }
+    const bool pointwise = g.fh == 1 && g.fw == 1 && g.sh == 1 && g.sw == 1;
+    if (pointwise && ctx->math == TFJSB_MATH_TF32 && ctx->encode_tiled) {
+        // df [Cin, Cout] = x^T . dy, a product whose summed index is the pixel.  The pixels are cut into B
+        // slices; slice b of x and of dy is transposed into scratch ([Cin, M/B] and [Cout, M/B]), the B small
+        // products run as one batched launch of the tensor-core GEMM (their tiles share the SMs), and the B
+        // partial results are added in slice order.
+        const int64_t M = pixels;
+        const int64_t tiles = ((g.C + 127) / 128) * ((g.Co + 31) / 32);
+        int64_t B = 0;
+        for (int64_t cand = 1024; cand >= 1; cand >>= 1) {
+            if (M % cand != 0 || (M / cand) % 4 != 0 || (cand > 1 && M / cand < 256)) continue;
+            if (cand > 1 && cand * tiles > 8 * (int64_t)ctx->sm_count) continue;
+            B = cand;
+            break;
+        }
+        if (B >= 1 && gemm_tf32_supported(g.C, g.Co, M / B) && M / B <= 65535LL * 32) {
+            const int64_t Ms = M / B;
+            if ((st = ensure_scratch(ctx, &ctx->scratch_a, (size_t)M * g.C * 4)) != TFJSB_OK) return st;
+            if ((st = ensure_scratch(ctx, &ctx->scratch_b, (size_t)M * g.Co * 4)) != TFJSB_OK) return st;
+            if (B > 1 && (st = ensure_scratch(ctx, &ctx->scratch_c, (size_t)B * g.C * g.Co * 4)) != TFJSB_OK) return st;
+            if ((e = launch_transpose_batched(px, ctx->scratch_a.ptr, B, Ms, g.C, s, &ctx->launches)) != cudaSuccess)
+                return cuda_fail(ctx, e, "transpose(x)");
+            if ((e = launch_transpose_batched(pg, ctx->scratch_b.ptr, B, Ms, g.Co, s, &ctx->launches)) != cudaSuccess)
+                return cuda_fail(ctx, e, "transpose(dy)");
+            GemmTf32Plan plan;
+            float* target = B > 1 ? ctx->scratch_c.ptr : pdf;
+            if ((st = gemm_tf32_plan(ctx, ctx->scratch_a.ptr, ctx->scratch_b.ptr, target, g.C, g.Co, Ms, &plan, B)) != TFJSB_OK) return st;
+            if ((e = launch_gemm_tf32(plan, nullptr, TFJSB_ACT_NONE, ctx->dev_status, s, &ctx->launches)) != cudaSuccess)
+                return cuda_fail(ctx, e, "tf32 gemm launch");
+            if (B > 1 && (e = launch_sum_rows(ctx->scratch_c.ptr, pdf, nullptr, B, (int64_t)g.C * g.Co, 1, s, &ctx->launches)) != cudaSuccess)
+                return cuda_fail(ctx, e, "partial-sum launch");
+            return TFJSB_OK;
+        }
+    }
+    int slices = backprop_slices(pixels, ctx->sm_count);
+    const int64_t tile_blocks = (int64_t)g.fh * g.fw * ((g.C + 31) / 32) * ((g.Co + 31) / 32);
+    while (slices > 1 && tile_blocks * slices > 16 * (int64_t)ctx->sm_count) slices >>= 1;
+    if (slices > 1 && (st = ensure_scratch(ctx, &ctx->scratch_c, (size_t)slices * numel(dfilter) * 4)) != TFJSB_OK) return st;
+    if ((e = launch_conv2d_backprop_filter(px, pg, pdf, ctx->scratch_c.ptr, slices, g, s, &ctx->launches)) != cudaSuccess)
+        return cuda_fail(ctx, e, "conv2d_backprop_filter launch");
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_depthwise_conv2d_backprop_input(tfjsb_ctx* ctx, const tfjsb_tensor* dy, const tfjsb_tensor* filter,
+                                                   const int strides[2], tfjsb_pad pad, const int dilations[2], tfjsb_tensor* dx,
+                                                   void* stream) {
+    TFJSB_REQUIRE_CTX(ctx);
+    tfjsb_status st;
+    if ((st = check_tensor(ctx, dy, "dy", 4, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, filter, "filter", 4, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, dx, "dx", 4, 4)) != TFJSB_OK) return st;
+    ConvGeom g;
+    if ((st = grad_geometry(ctx, dx, filter, dy, strides, pad, dilations, true, &g)) != TFJSB_OK) return st;
+    if (overlaps(dx, dy) || overlaps(dx, filter)) return fail(ctx, TFJSB_ERR_INVALID_ARG, "dx aliases an input");
+    if (numel(dx) == 0) return TFJSB_OK;
+    cudaError_t e = launch_depthwise_backprop_input(static_cast<const float*>(dy->data), static_cast<const float*>(filter->data),
+                                                    static_cast<float*>(dx->data), g, ctx->sm_count,
+                                                    static_cast<cudaStream_t>(stream), &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "depthwise_backprop_input launch");
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_depthwise_conv2d_backprop_filter(tfjsb_ctx* ctx, const tfjsb_tensor* x, const tfjsb_tensor* dy,
+                                                    const int strides[2], tfjsb_pad pad, const int dilations[2],
+                                                    tfjsb_tensor* dfilter, void* stream) {
+    TFJSB_REQUIRE_CTX(ctx);
+    tfjsb_status st;
+    if ((st = check_tensor(ctx, x, "x", 4, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, dy, "dy", 4, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, dfilter, "dfilter", 4, 4)) != TFJSB_OK) return st;
+    ConvGeom g;
+    if ((st = grad_geometry(ctx, x, dfilter, dy, strides, pad, dilations, true, &g)) != TFJSB_OK) return st;
+    if (overlaps(dfilter, dy) || overlaps(dfilter, x)) return fail(ctx, TFJSB_ERR_INVALID_ARG, "dfilter aliases an input");
+    if (numel(dfilter) == 0) return TFJSB_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int64_t pixels = g.N * g.Ho * g.Wo;
+    if (pixels == 0) {
+        cudaError_t e = cudaMemsetAsync(dfilter->data, 0, (size_t)numel(dfilter) * 4, s);
+        return e == cudaSuccess ? TFJSB_OK : cuda_fail(ctx, e, "cudaMemsetAsync");
+    }
+    int slices = backprop_slices(pixels, ctx->sm_count);
+    if (slices > 1 && (st = ensure_scratch(ctx, &ctx->scratch_c, (size_t)slices * numel(dfilter) * 4)) != TFJSB_OK) return st;
+    cudaError_t e = launch_depthwise_backprop_filter(static_cast<const float*>(x->data), static_cast<const float*>(dy->data),
+                                                     static_cast<float*>(dfilter->data), ctx->scratch_c.ptr, slices, g, s,
+                                                     &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "depthwise_backprop_filter launch");
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_act_backprop(tfjsb_ctx* ctx, const tfjsb_tensor* y, const tfjsb_tensor* dy, tfjsb_act act, tfjsb_tensor* dz,
+                                void* stream) {
+    TFJSB_REQUIRE_CTX(ctx);
+    tfjsb_status st;
+    if (act != TFJSB_ACT_NONE && act != TFJSB_ACT_RELU && act != TFJSB_ACT_RELU6) return fail(ctx, TFJSB_ERR_INVALID_ARG, "unknown activation");
+    if ((st = check_tensor(ctx, y, "y", 1, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, dy, "dy", 1, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, dz, "dz", 1, 4)) != TFJSB_OK) return st;
+    if (dy->rank != y->rank || dz->rank != y->rank) return fail(ctx, TFJSB_ERR_SHAPE, "y, dy and dz must have one shape");
+    for (int i = 0; i < y->rank; ++i)
+        if (dy->dims[i] != y->dims[i] || dz->dims[i] != y->dims[i]) return fail(ctx, TFJSB_ERR_SHAPE, "y, dy and dz must have one shape");
+    if (overlaps(dz, y) || overlaps(dz, dy)) return fail(ctx, TFJSB_ERR_INVALID_ARG, "dz aliases an input");
+    if (numel(y) == 0) return TFJSB_OK;
+    cudaError_t e = launch_act_backprop(static_cast<const float*>(y->data), static_cast<const float*>(dy->data),
+                                        static_cast<float*>(dz->data), numel(y), act, ctx->sm_count,
+                                        static_cast<cudaStream_t>(stream), &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "act_backprop launch");
+    return TFJSB_OK;
+}
+
+tfjsb_status tfjsb_bias_backprop(tfjsb_ctx* ctx, const tfjsb_tensor* dz, tfjsb_tensor* dbias, void* stream) {
+    TFJSB_REQUIRE_CTX(ctx);
+    tfjsb_status st;
+    if ((st = check_tensor(ctx, dz, "dz", 1, 4)) != TFJSB_OK) return st;
+    if ((st = check_tensor(ctx, dbias, "dbias", 1, 1)) != TFJSB_OK) return st;
+    const int64_t C = dz->dims[dz->rank - 1];
+    if (dbias->dims[0] != C) return fail(ctx, TFJSB_ERR_SHAPE, "dbias must have the length of dz's last dimension");
+    if (overlaps(dbias, dz)) return fail(ctx, TFJSB_ERR_INVALID_ARG, "dbias aliases the input");
+    if (C == 0) return TFJSB_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int64_t rows = numel(dz) / C;
+    if (rows == 0) {
+        cudaError_t e = cudaMemsetAsync(dbias->data, 0, (size_t)C * 4, s);
+        return e == cudaSuccess ? TFJSB_OK : cuda_fail(ctx, e, "cudaMemsetAsync");
+    }
+    const int slices = backprop_slices(rows, ctx->sm_count);
+    if (slices > 1 && (st = ensure_scratch(ctx, &ctx->scratch_c, (size_t)slices * C * 4)) != TFJSB_OK) return st;
+    cudaError_t e = launch_sum_rows(static_cast<const float*>(dz->data), static_cast<float*>(dbias->data), ctx->scratch_c.ptr, rows, C,
+                                    slices, s, &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "bias_backprop launch");
     return TFJSB_OK;
 }
 

@@ -8,6 +8,7 @@
 
 #include <string>
 #include <utility>
+#include <vector>
 
 #include "tfjsb.h"
 
@@ -86,6 +87,8 @@ struct tfjsb_ctx {
     unsigned int* dev_status = nullptr;  // device status word
     tfjsb::EncodeTiledFn encode_tiled = nullptr;
     tfjsb::Scratch scratch_a, scratch_b;  // transposed operands of tfjsb_matmul
+    tfjsb::Scratch scratch_c;             // partial sums of the filter / bias gradients
+    std::vector<void*> retired;            // outgrown scratch blocks, freed at shutdown
     int64_t launches = 0;
     int live_models = 0;
 };
@@ -94,7 +97,9 @@ namespace tfjsb {
 
 tfjsb_status fail(tfjsb_ctx* ctx, tfjsb_status st, const std::string& msg);
 tfjsb_status cuda_fail(tfjsb_ctx* ctx, cudaError_t err, const char* what);
-// Grows `s` to at least `bytes` (frees and reallocates; callers keep stream order in mind).
+// Grows `s` to at least `bytes`.  Never synchronises: an outgrown block may still be read by kernels in
+// flight on any stream, so it is kept until tfjsb_shutdown; growth is geometric, so all outgrown blocks
+// together are smaller than the live one.  tfjsb_reserve_scratch sizes the blocks up front.
 tfjsb_status ensure_scratch(tfjsb_ctx* ctx, Scratch* s, size_t bytes);
 
 // ---- kernel launch with optional programmatic dependent launch --------------------------------------
@@ -278,6 +283,28 @@ cudaError_t launch_bf16_to_f32(const void* in, float* out, int64_t n, cudaStream
 cudaError_t launch_round_to_bf16_in_place(float* v, int64_t n, cudaStream_t s, int64_t* launches);
 // out [r*N, r*K] = r copies of km [N, K] down the diagonal, zeros elsewhere
 cudaError_t launch_block_diagonal(const float* km, float* out, int64_t N, int64_t K, int r, cudaStream_t s, int64_t* launches);
+
+// ---- gradients (backprop.cu) ----------------------------------------------------------------------
+// `g` is the geometry of the FORWARD op (H, W, C the forward input; Ho, Wo, Co the forward output).
+int backprop_slices(int64_t rows, int sm_count);
+cudaError_t launch_conv2d_backprop_input(const float* dy, const float* f, float* dx, const ConvGeom& g, int sm_count,
+                                         cudaStream_t s, int64_t* launches);
+// `partial` holds slices * fh*fw*C*Co floats (unused when slices == 1)
+cudaError_t launch_conv2d_backprop_filter(const float* x, const float* dy, float* df, float* partial, int slices,
+                                          const ConvGeom& g, cudaStream_t s, int64_t* launches);
+cudaError_t launch_depthwise_backprop_input(const float* dy, const float* f, float* dx, const ConvGeom& g, int sm_count,
+                                            cudaStream_t s, int64_t* launches);
+// `partial` holds slices * fh*fw*Co floats (unused when slices == 1)
+cudaError_t launch_depthwise_backprop_filter(const float* x, const float* dy, float* df, float* partial, int slices,
+                                             const ConvGeom& g, cudaStream_t s, int64_t* launches);
+cudaError_t launch_act_backprop(const float* y, const float* dy, float* dz, int64_t n, int act, int sm_count, cudaStream_t s,
+                                int64_t* launches);
+// out[c] = sum_r in[r, c]; with slices > 1 in two steps through `partial` (slices * C floats)
+cudaError_t launch_sum_rows(const float* in, float* out, float* partial, int64_t rows, int64_t C, int slices, cudaStream_t s,
+                            int64_t* launches);
+// out[b, c, r] = in[b, r, c] for `batches` matrices [rows, cols] stored one after the other
+cudaError_t launch_transpose_batched(const float* in, float* out, int64_t batches, int64_t rows, int64_t cols, cudaStream_t s,
+                                     int64_t* launches);
 
 // Fused depthwise 3x3 (stride 1) + pointwise block: the depthwise output is produced straight into
 // the tensor-core operand layout in shared memory and never written to global memory.
