@@ -389,6 +389,16 @@ tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const float* x, const ConvGeom& g, D
     plan->smem_bytes = (size_t)stages * d.stage_bytes + 128;
     const int64_t max_grid = (int64_t)ctx->sm_count * 2;
     plan->grid = (int)(plan->num_tiles < max_grid ? plan->num_tiles : max_grid);
+    // A CTA walks tiles first, first + grid, ...; the channel block is the fastest tile coordinate, so a grid
+    // that is a multiple of the number of channel blocks keeps every CTA on ONE channel block: its nine filter
+    // vectors and the bias are loaded once instead of once per tile (a dependent global load in front of a
+    // tile's short burst of work), while the CTAs that run side by side still cover all channel blocks of the
+    // same pixels, so whole pixel vectors are read from DRAM at about the same time.  Measured on
+    // [128,14,14,512]: 22.7 -> 20.6 us; no change for the 7 x 7 and stride-2 layers.
+    if (plan->grid > plan->c_blocks && plan->grid % plan->c_blocks != 0) {
+        const int rounded = plan->grid / plan->c_blocks * plan->c_blocks;
+        if (rounded * 8 >= plan->grid * 7) plan->grid = rounded;
+    }
     plan->variant = v;
     return TFJSB_OK;
 }
