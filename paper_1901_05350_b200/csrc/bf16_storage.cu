@@ -452,7 +452,7 @@ __global__ void block_diagonal_kernel(const float* __restrict__ km, float* __res
 
 int grid_for(int64_t threads, int block) {
     const int64_t blocks = (threads + block - 1) / block;
-    const int64_t cap = 148LL * 64;
+    const int64_t cap = (int64_t)current_sm_count() * 64;
     return (int)(blocks < 1 ? 1 : (blocks > cap ? cap : blocks));
 }
 

@@ -102,6 +102,12 @@ tfjsb_status cuda_fail(tfjsb_ctx* ctx, cudaError_t err, const char* what);
 // together are smaller than the live one.  tfjsb_reserve_scratch sizes the blocks up front.
 tfjsb_status ensure_scratch(tfjsb_ctx* ctx, Scratch* s, size_t bytes);
 
+// Raises a kernel's dynamic shared-memory limit once per (kernel, device): function attributes belong to
+// a device's copy of the function, and contexts on several devices or host threads may launch the same kernel.
+cudaError_t smem_attr_once(const void* kernel, int bytes);
+// Number of SMs of the current device (cached per device): grid caps of the grid-stride kernels.
+int current_sm_count();
+
 // ---- kernel launch with optional programmatic dependent launch --------------------------------------
 // The executor sets this while it enqueues a model: its kernels all call pdl_wait() before reading
 // their inputs, so each may be launched while the previous one drains and only its prologue
@@ -320,6 +326,7 @@ struct DwPwPlan {
     int patch_bytes = 0, patch_stride = 0;
     // small-window convolution mode of the same kernel
     bool conv = false;
+    bool y_bf16 = false;  // the output tensor is bfloat16 (narrow storage): small-window mode only
     int row_floats = 0, patch_rows = 0;
 };
 bool dwpw_fused_supported(const ConvGeom& dw, int64_t Cout);
@@ -329,7 +336,8 @@ tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
 // memory); `bt` is the filter packed [Cout, 32].  Launched with launch_dwpw_fused (pw_bias / pw_act = the
 // convolution's bias and activation; the depthwise arguments are ignored).
 bool conv_patch_supported(const ConvGeom& g);
-tfjsb_status conv_patch_plan(tfjsb_ctx* ctx, const float* x, const float* bt, float* y, const ConvGeom& g, DwPwPlan* plan);
+tfjsb_status conv_patch_plan(tfjsb_ctx* ctx, const float* x, const float* bt, void* y, const ConvGeom& g, DwPwPlan* plan,
+                             bool y_bf16 = false);
 cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, const float* dw_bias, int dw_act,
                               const float* pw_bias, int pw_act, unsigned int* dev_status, cudaStream_t s,
                               int64_t* launches);

@@ -335,13 +335,9 @@ constexpr int DW_SMEM_BUDGET = 113 * 1024;  // two CTAs per SM
 template <int S, int TW, int R, int D = 1>
 cudaError_t launch_tma_instance(const DepthwisePlan& plan, const float* f, const float* bias, int act, float* y,
                                 const ConvGeom& g, unsigned int* dev_status, cudaStream_t s) {
-    static bool attr_set = false;
     auto kernel = depthwise3x3_tma_kernel<S, TW, R, D>;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DW_SMEM_BUDGET);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    cudaError_t ae = smem_attr_once(reinterpret_cast<const void*>(kernel), DW_SMEM_BUDGET);
+    if (ae != cudaSuccess) return ae;
     DwTiling t{plan.tiles_x, plan.tiles_y, plan.c_blocks, plan.stages, (long long)plan.num_tiles};
     return launch_k(kernel, dim3(plan.grid), dim3(DW_TMA_THREADS), plan.smem_bytes, s, plan.map_x, f, bias, act, y, g, t,
                     dev_status);
@@ -449,7 +445,7 @@ cudaError_t launch_depthwise(const DepthwisePlan& plan, const float* x, const fl
         }
     }
     int64_t blocks = (n_out + DW_THREADS - 1) / DW_THREADS;
-    if (blocks > 148 * 32) blocks = 148 * 32;
+    if (blocks > current_sm_count() * 32) blocks = current_sm_count() * 32;
     depthwise_generic_kernel<<<(unsigned)blocks, DW_THREADS, 0, s>>>(x, f, bias, act, y, g, n_out);
     ++*launches;
     return cudaGetLastError();

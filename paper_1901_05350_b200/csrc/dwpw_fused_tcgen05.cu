@@ -106,7 +106,11 @@ __device__ __forceinline__ void store_depthwise_block(const float2 (&acc)[F_TH /
     }
 }
 
-template <bool CONV>
+// NARROW (small-window mode only): the narrow-storage form of the convolution.  The fp32 input is rounded to
+// bfloat16 as it is rearranged into the A operand and the filter holds bfloat16 values, so every TF32
+// product is the exact product of two bfloat16 values (8 significand bits fit TF32's 11); the sum is fp32
+// and the result is stored as bfloat16 (rounded to nearest even after bias and activation).
+template <bool CONV, bool NARROW = false>
 __global__ void __launch_bounds__(CONV ? F_CONV_THREADS : F_THREADS, CONV ? 2 : 1)
 dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ CUtensorMap map_y, const FusedArgs args) {
@@ -359,7 +363,11 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 const uint32_t row_addr = slab + (uint32_t)lane * 128u;
                 const float* bias = (args.pw_bias != nullptr) ? args.pw_bias + col0 : nullptr;
                 const int cols_left = args.Co - col0;
-                if (args.pw_act == TFJSB_ACT_RELU6) stage_chunk<TFJSB_ACT_RELU6>(r, bias, cols_left, row_addr, lane);
+                if (NARROW) {  // 32 rows of 64 bytes in the 64-byte swizzle of the bfloat16 output map
+                    if (args.pw_act == TFJSB_ACT_RELU6) stage_chunk_bf16<TFJSB_ACT_RELU6>(r, bias, cols_left, slab, lane);
+                    else if (args.pw_act == TFJSB_ACT_RELU) stage_chunk_bf16<TFJSB_ACT_RELU>(r, bias, cols_left, slab, lane);
+                    else stage_chunk_bf16<TFJSB_ACT_NONE>(r, bias, cols_left, slab, lane);
+                } else if (args.pw_act == TFJSB_ACT_RELU6) stage_chunk<TFJSB_ACT_RELU6>(r, bias, cols_left, row_addr, lane);
                 else if (args.pw_act == TFJSB_ACT_RELU) stage_chunk<TFJSB_ACT_RELU>(r, bias, cols_left, row_addr, lane);
                 else stage_chunk<TFJSB_ACT_NONE>(r, bias, cols_left, row_addr, lane);
                 fence_async_smem();
@@ -407,7 +415,10 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 for (int h = 0; h < BLOCK_K / 4; ++h) {
                     float v[4];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) v[e] = 4 * h + e < args.k_total ? patch[args.koff[4 * h + e]] : 0.0f;
+                    for (int e = 0; e < 4; ++e) {
+                        v[e] = 4 * h + e < args.k_total ? patch[args.koff[4 * h + e]] : 0.0f;
+                        if (NARROW) v[e] = __bfloat162float(__float2bfloat16_rn(v[e]));  // what is stored is a bfloat16
+                    }
                     const uint32_t dst = row_addr + (uint32_t)((h ^ (p & 7)) << 4);
                     asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3])
                                  : "memory");
@@ -546,6 +557,7 @@ tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
     if (ps > 4) ps = 4;
     if (ps < 2) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "no room for the input patch ring");
     plan->conv = false;
+    plan->y_bf16 = false;
     plan->patch_stages = ps;
     plan->patch_bytes = F_PATCH_BYTES;
     plan->patch_stride = F_PATCH_STRIDE;
@@ -604,7 +616,10 @@ bool conv_patch_supported(const ConvGeom& g) {
            g.N < (1LL << 31);
 }
 
-tfjsb_status conv_patch_plan(tfjsb_ctx* ctx, const float* x, const float* bt, float* y, const ConvGeom& g, DwPwPlan* plan) {
+tfjsb_status conv_patch_plan(tfjsb_ctx* ctx, const float* x, const float* bt, void* y, const ConvGeom& g, DwPwPlan* plan,
+                             bool y_bf16) {
+    if (y_bf16 && g.Co % 8 != 0) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "a bfloat16 output needs a channel count that is a multiple of 8");
+    plan->y_bf16 = y_bf16;
     if (!conv_patch_supported(g)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the patch convolution kernel");
     if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
     plan->conv = true;
@@ -666,7 +681,16 @@ tfjsb_status conv_patch_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
         cuuint64_t dims[4] = {(cuuint64_t)g.Co, (cuuint64_t)g.Wo, (cuuint64_t)g.Ho, (cuuint64_t)g.N};
         cuuint64_t strides[3] = {(cuuint64_t)g.Co * 4u, (cuuint64_t)g.Wo * g.Co * 4u, (cuuint64_t)g.Ho * g.Wo * g.Co * 4u};
         cuuint32_t box[4] = {(cuuint32_t)EPI_COLS, (cuuint32_t)F_TW, 2u, 1u};
-        if ((st = encode(&plan->map_y, y, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, "the convolution output")) != TFJSB_OK) return st;
+        if (y_bf16) {
+            for (cuuint64_t& v : strides) v /= 2;  // two bytes per value
+            cuuint32_t elem[4] = {1u, 1u, 1u, 1u};
+            CUresult r = ctx->encode_tiled(&plan->map_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, y, dims, strides, box, elem,
+                                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+                                           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS)
+                return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled failed for the bfloat16 convolution output (CUresult " +
+                                                     std::to_string((int)r) + ")");
+        } else if ((st = encode(&plan->map_y, y, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, "the convolution output")) != TFJSB_OK) return st;
     }
     return TFJSB_OK;
 }
@@ -674,13 +698,12 @@ tfjsb_status conv_patch_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
 cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, const float* dw_bias, int dw_act,
                               const float* pw_bias, int pw_act, unsigned int* dev_status, cudaStream_t s,
                               int64_t* launches) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(dwpw_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 2048);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(dwpw_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, F_CONV_SMEM);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
+    {
+        cudaError_t ae = cudaSuccess;
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<false>), SMEM_LIMIT - 2048);
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<true>), F_CONV_SMEM);
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<true, true>), F_CONV_SMEM);
+        if (ae != cudaSuccess) return ae;
     }
     FusedArgs a;
     a.C = plan.g.C; a.Co = plan.Co;
@@ -703,7 +726,10 @@ cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, cons
     a.dw_filter = dw_filter; a.dw_bias = dw_bias; a.dw_act = dw_act;
     a.pw_bias = pw_bias; a.pw_act = pw_act;
     a.dev_status = dev_status;
-    cudaError_t e = plan.conv ? launch_k(dwpw_fused_kernel<true>, dim3(plan.grid), dim3(F_CONV_THREADS), plan.smem_bytes, s,
+    cudaError_t e = (plan.conv && plan.y_bf16)
+                        ? launch_k(dwpw_fused_kernel<true, true>, dim3(plan.grid), dim3(F_CONV_THREADS), plan.smem_bytes, s,
+                                   plan.map_x, plan.map_b, plan.map_y, a)
+                    : plan.conv ? launch_k(dwpw_fused_kernel<true>, dim3(plan.grid), dim3(F_CONV_THREADS), plan.smem_bytes, s,
                                          plan.map_x, plan.map_b, plan.map_y, a)
                               : launch_k(dwpw_fused_kernel<false>, dim3(plan.grid), dim3(F_THREADS), plan.smem_bytes, s,
                                          plan.map_x, plan.map_b, plan.map_y, a);

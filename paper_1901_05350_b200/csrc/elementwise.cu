@@ -302,7 +302,7 @@ cudaError_t launch_pack_filter(const float* f, float* out, int64_t K, int64_t N,
                                int64_t* launches) {
     const int64_t total = N * k_pad;
     if (total == 0) return cudaSuccess;
-    pack_filter_kernel<<<grid_for(total, kThreads, 148 * 8), kThreads, 0, s>>>(f, out, K, N, k_pad);
+    pack_filter_kernel<<<grid_for(total, kThreads, current_sm_count() * 8), kThreads, 0, s>>>(f, out, K, N, k_pad);
     ++*launches;
     return cudaGetLastError();
 }
@@ -313,10 +313,10 @@ cudaError_t launch_bias_act(const float* x, const float* bias, float* y, int64_t
     if (n == 0) return cudaSuccess;
     if (C % 4 == 0) {
         const int64_t n_vec = n / 4;
-        bias_act_vec4_kernel<<<grid_for(n_vec, kThreads, 148 * 16), kThreads, 0, s>>>(
+        bias_act_vec4_kernel<<<grid_for(n_vec, kThreads, current_sm_count() * 16), kThreads, 0, s>>>(
             reinterpret_cast<const float4*>(x), bias, reinterpret_cast<float4*>(y), n_vec, (int)(C / 4), act);
     } else {
-        bias_act_scalar_kernel<<<grid_for(n, kThreads, 148 * 16), kThreads, 0, s>>>(x, bias, y, n, C, act);
+        bias_act_scalar_kernel<<<grid_for(n, kThreads, current_sm_count() * 16), kThreads, 0, s>>>(x, bias, y, n, C, act);
     }
     ++*launches;
     return cudaGetLastError();
@@ -339,7 +339,7 @@ cudaError_t launch_avg_pool(const float* x, float* y, const ConvGeom& g, cudaStr
         ++*launches;
         return e;
     } else {
-        avg_pool_window_kernel<<<grid_for(n_out, kThreads, 148 * 16), kThreads, 0, s>>>(x, y, g, n_out);
+        avg_pool_window_kernel<<<grid_for(n_out, kThreads, current_sm_count() * 16), kThreads, 0, s>>>(x, y, g, n_out);
     }
     ++*launches;
     return cudaGetLastError();
@@ -349,9 +349,9 @@ cudaError_t launch_max_pool(const float* x, float* y, const ConvGeom& g, cudaStr
     const int64_t n_out = g.N * g.Ho * g.Wo * g.C;
     if (n_out == 0) return cudaSuccess;
     if (g.C % 4 == 0)
-        max_pool_vec4_kernel<<<grid_for(n_out / 4, kThreads, 148 * 32), kThreads, 0, s>>>(x, y, g, n_out / 4);
+        max_pool_vec4_kernel<<<grid_for(n_out / 4, kThreads, current_sm_count() * 32), kThreads, 0, s>>>(x, y, g, n_out / 4);
     else
-        max_pool_window_kernel<<<grid_for(n_out, kThreads, 148 * 16), kThreads, 0, s>>>(x, y, g, n_out);
+        max_pool_window_kernel<<<grid_for(n_out, kThreads, current_sm_count() * 16), kThreads, 0, s>>>(x, y, g, n_out);
     ++*launches;
     return cudaGetLastError();
 }
@@ -359,10 +359,10 @@ cudaError_t launch_max_pool(const float* x, float* y, const ConvGeom& g, cudaStr
 template <int OP>
 static cudaError_t launch_binary_op(const float* a, const float* b, float* out, int64_t n, int64_t b_len, cudaStream_t s) {
     if (n % 4 == 0 && b_len % 4 == 0)
-        binary_vec4_kernel<OP><<<grid_for(n / 4, kThreads, 148 * 16), kThreads, 0, s>>>(
+        binary_vec4_kernel<OP><<<grid_for(n / 4, kThreads, current_sm_count() * 16), kThreads, 0, s>>>(
             reinterpret_cast<const float4*>(a), reinterpret_cast<const float4*>(b), reinterpret_cast<float4*>(out), n / 4, b_len / 4);
     else
-        binary_scalar_kernel<OP><<<grid_for(n, kThreads, 148 * 16), kThreads, 0, s>>>(a, b, out, n, b_len);
+        binary_scalar_kernel<OP><<<grid_for(n, kThreads, current_sm_count() * 16), kThreads, 0, s>>>(a, b, out, n, b_len);
     return cudaGetLastError();
 }
 

@@ -155,6 +155,11 @@ tfjsb_status bind_step(tfjsb_model* m, Step& st, const float* in, float* out) {
         if (rc != TFJSB_OK) return rc;
         st.plan_built = true;
     }
+    if (st.kind == STEP_CONV_NARROW && st.conv_patch && (changed || !st.plan_built)) {
+        tfjsb_status rc = conv_patch_plan(m->ctx, in, st.filter_km, out, st.g, &st.fused_plan, true);
+        if (rc != TFJSB_OK) return rc;
+        st.plan_built = true;
+    }
     if (st.kind == STEP_DEPTHWISE && (changed || !st.plan_built)) {
         tfjsb_status rc = depthwise_plan(m->ctx, in, st.g, &st.dw_plan);
         if (rc != TFJSB_OK) return rc;
@@ -228,6 +233,9 @@ cudaError_t launch_step(tfjsb_model* m, const Step& st, cudaStream_t s) {
             return launch_gemm_bf16(st.plan16, st.pack_r > 1 ? st.bias_packed : st.bias, st.act, ctx->dev_status, s,
                                     &ctx->launches);
         case STEP_CONV_NARROW:
+            if (st.conv_patch)
+                return launch_dwpw_fused(st.fused_plan, nullptr, nullptr, TFJSB_ACT_NONE, st.bias, st.act, ctx->dev_status, s,
+                                         &ctx->launches);
             return launch_conv_narrow(st.in, st.in_f32, st.filter, st.bias, st.act, st.out, st.out_bf16, st.g, s,
                                       &ctx->launches);
         case STEP_DEPTHWISE_NARROW:
@@ -573,6 +581,18 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
             if (sp.in_f32 && (sp.kind == STEP_GEMM_NARROW || sp.kind == STEP_DEPTHWISE_NARROW || sp.kind == STEP_POOL_NARROW))
                 return bail(TFJSB_ERR_UNSUPPORTED, "layer " + std::to_string(i) + ": in the bfloat16 storage mode only conv2d and "
                                                    "softmax layers read an fp32 tensor");
+            // A small-window first layer (the 3x3 stem on RGB input) runs on the tensor cores: the patch kernel
+            // rounds the fp32 image as it builds the operand tile, multiplies in TF32 (exact for bfloat16
+            // values) and stores bfloat16.
+            if (sp.kind == STEP_CONV_NARROW && sp.in_f32 && sp.out_bf16 && !sp.is_dense && sp.g.Co % 8 == 0 &&
+                conv_patch_supported(sp.g) && !getenv("TFJSB_NO_PATCH_CONV")) {
+                const int64_t k_pad = conv_igemm_k_pad(sp.g);
+                if ((st = dev_alloc(m, (size_t)(k_pad * sp.g.Co), &sp.filter_km)) != TFJSB_OK) return bail(st, ctx->last_error);
+                cudaError_t e = launch_pack_filter(sp.filter, sp.filter_km, (int64_t)sp.g.fh * sp.g.fw * sp.g.C, sp.g.Co, k_pad, 0,
+                                                   &ctx->launches);
+                if (e != cudaSuccess) return bail(TFJSB_ERR_CUDA, std::string("packing weights: ") + cudaGetErrorString(e));
+                sp.conv_patch = true;
+            }
         }
     }
     // arena: two regions, each large enough for the largest intermediate
@@ -838,7 +858,7 @@ tfjsb_status tfjsb_model_layer_kernel(tfjsb_model* m, int layer, char* name, int
         case STEP_POOL: k = (st.g.Ho == 1 && st.g.Wo == 1 && st.g.fh == st.g.H && st.g.fw == st.g.W) ? "avg_pool_global_kernel" : "avg_pool_window_kernel"; break;
         case STEP_SOFTMAX: k = "softmax_rows_kernel"; break;
         case STEP_GEMM_NARROW: k = st.plan16.pair ? "gemm_bf16_pair_kernel" : "gemm_bf16_kernel"; break;
-        case STEP_CONV_NARROW: k = "conv_narrow_kernel"; break;
+        case STEP_CONV_NARROW: k = st.conv_patch ? "dwpw_fused_kernel<true, true>" : "conv_narrow_kernel"; break;
         case STEP_DEPTHWISE_NARROW: k = "depthwise3x3_narrow_kernel"; break;
         case STEP_POOL_NARROW: k = "avg_pool_global_narrow_kernel"; break;
     }

@@ -355,12 +355,10 @@ tfjsb_status gemm_bf16_pair_plan(tfjsb_ctx* ctx, const void* a, const void* bt, 
 
 cudaError_t launch_gemm_bf16_pair(const GemmBf16Plan& plan, const float* bias, int act, unsigned int* dev_status,
                                   cudaStream_t s, int64_t* launches) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_bf16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             SMEM_LIMIT - 2048);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
+    {
+        cudaError_t ae = cudaSuccess;
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&gemm_bf16_pair_kernel), SMEM_LIMIT - 2048);
+        if (ae != cudaSuccess) return ae;
     }
     PairArgs16 args;
     args.M = (int)plan.M; args.N = (int)plan.N; args.K = (int)plan.K;

@@ -361,12 +361,10 @@ tfjsb_status gemm_tf32_splitk_plan(tfjsb_ctx* ctx, const float* a, const float* 
 
 cudaError_t launch_gemm_tf32_splitk(const GemmTf32Plan& plan, const float* bias, int act, unsigned int* dev_status,
                                     cudaStream_t s, int64_t* launches) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tf32_splitk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             SMEM_LIMIT - 2048);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
+    {
+        cudaError_t ae = cudaSuccess;
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&gemm_tf32_splitk_kernel), SMEM_LIMIT - 2048);
+        if (ae != cudaSuccess) return ae;
     }
     SplitArgs args;
     args.M = (int)plan.M; args.N = (int)plan.N; args.K = (int)plan.K;

@@ -590,15 +590,11 @@ cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int ac
                              cudaStream_t s, int64_t* launches) {
     if (plan.pair) return launch_gemm_tf32_pair(plan, bias, act, dev_status, s, launches);
     if (plan.cluster_split) return launch_gemm_tf32_splitk(plan, bias, act, dev_status, s, launches);
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tf32_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             SMEM_LIMIT - 2048);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(gemm_tf32_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     SMEM_LIMIT - 2048);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
+    {
+        cudaError_t ae = cudaSuccess;
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&gemm_tf32_kernel<false>), SMEM_LIMIT - 2048);
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&gemm_tf32_kernel<true>), SMEM_LIMIT - 2048);
+        if (ae != cudaSuccess) return ae;
     }
     cudaError_t e;
     KernelArgs args;

@@ -286,9 +286,19 @@ def test_config4_mobilenet_100_224_narrow_every_layer(ctx, oracle):
         assert rel_fro(got, want[i]) <= 1e-2, f"layer {i} ({layer.name}) diverges: {rel_fro(got, want[i]):.3e}"
         if i < len(layers) - 2:
             assert np.all((got.view(np.uint32) & 0xFFFF) == 0), layer.name
-    for i in (0, 1, 2):  # no accumulated noise yet: at most one bfloat16 step, on few elements
-        steps = bf16_steps(host(model.layer_output_f32(i)), want[i])
-        assert steps.max() <= 1 and np.count_nonzero(steps) <= 0.01 * steps.size, i
+    # Each of the first layers on its own: the oracle applied to the input the GPU layer actually read (its own
+    # previous output), so that a one-step difference in an earlier layer, which a later sum can turn into
+    # several steps of a small result, is not in the comparison.  What remains is one bfloat16 step of the value
+    # plus the fp32 summation error (absolute, relative to the largest values of the layer), on few elements.
+    prev = x
+    for i in (0, 1, 2, 3, 4):
+        got = host(model.layer_output_f32(i))
+        alone = oracle.round_bf16(oracle.run_model([layers[i]], prev, storage="bf16"))
+        assert np.all(np.abs(got - alone) <= 2.0 ** -7 * np.abs(alone) + 2e-6 * np.abs(alone).max()), layers[i].name
+        assert np.count_nonzero(got != alone) <= 0.01 * got.size, layers[i].name
+        prev = got
+    steps = bf16_steps(host(model.layer_output_f32(0)), want[0])
+    assert steps.max() <= 1 and np.count_nonzero(steps) <= 0.01 * steps.size
     check_logits(host(model.layer_output_f32(28)), probs, want[28], want[29])
     model.close()
 
