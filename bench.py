@@ -466,7 +466,7 @@ def run_ours(args):
             "sm_mhz_during_timed_region": clocks["sm_mhz"],
             "how": "algorithmic bytes (or flops) of the listed launches / their summed CUDA-event durations, per pass; "
                    "kernel names come from the library (tfjsb_model_layer_kernel); traffic = ncu DRAM read+write bytes "
-                   "per pass for the same launches, scaled from a small-batch capture (null: kernel changed since)",
+                   "per pass for the same launches, from a one-pass capture at the same batch (null: kernel changed since)",
         }
         line["roofline_step"] = {"sum_roofline_us": sum(r["roofline_us"] for r in rows), "sum_measured_us": total_ms * 1e3,
                                  "frac": sum(r["roofline_us"] for r in rows) / (total_ms * 1e3),
@@ -612,10 +612,19 @@ def run_ours(args):
     return 0
 
 
-# DRAM bytes (read + write) per image of one launch, from an ncu capture of the same kernel on the same layer
-# at a small batch (traffic grows in proportion to the batch: every tile streams its own pixels, the weights
-# are a fixed few hundred KB).  Keyed by (kernel, launch name); an entry is dropped when its kernel changes.
-TRAFFIC_BYTES_PER_IMAGE = {}
+# DRAM bytes (read + write) per image of one launch, from a one-pass ncu capture (two DRAM byte counters and the
+# duration, nothing saved or restored) of the same kernels on the same layers at batch 128, divided by 128.
+# Reads are cold and equal the layer's input; writes are counted when L2 evicts them, so layers whose output is
+# smaller than L2 under-count their writes.  Keyed by (kernel, launch name); an entry is dropped when its kernel changes.
+TRAFFIC_BYTES_PER_IMAGE = {
+    ("dwpw_fused_kernel<false>", "dw1+pw1"): 4323550, ("dwpw_fused_kernel<false>", "dw3+pw3"): 2801264,
+    ("dwpw_fused_kernel<false>", "dw5+pw5"): 1191094,
+    ("depthwise3x3_tma_kernel", "dw2"): 3848786, ("depthwise3x3_tma_kernel", "dw4"): 1831464,
+    ("depthwise3x3_tma_kernel", "dw6"): 843858, ("depthwise3x3_tma_kernel", "dw7"): 417474,
+    ("depthwise3x3_tma_kernel", "dw8"): 418886, ("depthwise3x3_tma_kernel", "dw9"): 417810,
+    ("depthwise3x3_tma_kernel", "dw10"): 418432, ("depthwise3x3_tma_kernel", "dw11"): 418440,
+    ("depthwise3x3_tma_kernel", "dw12"): 401696, ("depthwise3x3_tma_kernel", "dw13"): 201150,
+}
 
 
 def traffic_of(kernel, rows):
