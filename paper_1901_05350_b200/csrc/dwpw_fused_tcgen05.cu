@@ -110,7 +110,10 @@ __device__ __forceinline__ void store_depthwise_block(const float2 (&acc)[F_TH /
 // bfloat16 as it is rearranged into the A operand and the filter holds bfloat16 values, so every TF32
 // product is the exact product of two bfloat16 values (8 significand bits fit TF32's 11); the sum is fp32
 // and the result is stored as bfloat16 (rounded to nearest even after bias and activation).
-template <bool CONV, bool NARROW = false>
+// STREAM_B: the weight slices do not stay resident (more k-blocks than the ring has stages) and are fetched
+// again for every tile; the producer then feeds two rings that drain at different rates and must not block on
+// either (a kernel instance of its own, so that the common case keeps its register allocation).
+template <bool CONV, bool NARROW = false, bool STREAM_B = false>
 __global__ void __launch_bounds__(CONV ? F_CONV_THREADS : F_THREADS, CONV ? 2 : 1)
 dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ CUtensorMap map_y, const FusedArgs args) {
@@ -191,7 +194,77 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 
     if (warp == 0) {
         // ---------------------------------------------------------------- producer
-        if (lane == 0) {
+        if (STREAM_B && lane == 0) {
+            // One thread, two rings (input patches for the depthwise warps, weight slices for the tensor core):
+            // it probes both "empty" barriers in turn and issues whichever copy has room.  Issued in program
+            // order, a full weight ring held back the next patch and the depthwise warps spent half their
+            // time waiting for input (28x28x256 -> 256 at batch 128: 78 -> 71 us).
+            int ps = 0, bs = 0;
+            uint32_t pphase = 0, bphase = 0;
+            const int my_tiles = (int)blockIdx.x < args.num_tiles ? (args.num_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+            const int total_p = my_tiles * num_k_blocks, total_b = total_p * args.n_sub;
+            int pk = 0, bk = 0;                  // copies issued so far
+            int p_tile = blockIdx.x, p_kb = 0;   // next patch: tile and k-block
+            int p_n = 0, p_ty = 0, p_tx = 0;
+            bool p_coords = false;
+            int b_kb = 0, b_h = 0;               // next weight slice: k-block and column half
+            bool ok = true;
+            unsigned long long idle_since = 0;
+            while (ok && (pk < total_p || bk < total_b)) {
+                bool progressed = false;
+                // a single ring left to feed: sleep on its barrier instead of probing
+                if (bk == total_b && !bounded_wait(smem_u32(&bar_patch_empty[ps]), pphase ^ 1u, abort_flag)) { ok = false; break; }
+                if (pk == total_p && !bounded_wait(smem_u32(&bar_b_empty[bs]), bphase ^ 1u, abort_flag)) { ok = false; break; }
+                if (pk < total_p && mbar_test_wait(smem_u32(&bar_patch_empty[ps]), pphase ^ 1u)) {
+                    if (!p_coords) {
+                        p_n = p_tile / tiles_per_image;
+                        const int rem = p_tile - p_n * tiles_per_image;
+                        p_ty = rem / args.tiles_x;
+                        p_tx = rem - p_ty * args.tiles_x;
+                        p_coords = true;
+                    }
+                    const uint32_t pf = smem_u32(&bar_patch_full[ps]);
+                    mbar_arrive_expect_tx(pf, (uint32_t)args.patch_bytes);
+                    tma_load_4d(patch_base + (uint32_t)(ps * args.patch_stride), &map_x, pf, p_kb * BLOCK_K,
+                                p_tx * F_TW - args.pl, p_ty * F_TH - args.pt, p_n);
+                    if (++ps == args.patch_stages) { ps = 0; pphase ^= 1u; }
+                    if (++p_kb == num_k_blocks) { p_kb = 0; p_tile += gridDim.x; p_coords = false; }
+                    ++pk;
+                    progressed = true;
+                }
+                if (bk < total_b && mbar_test_wait(smem_u32(&bar_b_empty[bs]), bphase ^ 1u)) {
+                    const uint32_t bf = smem_u32(&bar_b_full[bs]);
+                    mbar_arrive_expect_tx(bf, (uint32_t)b_stage_bytes);
+                    tma_load_2d(b_base + (uint32_t)bs * (uint32_t)b_stage_bytes, &map_b, bf, b_kb * BLOCK_K, b_h * block_n);
+                    if (++bs == args.b_stages) { bs = 0; bphase ^= 1u; }
+                    if (++b_h == args.n_sub) { b_h = 0; if (++b_kb == num_k_blocks) b_kb = 0; }
+                    ++bk;
+                    progressed = true;
+                }
+                if (progressed) { idle_since = 0; continue; }
+                __nanosleep(32);
+                if (*abort_flag) ok = false;
+                else if (idle_since == 0) idle_since = global_ns();
+                else if (global_ns() - idle_since > WAIT_LIMIT_NS) ok = false;
+            }
+            if (!ok || *abort_flag) {
+                if (!*abort_flag) {
+                    *abort_flag = 1;
+                    atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_PRODUCER);
+                }
+                // copies in flight must land before the CTA's shared memory is released
+                const unsigned long long t0 = global_ns();
+                bool all = true;
+                for (int k = (pk > args.patch_stages ? pk - args.patch_stages : 0); k < pk; ++k)
+                    while (!mbar_try_wait(smem_u32(&bar_patch_full[k % args.patch_stages]), (uint32_t)((k / args.patch_stages) & 1)))
+                        if (global_ns() - t0 > WAIT_LIMIT_NS) { all = false; break; }
+                for (int k = (bk > args.b_stages ? bk - args.b_stages : 0); k < bk; ++k)
+                    while (!mbar_try_wait(smem_u32(&bar_b_full[k % args.b_stages]), (uint32_t)((k / args.b_stages) & 1)))
+                        if (global_ns() - t0 > WAIT_LIMIT_NS) { all = false; break; }
+                if (!all) atomicOr(args.dev_status, DEV_STATUS_TIMEOUT_DRAIN);
+            }
+        }
+        if (!STREAM_B && lane == 0) {
             int ps = 0, bs = 0;
             uint32_t pphase = 0, bphase = 0;
             int issued = 0;
@@ -702,6 +775,7 @@ cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, cons
         cudaError_t ae = cudaSuccess;
         if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<false>), SMEM_LIMIT - 2048);
         if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<true>), F_CONV_SMEM);
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<false, false, true>), SMEM_LIMIT - 2048);
         if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<true, true>), F_CONV_SMEM);
         if (ae != cudaSuccess) return ae;
     }
@@ -728,6 +802,9 @@ cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, cons
     a.dev_status = dev_status;
     cudaError_t e = (plan.conv && plan.y_bf16)
                         ? launch_k(dwpw_fused_kernel<true, true>, dim3(plan.grid), dim3(F_CONV_THREADS), plan.smem_bytes, s,
+                                   plan.map_x, plan.map_b, plan.map_y, a)
+                    : (!plan.conv && !plan.b_resident)
+                        ? launch_k(dwpw_fused_kernel<false, false, true>, dim3(plan.grid), dim3(F_THREADS), plan.smem_bytes, s,
                                    plan.map_x, plan.map_b, plan.map_y, a)
                     : plan.conv ? launch_k(dwpw_fused_kernel<true>, dim3(plan.grid), dim3(F_CONV_THREADS), plan.smem_bytes, s,
                                          plan.map_x, plan.map_b, plan.map_y, a)

@@ -40,6 +40,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
+// Non-blocking probe of the same condition (try_wait may suspend the thread for a while before it
+// answers; a thread that watches two barriers must not sleep on one of them).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
 // Waits for the phase with the given parity; gives up after WAIT_LIMIT_NS or when another role
 // has raised the abort flag.  Returns false on giving up.  The first probe is inlined: a wait that
 // is already satisfied costs one try_wait (a call here doubled the cost of every pipeline step of
