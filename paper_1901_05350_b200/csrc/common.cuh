@@ -321,6 +321,7 @@ struct DwPwPlan {
     int Co = 0;
     int block_n = 0, n_sub = 1, acc_stages = 0, patch_stages = 0, a_stages = 0, b_stages = 0;
     bool b_resident = false;  // the B ring holds all of Bt for the whole kernel
+    bool wide_epi = false;    // sixteen epilogue warps and one depthwise group (one k-block per tile)
     int tiles_x = 0, tiles_y = 0, num_tiles = 0, grid = 0;
     size_t smem_bytes = 0;
     int patch_bytes = 0, patch_stride = 0;

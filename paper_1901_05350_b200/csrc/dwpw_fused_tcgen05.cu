@@ -30,6 +30,8 @@
 // rearrange it into the A operand (thread = pixel), the packed filter [Cout, 32] stays resident as
 // B, and the block is 14 warps so that two CTAs share an SM: per tile every role costs mostly its
 // own synchronisation, and two CTAs double each of them.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "ptx_sm100.cuh"
 #include "umma_tile.cuh"
@@ -113,7 +115,10 @@ __device__ __forceinline__ void store_depthwise_block(const float2 (&acc)[F_TH /
 // STREAM_B: the weight slices do not stay resident (more k-blocks than the ring has stages) and are fetched
 // again for every tile; the producer then feeds two rings that drain at different rates and must not block on
 // either (a kernel instance of its own, so that the common case keeps its register allocation).
-template <bool CONV, bool NARROW = false, bool STREAM_B = false>
+// WIDE_EPI: blocks with few input channels (one k-block per tile) are paced by the epilogue, not by the
+// depthwise stage: sixteen epilogue warps (four per tensor-memory lane quarter, taking tiles in turn) and a
+// single group of eight depthwise warps, instead of eight and two groups of eight.
+template <bool CONV, bool NARROW = false, bool STREAM_B = false, bool WIDE_EPI = false>
 __global__ void __launch_bounds__(CONV ? F_CONV_THREADS : F_THREADS, CONV ? 2 : 1)
 dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ CUtensorMap map_y, const FusedArgs args) {
@@ -132,8 +137,10 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     // little arithmetic per tile: what bounds a tile there is the fixed cost of each role's
     // synchronisation (barrier waits, fences, MMA issue), so it runs as two small CTAs per SM, which
     // doubles every role, instead of one large CTA.
-    constexpr int EPI_WARPS = 8;
-    constexpr int CMP_WARPS = CONV ? F_CONV_CMP_WARPS : F_DW_WARPS;
+    static_assert(!(WIDE_EPI && CONV), "the wide epilogue belongs to the depthwise + pointwise mode");
+    constexpr int EPI_WARPS = WIDE_EPI ? 16 : 8;
+    constexpr int DW_GROUPS = WIDE_EPI ? 1 : F_DW_GROUPS;
+    constexpr int CMP_WARPS = CONV ? F_CONV_CMP_WARPS : DW_GROUPS * F_DW_GROUP_WARPS;
     constexpr int GROUP_WARPS = CONV ? F_CONV_CMP_WARPS : F_DW_GROUP_WARPS;  // warps that fill one A stage
     constexpr int CMP_WARP0 = 2 + EPI_WARPS;
     constexpr int EPI_GROUPS = EPI_WARPS / 4;
@@ -579,7 +586,7 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                         mbar_arrive(smem_u32(&bar_patch_empty[ps]));
                     }
                 }
-                if (++turn == F_DW_GROUPS) turn = 0;
+                if (++turn == DW_GROUPS) turn = 0;
                 if (++ps == args.patch_stages) { ps = 0; pphase ^= 1u; }
                 if (++as == args.a_stages) { as = 0; aphase ^= 1u; }
             }
@@ -622,10 +629,13 @@ tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
     plan->b_stages = plan->n_sub == 2 ? 3 : (bn == 256 ? 2 : 3);
     // all of Bt resident when its k-blocks fit the B ring's four barriers and leave room for three patches
     const int k_blocks = dw.C / BLOCK_K;
+    // one k-block per tile and a narrow output: the epilogue paces the kernel (see WIDE_EPI)
+    plan->wide_epi = k_blocks == 1 && bn <= 128 && !getenv("TFJSB_NO_WIDE_EPI");
+    const int epi_bytes = plan->wide_epi ? 2 * EPI_BYTES : EPI_BYTES;
     plan->b_resident = plan->n_sub == 1 && k_blocks <= 4 &&
-                       EPI_BYTES + plan->a_stages * A_STAGE_BYTES + k_blocks * bn * BLOCK_K * 4 + 3 * F_PATCH_STRIDE <= SMEM_LIMIT - 2048;
+                       epi_bytes + plan->a_stages * A_STAGE_BYTES + k_blocks * bn * BLOCK_K * 4 + 3 * F_PATCH_STRIDE <= SMEM_LIMIT - 2048;
     if (plan->b_resident) plan->b_stages = k_blocks;
-    const int fixed = EPI_BYTES + plan->a_stages * A_STAGE_BYTES + plan->b_stages * bn * BLOCK_K * 4;
+    const int fixed = epi_bytes + plan->a_stages * A_STAGE_BYTES + plan->b_stages * bn * BLOCK_K * 4;
     int ps = (SMEM_LIMIT - 2048 - fixed) / F_PATCH_STRIDE;
     if (ps > 4) ps = 4;
     if (ps < 2) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "no room for the input patch ring");
@@ -696,6 +706,7 @@ tfjsb_status conv_patch_plan(tfjsb_ctx* ctx, const float* x, const float* bt, vo
     if (!conv_patch_supported(g)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the patch convolution kernel");
     if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
     plan->conv = true;
+    plan->wide_epi = false;
     plan->g = g;
     plan->Co = g.Co;
     int bn = 32;
@@ -776,6 +787,7 @@ cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, cons
         if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<false>), SMEM_LIMIT - 2048);
         if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<true>), F_CONV_SMEM);
         if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<false, false, true>), SMEM_LIMIT - 2048);
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<false, false, false, true>), SMEM_LIMIT - 2048);
         if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<true, true>), F_CONV_SMEM);
         if (ae != cudaSuccess) return ae;
     }
@@ -802,6 +814,9 @@ cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, cons
     a.dev_status = dev_status;
     cudaError_t e = (plan.conv && plan.y_bf16)
                         ? launch_k(dwpw_fused_kernel<true, true>, dim3(plan.grid), dim3(F_CONV_THREADS), plan.smem_bytes, s,
+                                   plan.map_x, plan.map_b, plan.map_y, a)
+                    : (!plan.conv && plan.wide_epi && plan.b_resident)
+                        ? launch_k(dwpw_fused_kernel<false, false, false, true>, dim3(plan.grid), dim3(F_THREADS), plan.smem_bytes, s,
                                    plan.map_x, plan.map_b, plan.map_y, a)
                     : (!plan.conv && !plan.b_resident)
                         ? launch_k(dwpw_fused_kernel<false, false, true>, dim3(plan.grid), dim3(F_THREADS), plan.smem_bytes, s,
