@@ -317,8 +317,12 @@ tfjsb_status tfjsb_model_host_wait(tfjsb_model* model);
  * channels a multiple of 32) can run as ONE kernel that keeps the depthwise output in shared
  * memory as the tensor-core operand, so the intermediate tensor is neither written nor read back.
  * mode 0: never; 1 (default): where the pair has enough 8x16-pixel tiles for the fused kernel to be
- * the faster choice; 2: wherever the shapes allow.  Results are bit-identical in every mode.  The
- * keep-all debug mode always runs the layers separately. */
+ * the faster choice; 2: wherever the shapes allow.  In the fp32 storage modes results are bit-identical
+ * in every mode.  Models in the BF16 storage mode have the same kernel in that format (bfloat16 in and
+ * out, the depthwise result rounded to bfloat16 on its way into the operand tile); there it is never
+ * the default (the separate narrow kernels are faster) and agrees with the separate kernels to the
+ * rounding of a stored value, not bit for bit.  The keep-all debug mode always runs the layers
+ * separately. */
 tfjsb_status tfjsb_model_set_fusion(tfjsb_model* model, int mode);
 
 /* Replays one run as a CUDA graph instead of enqueueing the layers one by one (the enqueue cost per

@@ -331,8 +331,9 @@ struct DwPwPlan {
     int row_floats = 0, patch_rows = 0;
 };
 bool dwpw_fused_supported(const ConvGeom& dw, int64_t Cout);
-tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, float* y, const ConvGeom& dw,
-                             int64_t Cout, DwPwPlan* plan);
+// `narrow`: x and y are bfloat16 (narrow storage), bt holds bfloat16 values as fp32
+tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const void* x, const float* bt, void* y, const ConvGeom& dw,
+                             int64_t Cout, DwPwPlan* plan, bool narrow = false);
 // conv2d with fh*fw*Cin <= 32 on the same kernel (input patch by bulk tensor copy, im2col in shared
 // memory); `bt` is the filter packed [Cout, 32].  Launched with launch_dwpw_fused (pw_bias / pw_act = the
 // convolution's bias and activation; the depthwise arguments are ignored).

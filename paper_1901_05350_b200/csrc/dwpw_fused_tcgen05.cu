@@ -91,7 +91,7 @@ __device__ __forceinline__ void fma4s(float4& acc, const float4& a, const float4
 // into the A operand (GEMM row of a pixel = row*16 + column).  The activation is a template parameter:
 // the kernel is close to instruction-issue bound, and a run-time choice costs two extra instructions
 // per value.
-template <int ACT>
+template <int ACT, bool ROUND_BF16 = false>
 __device__ __forceinline__ void store_depthwise_block(const float2 (&acc)[F_TH / 2][2], const float2 b, uint32_t a_stage,
                                                       int rg, int colg, int c2) {
     constexpr int R = F_TH / 2;
@@ -99,8 +99,12 @@ __device__ __forceinline__ void store_depthwise_block(const float2 (&acc)[F_TH /
     for (int r = 0; r < R; ++r) {
 #pragma unroll
         for (int cc = 0; cc < 2; ++cc) {
-            const float vx = apply_act_t<ACT>(acc[r][cc].x + b.x);
-            const float vy = apply_act_t<ACT>(acc[r][cc].y + b.y);
+            float vx = apply_act_t<ACT>(acc[r][cc].x + b.x);
+            float vy = apply_act_t<ACT>(acc[r][cc].y + b.y);
+            if (ROUND_BF16) {  // narrow storage: the depthwise layer's output is a bfloat16 (an exact TF32 operand)
+                vx = __bfloat162float(__float2bfloat16_rn(vx));
+                vy = __bfloat162float(__float2bfloat16_rn(vy));
+            }
             const int p = (rg * R + r) * F_TW + colg * 2 + cc;
             const uint32_t dst = a_stage + (uint32_t)p * 128u + (uint32_t)(((c2 >> 1) ^ (p & 7)) << 4) + (uint32_t)((c2 & 1) << 3);
             asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(dst), "f"(vx), "f"(vy) : "memory");
@@ -108,7 +112,10 @@ __device__ __forceinline__ void store_depthwise_block(const float2 (&acc)[F_TH /
     }
 }
 
-// NARROW (small-window mode only): the narrow-storage form of the convolution.  The fp32 input is rounded to
+// NARROW: the narrow-storage forms.  Depthwise + pointwise: the block input is bfloat16 (the patch is copied as
+// such and widened by the depthwise threads), the depthwise result is rounded to bfloat16 before it becomes the
+// A operand, the pointwise filter holds bfloat16 values, the output is stored as bfloat16.  Small-window mode: the
+// narrow-storage form of the convolution.  The fp32 input is rounded to
 // bfloat16 as it is rearranged into the A operand and the filter holds bfloat16 values, so every TF32
 // product is the exact product of two bfloat16 values (8 significand bits fit TF32's 11); the sum is fp32
 // and the result is stored as bfloat16 (rounded to nearest even after bias and activation).
@@ -555,13 +562,22 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     float2 acc[R][2];
 #pragma unroll
                     for (int r = 0; r < R; ++r) acc[r][0] = acc[r][1] = make_float2(0.f, 0.f);
-                    const float* patch = patch_ptr + (size_t)ps * (F_PATCH_STRIDE / 4) + ((rg * R) * F_PW + colg * 2) * BLOCK_K + c2 * 2;
+                    // element (two channels) index of this thread's first sample in the patch [10][18][32 channels]
+                    const int origin = ((rg * R) * F_PW + colg * 2) * BLOCK_K + c2 * 2;
+                    const float* patch = patch_ptr + (size_t)ps * (F_PATCH_STRIDE / 4) + origin;
+                    const uint32_t* patch16 = reinterpret_cast<const uint32_t*>(reinterpret_cast<const uint8_t*>(patch_ptr) +
+                                                                                (size_t)ps * args.patch_stride) + (origin >> 1);
 #pragma unroll
                     for (int j = 0; j < R + 2; ++j) {
                         const float* row = patch + j * F_PW * BLOCK_K;
                         float2 v[4];
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) v[q] = *reinterpret_cast<const float2*>(row + q * BLOCK_K);
+                        for (int q = 0; q < 4; ++q) {
+                            if (NARROW) {  // two bfloat16 channels in 32 bits: each is the upper half of its fp32
+                                const uint32_t pair = patch16[(j * F_PW * BLOCK_K + q * BLOCK_K) >> 1];
+                                v[q] = make_float2(__uint_as_float(pair << 16), __uint_as_float(pair & 0xffff0000u));
+                            } else v[q] = *reinterpret_cast<const float2*>(row + q * BLOCK_K);
+                        }
 #pragma unroll
                         for (int ky = 0; ky < 3; ++ky) {
                             const int d = j - ky;
@@ -576,9 +592,9 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                         }
                     }
                     const uint32_t a_stage = a_base + (uint32_t)as * A_STAGE_BYTES;
-                    if (args.dw_act == TFJSB_ACT_RELU6) store_depthwise_block<TFJSB_ACT_RELU6>(acc, b, a_stage, rg, colg, c2);
-                    else if (args.dw_act == TFJSB_ACT_RELU) store_depthwise_block<TFJSB_ACT_RELU>(acc, b, a_stage, rg, colg, c2);
-                    else store_depthwise_block<TFJSB_ACT_NONE>(acc, b, a_stage, rg, colg, c2);
+                    if (args.dw_act == TFJSB_ACT_RELU6) store_depthwise_block<TFJSB_ACT_RELU6, NARROW>(acc, b, a_stage, rg, colg, c2);
+                    else if (args.dw_act == TFJSB_ACT_RELU) store_depthwise_block<TFJSB_ACT_RELU, NARROW>(acc, b, a_stage, rg, colg, c2);
+                    else store_depthwise_block<TFJSB_ACT_NONE, NARROW>(acc, b, a_stage, rg, colg, c2);
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0) {
@@ -613,8 +629,9 @@ bool dwpw_fused_supported(const ConvGeom& dw, int64_t Cout) {
            tiles < (1LL << 31) && dw.N < (1LL << 31);
 }
 
-tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, float* y, const ConvGeom& dw,
-                             int64_t Cout, DwPwPlan* plan) {
+tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const void* x, const float* bt, void* y, const ConvGeom& dw,
+                             int64_t Cout, DwPwPlan* plan, bool narrow) {
+    if (narrow && Cout % 8 != 0) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "a bfloat16 output needs a channel count that is a multiple of 8");
     if (!dwpw_fused_supported(dw, Cout)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the fused block kernel");
     if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
     plan->g = dw;
@@ -629,22 +646,24 @@ tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
     plan->b_stages = plan->n_sub == 2 ? 3 : (bn == 256 ? 2 : 3);
     // all of Bt resident when its k-blocks fit the B ring's four barriers and leave room for three patches
     const int k_blocks = dw.C / BLOCK_K;
+    // a bfloat16 patch is half the bytes (12 KiB keeps the stages 1024-aligned)
+    const int patch_bytes = narrow ? F_PATCH_BYTES / 2 : F_PATCH_BYTES, patch_stride = narrow ? 12 * 1024 : F_PATCH_STRIDE;
     // one k-block per tile and a narrow output: the epilogue paces the kernel (see WIDE_EPI)
     plan->wide_epi = k_blocks == 1 && bn <= 128 && !getenv("TFJSB_NO_WIDE_EPI");
     const int epi_bytes = plan->wide_epi ? 2 * EPI_BYTES : EPI_BYTES;
     plan->b_resident = plan->n_sub == 1 && k_blocks <= 4 &&
-                       epi_bytes + plan->a_stages * A_STAGE_BYTES + k_blocks * bn * BLOCK_K * 4 + 3 * F_PATCH_STRIDE <= SMEM_LIMIT - 2048;
+                       epi_bytes + plan->a_stages * A_STAGE_BYTES + k_blocks * bn * BLOCK_K * 4 + 3 * patch_stride <= SMEM_LIMIT - 2048;
     if (plan->b_resident) plan->b_stages = k_blocks;
     const int fixed = epi_bytes + plan->a_stages * A_STAGE_BYTES + plan->b_stages * bn * BLOCK_K * 4;
-    int ps = (SMEM_LIMIT - 2048 - fixed) / F_PATCH_STRIDE;
+    int ps = (SMEM_LIMIT - 2048 - fixed) / patch_stride;
     if (ps > 4) ps = 4;
     if (ps < 2) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "no room for the input patch ring");
     plan->conv = false;
-    plan->y_bf16 = false;
+    plan->y_bf16 = narrow;
     plan->patch_stages = ps;
-    plan->patch_bytes = F_PATCH_BYTES;
-    plan->patch_stride = F_PATCH_STRIDE;
-    plan->smem_bytes = (size_t)1024 + fixed + (size_t)ps * F_PATCH_STRIDE;
+    plan->patch_bytes = patch_bytes;
+    plan->patch_stride = patch_stride;
+    plan->smem_bytes = (size_t)1024 + fixed + (size_t)ps * patch_stride;
     plan->tiles_x = (dw.Wo + F_TW - 1) / F_TW;
     plan->tiles_y = (dw.Ho + F_TH - 1) / F_TH;
     const int64_t tiles = dw.N * plan->tiles_x * plan->tiles_y;
@@ -652,9 +671,10 @@ tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
     plan->grid = (int)(tiles < ctx->sm_count ? tiles : ctx->sm_count);
 
     auto encode = [&](CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides,
-                      const cuuint32_t* box, CUtensorMapSwizzle swz, const char* what) -> tfjsb_status {
+                      const cuuint32_t* box, CUtensorMapSwizzle swz, const char* what, bool bf16 = false) -> tfjsb_status {
         cuuint32_t elem[4] = {1u, 1u, 1u, 1u};
-        CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<void*>(base), dims,
+        CUresult r = ctx->encode_tiled(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                                       (cuuint32_t)rank, const_cast<void*>(base), dims,
                                        strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS)
@@ -665,9 +685,10 @@ tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
     tfjsb_status st;
     {
         cuuint64_t dims[4] = {(cuuint64_t)dw.C, (cuuint64_t)dw.W, (cuuint64_t)dw.H, (cuuint64_t)dw.N};
-        cuuint64_t strides[3] = {(cuuint64_t)dw.C * 4u, (cuuint64_t)dw.W * dw.C * 4u, (cuuint64_t)dw.H * dw.W * dw.C * 4u};
+        const cuuint64_t eb = narrow ? 2u : 4u;  // bytes per stored value
+        cuuint64_t strides[3] = {(cuuint64_t)dw.C * eb, (cuuint64_t)dw.W * dw.C * eb, (cuuint64_t)dw.H * dw.W * dw.C * eb};
         cuuint32_t box[4] = {(cuuint32_t)BLOCK_K, (cuuint32_t)F_PW, (cuuint32_t)F_PH, 1u};
-        if ((st = encode(&plan->map_x, x, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE, "the block input")) != TFJSB_OK) return st;
+        if ((st = encode(&plan->map_x, x, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE, "the block input", narrow)) != TFJSB_OK) return st;
     }
     {
         cuuint64_t dims[2] = {(cuuint64_t)dw.C, (cuuint64_t)Cout};
@@ -677,9 +698,11 @@ tfjsb_status dwpw_fused_plan(tfjsb_ctx* ctx, const float* x, const float* bt, fl
     }
     {
         cuuint64_t dims[4] = {(cuuint64_t)Cout, (cuuint64_t)dw.Wo, (cuuint64_t)dw.Ho, (cuuint64_t)dw.N};
-        cuuint64_t strides[3] = {(cuuint64_t)Cout * 4u, (cuuint64_t)dw.Wo * Cout * 4u, (cuuint64_t)dw.Ho * dw.Wo * Cout * 4u};
+        const cuuint64_t eb = narrow ? 2u : 4u;
+        cuuint64_t strides[3] = {(cuuint64_t)Cout * eb, (cuuint64_t)dw.Wo * Cout * eb, (cuuint64_t)dw.Ho * dw.Wo * Cout * eb};
         cuuint32_t box[4] = {(cuuint32_t)EPI_COLS, (cuuint32_t)F_TW, 2u, 1u};
-        if ((st = encode(&plan->map_y, y, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B, "the block output")) != TFJSB_OK) return st;
+        if ((st = encode(&plan->map_y, y, 4, dims, strides, box, narrow ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                         "the block output", narrow)) != TFJSB_OK) return st;
     }
     return TFJSB_OK;
 }
@@ -788,6 +811,9 @@ cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, cons
         if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<true>), F_CONV_SMEM);
         if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<false, false, true>), SMEM_LIMIT - 2048);
         if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<false, false, false, true>), SMEM_LIMIT - 2048);
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<false, true>), SMEM_LIMIT - 2048);
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<false, true, true>), SMEM_LIMIT - 2048);
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<false, true, false, true>), SMEM_LIMIT - 2048);
         if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&dwpw_fused_kernel<true, true>), F_CONV_SMEM);
         if (ae != cudaSuccess) return ae;
     }
@@ -812,6 +838,20 @@ cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, cons
     a.dw_filter = dw_filter; a.dw_bias = dw_bias; a.dw_act = dw_act;
     a.pw_bias = pw_bias; a.pw_act = pw_act;
     a.dev_status = dev_status;
+    if (!plan.conv && plan.y_bf16) {
+        cudaError_t en;
+        if (plan.wide_epi && plan.b_resident)
+            en = launch_k(dwpw_fused_kernel<false, true, false, true>, dim3(plan.grid), dim3(F_THREADS), plan.smem_bytes, s, plan.map_x,
+                          plan.map_b, plan.map_y, a);
+        else if (!plan.b_resident)
+            en = launch_k(dwpw_fused_kernel<false, true, true>, dim3(plan.grid), dim3(F_THREADS), plan.smem_bytes, s, plan.map_x,
+                          plan.map_b, plan.map_y, a);
+        else
+            en = launch_k(dwpw_fused_kernel<false, true>, dim3(plan.grid), dim3(F_THREADS), plan.smem_bytes, s, plan.map_x, plan.map_b,
+                          plan.map_y, a);
+        ++*launches;
+        return en;
+    }
     cudaError_t e = (plan.conv && plan.y_bf16)
                         ? launch_k(dwpw_fused_kernel<true, true>, dim3(plan.grid), dim3(F_CONV_THREADS), plan.smem_bytes, s,
                                    plan.map_x, plan.map_b, plan.map_y, a)

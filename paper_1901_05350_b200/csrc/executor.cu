@@ -198,7 +198,7 @@ tfjsb_status bind_all(tfjsb_model* m, const float* input, float* output) {
             Step& st = m->steps[i];
             if (!st.fuse_next) continue;
             Step& pw = m->steps[i + 1];
-            tfjsb_status rc = dwpw_fused_plan(m->ctx, st.in, pw.filter_km, pw.out, st.g, pw.N, &st.fused_plan);
+            tfjsb_status rc = dwpw_fused_plan(m->ctx, st.in, pw.filter_km, pw.out, st.g, pw.N, &st.fused_plan, m->narrow);
             if (rc != TFJSB_OK) return rc;
         }
     }
@@ -543,6 +543,7 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
             float* km16 = nullptr;
             if ((st = dev_alloc(m, (w_elems + 1) / 2, &km16)) != TFJSB_OK) return bail(st, ctx->last_error);
             cudaError_t e = launch_transpose(step.filter, km32, step.K, step.N, 0, &ctx->launches);
+            step.filter_km = km32;  // [N, K] fp32 holding bfloat16 values: the B operand of the fused block kernel
             if (r > 1) {
                 float* diag = nullptr;
                 if ((st = dev_alloc(m, w_elems, &diag)) != TFJSB_OK) return bail(st, ctx->last_error);
@@ -613,6 +614,25 @@ tfjsb_status tfjsb_model_create(tfjsb_ctx* ctx, const tfjsb_layer_desc* layers, 
                 dw.fusable = true;
                 dw.fuse_pays = tiles >= 4 * (int64_t)ctx->sm_count;
                 dw.fuse_next = dw.fuse_pays;
+            }
+        }
+    }
+    if (m->narrow && !getenv("TFJSB_NO_FUSION")) {
+        // The same fused kernel in the narrow format: bfloat16 patches in, the depthwise result rounded to
+        // bfloat16 on its way into the operand tile, TF32 multiplies (exact for bfloat16 values), bfloat16 out.
+        for (size_t i = 0; i + 1 < m->steps.size(); ++i) {
+            Step& dw = m->steps[i];
+            const Step& pw = m->steps[i + 1];
+            if (dw.kind == STEP_DEPTHWISE_NARROW && pw.kind == STEP_GEMM_NARROW && !pw.is_dense && pw.filter_km && pw.K == dw.g.Co &&
+                pw.M == dw.g.N * dw.g.Ho * dw.g.Wo && pw.N % 8 == 0 && dw.out_bf16 && pw.out_bf16 && dwpw_fused_supported(dw.g, pw.N)) {
+                const int64_t tiles = dw.g.N * ((dw.g.Ho + 7) / 8) * ((dw.g.Wo + 15) / 16);
+                // Available (tfjsb_model_set_fusion(model, 2)) but not chosen: the fused kernel is paced by its own
+                // pipeline, not by memory traffic, so halving the bytes does not speed it up, while the separate
+                // narrow kernels do gain from it (batch 128: 118 / 106 / 66 us fused against 66+55 / 63+37 / 35+26).
+                (void)tiles;
+                dw.fusable = true;
+                dw.fuse_pays = false;
+                dw.fuse_next = false;
             }
         }
     }

@@ -257,6 +257,83 @@ def test_small_integer_model_is_bit_exact(ctx, oracle):
     model.close()
 
 
+FUSED_BLOCKS = [
+    # N, H, W, C, Cout: depthwise 3x3 + pointwise as ONE kernel in the narrow format
+    (2, 40, 52, 32, 64),     # one k-block per tile: the sixteen-epilogue-warp instance; ragged tiles (40 = 5 x 8, 52 = 3 x 16 + 4)
+    (2, 24, 40, 128, 128),   # four k-blocks, weights resident in shared memory
+    (1, 20, 24, 256, 256),   # eight k-blocks, weights streamed per tile
+    (3, 9, 17, 64, 40),      # images barely larger than a tile, Cout not a power of two
+]
+
+
+def block_model(si_mod, seed, N, H, W, C, Cout, integers):
+    """conv 3x3 (3 -> C) -> depthwise 3x3 -> pointwise (C -> Cout) -> global pool; the pair in the middle fuses."""
+    L = si_mod.Layer
+    layers = [L(kind="conv2d", filter_hw=(3, 3), strides=(1, 1), pad="same", act="relu6", out_channels=C, name="stem"),
+              L(kind="depthwise_conv2d", filter_hw=(3, 3), strides=(1, 1), pad="same", act="relu6", out_channels=1, name="dw"),
+              L(kind="conv2d", filter_hw=(1, 1), strides=(1, 1), pad="same", act="relu6", out_channels=Cout, name="pw"),
+              L(kind="global_avg_pool", name="pool")]
+    if integers:
+        x = si_mod.small_integers(seed, 0, (N, H, W, 3), -2, 2)
+        # sparse small filters keep every sum an integer below 2^8, which bfloat16 holds exactly
+        layers[0].filter = si_mod.small_integers(seed, 1, (3, 3, 3, C), -1, 1)
+        layers[0].bias = si_mod.small_integers(seed, 2, (C,), -1, 1)
+        layers[1].filter = si_mod.small_integers(seed, 3, (3, 3, C, 1), -1, 1) * (si_mod.small_integers(seed, 4, (3, 3, C, 1), 0, 2) == 0)
+        layers[1].bias = si_mod.small_integers(seed, 5, (C,), -1, 1)
+        layers[2].filter = si_mod.small_integers(seed, 6, (1, 1, C, Cout), -1, 1) * (si_mod.small_integers(seed, 7, (1, 1, C, Cout), 0, 7) == 0)
+        layers[2].bias = si_mod.small_integers(seed, 8, (Cout,), -1, 1)
+    else:
+        x = si_mod.uniform(seed, 0, (N, H, W, 3), -1, 1)
+        si_mod.make_model_weights(layers, 3, seed)
+    return x, layers
+
+
+@pytest.mark.parametrize("case", FUSED_BLOCKS)
+def test_fused_depthwise_pointwise_block_narrow(ctx, oracle, case):
+    """The fused block kernel in the narrow format (bfloat16 patches in, depthwise result rounded to bfloat16 into
+    the operand tile, TF32 multiplies of bfloat16 values, bfloat16 out): bit for bit on small integers, within the
+    stored-result bars on random values, and against the same model run layer by layer."""
+    N, H, W, C, Cout = case
+    # small integers: every product, sum and stored value is exact on both sides
+    x, layers = block_model(si, 620, N, H, W, C, Cout, integers=True)
+    want = oracle.run_model(layers, x, keep_all=True, storage="bf16")
+    assert all(np.array_equal(a, b) for a, b in zip(want, oracle.run_model(layers, x, keep_all=True)))
+    assert np.abs(want[2]).max() > 0
+    model = narrow_model(ctx, layers, x.shape)
+    model.set_fusion("always")
+    out = host(model.run(dev(x)))
+    ctx.check_device_status()
+    assert model.layer_kernels()[1:3] == ["dwpw_fused_kernel<false>", "(in the previous layer's kernel)"]
+    assert model.launches_per_run == 3
+    assert same_bits(host(model.layer_output_f32(2)), want[2])
+    assert same_bits(out, want[3])
+    model.close()
+    # random values
+    x, layers = block_model(si, 621, N, H, W, C, Cout, integers=False)
+    want = oracle.run_model(layers, x, keep_all=True, storage="bf16")
+    model = narrow_model(ctx, layers, x.shape)
+    model.set_fusion("always")
+    out = host(model.run(dev(x)))
+    fused_pw = host(model.layer_output_f32(2))
+    ctx.check_device_status()
+    assert np.all((fused_pw.view(np.uint32) & 0xFFFF) == 0)
+    assert rel_fro(fused_pw, want[2]) <= 1e-2
+    assert fused_pw.min() >= 0 and fused_pw.max() <= 6
+    assert rel_fro(out, want[3]) <= 5e-3
+    # the pointwise layer on the input it actually saw: the oracle's pointwise layer applied to the oracle's
+    # depthwise layer of the GPU's own first-layer output (one bfloat16 step plus the fp32 summation error)
+    model.set_keep_all(True)
+    model.run(dev(x))
+    stem = host(model.layer_output_f32(0))
+    unfused_pw = host(model.layer_output_f32(2))
+    alone = oracle.run_model(layers[1:3], stem, keep_all=True, storage="bf16")
+    alone_pw = oracle.round_bf16(alone[1])
+    for got in (fused_pw, unfused_pw):
+        assert rel_fro(got, alone_pw) <= 4e-3
+        assert np.count_nonzero(np.abs(got - alone_pw) > 2.0 ** -6 * np.abs(alone_pw) + 2e-5 * np.abs(alone_pw).max()) <= 2e-3 * got.size
+    model.close()
+
+
 def test_config3_mobilenet_025_128_narrow(ctx, oracle):
     x, layers = si.config_mobilenet(0.25, 128, 1, seed=si.CONFIG_SEEDS["mobilenet_025_128"])
     want = oracle.run_model(layers, x, keep_all=True, storage="bf16")
