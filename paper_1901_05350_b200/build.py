@@ -27,14 +27,13 @@ SOURCES = [
     "elementwise.cu",
     "gemm_fp32_simt.cu",
     "gemm_tf32_tcgen05.cu",
-    "gemm_tf32_pair.cu",
+    "gemm_pair.cu",
     "gemm_tf32_splitk.cu",
     "conv2d_fp32_simt.cu",
     "depthwise.cu",
     "matmul_static_scratch.cu",
     "dwpw_fused_tcgen05.cu",
     "gemm_bf16_tcgen05.cu",
-    "gemm_bf16_pair.cu",
     "bf16_storage.cu",
     "backprop.cu",
 ]

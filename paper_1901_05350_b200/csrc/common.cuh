@@ -213,7 +213,7 @@ struct GemmTf32Plan {
     int num_tiles;
     int grid;
     size_t smem_bytes;
-    // CTA-pair kernel (gemm_tf32_pair.cu): 256 x block_n tiles shared by two CTAs
+    // CTA-pair kernel (gemm_pair.cu): 256 x block_n tiles shared by two CTAs
     bool pair = false;
     // cluster split-K kernel (gemm_tf32_splitk.cu): `splits` CTAs per tile, reduced through shared memory
     bool cluster_split = false;
@@ -259,7 +259,7 @@ struct GemmBf16Plan {
     CUtensorMap map_a, map_b, map_c;
     int64_t M = 0, N = 0, K = 0;
     bool c_is_bf16 = true;
-    bool pair = false;  // CTA-pair kernel (gemm_bf16_pair.cu): 256 x block_n tiles shared by two CTAs
+    bool pair = false;  // CTA-pair kernel (gemm_pair.cu): 256 x block_n tiles shared by two CTAs
     int block_n = 0, stages = 0, acc_stages = 0, num_tiles = 0, grid = 0;
     int epi_warps = 16;  // epilogue warps of the single-CTA kernel: 16 for short K loops, 8 otherwise
     size_t smem_bytes = 0;

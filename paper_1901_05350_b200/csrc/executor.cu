@@ -869,7 +869,7 @@ tfjsb_status tfjsb_model_layer_kernel(tfjsb_model* m, int layer, char* name, int
     else if (fused_mode && st.fuse_next) k = "dwpw_fused_kernel<false>";
     else switch (st.kind) {
         case STEP_GEMM_TF32:
-            k = st.plan.pair ? "gemm_tf32_pair_kernel" : st.plan.cluster_split ? "gemm_tf32_splitk_kernel" : "gemm_tf32_kernel<false>";
+            k = st.plan.pair ? "gemm_pair_kernel<false>" : st.plan.cluster_split ? "gemm_tf32_splitk_kernel" : "gemm_tf32_kernel<false>";
             break;
         case STEP_CONV_TF32: k = st.conv_patch ? "dwpw_fused_kernel<true>" : "gemm_tf32_kernel<true>"; break;
         case STEP_GEMM_FP32: k = "gemm_fp32_kernel"; break;
@@ -877,7 +877,7 @@ tfjsb_status tfjsb_model_layer_kernel(tfjsb_model* m, int layer, char* name, int
         case STEP_DEPTHWISE: k = st.dw_plan.variant >= 0 ? "depthwise3x3_tma_kernel" : "depthwise3x3_kernel"; break;
         case STEP_POOL: k = (st.g.Ho == 1 && st.g.Wo == 1 && st.g.fh == st.g.H && st.g.fw == st.g.W) ? "avg_pool_global_kernel" : "avg_pool_window_kernel"; break;
         case STEP_SOFTMAX: k = "softmax_rows_kernel"; break;
-        case STEP_GEMM_NARROW: k = st.plan16.pair ? "gemm_bf16_pair_kernel" : "gemm_bf16_kernel"; break;
+        case STEP_GEMM_NARROW: k = st.plan16.pair ? "gemm_pair_kernel<true>" : "gemm_bf16_kernel"; break;
         case STEP_CONV_NARROW: k = st.conv_patch ? "dwpw_fused_kernel<true, true>" : "conv_narrow_kernel"; break;
         case STEP_DEPTHWISE_NARROW: k = "depthwise3x3_narrow_kernel"; break;
         case STEP_POOL_NARROW: k = "avg_pool_global_narrow_kernel"; break;

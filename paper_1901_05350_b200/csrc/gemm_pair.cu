@@ -1,8 +1,13 @@
 // Tensor-core GEMM on CTA pairs (tcgen05 cta_group::2) with the fused bias + activation epilogue:
 //
-//     C[M,N] = act( A[M,K] . Bt[N,K]^T + bias[N] )        fp32 in, fp32 out, TF32 multiplies
+//     C[M,N] = act( A[M,K] . Bt[N,K]^T + bias[N] )
 //
-// Same contract as the single-CTA kernel (gemm_tf32_tcgen05.cu); this one is for the shapes whose
+// One kernel template, two element types: fp32 in and out with TF32 multiplies (the fp32-storage path), and
+// bfloat16 in and out (the narrow-storage path: a k-block is 64 elements in the same 128-byte swizzled rows,
+// consumed by four `kind::f16` MMAs of K = 16; the epilogue rounds to bfloat16 and stores through
+// 64-byte-swizzled slabs).  Sums are fp32 in tensor memory in both.
+//
+// Same contract as the single-CTA kernels (gemm_tf32_tcgen05.cu, gemm_bf16_tcgen05.cu); this one is for the shapes whose
 // time is set by the K loop (large K and N, many tiles).  With fp32 operands a single CTA must bring
 // 128 + 256 operand rows of 128 bytes into shared memory for every 128 x 256 x 32 block of
 // multiply-adds and read them back out for the tensor core, which saturates the shared memory's
@@ -39,6 +44,21 @@ constexpr int P_MAX_STAGES = 8;
 constexpr int P_ACC_STAGES = 2;     // 2 x 256 columns = all of tensor memory
 constexpr int P_TILE_M = 2 * BLOCK_M;
 
+// D[tmem of both CTAs] (+)= A . B^T over the pair, bfloat16 operands: M = 256, issued by the even CTA.
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// elements per k-block (one 128-byte swizzled row) and per MMA, by element type
+template <bool BF16> struct PairElem { static constexpr int BK = BLOCK_K, MMA_K = UMMA_K; };
+template <> struct PairElem<true> { static constexpr int BK = 64, MMA_K = 16; };
+
 struct PairArgs {
     int M, N, K;
     int block_n;    // columns of the pair's tile: a multiple of 32, 64..256
@@ -50,8 +70,9 @@ struct PairArgs {
     unsigned int* dev_status;
 };
 
+template <bool BF16>
 __global__ void __launch_bounds__(P_THREADS, 1)
-gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                       const __grid_constant__ CUtensorMap map_c, const PairArgs args) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[P_MAX_STAGES];        // used in the even CTA only
@@ -68,8 +89,9 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     const bool leader = rank == 0;
     const int block_n = args.block_n, stages = args.stages;
     const int half_n = block_n >> 1;
-    const int stage_bytes = A_STAGE_BYTES + half_n * BLOCK_K * 4;
-    const int num_k_blocks = (args.K + BLOCK_K - 1) / BLOCK_K;
+    constexpr int BK = PairElem<BF16>::BK, MMA_K = PairElem<BF16>::MMA_K;
+    const int stage_bytes = A_STAGE_BYTES + half_n * 128;  // rows of 128 bytes whatever the element type
+    const int num_k_blocks = (args.K + BK - 1) / BK;
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
 
     // dynamic shared memory, identical in both CTAs (the MMA descriptors address both by offset):
@@ -135,8 +157,8 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                     const uint32_t full = map_to_cta(smem_u32(&bar_full[stage]), 0u);
                     if (leader) mbar_arrive_expect_tx(smem_u32(&bar_full[stage]), (uint32_t)(2 * stage_bytes));
                     const uint32_t a_dst = stage_base + (uint32_t)stage * (uint32_t)stage_bytes;
-                    tma_load_2d_pair(a_dst, &map_a, full, kb * BLOCK_K, m0);
-                    tma_load_2d_pair(a_dst + A_STAGE_BYTES, &map_b, full, kb * BLOCK_K, n0);
+                    tma_load_2d_pair(a_dst, &map_a, full, kb * BK, m0);
+                    tma_load_2d_pair(a_dst + A_STAGE_BYTES, &map_b, full, kb * BK, n0);
                     ++issued;
                     if (++stage == stages) { stage = 0; phase ^= 1u; }
                 }
@@ -163,7 +185,7 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer (even CTA only)
         if (lane == 0 && leader) {
-            const uint32_t idesc = make_idesc_tf32(P_TILE_M, block_n);
+            const uint32_t idesc = BF16 ? make_idesc_bf16(P_TILE_M, block_n) : make_idesc_tf32(P_TILE_M, block_n);
             const uint16_t both = 3;
             int stage = 0;
             uint32_t phase = 0;
@@ -182,9 +204,10 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                     const uint64_t a_desc = make_kmajor_sw128_desc(a_addr);
                     const uint64_t b_desc = make_kmajor_sw128_desc(a_addr + A_STAGE_BYTES);
 #pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                        tc_mma_tf32_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                         (kb | k) != 0 ? 1u : 0u);
+                    for (int k = 0; k < BK / MMA_K; ++k) {  // 32 bytes along K per MMA: 2 descriptor units
+                        if (BF16) tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+                        else tc_mma_tf32_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
                     issued_any = true;
                     tc_commit_pair(smem_u32(&bar_empty[stage]), both);
                     if (++stage == stages) { stage = 0; phase ^= 1u; }
@@ -262,7 +285,11 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                 const uint32_t row_addr = slab + (uint32_t)lane * 128u;
                 const float* bias = (args.bias != nullptr) ? args.bias + col0 : nullptr;
                 const int cols_left = args.N - col0;
-                if (args.act == TFJSB_ACT_RELU6) stage_chunk<TFJSB_ACT_RELU6>(r, bias, cols_left, row_addr, lane);
+                if (BF16) {
+                    if (args.act == TFJSB_ACT_RELU6) stage_chunk_bf16<TFJSB_ACT_RELU6>(r, bias, cols_left, slab, lane);
+                    else if (args.act == TFJSB_ACT_RELU) stage_chunk_bf16<TFJSB_ACT_RELU>(r, bias, cols_left, slab, lane);
+                    else stage_chunk_bf16<TFJSB_ACT_NONE>(r, bias, cols_left, slab, lane);
+                } else if (args.act == TFJSB_ACT_RELU6) stage_chunk<TFJSB_ACT_RELU6>(r, bias, cols_left, row_addr, lane);
                 else if (args.act == TFJSB_ACT_RELU) stage_chunk<TFJSB_ACT_RELU>(r, bias, cols_left, row_addr, lane);
                 else stage_chunk<TFJSB_ACT_NONE>(r, bias, cols_left, row_addr, lane);
                 fence_async_smem();
@@ -296,13 +323,13 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 }
 
 tfjsb_status encode_pair_2d(tfjsb_ctx* ctx, CUtensorMap* map, const void* base, int64_t inner, int64_t outer, int box_inner,
-                            int box_outer, const char* what) {
+                            int box_outer, const char* what, bool bf16 = false, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
-    cuuint64_t strides[1] = {(cuuint64_t)inner * 4u};
+    cuuint64_t strides[1] = {(cuuint64_t)inner * (bf16 ? 2u : 4u)};
     cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
     cuuint32_t elem[2] = {1u, 1u};
-    CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, elem,
-                                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+    CUresult r = ctx->encode_tiled(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                                   const_cast<void*>(base), dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS)
         return fail(ctx, TFJSB_ERR_CUDA,
@@ -359,26 +386,27 @@ tfjsb_status gemm_tf32_pair_plan(tfjsb_ctx* ctx, const float* a, const float* bt
     return encode_pair_2d(ctx, &plan->map_c, c, N, M, EPI_COLS, 32, "C");
 }
 
-cudaError_t launch_gemm_tf32_pair(const GemmTf32Plan& plan, const float* bias, int act, unsigned int* dev_status,
-                                  cudaStream_t s, int64_t* launches) {
-    {
-        cudaError_t ae = cudaSuccess;
-        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&gemm_tf32_pair_kernel), SMEM_LIMIT - 2048);
-        if (ae != cudaSuccess) return ae;
-    }
+namespace {
+
+template <bool BF16>
+cudaError_t launch_pair(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c, int64_t M, int64_t N, int64_t K,
+                        int block_n, int stages, int num_tiles, int grid, size_t smem_bytes, const float* bias, int act,
+                        unsigned int* dev_status, cudaStream_t s, int64_t* launches) {
+    cudaError_t ae = smem_attr_once(reinterpret_cast<const void*>(&gemm_pair_kernel<BF16>), SMEM_LIMIT - 2048);
+    if (ae != cudaSuccess) return ae;
     PairArgs args;
-    args.M = (int)plan.M; args.N = (int)plan.N; args.K = (int)plan.K;
-    args.block_n = plan.block_n;
-    args.stages = plan.stages;
-    args.n_tiles = (int)((plan.N + plan.block_n - 1) / plan.block_n);
-    args.num_tiles = plan.num_tiles;
+    args.M = (int)M; args.N = (int)N; args.K = (int)K;
+    args.block_n = block_n;
+    args.stages = stages;
+    args.n_tiles = (int)((N + block_n - 1) / block_n);
+    args.num_tiles = num_tiles;
     args.bias = bias;
     args.act = act;
     args.dev_status = dev_status;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(plan.grid);
+    cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(P_THREADS);
-    cfg.dynamicSmemBytes = plan.smem_bytes;
+    cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = s;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -389,9 +417,63 @@ cudaError_t launch_gemm_tf32_pair(const GemmTf32Plan& plan, const float* bias, i
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = g_launch_pdl ? 2 : 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_tf32_pair_kernel, plan.map_a, plan.map_b, plan.map_c, args);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_pair_kernel<BF16>, map_a, map_b, map_c, args);
     ++*launches;
     return e;
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_tf32_pair(const GemmTf32Plan& plan, const float* bias, int act, unsigned int* dev_status,
+                                  cudaStream_t s, int64_t* launches) {
+    return launch_pair<false>(plan.map_a, plan.map_b, plan.map_c, plan.M, plan.N, plan.K, plan.block_n, plan.stages, plan.num_tiles,
+                              plan.grid, plan.smem_bytes, bias, act, dev_status, s, launches);
+}
+
+// Where the pair pays: nowhere yet.  On the shape it was written for (25088 x 512 x 512, the 14 x 14
+// pointwise layers at batch 128) it measures 19.6 us alone against 19.7 us for the single-CTA kernel,
+// and 23 us against 21.5 us inside the model: with 16-bit operands that GEMM is eight k-blocks per
+// tile and three rounds of tiles, and its fixed costs (first loads, last epilogue, 52 MB of HBM
+// traffic in 8 us) outweigh the K loop the pair shortens.  The planner therefore never picks it by
+// itself; TFJSB_GEMM_PAIR=1 selects it wherever the shape allows (the parity tests do), for shapes
+// with long K loops and many tiles, where its fp32-storage sibling wins 6-10 %.
+bool gemm_bf16_pair_preferred(int64_t M, int64_t N, int64_t K, int sm_count) {
+    (void)M; (void)N; (void)K; (void)sm_count;
+    return false;
+}
+
+tfjsb_status gemm_bf16_pair_plan(tfjsb_ctx* ctx, const void* a, const void* bt, void* c, int64_t M, int64_t N, int64_t K,
+                                 GemmBf16Plan* plan) {
+    if (!gemm_bf16_supported(M, N, K)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the bfloat16 GEMM");
+    if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+    plan->M = M; plan->N = N; plan->K = K;
+    plan->c_is_bf16 = true;
+    plan->pair = true;
+    int bn = 256;
+    while (bn > 64 && bn / 2 >= N) bn >>= 1;
+    plan->block_n = bn;
+    plan->acc_stages = P_ACC_STAGES;
+    const int stage_bytes = A_STAGE_BYTES + (bn / 2) * 128;
+    int stages = (SMEM_LIMIT - 1024 - EPI_BYTES - 512) / stage_bytes;
+    if (stages > P_MAX_STAGES) stages = P_MAX_STAGES;
+    plan->stages = stages;
+    plan->smem_bytes = (size_t)1024 + EPI_BYTES + (size_t)stages * stage_bytes;
+    const int64_t n_tiles = (N + bn - 1) / bn;
+    const int64_t tiles = ((M + P_TILE_M - 1) / P_TILE_M) * n_tiles;
+    if (tiles >= (1LL << 31)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "too many tiles");
+    plan->num_tiles = (int)tiles;
+    const int64_t pairs = ctx->sm_count / 2;
+    plan->grid = 2 * (int)(tiles < pairs ? tiles : pairs);
+    tfjsb_status st;
+    if ((st = encode_pair_2d(ctx, &plan->map_a, a, K, M, PairElem<true>::BK, BLOCK_M, "A", true)) != TFJSB_OK) return st;
+    if ((st = encode_pair_2d(ctx, &plan->map_b, bt, K, N, PairElem<true>::BK, bn / 2, "B", true)) != TFJSB_OK) return st;
+    return encode_pair_2d(ctx, &plan->map_c, c, N, M, EPI_COLS, 32, "C", true, CU_TENSOR_MAP_SWIZZLE_64B);
+}
+
+cudaError_t launch_gemm_bf16_pair(const GemmBf16Plan& plan, const float* bias, int act, unsigned int* dev_status,
+                                  cudaStream_t s, int64_t* launches) {
+    return launch_pair<true>(plan.map_a, plan.map_b, plan.map_c, plan.M, plan.N, plan.K, plan.block_n, plan.stages, plan.num_tiles,
+                             plan.grid, plan.smem_bytes, bias, act, dev_status, s, launches);
 }
 
 }  // namespace tfjsb
