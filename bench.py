@@ -190,7 +190,7 @@ def narrow_layer_work(layers, in_shape, window_out_shape):
 
 
 FUSED_INTO_PREVIOUS = "(in the previous layer's kernel)"
-TENSOR_CORE_KERNELS = ("gemm_tf32", "gemm_bf16", "dwpw_fused")
+TENSOR_CORE_KERNELS = ("gemm_tf32", "gemm_bf16", "gemm_pair", "dwpw_fused")
 
 
 def label_and_merge(rows, ms, kernels):
@@ -621,13 +621,13 @@ def run_ours(args):
 # Reads are cold and equal the layer's input; writes are counted when L2 evicts them, so layers whose output is
 # smaller than L2 under-count their writes.  Keyed by (kernel, launch name); an entry is dropped when its kernel changes.
 TRAFFIC_BYTES_PER_IMAGE = {
-    ("dwpw_fused_kernel<false>", "dw1+pw1"): 4325620, ("dwpw_fused_kernel<false>", "dw3+pw3"): 2800432,
-    ("dwpw_fused_kernel<false>", "dw5+pw5"): 1184820,
-    ("depthwise3x3_tma_kernel", "dw2"): 3853964, ("depthwise3x3_tma_kernel", "dw4"): 1831340,
-    ("depthwise3x3_tma_kernel", "dw6"): 846060, ("depthwise3x3_tma_kernel", "dw7"): 417200,
-    ("depthwise3x3_tma_kernel", "dw8"): 420342, ("depthwise3x3_tma_kernel", "dw9"): 420150,
-    ("depthwise3x3_tma_kernel", "dw10"): 417732, ("depthwise3x3_tma_kernel", "dw11"): 419190,
-    ("depthwise3x3_tma_kernel", "dw12"): 401774, ("depthwise3x3_tma_kernel", "dw13"): 201146,
+    ("dwpw_fused_kernel<false>", "dw1+pw1"): 4325282, ("dwpw_fused_kernel<false>", "dw3+pw3"): 2801262,
+    ("dwpw_fused_kernel<false>", "dw5+pw5"): 1186080,
+    ("depthwise3x3_tma_kernel", "dw2"): 3848518, ("depthwise3x3_tma_kernel", "dw4"): 1832338,
+    ("depthwise3x3_tma_kernel", "dw6"): 845540, ("depthwise3x3_tma_kernel", "dw7"): 432686,
+    ("depthwise3x3_tma_kernel", "dw8"): 432552, ("depthwise3x3_tma_kernel", "dw9"): 434704,
+    ("depthwise3x3_tma_kernel", "dw10"): 433112, ("depthwise3x3_tma_kernel", "dw11"): 431666,
+    ("depthwise3x3_tma_kernel", "dw12"): 401718, ("depthwise3x3_tma_kernel", "dw13"): 201164,
 }
 
 

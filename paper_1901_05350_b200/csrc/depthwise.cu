@@ -24,6 +24,8 @@
 // 'same' padding) into a ring of stages (full / empty mbarriers) while eight compute warps work
 // on the landed tiles from shared memory with the same sliding-row scheme and store float4s
 // straight to global memory.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "ptx_sm100.cuh"
 
@@ -149,7 +151,7 @@ __device__ __forceinline__ void store_rows(const float4 (&acc)[R], const float4 
 }
 
 // ---- pipelined kernel ---------------------------------------------------------------------------
-constexpr int DW_CB = 32;          // channels per tile: one 128-byte line per pixel
+constexpr int DW_CB = 32;          // channels per tile of the narrow instances: one 128-byte line per pixel
 constexpr int DW_MAX_STAGES = 4;
 
 struct DwTiling {
@@ -157,24 +159,25 @@ struct DwTiling {
     long long num_tiles;
 };
 
-template <int S, int TW, int R, int D = 1>
+template <int S, int TW, int R, int D = 1, int CB = DW_CB>
 struct DwTile {
-    static constexpr int RG = 32 / TW;                 // row groups of threads: 256 = 8 quads x TW x RG
+    static constexpr int QUADS = CB / 4;               // threads across a pixel's channels (4 channels each)
+    static constexpr int RG = DW_THREADS / QUADS / TW; // row groups of threads: 256 = QUADS x TW x RG
     static constexpr int TH = RG * R;                  // output rows per tile
     static constexpr int TWIN = (TW - 1) * S + 2 * D + 1;  // input patch (D: dilation, taps D pixels apart)
     static constexpr int THIN = (TH - 1) * S + 2 * D + 1;
-    static constexpr int STAGE_FLOATS = THIN * TWIN * DW_CB;
+    static constexpr int STAGE_FLOATS = THIN * TWIN * CB;
     static constexpr int STAGE_BYTES = STAGE_FLOATS * 4;
 };
 
 constexpr int DW_TMA_THREADS = DW_THREADS + 32;  // eight compute warps and the warp that issues the copies
 
-template <int S, int TW, int R, int D = 1>
+template <int S, int TW, int R, int D = 1, int CB = DW_CB>
 __global__ void __launch_bounds__(DW_TMA_THREADS, 2)
 depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __restrict__ f,
                         const float* __restrict__ bias, int act, float* __restrict__ y, ConvGeom g, DwTiling t,
                         unsigned int* dev_status) {
-    using T = DwTile<S, TW, R, D>;
+    using T = DwTile<S, TW, R, D, CB>;
     extern __shared__ uint8_t dw_smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[DW_MAX_STAGES];   // copy landed (1 arrival + bytes)
     __shared__ __align__(8) uint64_t bar_empty[DW_MAX_STAGES];  // the eight compute warps are done with the stage
@@ -225,7 +228,7 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
                 tile_info[slot] = make_int4(cb, tx, ty, n);
                 const uint32_t bar = ptx::smem_u32(&bar_full[slot]);
                 ptx::mbar_arrive_expect_tx(bar, (uint32_t)T::STAGE_BYTES);
-                ptx::tma_load_4d(smem_base + (uint32_t)slot * (uint32_t)T::STAGE_BYTES, &map_x, bar, cb * DW_CB,
+                ptx::tma_load_4d(smem_base + (uint32_t)slot * (uint32_t)T::STAGE_BYTES, &map_x, bar, cb * CB,
                                  tx * TW * S - g.pl, ty * T::TH * S - g.pt, n);
                 if (++slot == t.stages) { slot = 0; parity ^= 1u; }
             }
@@ -251,9 +254,9 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
     // ---------------------------------------------------------------- compute warps
     // The warps never synchronise with each other: each waits for the stage, does its share of the
     // tile and reports the stage free, so a fast warp can run up to `stages` tiles ahead of a slow one.
-    const int c4 = tid & 7;
-    const int col = (tid >> 3) % TW;
-    const int rg = tid / (8 * TW);
+    const int c4 = tid % T::QUADS;
+    const int col = (tid / T::QUADS) % TW;
+    const int rg = tid / (T::QUADS * TW);
     const int64_t row_pitch = (int64_t)g.Wo * g.Co;
 
     float4 w[9];
@@ -269,7 +272,7 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
         }
         const int4 info = tile_info[slot];
         const int cb = info.x, tx = info.y, ty = info.z;
-        const int c = cb * DW_CB + c4 * 4;
+        const int c = cb * CB + c4 * 4;
         const int ox = tx * TW + col;
         const int oy0 = ty * T::TH + rg * R;
         const bool live = c < g.C && ox < g.Wo && oy0 < g.Ho;
@@ -284,12 +287,12 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
             float4 acc[R];
 #pragma unroll
             for (int r = 0; r < R; ++r) acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-            const float* patch = smem_f + (size_t)slot * T::STAGE_FLOATS + ((rg * R * S) * T::TWIN + col * S) * DW_CB + c4 * 4;
+            const float* patch = smem_f + (size_t)slot * T::STAGE_FLOATS + ((rg * R * S) * T::TWIN + col * S) * CB + c4 * 4;
             constexpr int IN_ROWS = (R - 1) * S + 2 * D + 1;
 #pragma unroll
             for (int j = 0; j < IN_ROWS; ++j) {
-                const float* row = patch + j * T::TWIN * DW_CB;
-                const float4 v0 = ld4(row), v1 = ld4(row + D * DW_CB), v2 = ld4(row + 2 * D * DW_CB);
+                const float* row = patch + j * T::TWIN * CB;
+                const float4 v0 = ld4(row), v1 = ld4(row + D * CB), v2 = ld4(row + 2 * D * CB);
 #pragma unroll
                 for (int ky = 0; ky < 3; ++ky) {
                     const int d = j - ky * D;
@@ -317,25 +320,30 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
     }
 }
 
-// the instances: {stride, tile width, rows per thread}
+// the instances: {stride, tile width, tile height, bytes of a stage, channels per tile}
 struct DwVariant {
-    int S, TW, TH, stage_bytes;
+    int S, TW, TH, stage_bytes, cb;
 };
 constexpr DwVariant kDwVariants[] = {
-    {1, 16, DwTile<1, 16, 4>::TH, DwTile<1, 16, 4>::STAGE_BYTES},  // 0: large stride-1 images
-    {1, 16, DwTile<1, 16, 7>::TH, DwTile<1, 16, 7>::STAGE_BYTES},  // 1: 9..14 output rows in one tile
-    {1, 8, DwTile<1, 8, 2>::TH, DwTile<1, 8, 2>::STAGE_BYTES},     // 2: images up to 8 wide
-    {2, 16, DwTile<2, 16, 2>::TH, DwTile<2, 16, 2>::STAGE_BYTES},  // 3: stride 2
-    {2, 8, DwTile<2, 8, 2>::TH, DwTile<2, 8, 2>::STAGE_BYTES},     // 4: stride 2, outputs up to 8 wide
-    {1, 16, DwTile<1, 16, 4, 2>::TH, DwTile<1, 16, 4, 2>::STAGE_BYTES},  // 5: stride 1, dilation 2
-    {1, 16, DwTile<1, 16, 4, 4>::TH, DwTile<1, 16, 4, 4>::STAGE_BYTES},  // 6: stride 1, dilation 4
+    {1, 16, DwTile<1, 16, 4>::TH, DwTile<1, 16, 4>::STAGE_BYTES, DW_CB},  // 0: large stride-1 images
+    {1, 16, DwTile<1, 16, 7>::TH, DwTile<1, 16, 7>::STAGE_BYTES, DW_CB},  // 1: 9..14 output rows in one tile
+    {1, 8, DwTile<1, 8, 2>::TH, DwTile<1, 8, 2>::STAGE_BYTES, DW_CB},     // 2: images up to 8 wide
+    {2, 16, DwTile<2, 16, 2>::TH, DwTile<2, 16, 2>::STAGE_BYTES, DW_CB},  // 3: stride 2
+    {2, 8, DwTile<2, 8, 2>::TH, DwTile<2, 8, 2>::STAGE_BYTES, DW_CB},     // 4: stride 2, outputs up to 8 wide
+    {1, 16, DwTile<1, 16, 4, 2>::TH, DwTile<1, 16, 4, 2>::STAGE_BYTES, DW_CB},  // 5: stride 1, dilation 2
+    {1, 16, DwTile<1, 16, 4, 4>::TH, DwTile<1, 16, 4, 4>::STAGE_BYTES, DW_CB},  // 6: stride 1, dilation 4
+    // 64 channels per tile (256-byte lines): half as many box rows for the copy unit per byte moved
+    {1, 16, DwTile<1, 16, 4, 1, 64>::TH, DwTile<1, 16, 4, 1, 64>::STAGE_BYTES, 64},  // 7: as 0
+    {1, 16, DwTile<1, 16, 7, 1, 64>::TH, DwTile<1, 16, 7, 1, 64>::STAGE_BYTES, 64},  // 8: as 1 (two tiles down a 14-row image)
+    {1, 8, DwTile<1, 8, 4, 1, 64>::TH, DwTile<1, 8, 4, 1, 64>::STAGE_BYTES, 64},     // 9: as 2 (a whole 7 x 7 image)
+    {2, 8, DwTile<2, 8, 2, 1, 64>::TH, DwTile<2, 8, 2, 1, 64>::STAGE_BYTES, 64},     // 10: stride 2
 };
 constexpr int DW_SMEM_BUDGET = 113 * 1024;  // two CTAs per SM
 
-template <int S, int TW, int R, int D = 1>
+template <int S, int TW, int R, int D = 1, int CB = DW_CB>
 cudaError_t launch_tma_instance(const DepthwisePlan& plan, const float* f, const float* bias, int act, float* y,
                                 const ConvGeom& g, unsigned int* dev_status, cudaStream_t s) {
-    auto kernel = depthwise3x3_tma_kernel<S, TW, R, D>;
+    auto kernel = depthwise3x3_tma_kernel<S, TW, R, D, CB>;
     cudaError_t ae = smem_attr_once(reinterpret_cast<const void*>(kernel), DW_SMEM_BUDGET);
     if (ae != cudaSuccess) return ae;
     DwTiling t{plan.tiles_x, plan.tiles_y, plan.c_blocks, plan.stages, (long long)plan.num_tiles};
@@ -361,11 +369,20 @@ tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const float* x, const ConvGeom& g, D
     if (dilated) v = g.dh == 2 ? 5 : 6;
     else if (g.sh == 1) v = g.Wo <= 8 ? 2 : ((g.Ho > 8 && g.Ho <= 14) ? 1 : 0);
     else v = g.Wo <= 8 ? 4 : 3;
+    static const bool wide_off = std::getenv("TFJSB_DW_CB32") != nullptr;
+    // 64-channel tiles where the channel count allows.  Measured at batch 128: [112,112,64] stride 2
+    // 90.1 -> 86.9 us, [7,7,1024] 19.5 -> 15.4 us, the 14 x 14 x 512 layers unchanged; the stride-2 form is
+    // 8 outputs wide, so it is taken only where that wastes fewer columns than the 16-wide 32-channel one
+    // ([28,28,256] stride 2 ran 27.3 -> 29.1 us with it).
+    if (!dilated && g.C % 64 == 0 && !wide_off) {
+        if (g.sh == 1) v = v == 0 ? 7 : (v == 1 ? 8 : 9);
+        else if ((g.Wo + 7) / 8 * 8 < (g.Wo + 15) / 16 * 16) v = 10;
+    }
     const DwVariant& d = kDwVariants[v];
     const int twin = (d.TW - 1) * d.S + 2 * g.dw + 1, thin = (d.TH - 1) * d.S + 2 * g.dh + 1;
     cuuint64_t dims[4] = {(cuuint64_t)g.C, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
     cuuint64_t strides[3] = {(cuuint64_t)g.C * 4u, (cuuint64_t)g.W * g.C * 4u, (cuuint64_t)g.H * g.W * g.C * 4u};
-    cuuint32_t box[4] = {(cuuint32_t)DW_CB, (cuuint32_t)twin, (cuuint32_t)thin, 1u};
+    cuuint32_t box[4] = {(cuuint32_t)d.cb, (cuuint32_t)twin, (cuuint32_t)thin, 1u};
     cuuint32_t elem[4] = {1u, 1u, 1u, 1u};
     CUresult r = ctx->encode_tiled(&plan->map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(x), dims, strides,
                                    box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
@@ -375,7 +392,7 @@ tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const float* x, const ConvGeom& g, D
                                              std::to_string((int)r) + ")");
     plan->tiles_x = (g.Wo + d.TW - 1) / d.TW;
     plan->tiles_y = (g.Ho + d.TH - 1) / d.TH;
-    plan->c_blocks = (g.C + DW_CB - 1) / DW_CB;
+    plan->c_blocks = (g.C + d.cb - 1) / d.cb;
     plan->num_tiles = (int64_t)plan->tiles_x * plan->tiles_y * plan->c_blocks * g.N;
     if (plan->num_tiles > 0x7fffffff) return TFJSB_OK;  // tile indices are 32-bit in the kernel
     int stages = (DW_SMEM_BUDGET - 256) / d.stage_bytes;
@@ -413,6 +430,10 @@ cudaError_t launch_depthwise(const DepthwisePlan& plan, const float* x, const fl
             case 3: e = launch_tma_instance<2, 16, 2>(plan, f, bias, act, y, g, dev_status, s); break;
             case 4: e = launch_tma_instance<2, 8, 2>(plan, f, bias, act, y, g, dev_status, s); break;
             case 5: e = launch_tma_instance<1, 16, 4, 2>(plan, f, bias, act, y, g, dev_status, s); break;
+            case 7: e = launch_tma_instance<1, 16, 4, 1, 64>(plan, f, bias, act, y, g, dev_status, s); break;
+            case 8: e = launch_tma_instance<1, 16, 7, 1, 64>(plan, f, bias, act, y, g, dev_status, s); break;
+            case 9: e = launch_tma_instance<1, 8, 4, 1, 64>(plan, f, bias, act, y, g, dev_status, s); break;
+            case 10: e = launch_tma_instance<2, 8, 2, 1, 64>(plan, f, bias, act, y, g, dev_status, s); break;
             default: e = launch_tma_instance<1, 16, 4, 4>(plan, f, bias, act, y, g, dev_status, s); break;
         }
         ++*launches;

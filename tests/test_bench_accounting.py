@@ -60,3 +60,23 @@ def test_narrow_accounting_halves_what_is_stored_narrow(bench, oracle):
         assert n["flops"] == w["flops"]
         assert n["bytes"] <= w["bytes"]
     assert by["pw7"]["tensor"] and by["dense"]["tensor"] and not by["dw2"]["tensor"] and not by["stem"]["tensor"]
+
+
+def test_roofline_bound_of_the_kernels_the_library_names(bench):
+    """The compute leg of a row's roofline uses the tensor-core peak exactly for the kernels that run on
+    the tensor cores: a GEMM kernel left off that list would be judged against the CUDA-core peak and read
+    several times above its roofline."""
+    peaks = {"hbm_gbs": 6500.0, "bf16_tflops": 1600.0, "bf16_tflops_sustained": 1400.0}
+    pw7 = dict(name="pw7", flops=2 * 25088 * 512 * 512, bytes=4 * (2 * 25088 * 512 + 512 * 512 + 512), units=25088 * 512)
+    for kernel in ("gemm_pair_kernel<false>", "gemm_pair_kernel<true>", "gemm_tf32_kernel<false>", "gemm_tf32_kernel<true>",
+                   "gemm_tf32_splitk_kernel", "gemm_bf16_kernel", "dwpw_fused_kernel<false>", "dwpw_fused_kernel<true, true>"):
+        (row,) = bench.roofline_rows([dict(pw7, kernel=kernel)], [0.030], peaks, fp32_tflops=75.0)
+        assert row["bound"] == "tensor", kernel
+        assert abs(row["roofline_us"] - pw7["flops"] / 800e12 * 1e6) < 1e-6, kernel
+        assert row["frac"] < 1.0
+    for kernel in ("gemm_fp32_kernel", "conv2d_fp32_kernel"):
+        (row,) = bench.roofline_rows([dict(pw7, kernel=kernel)], [0.300], peaks, fp32_tflops=75.0)
+        assert row["bound"] == "alu", kernel
+    dw = dict(name="dw7", flops=18 * 25088 * 512, bytes=4 * (2 * 25088 * 512 + 10 * 512), units=25088 * 512)
+    (row,) = bench.roofline_rows([dict(dw, kernel="depthwise3x3_tma_kernel")], [0.020], peaks, fp32_tflops=75.0)
+    assert row["bound"] == "hbm"
