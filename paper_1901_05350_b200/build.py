@@ -26,14 +26,13 @@ SOURCES = [
     "executor.cu",
     "elementwise.cu",
     "gemm_fp32_simt.cu",
-    "gemm_tf32_tcgen05.cu",
+    "gemm_cta.cu",
     "gemm_pair.cu",
     "gemm_tf32_splitk.cu",
     "conv2d_fp32_simt.cu",
     "depthwise.cu",
     "matmul_static_scratch.cu",
     "dwpw_fused_tcgen05.cu",
-    "gemm_bf16_tcgen05.cu",
     "bf16_storage.cu",
     "backprop.cu",
 ]

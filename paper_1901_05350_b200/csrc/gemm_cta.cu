@@ -31,6 +31,18 @@
 // Every wait is bounded: a wait that exceeds WAIT_LIMIT_NS raises an abort flag that all roles
 // poll, ORs a code into the context's device status word, and the CTA drains its copies, frees
 // its tensor memory and returns.
+//
+// The same pipeline serves bfloat16 storage (the narrow-storage mode, the 16-bit analogue of the
+// paper's half-float textures, Sec. 4.1.3): `gemm_pipeline` is a template on the element format and
+// `gemm_tf32_kernel` / `gemm_bf16_kernel` are its instances.  With bfloat16 a k-block is 64 elements
+// (still one 128-byte swizzle row, consumed by four `kind::f16` MMAs of K = 16), products of two
+// bfloat16 are exact in fp32, the sums are fp32 in tensor memory, and the result gets the fp32 bias,
+// the activation and one rounding (to nearest even) when it is stored as bfloat16.  Half the bytes per
+// tile leave the layers with one or two k-blocks per tile bound by the epilogue's latency per 32 x 32
+// block, so those run with sixteen epilogue warps, four per lane quadrant, taking every fourth block;
+// long K loops keep eight (the extra warps' polling costs them about 4 %).
+#include <cuda_bf16.h>
+
 #include <cstdlib>
 
 #include "common.cuh"
@@ -45,9 +57,27 @@ using namespace tile;
 namespace {
 
 constexpr int MAX_STAGES = 8;
-constexpr int GEMM_THREADS = 320;    // producer warp, MMA warp, 8 epilogue warps
+constexpr int MAX_EPI_WARPS = 16;    // eight or sixteen epilogue warps: two or four per tensor-memory lane quadrant
+constexpr int GEMM_MAX_THREADS = 64 + MAX_EPI_WARPS * 32;  // producer warp, MMA warp, the epilogue warps
+constexpr int GATHER_EPI_WARPS = 8;
 constexpr int GATHER_GROUPS = 3;     // implicit-GEMM convolution: groups of 4 warps that build A tiles
-constexpr int CONV_THREADS = GEMM_THREADS + GATHER_GROUPS * 128;
+constexpr int CONV_THREADS = 64 + GATHER_EPI_WARPS * 32 + GATHER_GROUPS * 128;
+
+// element formats of the pipeline: what A and Bt are stored as, and what C is stored as
+constexpr int IO_F32 = 0;        // fp32 in (multiplied as TF32), fp32 out
+constexpr int IO_BF16 = 1;       // bfloat16 in, bfloat16 out
+constexpr int IO_BF16_F32 = 2;   // bfloat16 in, fp32 out
+
+// D[tmem] (+)= A[smem] . B[smem]^T, single CTA, bfloat16 operands, fp32 accumulate.
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 
 // ---- A-row gathers of the implicit-GEMM convolution ---------------------------------------------
 // Each fills v[0..31] with columns k0..k0+31 of one row of the im2col matrix: k = (ky*fw + kx)*Cin + ci
@@ -137,6 +167,7 @@ struct KernelArgs {
     int tiles_per_batch;  // tiles of one product (rows x columns)
     int num_tiles;  // total, over all products of the batch
     int acc_stages;  // accumulator stages in tensor memory: 2 (block_n 256) or 4
+    int epi_warps;   // 8 or 16
     const float* bias;
     int act;
     unsigned int* dev_status;
@@ -145,10 +176,15 @@ struct KernelArgs {
     ConvGeom g;
 };
 
-template <bool GATHER>
-__global__ void __launch_bounds__(GATHER ? CONV_THREADS : GEMM_THREADS, 1)
-gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                 const __grid_constant__ CUtensorMap map_c, const KernelArgs args) {
+template <bool GATHER, int IO, bool BATCHED>
+__device__ __forceinline__ void gemm_pipeline(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c,
+                                              const KernelArgs& args) {
+    static_assert(!GATHER || IO == IO_F32, "the gathering producer builds fp32 tiles");
+    constexpr bool IN_BF16 = IO != IO_F32;
+    constexpr bool OUT_BF16 = IO == IO_BF16;
+    constexpr int BK = IN_BF16 ? 64 : BLOCK_K;        // elements per k-block: 128 bytes either way
+    constexpr int MMAS_PER_KB = 4;                    // 32 bytes of K per tcgen05.mma in both formats
+    constexpr uint32_t SLAB_BYTES = OUT_BF16 ? 2048u : (uint32_t)EPI_SLAB_BYTES;  // 32 rows x 32 columns of the output type
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[MAX_STAGES];
     __shared__ __align__(8) uint64_t bar_empty[MAX_STAGES];
@@ -161,14 +197,15 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     volatile int* abort_flag = &abort_flag_s;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int block_n = args.block_n, stages = args.stages, acc_stages = args.acc_stages;
-    const int stage_bytes = A_STAGE_BYTES + block_n * BLOCK_K * 4;
-    const int num_k_blocks = (args.K + BLOCK_K - 1) / BLOCK_K;
+    const int epi_warps = GATHER ? GATHER_EPI_WARPS : args.epi_warps;
+    const int stage_bytes = A_STAGE_BYTES + block_n * 128;
+    const int num_k_blocks = (args.K + BK - 1) / BK;
 
     // dynamic shared memory, aligned to the 1024-byte swizzle pattern:
-    //   [epilogue slabs: 32 KiB][stage 0: A | B][stage 1] ...
+    //   [epilogue slabs, one per epilogue warp][stage 0: A | B][stage 1] ...
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t epi_base = smem_base;
-    const uint32_t stage_base = smem_base + EPI_BYTES;
+    const uint32_t stage_base = smem_base + (uint32_t)epi_warps * SLAB_BYTES;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -179,7 +216,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         }
         for (int s = 0; s < acc_stages; ++s) {
             mbar_init(smem_u32(&bar_acc_full[s]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[s]), 8);
+            mbar_init(smem_u32(&bar_acc_empty[s]), (uint32_t)epi_warps);
         }
         mbar_init(smem_u32(&bar_drain), 1);
         abort_flag_s = 0;
@@ -216,7 +253,8 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             for (int s = 0; s < MAX_STAGES; ++s) armed[s] = -1;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
-                const int batch = tile / args.tiles_per_batch, in_batch = tile - batch * args.tiles_per_batch;
+                const int batch = BATCHED ? tile / args.tiles_per_batch : 0;
+                const int in_batch = tile - batch * args.tiles_per_batch;
                 const int m0 = (in_batch / args.n_tiles) * BLOCK_M;
                 const int n0 = (in_batch % args.n_tiles) * block_n;
                 (void)m0;
@@ -235,9 +273,11 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         mbar_arrive_expect_tx(full, (uint32_t)(stage_bytes - A_STAGE_BYTES));
                     } else {
                         mbar_arrive_expect_tx(full, (uint32_t)stage_bytes);
-                        tma_load_3d(a_dst, &map_a, full, kb * BLOCK_K, m0, batch);
+                        if (BATCHED) tma_load_3d(a_dst, &map_a, full, kb * BK, m0, batch);
+                        else tma_load_2d(a_dst, &map_a, full, kb * BK, m0);
                     }
-                    tma_load_3d(a_dst + A_STAGE_BYTES, &map_b, full, kb * BLOCK_K, n0, batch);
+                    if (BATCHED) tma_load_3d(a_dst + A_STAGE_BYTES, &map_b, full, kb * BK, n0, batch);
+                    else tma_load_2d(a_dst + A_STAGE_BYTES, &map_b, full, kb * BK, n0);
 #pragma unroll
                     for (int s = 0; s < MAX_STAGES; ++s)
                         if (s == stage) armed[s] = (int)phase;
@@ -264,7 +304,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = make_idesc_tf32(BLOCK_M, block_n);
+            const uint32_t idesc = IN_BF16 ? make_idesc_bf16(BLOCK_M, block_n) : make_idesc_tf32(BLOCK_M, block_n);
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
@@ -282,10 +322,14 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     const uint64_t a_desc = make_kmajor_sw128_desc(a_addr);
                     const uint64_t b_desc = make_kmajor_sw128_desc(a_addr + A_STAGE_BYTES);
 #pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+                    for (int k = 0; k < MMAS_PER_KB; ++k) {
                         // step along K inside the 128-byte swizzled row: 32 bytes = 2 descriptor units
-                        tc_mma_tf32(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                    (kb | k) != 0 ? 1u : 0u);
+                        if (IN_BF16)
+                            tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                        (kb | k) != 0 ? 1u : 0u);
+                        else
+                            tc_mma_tf32(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                        (kb | k) != 0 ? 1u : 0u);
                     }
                     issued_any = true;
                     tc_commit(smem_u32(&bar_empty[stage]));
@@ -313,22 +357,24 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 }
             }
         }
-    } else if (warp < 10) {
-        // ---------------------------------------------------------------- epilogue (warps 2..9)
-        // Two warps share each TMEM lane quadrant (a warp may only read lanes 32*(warp%4)..+31) and
-        // take alternate 32-column chunks, counted across tiles so that with one chunk per tile they
-        // alternate tiles.
+    } else if (warp < 2 + epi_warps) {
+        // ---------------------------------------------------------------- epilogue (warps 2..)
+        // Two or four warps share each TMEM lane quadrant (a warp may only read lanes 32*(warp%4)..+31)
+        // and take every second or fourth 32-column chunk, counted across tiles so that with one chunk
+        // per tile they take tiles in turn.
         const int ew = warp - 2;
         const int quad = warp & 3;
-        const int half = ew >> 2;
-        const uint32_t slab = epi_base + (uint32_t)ew * EPI_SLAB_BYTES;
+        const int sub = ew >> 2;  // which of the quadrant's warps
+        const int per_quad_mask = (epi_warps >> 2) - 1;  // 1 or 3
+        const uint32_t slab = epi_base + (uint32_t)ew * SLAB_BYTES;
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
         const int chunks_per_tile = block_n / EPI_COLS;
-        int first_chunk = half;  // parity bookkeeping: chunk `ch` of this tile is ours when (ch - first_chunk) is even
+        int chunk_base = 0;  // chunks of earlier tiles, modulo the quadrant's warps
         for (int tile = blockIdx.x; ok && tile < args.num_tiles; tile += gridDim.x) {
-            const int batch = tile / args.tiles_per_batch, in_batch = tile - batch * args.tiles_per_batch;
+            const int batch = BATCHED ? tile / args.tiles_per_batch : 0;
+            const int in_batch = tile - batch * args.tiles_per_batch;
             const int m0 = (in_batch / args.n_tiles) * BLOCK_M;
             const int n0 = (in_batch % args.n_tiles) * block_n;
             // every lane polls (each needs the acquire), the vote keeps the warp uniform
@@ -349,12 +395,12 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             if (live_cols < block_n) n_chunks = (live_cols + EPI_COLS - 1) / EPI_COLS;
             const bool rows_live = row0 < args.M;
             bool released = false;
-            for (int ch = first_chunk; ch < n_chunks; ch += 2) {
+            for (int ch = (sub - chunk_base) & per_quad_mask; ch < n_chunks; ch += per_quad_mask + 1) {
                 uint32_t r[32];
                 const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * block_n + ch * EPI_COLS);
                 tc_ld_32x32(taddr, r);
                 tc_ld_wait();
-                if (ch + 2 >= n_chunks) {
+                if (ch + per_quad_mask + 1 >= n_chunks) {
                     // this warp has read its share of the accumulator: hand it back to the MMA issuer
                     tc_fence_before();
                     __syncwarp();
@@ -366,16 +412,23 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 // the slab is free once the previous store issued from it has read it
                 if (lane == 0) tma_store_wait_read<0>();
                 __syncwarp();
-                const uint32_t row_addr = slab + (uint32_t)lane * 128u;
                 const float* bias = (args.bias != nullptr) ? args.bias + col0 : nullptr;
                 const int cols_left = args.N - col0;
-                if (args.act == TFJSB_ACT_RELU6) stage_chunk<TFJSB_ACT_RELU6>(r, bias, cols_left, row_addr, lane);
-                else if (args.act == TFJSB_ACT_RELU) stage_chunk<TFJSB_ACT_RELU>(r, bias, cols_left, row_addr, lane);
-                else stage_chunk<TFJSB_ACT_NONE>(r, bias, cols_left, row_addr, lane);
+                if (OUT_BF16) {
+                    if (args.act == TFJSB_ACT_RELU6) stage_chunk_bf16<TFJSB_ACT_RELU6>(r, bias, cols_left, slab, lane);
+                    else if (args.act == TFJSB_ACT_RELU) stage_chunk_bf16<TFJSB_ACT_RELU>(r, bias, cols_left, slab, lane);
+                    else stage_chunk_bf16<TFJSB_ACT_NONE>(r, bias, cols_left, slab, lane);
+                } else {
+                    const uint32_t row_addr = slab + (uint32_t)lane * 128u;
+                    if (args.act == TFJSB_ACT_RELU6) stage_chunk<TFJSB_ACT_RELU6>(r, bias, cols_left, row_addr, lane);
+                    else if (args.act == TFJSB_ACT_RELU) stage_chunk<TFJSB_ACT_RELU>(r, bias, cols_left, row_addr, lane);
+                    else stage_chunk<TFJSB_ACT_NONE>(r, bias, cols_left, row_addr, lane);
+                }
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    tma_store_3d(&map_c, slab, col0, row0, batch);
+                    if (BATCHED) tma_store_3d(&map_c, slab, col0, row0, batch);
+                    else tma_store_2d(&map_c, slab, col0, row0);
                     tma_store_commit();
                 }
             }
@@ -384,7 +437,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
             }
-            if (chunks_per_tile & 1) first_chunk ^= 1;
+            chunk_base = (chunk_base + chunks_per_tile) & per_quad_mask;
             if (++acc == acc_stages) { acc = 0; acc_phase ^= 1u; }
         }
         if (lane == 0) tma_store_wait_all();
@@ -399,7 +452,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         // flight) and writes it in the 128-byte-swizzled layout the tensor core reads; the groups take
         // k-blocks in turn so that several tiles' loads are outstanding at once.
         const ConvGeom& g = args.g;
-        const int gw = warp - 10;
+        const int gw = warp - (2 + GATHER_EPI_WARPS);
         const int group = gw >> 2;
         const int row = ((gw & 3) << 5) + lane;
         const bool vec4 = (g.C & 3) == 0;
@@ -467,6 +520,30 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     }
 }
 
+// The instances.  The tensor maps stay kernel parameters (`__grid_constant__`): the copy unit reads them
+// from parameter space, and the pipeline, inlined, takes their addresses there.
+template <bool GATHER>
+__global__ void __launch_bounds__(GATHER ? CONV_THREADS : GEMM_MAX_THREADS, 1)
+gemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const __grid_constant__ CUtensorMap map_c, const KernelArgs args) {
+    gemm_pipeline<GATHER, IO_F32, false>(map_a, map_b, map_c, args);
+}
+
+// A batch of independent products of one shape (rank-3 matMul): the tensor maps carry the batch as a third
+// dimension and a tile is (product, rows, columns).
+__global__ void __launch_bounds__(GEMM_MAX_THREADS, 1)
+gemm_tf32_batched_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                         const __grid_constant__ CUtensorMap map_c, const KernelArgs args) {
+    gemm_pipeline<false, IO_F32, true>(map_a, map_b, map_c, args);
+}
+
+template <bool OUT_BF16>
+__global__ void __launch_bounds__(GEMM_MAX_THREADS, 1)
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const __grid_constant__ CUtensorMap map_c, const KernelArgs args) {
+    gemm_pipeline<false, OUT_BF16 ? IO_BF16 : IO_BF16_F32, false>(map_a, map_b, map_c, args);
+}
+
 int choose_block_n(int64_t M, int64_t N, int sm_count, int64_t batches) {
     int bn = 32;
     while (bn < 256 && bn < N) bn <<= 1;
@@ -482,15 +559,19 @@ int choose_block_n(int64_t M, int64_t N, int sm_count, int64_t batches) {
     return bn;
 }
 
-// A batch of `batches` row-major matrices [outer, inner] stored one after the other, box = one tile of one matrix.
+// A row-major matrix [outer, inner], or (batches > 1: a rank-3 map) that many of them stored one after the other;
+// box = one tile of one matrix.  fp32 elements with the 128-byte swizzle unless `bf16` (then bfloat16, and `swizzle` as given: 128 bytes for
+// the operand tiles, 64 for the 32-column output slab).
 tfjsb_status encode_2d(tfjsb_ctx* ctx, CUtensorMap* map, const void* base, int64_t inner, int64_t outer,
-                       int box_inner, int box_outer, const char* what, int64_t batches = 1) {
+                       int box_inner, int box_outer, const char* what, int64_t batches = 1, bool bf16 = false,
+                       CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
+    const cuuint64_t eb = bf16 ? 2u : 4u;
     cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)batches};
-    cuuint64_t strides[2] = {(cuuint64_t)inner * 4u, (cuuint64_t)inner * (cuuint64_t)outer * 4u};
+    cuuint64_t strides[2] = {(cuuint64_t)inner * eb, (cuuint64_t)inner * (cuuint64_t)outer * eb};
     cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer, 1u};
     cuuint32_t elem[3] = {1u, 1u, 1u};
-    CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides,
-                                   box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+    CUresult r = ctx->encode_tiled(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, batches > 1 ? 3 : 2,
+                                   const_cast<void*>(base), dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS)
         return fail(ctx, TFJSB_ERR_CUDA,
@@ -594,6 +675,7 @@ cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int ac
         cudaError_t ae = cudaSuccess;
         if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&gemm_tf32_kernel<false>), SMEM_LIMIT - 2048);
         if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&gemm_tf32_kernel<true>), SMEM_LIMIT - 2048);
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&gemm_tf32_batched_kernel), SMEM_LIMIT - 2048);
         if (ae != cudaSuccess) return ae;
     }
     cudaError_t e;
@@ -605,6 +687,7 @@ cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int ac
     args.tiles_per_batch = (int)(plan.num_tiles / (plan.batches > 0 ? plan.batches : 1));
     args.num_tiles = plan.num_tiles;
     args.acc_stages = plan.acc_stages;
+    args.epi_warps = GATHER_EPI_WARPS;  // sixteen measured slower with fp32 tiles
     args.bias = bias;
     args.act = act;
     args.dev_status = dev_status;
@@ -613,9 +696,84 @@ cudaError_t launch_gemm_tf32(const GemmTf32Plan& plan, const float* bias, int ac
     if (plan.gather)
         e = launch_k(gemm_tf32_kernel<true>, dim3(plan.grid), dim3(CONV_THREADS), plan.smem_bytes, s, plan.map_a, plan.map_b,
                      plan.map_c, args);
+    else if (plan.batches > 1)
+        e = launch_k(gemm_tf32_batched_kernel, dim3(plan.grid), dim3(64 + 32 * args.epi_warps), plan.smem_bytes, s, plan.map_a,
+                     plan.map_b, plan.map_c, args);
     else
-        e = launch_k(gemm_tf32_kernel<false>, dim3(plan.grid), dim3(GEMM_THREADS), plan.smem_bytes, s, plan.map_a, plan.map_b,
+        e = launch_k(gemm_tf32_kernel<false>, dim3(plan.grid), dim3(64 + 32 * args.epi_warps), plan.smem_bytes, s, plan.map_a, plan.map_b,
                      plan.map_c, args);
+    ++*launches;
+    return e;
+}
+
+// ---- bfloat16 storage ------------------------------------------------------------------------------
+bool gemm_bf16_supported(int64_t M, int64_t N, int64_t K) {
+    // row pitches of A, Bt (K bfloat16) and C (N bfloat16) must be multiples of 16 bytes; coordinates are 32-bit
+    return M >= 1 && N >= 8 && K >= 8 && (K % 8 == 0) && (N % 8 == 0) && M < (1LL << 31) - 256 && N < (1LL << 31) - 256 &&
+           K < (1LL << 31) - 256 && ((M + BLOCK_M - 1) / BLOCK_M) * ((N + 31) / 32) < (1LL << 31);
+}
+
+tfjsb_status gemm_bf16_plan(tfjsb_ctx* ctx, const void* a, const void* bt, void* c, bool c_is_bf16, int64_t M, int64_t N,
+                            int64_t K, GemmBf16Plan* plan) {
+    if (!gemm_bf16_supported(M, N, K)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "shape not supported by the bfloat16 GEMM");
+    if (!ctx->encode_tiled) return fail(ctx, TFJSB_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+    if (c_is_bf16) {
+        const char* pair_env = getenv("TFJSB_GEMM_PAIR");
+        const bool use_pair = pair_env ? (pair_env[0] == '1' && N >= 64) : gemm_bf16_pair_preferred(M, N, K, ctx->sm_count);
+        if (use_pair) return gemm_bf16_pair_plan(ctx, a, bt, c, M, N, K, plan);
+    }
+    constexpr int BK16 = 64;  // bfloat16 elements per k-block
+    plan->M = M; plan->N = N; plan->K = K;
+    plan->c_is_bf16 = c_is_bf16;
+    plan->pair = false;
+    plan->block_n = choose_block_n(M, N, ctx->sm_count, 1);
+    plan->acc_stages = plan->block_n > 128 ? 2 : MAX_ACC_STAGES;
+    const int stage_bytes = A_STAGE_BYTES + plan->block_n * 128;
+    plan->epi_warps = (K + BK16 - 1) / BK16 <= 4 ? 16 : 8;
+    const int epi_bytes = plan->epi_warps * (c_is_bf16 ? 2048 : EPI_SLAB_BYTES);
+    int stages = (SMEM_LIMIT - 1024 - epi_bytes - 512) / stage_bytes;
+    if (stages > MAX_STAGES) stages = MAX_STAGES;
+    plan->stages = stages;
+    plan->smem_bytes = (size_t)1024 + epi_bytes + (size_t)stages * stage_bytes;
+    const int64_t n_tiles = (N + plan->block_n - 1) / plan->block_n;
+    const int64_t tiles = ((M + BLOCK_M - 1) / BLOCK_M) * n_tiles;
+    if (tiles >= (1LL << 31)) return fail(ctx, TFJSB_ERR_UNSUPPORTED, "too many tiles");
+    plan->num_tiles = (int)tiles;
+    plan->grid = (int)(tiles < ctx->sm_count ? tiles : ctx->sm_count);
+    tfjsb_status st;
+    if ((st = encode_2d(ctx, &plan->map_a, a, K, M, BK16, BLOCK_M, "A", 1, true)) != TFJSB_OK) return st;
+    if ((st = encode_2d(ctx, &plan->map_b, bt, K, N, BK16, plan->block_n, "B", 1, true)) != TFJSB_OK) return st;
+    if (c_is_bf16) return encode_2d(ctx, &plan->map_c, c, N, M, EPI_COLS, 32, "C", 1, true, CU_TENSOR_MAP_SWIZZLE_64B);
+    return encode_2d(ctx, &plan->map_c, c, N, M, EPI_COLS, 32, "C");
+}
+
+cudaError_t launch_gemm_bf16(const GemmBf16Plan& plan, const float* bias, int act, unsigned int* dev_status,
+                             cudaStream_t s, int64_t* launches) {
+    if (plan.pair) return launch_gemm_bf16_pair(plan, bias, act, dev_status, s, launches);
+    {
+        cudaError_t ae = cudaSuccess;
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&gemm_bf16_kernel<false>), SMEM_LIMIT - 2048);
+        if (ae == cudaSuccess) ae = smem_attr_once(reinterpret_cast<const void*>(&gemm_bf16_kernel<true>), SMEM_LIMIT - 2048);
+        if (ae != cudaSuccess) return ae;
+    }
+    KernelArgs args{};
+    args.M = (int)plan.M; args.N = (int)plan.N; args.K = (int)plan.K;
+    args.block_n = plan.block_n;
+    args.stages = plan.stages;
+    args.n_tiles = (int)((plan.N + plan.block_n - 1) / plan.block_n);
+    args.tiles_per_batch = plan.num_tiles;
+    args.num_tiles = plan.num_tiles;
+    args.acc_stages = plan.acc_stages;
+    args.epi_warps = plan.epi_warps;
+    args.bias = bias;
+    args.act = act;
+    args.dev_status = dev_status;
+    const dim3 block(64 + 32 * plan.epi_warps);
+    cudaError_t e;
+    if (plan.c_is_bf16)
+        e = launch_k(gemm_bf16_kernel<true>, dim3(plan.grid), block, plan.smem_bytes, s, plan.map_a, plan.map_b, plan.map_c, args);
+    else
+        e = launch_k(gemm_bf16_kernel<false>, dim3(plan.grid), block, plan.smem_bytes, s, plan.map_a, plan.map_b, plan.map_c, args);
     ++*launches;
     return e;
 }

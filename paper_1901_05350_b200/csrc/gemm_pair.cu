@@ -7,7 +7,7 @@
 // consumed by four `kind::f16` MMAs of K = 16; the epilogue rounds to bfloat16 and stores through
 // 64-byte-swizzled slabs).  Sums are fp32 in tensor memory in both.
 //
-// Same contract as the single-CTA kernels (gemm_tf32_tcgen05.cu, gemm_bf16_tcgen05.cu); this one is for the shapes whose
+// Same contract as the single-CTA kernels (gemm_cta.cu); this one is for the shapes whose
 // time is set by the K loop (large K and N, many tiles).  With fp32 operands a single CTA must bring
 // 128 + 256 operand rows of 128 bytes into shared memory for every 128 x 256 x 32 block of
 // multiply-adds and read them back out for the tensor core, which saturates the shared memory's
