@@ -194,8 +194,14 @@ struct DepthwisePlan {
     int64_t num_tiles = 0;
     int grid = 0, stages = 0;
     size_t smem_bytes = 0;
+    bool narrow = false;  // planned for bfloat16 storage
 };
-tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const float* x, const ConvGeom& g, DepthwisePlan* plan);
+// `narrow`: x is bfloat16 (narrow storage); the plan then runs through launch_depthwise_tma_narrow, and
+// variant stays -1 where the pipelined kernel has no instance for the shape.
+tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const void* x, const ConvGeom& g, DepthwisePlan* plan, bool narrow = false);
+cudaError_t launch_depthwise_tma_narrow(const DepthwisePlan& plan, const float* f, const float* bias, int act, void* y,
+                                        bool y_is_bf16, const ConvGeom& g, unsigned int* dev_status, cudaStream_t s,
+                                        int64_t* launches);
 cudaError_t launch_depthwise(const DepthwisePlan& plan, const float* x, const float* f, const float* bias, int act,
                              float* y, const ConvGeom& g, unsigned int* dev_status, cudaStream_t s,
                              int64_t* launches);

@@ -24,6 +24,8 @@
 // 'same' padding) into a ring of stages (full / empty mbarriers) while eight compute warps work
 // on the landed tiles from shared memory with the same sliding-row scheme and store float4s
 // straight to global memory.
+#include <cuda_bf16.h>
+
 #include <cstdlib>
 
 #include "common.cuh"
@@ -135,19 +137,49 @@ __global__ void depthwise_generic_kernel(const float* __restrict__ x, const floa
     }
 }
 
-// Bias, activation and store of one thread's R output rows (4 channels each) of the pipelined kernel.
-template <int ACT, int R>
-__device__ __forceinline__ void store_rows(const float4 (&acc)[R], const float4 b, float* yp, int64_t row_pitch, int rows) {
+// Bias, activation and store of one thread's R output rows (4 channels each) of the pipelined kernel;
+// `idx` is the element index of the first row's first channel, OUT16 stores bfloat16 (rounded to nearest even).
+template <int ACT, int R, bool OUT16>
+__device__ __forceinline__ void store_rows(const float4 (&acc)[R], const float4 b, void* y, int64_t idx, int64_t row_pitch, int rows) {
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         if (r < rows) {
             float4 v = acc[r];
             v.x = apply_act_t<ACT>(v.x + b.x); v.y = apply_act_t<ACT>(v.y + b.y);
             v.z = apply_act_t<ACT>(v.z + b.z); v.w = apply_act_t<ACT>(v.w + b.w);
-            *reinterpret_cast<float4*>(yp) = v;
+            if (OUT16) {
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+                uint2 o;
+                o.x = *reinterpret_cast<const uint32_t*>(&lo);
+                o.y = *reinterpret_cast<const uint32_t*>(&hi);
+                *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(y) + idx) = o;
+            } else {
+                *reinterpret_cast<float4*>(static_cast<float*>(y) + idx) = v;
+            }
         }
-        yp += row_pitch;
+        idx += row_pitch;
     }
+}
+
+template <int R, bool OUT16>
+__device__ __forceinline__ void store_rows_act(int act, const float4 (&acc)[R], const float4 b, void* y, int64_t idx,
+                                               int64_t row_pitch, int rows) {
+    // the activation is chosen once per tile, not once per value: the kernel is close to issue bound
+    if (act == TFJSB_ACT_RELU6) store_rows<TFJSB_ACT_RELU6, R, OUT16>(acc, b, y, idx, row_pitch, rows);
+    else if (act == TFJSB_ACT_RELU) store_rows<TFJSB_ACT_RELU, R, OUT16>(acc, b, y, idx, row_pitch, rows);
+    else store_rows<TFJSB_ACT_NONE, R, OUT16>(acc, b, y, idx, row_pitch, rows);
+}
+
+// Four consecutive channels of one patch sample as fp32: one 16-byte load, or one 8-byte load of four
+// bfloat16 (each is the upper half of its fp32).
+template <bool NARROW>
+__device__ __forceinline__ float4 ld_quad(const uint8_t* p) {
+    if (NARROW) {
+        const uint2 raw = *reinterpret_cast<const uint2*>(p);
+        return make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u),
+                           __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u));
+    }
+    return *reinterpret_cast<const float4*>(p);
 }
 
 // ---- pipelined kernel ---------------------------------------------------------------------------
@@ -159,25 +191,28 @@ struct DwTiling {
     long long num_tiles;
 };
 
-template <int S, int TW, int R, int D = 1, int CB = DW_CB>
+template <int S, int TW, int R, int D = 1, int CB = DW_CB, bool NARROW = false>
 struct DwTile {
     static constexpr int QUADS = CB / 4;               // threads across a pixel's channels (4 channels each)
     static constexpr int RG = DW_THREADS / QUADS / TW; // row groups of threads: 256 = QUADS x TW x RG
     static constexpr int TH = RG * R;                  // output rows per tile
     static constexpr int TWIN = (TW - 1) * S + 2 * D + 1;  // input patch (D: dilation, taps D pixels apart)
     static constexpr int THIN = (TH - 1) * S + 2 * D + 1;
-    static constexpr int STAGE_FLOATS = THIN * TWIN * CB;
-    static constexpr int STAGE_BYTES = STAGE_FLOATS * 4;
+    static constexpr int EB = NARROW ? 2 : 4;                    // bytes per stored value (bfloat16 or fp32)
+    static constexpr int STAGE_BYTES = THIN * TWIN * CB * EB;    // what one copy delivers
+    static constexpr int STAGE_STRIDE = (STAGE_BYTES + 127) / 128 * 128;  // pitch of the ring
 };
 
 constexpr int DW_TMA_THREADS = DW_THREADS + 32;  // eight compute warps and the warp that issues the copies
 
-template <int S, int TW, int R, int D = 1, int CB = DW_CB>
+// NARROW: the input is bfloat16 (the patch is copied as such and widened by the compute threads; filter and bias
+// stay fp32, the sums are fp32 in the same order) and the output is bfloat16 or, with y_f32, fp32.
+template <int S, int TW, int R, int D = 1, int CB = DW_CB, bool NARROW = false>
 __global__ void __launch_bounds__(DW_TMA_THREADS, 2)
 depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* __restrict__ f,
-                        const float* __restrict__ bias, int act, float* __restrict__ y, ConvGeom g, DwTiling t,
+                        const float* __restrict__ bias, int act, void* __restrict__ y, int y_f32, ConvGeom g, DwTiling t,
                         unsigned int* dev_status) {
-    using T = DwTile<S, TW, R, D, CB>;
+    using T = DwTile<S, TW, R, D, CB, NARROW>;
     extern __shared__ uint8_t dw_smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[DW_MAX_STAGES];   // copy landed (1 arrival + bytes)
     __shared__ __align__(8) uint64_t bar_empty[DW_MAX_STAGES];  // the eight compute warps are done with the stage
@@ -186,7 +221,7 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
     volatile int* abort_flag = &abort_flag_s;
 
     const uint32_t smem_base = (ptx::smem_u32(dw_smem_raw) + 127u) & ~127u;
-    const float* smem_f = reinterpret_cast<const float*>(dw_smem_raw + (smem_base - ptx::smem_u32(dw_smem_raw)));
+    const uint8_t* smem_p = dw_smem_raw + (smem_base - ptx::smem_u32(dw_smem_raw));
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
 
@@ -228,7 +263,7 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
                 tile_info[slot] = make_int4(cb, tx, ty, n);
                 const uint32_t bar = ptx::smem_u32(&bar_full[slot]);
                 ptx::mbar_arrive_expect_tx(bar, (uint32_t)T::STAGE_BYTES);
-                ptx::tma_load_4d(smem_base + (uint32_t)slot * (uint32_t)T::STAGE_BYTES, &map_x, bar, cb * CB,
+                ptx::tma_load_4d(smem_base + (uint32_t)slot * (uint32_t)T::STAGE_STRIDE, &map_x, bar, cb * CB,
                                  tx * TW * S - g.pl, ty * T::TH * S - g.pt, n);
                 if (++slot == t.stages) { slot = 0; parity ^= 1u; }
             }
@@ -287,12 +322,15 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
             float4 acc[R];
 #pragma unroll
             for (int r = 0; r < R; ++r) acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-            const float* patch = smem_f + (size_t)slot * T::STAGE_FLOATS + ((rg * R * S) * T::TWIN + col * S) * CB + c4 * 4;
+            // byte offsets into the patch [THIN][TWIN][CB values]
+            const uint8_t* patch = smem_p + (size_t)slot * T::STAGE_STRIDE +
+                                   (size_t)((((rg * R * S) * T::TWIN + col * S) * CB + c4 * 4) * T::EB);
             constexpr int IN_ROWS = (R - 1) * S + 2 * D + 1;
 #pragma unroll
             for (int j = 0; j < IN_ROWS; ++j) {
-                const float* row = patch + j * T::TWIN * CB;
-                const float4 v0 = ld4(row), v1 = ld4(row + D * CB), v2 = ld4(row + 2 * D * CB);
+                const uint8_t* row = patch + j * T::TWIN * CB * T::EB;
+                const float4 v0 = ld_quad<NARROW>(row), v1 = ld_quad<NARROW>(row + D * CB * T::EB),
+                             v2 = ld_quad<NARROW>(row + 2 * D * CB * T::EB);
 #pragma unroll
                 for (int ky = 0; ky < 3; ++ky) {
                     const int d = j - ky * D;
@@ -306,12 +344,10 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
             // the stage has been read: hand it back before the stores go out
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bar_empty[slot]));
-            float* yp = y + (((int64_t)info.w * g.Ho + oy0) * g.Wo + ox) * g.Co + c;
+            const int64_t idx = (((int64_t)info.w * g.Ho + oy0) * g.Wo + ox) * g.Co + c;
             const int rows = g.Ho - oy0;
-            // the activation is chosen once per tile, not once per value: the kernel is close to issue bound
-            if (act == TFJSB_ACT_RELU6) store_rows<TFJSB_ACT_RELU6, R>(acc, b, yp, row_pitch, rows);
-            else if (act == TFJSB_ACT_RELU) store_rows<TFJSB_ACT_RELU, R>(acc, b, yp, row_pitch, rows);
-            else store_rows<TFJSB_ACT_NONE, R>(acc, b, yp, row_pitch, rows);
+            if (NARROW && !y_f32) store_rows_act<R, true>(act, acc, b, y, idx, row_pitch, rows);
+            else store_rows_act<R, false>(act, acc, b, y, idx, row_pitch, rows);
         } else {
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&bar_empty[slot]));
@@ -320,35 +356,81 @@ depthwise3x3_tma_kernel(const __grid_constant__ CUtensorMap map_x, const float* 
     }
 }
 
-// the instances: {stride, tile width, tile height, bytes of a stage, channels per tile}
+// the instances: {stride, tile width, tile height, bytes of a stage, pitch of the ring, channels per tile}
 struct DwVariant {
-    int S, TW, TH, stage_bytes, cb;
+    int S, TW, TH, stage_bytes, stage_stride, cb;
 };
+#define DW_VARIANT(S, TW, R, D, CB, NARROW)                                                       \
+    {S, TW, DwTile<S, TW, R, D, CB, NARROW>::TH, DwTile<S, TW, R, D, CB, NARROW>::STAGE_BYTES,    \
+     DwTile<S, TW, R, D, CB, NARROW>::STAGE_STRIDE, CB}
 constexpr DwVariant kDwVariants[] = {
-    {1, 16, DwTile<1, 16, 4>::TH, DwTile<1, 16, 4>::STAGE_BYTES, DW_CB},  // 0: large stride-1 images
-    {1, 16, DwTile<1, 16, 7>::TH, DwTile<1, 16, 7>::STAGE_BYTES, DW_CB},  // 1: 9..14 output rows in one tile
-    {1, 8, DwTile<1, 8, 2>::TH, DwTile<1, 8, 2>::STAGE_BYTES, DW_CB},     // 2: images up to 8 wide
-    {2, 16, DwTile<2, 16, 2>::TH, DwTile<2, 16, 2>::STAGE_BYTES, DW_CB},  // 3: stride 2
-    {2, 8, DwTile<2, 8, 2>::TH, DwTile<2, 8, 2>::STAGE_BYTES, DW_CB},     // 4: stride 2, outputs up to 8 wide
-    {1, 16, DwTile<1, 16, 4, 2>::TH, DwTile<1, 16, 4, 2>::STAGE_BYTES, DW_CB},  // 5: stride 1, dilation 2
-    {1, 16, DwTile<1, 16, 4, 4>::TH, DwTile<1, 16, 4, 4>::STAGE_BYTES, DW_CB},  // 6: stride 1, dilation 4
+    DW_VARIANT(1, 16, 4, 1, 32, false),   // 0: large stride-1 images
+    DW_VARIANT(1, 16, 7, 1, 32, false),   // 1: 9..14 output rows in one tile
+    DW_VARIANT(1, 8, 2, 1, 32, false),    // 2: images up to 8 wide
+    DW_VARIANT(2, 16, 2, 1, 32, false),   // 3: stride 2
+    DW_VARIANT(2, 8, 2, 1, 32, false),    // 4: stride 2, outputs up to 8 wide
+    DW_VARIANT(1, 16, 4, 2, 32, false),   // 5: stride 1, dilation 2
+    DW_VARIANT(1, 16, 4, 4, 32, false),   // 6: stride 1, dilation 4
     // 64 channels per tile (256-byte lines): half as many box rows for the copy unit per byte moved
-    {1, 16, DwTile<1, 16, 4, 1, 64>::TH, DwTile<1, 16, 4, 1, 64>::STAGE_BYTES, 64},  // 7: as 0
-    {1, 16, DwTile<1, 16, 7, 1, 64>::TH, DwTile<1, 16, 7, 1, 64>::STAGE_BYTES, 64},  // 8: as 1 (two tiles down a 14-row image)
-    {1, 8, DwTile<1, 8, 4, 1, 64>::TH, DwTile<1, 8, 4, 1, 64>::STAGE_BYTES, 64},     // 9: as 2 (a whole 7 x 7 image)
-    {2, 8, DwTile<2, 8, 2, 1, 64>::TH, DwTile<2, 8, 2, 1, 64>::STAGE_BYTES, 64},     // 10: stride 2
+    DW_VARIANT(1, 16, 4, 1, 64, false),   // 7: as 0
+    DW_VARIANT(1, 16, 7, 1, 64, false),   // 8: as 1 (two tiles down a 14-row image)
+    DW_VARIANT(1, 8, 4, 1, 64, false),    // 9: as 2 (a whole 7 x 7 image)
+    DW_VARIANT(2, 8, 2, 1, 64, false),    // 10: stride 2, 8 outputs wide
+    // bfloat16 storage: the same tiles on 2-byte values (64 channels = one 128-byte line), then 32 channels
+    DW_VARIANT(1, 16, 4, 1, 64, true),    // 11
+    DW_VARIANT(1, 16, 7, 1, 64, true),    // 12
+    DW_VARIANT(1, 8, 4, 1, 64, true),     // 13
+    DW_VARIANT(2, 16, 2, 1, 64, true),    // 14
+    DW_VARIANT(2, 8, 2, 1, 64, true),     // 15
+    DW_VARIANT(1, 16, 4, 1, 32, true),    // 16
+    DW_VARIANT(1, 16, 7, 1, 32, true),    // 17
+    DW_VARIANT(1, 8, 2, 1, 32, true),     // 18
+    DW_VARIANT(2, 16, 2, 1, 32, true),    // 19
+    DW_VARIANT(2, 8, 2, 1, 32, true),     // 20
 };
+#undef DW_VARIANT
+constexpr int DW_FIRST_NARROW = 11;
 constexpr int DW_SMEM_BUDGET = 113 * 1024;  // two CTAs per SM
 
-template <int S, int TW, int R, int D = 1, int CB = DW_CB>
-cudaError_t launch_tma_instance(const DepthwisePlan& plan, const float* f, const float* bias, int act, float* y,
+template <int S, int TW, int R, int D = 1, int CB = DW_CB, bool NARROW = false>
+cudaError_t launch_tma_instance(const DepthwisePlan& plan, const float* f, const float* bias, int act, void* y, bool y_f32,
                                 const ConvGeom& g, unsigned int* dev_status, cudaStream_t s) {
-    auto kernel = depthwise3x3_tma_kernel<S, TW, R, D, CB>;
+    auto kernel = depthwise3x3_tma_kernel<S, TW, R, D, CB, NARROW>;
     cudaError_t ae = smem_attr_once(reinterpret_cast<const void*>(kernel), DW_SMEM_BUDGET);
     if (ae != cudaSuccess) return ae;
     DwTiling t{plan.tiles_x, plan.tiles_y, plan.c_blocks, plan.stages, (long long)plan.num_tiles};
-    return launch_k(kernel, dim3(plan.grid), dim3(DW_TMA_THREADS), plan.smem_bytes, s, plan.map_x, f, bias, act, y, g, t,
-                    dev_status);
+    return launch_k(kernel, dim3(plan.grid), dim3(DW_TMA_THREADS), plan.smem_bytes, s, plan.map_x, f, bias, act, y,
+                    y_f32 ? 1 : 0, g, t, dev_status);
+}
+
+cudaError_t launch_tma_variant(const DepthwisePlan& plan, const float* f, const float* bias, int act, void* y, bool y_f32,
+                               const ConvGeom& g, unsigned int* dev_status, cudaStream_t s) {
+#define DW_CASE(V, ...) case V: return launch_tma_instance<__VA_ARGS__>(plan, f, bias, act, y, y_f32, g, dev_status, s)
+    switch (plan.variant) {
+        DW_CASE(0, 1, 16, 4, 1, 32, false);
+        DW_CASE(1, 1, 16, 7, 1, 32, false);
+        DW_CASE(2, 1, 8, 2, 1, 32, false);
+        DW_CASE(3, 2, 16, 2, 1, 32, false);
+        DW_CASE(4, 2, 8, 2, 1, 32, false);
+        DW_CASE(5, 1, 16, 4, 2, 32, false);
+        DW_CASE(6, 1, 16, 4, 4, 32, false);
+        DW_CASE(7, 1, 16, 4, 1, 64, false);
+        DW_CASE(8, 1, 16, 7, 1, 64, false);
+        DW_CASE(9, 1, 8, 4, 1, 64, false);
+        DW_CASE(10, 2, 8, 2, 1, 64, false);
+        DW_CASE(11, 1, 16, 4, 1, 64, true);
+        DW_CASE(12, 1, 16, 7, 1, 64, true);
+        DW_CASE(13, 1, 8, 4, 1, 64, true);
+        DW_CASE(14, 2, 16, 2, 1, 64, true);
+        DW_CASE(15, 2, 8, 2, 1, 64, true);
+        DW_CASE(16, 1, 16, 4, 1, 32, true);
+        DW_CASE(17, 1, 16, 7, 1, 32, true);
+        DW_CASE(18, 1, 8, 2, 1, 32, true);
+        DW_CASE(19, 2, 16, 2, 1, 32, true);
+        DW_CASE(20, 2, 8, 2, 1, 32, true);
+        default: return cudaErrorInvalidValue;
+    }
+#undef DW_CASE
 }
 
 int pow2_at_most(int v, int cap) {
@@ -359,12 +441,14 @@ int pow2_at_most(int v, int cap) {
 
 }  // namespace
 
-tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const float* x, const ConvGeom& g, DepthwisePlan* plan) {
+tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const void* x, const ConvGeom& g, DepthwisePlan* plan, bool narrow) {
     plan->variant = -1;
+    plan->narrow = narrow;
     const bool dilated = g.dh == g.dw && (g.dh == 2 || g.dh == 4) && g.sh == 1;  // atrous layers
     const bool shape_ok = g.fh == 3 && g.fw == 3 && g.mult == 1 && ((g.dh == 1 && g.dw == 1) || dilated) && g.sh == g.sw &&
                           (g.sh == 1 || g.sh == 2) && (g.C % 4 == 0) && g.C >= DW_CB;
     if (!shape_ok || !ctx->encode_tiled) return TFJSB_OK;
+    if (narrow && (dilated || g.C % 8 != 0)) return TFJSB_OK;  // 16-byte row pitches; no dilated instances in this format
     int v;
     if (dilated) v = g.dh == 2 ? 5 : 6;
     else if (g.sh == 1) v = g.Wo <= 8 ? 2 : ((g.Ho > 8 && g.Ho <= 14) ? 1 : 0);
@@ -378,13 +462,20 @@ tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const float* x, const ConvGeom& g, D
         if (g.sh == 1) v = v == 0 ? 7 : (v == 1 ? 8 : 9);
         else if ((g.Wo + 7) / 8 * 8 < (g.Wo + 15) / 16 * 16) v = 10;
     }
+    if (narrow) {
+        const bool wide8 = g.Wo <= 8 || (g.Wo + 7) / 8 * 8 < (g.Wo + 15) / 16 * 16;  // stride 2: the 8-wide tile wastes fewer columns
+        const int base = g.sh == 1 ? (g.Wo <= 8 ? 2 : ((g.Ho > 8 && g.Ho <= 14) ? 1 : 0)) : (wide8 ? 4 : 3);
+        v = DW_FIRST_NARROW + (g.C % 64 == 0 ? 0 : 5) + base;
+    }
     const DwVariant& d = kDwVariants[v];
+    const cuuint64_t eb = narrow ? 2u : 4u;
     const int twin = (d.TW - 1) * d.S + 2 * g.dw + 1, thin = (d.TH - 1) * d.S + 2 * g.dh + 1;
     cuuint64_t dims[4] = {(cuuint64_t)g.C, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
-    cuuint64_t strides[3] = {(cuuint64_t)g.C * 4u, (cuuint64_t)g.W * g.C * 4u, (cuuint64_t)g.H * g.W * g.C * 4u};
+    cuuint64_t strides[3] = {(cuuint64_t)g.C * eb, (cuuint64_t)g.W * g.C * eb, (cuuint64_t)g.H * g.W * g.C * eb};
     cuuint32_t box[4] = {(cuuint32_t)d.cb, (cuuint32_t)twin, (cuuint32_t)thin, 1u};
     cuuint32_t elem[4] = {1u, 1u, 1u, 1u};
-    CUresult r = ctx->encode_tiled(&plan->map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(x), dims, strides,
+    CUresult r = ctx->encode_tiled(&plan->map_x, narrow ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4,
+                                   const_cast<void*>(x), dims, strides,
                                    box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS)
@@ -395,11 +486,11 @@ tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const float* x, const ConvGeom& g, D
     plan->c_blocks = (g.C + d.cb - 1) / d.cb;
     plan->num_tiles = (int64_t)plan->tiles_x * plan->tiles_y * plan->c_blocks * g.N;
     if (plan->num_tiles > 0x7fffffff) return TFJSB_OK;  // tile indices are 32-bit in the kernel
-    int stages = (DW_SMEM_BUDGET - 256) / d.stage_bytes;
+    int stages = (DW_SMEM_BUDGET - 256) / d.stage_stride;
     if (stages > DW_MAX_STAGES) stages = DW_MAX_STAGES;
     if (stages < 2) return TFJSB_OK;  // cannot happen with the instances above
     plan->stages = stages;
-    plan->smem_bytes = (size_t)stages * d.stage_bytes + 128;
+    plan->smem_bytes = (size_t)stages * d.stage_stride + 128;
     const int64_t max_grid = (int64_t)ctx->sm_count * 2;
     plan->grid = (int)(plan->num_tiles < max_grid ? plan->num_tiles : max_grid);
     // A CTA walks tiles first, first + grid, ...; the channel block is the fastest tile coordinate, so a grid
@@ -422,20 +513,8 @@ cudaError_t launch_depthwise(const DepthwisePlan& plan, const float* x, const fl
     const int64_t n_out = g.N * g.Ho * g.Wo * g.Co;
     if (n_out == 0) return cudaSuccess;
     if (plan.variant >= 0) {
-        cudaError_t e;
-        switch (plan.variant) {
-            case 0: e = launch_tma_instance<1, 16, 4>(plan, f, bias, act, y, g, dev_status, s); break;
-            case 1: e = launch_tma_instance<1, 16, 7>(plan, f, bias, act, y, g, dev_status, s); break;
-            case 2: e = launch_tma_instance<1, 8, 2>(plan, f, bias, act, y, g, dev_status, s); break;
-            case 3: e = launch_tma_instance<2, 16, 2>(plan, f, bias, act, y, g, dev_status, s); break;
-            case 4: e = launch_tma_instance<2, 8, 2>(plan, f, bias, act, y, g, dev_status, s); break;
-            case 5: e = launch_tma_instance<1, 16, 4, 2>(plan, f, bias, act, y, g, dev_status, s); break;
-            case 7: e = launch_tma_instance<1, 16, 4, 1, 64>(plan, f, bias, act, y, g, dev_status, s); break;
-            case 8: e = launch_tma_instance<1, 16, 7, 1, 64>(plan, f, bias, act, y, g, dev_status, s); break;
-            case 9: e = launch_tma_instance<1, 8, 4, 1, 64>(plan, f, bias, act, y, g, dev_status, s); break;
-            case 10: e = launch_tma_instance<2, 8, 2, 1, 64>(plan, f, bias, act, y, g, dev_status, s); break;
-            default: e = launch_tma_instance<1, 16, 4, 4>(plan, f, bias, act, y, g, dev_status, s); break;
-        }
+        if (plan.narrow) return cudaErrorInvalidValue;  // a plan made for bfloat16 storage: launch_depthwise_tma_narrow
+        cudaError_t e = launch_tma_variant(plan, f, bias, act, y, true, g, dev_status, s);
         ++*launches;
         return e;
     }
@@ -470,6 +549,16 @@ cudaError_t launch_depthwise(const DepthwisePlan& plan, const float* x, const fl
     depthwise_generic_kernel<<<(unsigned)blocks, DW_THREADS, 0, s>>>(x, f, bias, act, y, g, n_out);
     ++*launches;
     return cudaGetLastError();
+}
+
+cudaError_t launch_depthwise_tma_narrow(const DepthwisePlan& plan, const float* f, const float* bias, int act, void* y,
+                                        bool y_is_bf16, const ConvGeom& g, unsigned int* dev_status, cudaStream_t s,
+                                        int64_t* launches) {
+    if (g.N * g.Ho * g.Wo * g.Co == 0) return cudaSuccess;
+    if (plan.variant < DW_FIRST_NARROW || !plan.narrow) return cudaErrorInvalidValue;
+    cudaError_t e = launch_tma_variant(plan, f, bias, act, y, !y_is_bf16, g, dev_status, s);
+    ++*launches;
+    return e;
 }
 
 }  // namespace tfjsb

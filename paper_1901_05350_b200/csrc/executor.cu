@@ -165,6 +165,13 @@ tfjsb_status bind_step(tfjsb_model* m, Step& st, const float* in, float* out) {
         if (rc != TFJSB_OK) return rc;
         st.plan_built = true;
     }
+    if (st.kind == STEP_DEPTHWISE_NARROW && (changed || !st.plan_built)) {
+        // the pipelined kernel where it has an instance for the shape (variant >= 0), else the register kernel
+        tfjsb_status rc = depthwise_plan(m->ctx, in, st.g, &st.dw_plan, !st.in_f32);
+        if (rc != TFJSB_OK) return rc;
+        if (st.in_f32) st.dw_plan.variant = -1;
+        st.plan_built = true;
+    }
     return TFJSB_OK;
 }
 
@@ -239,6 +246,9 @@ cudaError_t launch_step(tfjsb_model* m, const Step& st, cudaStream_t s) {
             return launch_conv_narrow(st.in, st.in_f32, st.filter, st.bias, st.act, st.out, st.out_bf16, st.g, s,
                                       &ctx->launches);
         case STEP_DEPTHWISE_NARROW:
+            if (st.dw_plan.variant >= 0)
+                return launch_depthwise_tma_narrow(st.dw_plan, st.filter, st.bias, st.act, st.out, st.out_bf16, st.g, ctx->dev_status, s,
+                                                   &ctx->launches);
             return launch_depthwise_narrow(st.in, st.filter, st.bias, st.act, st.out, st.out_bf16, st.g, s, &ctx->launches);
         case STEP_POOL_NARROW:
             return launch_avg_pool_global_narrow(st.in, st.out, st.out_bf16, st.g.N, st.g.H * st.g.W, st.g.C, s,
@@ -879,7 +889,7 @@ tfjsb_status tfjsb_model_layer_kernel(tfjsb_model* m, int layer, char* name, int
         case STEP_SOFTMAX: k = "softmax_rows_kernel"; break;
         case STEP_GEMM_NARROW: k = st.plan16.pair ? "gemm_pair_kernel<true>" : "gemm_bf16_kernel"; break;
         case STEP_CONV_NARROW: k = st.conv_patch ? "dwpw_fused_kernel<true, true>" : "conv_narrow_kernel"; break;
-        case STEP_DEPTHWISE_NARROW: k = "depthwise3x3_narrow_kernel"; break;
+        case STEP_DEPTHWISE_NARROW: k = st.dw_plan.variant >= 0 ? "depthwise3x3_tma_kernel" : "depthwise3x3_narrow_kernel"; break;
         case STEP_POOL_NARROW: k = "avg_pool_global_narrow_kernel"; break;
     }
     snprintf(name, (size_t)name_len, "%s", k);

@@ -98,6 +98,13 @@ DW_CASES = [
     (2, 29, 31, 32, 3, 3, 1, (2, 2), "same", (1, 1)),     # pipelined kernel: stride 2, odd sizes
     (1, 14, 14, 160, 3, 3, 1, (2, 2), "same", (1, 1)),    # pipelined kernel: stride 2, narrow output
     (1, 9, 40, 32, 3, 3, 1, (1, 1), "valid", (1, 1)),     # pipelined kernel: 'valid' (no padding offset)
+    # the 64-channel instances of the pipelined kernel (channel count a multiple of 64)
+    (2, 21, 37, 128, 3, 3, 1, (1, 1), "same", (1, 1)),    # large stride-1 images: ragged tiles both ways, two channel blocks
+    (3, 13, 20, 128, 3, 3, 1, (1, 1), "same", (1, 1)),    # 9..14 rows: two tiles down, two across, ragged
+    (3, 7, 7, 192, 3, 3, 1, (1, 1), "same", (1, 1)),      # whole 7 x 7 image per tile, three channel blocks
+    (2, 11, 6, 64, 3, 3, 1, (1, 1), "same", (1, 1)),      # narrow image taller than one tile
+    (2, 29, 47, 64, 3, 3, 1, (2, 2), "same", (1, 1)),     # stride 2, 8-wide tiles (24 outputs across), odd sizes
+    (1, 33, 50, 128, 3, 3, 1, (2, 2), "valid", (1, 1)),   # stride 2, 'valid', 8-wide tiles
     (5, 33, 18, 36, 3, 3, 1, (2, 2), "valid", (1, 1)),
     (3, 13, 11, 24, 3, 3, 1, (1, 1), "same", (1, 1)),     # channel quads not a power of two, ragged rows
     (2, 15, 9, 8, 3, 3, 1, (2, 2), "same", (1, 1)),       # odd sizes at stride 2 (symmetric padding)

@@ -334,6 +334,71 @@ def test_fused_depthwise_pointwise_block_narrow(ctx, oracle, case):
     model.close()
 
 
+NARROW_DEPTHWISE = [
+    # N, H, W, C, stride: one case per instance of the pipelined depthwise kernel in the narrow format
+    (2, 21, 37, 128, 1),   # 64-channel tiles, large stride-1 image, ragged tiles both ways
+    (3, 13, 20, 64, 1),    # 9..14 rows: two tiles down
+    (3, 7, 7, 192, 1),     # whole 7 x 7 image per tile, three channel blocks
+    (2, 11, 6, 64, 1),     # narrow image taller than one tile
+    (2, 29, 47, 64, 2),    # stride 2, 8-wide tiles
+    (1, 40, 61, 128, 2),   # stride 2, 16-wide tiles
+    (2, 21, 37, 40, 1),    # 32-channel tiles (channel count not a multiple of 64), partial channel block
+    (3, 13, 20, 96, 1),
+    (3, 7, 7, 40, 1),
+    (2, 29, 47, 32, 2),
+    (1, 40, 61, 48, 2),
+]
+
+
+@pytest.mark.parametrize("case", NARROW_DEPTHWISE)
+def test_depthwise_pipelined_kernel_narrow(ctx, oracle, case):
+    """conv 3x3 -> depthwise 3x3 -> global pool with bfloat16 storage; the depthwise layer runs on the bulk-copy
+    pipelined kernel: bit for bit on small integers, and on random values against the oracle's depthwise layer
+    applied to the GPU's own first-layer output (fp32 sums in another order, then one rounding to bfloat16)."""
+    N, H, W, C, stride = case
+    L = si.Layer
+
+    def build(seed, integers):
+        layers = [L(kind="conv2d", filter_hw=(3, 3), strides=(1, 1), pad="same", act="relu6", out_channels=C, name="stem"),
+                  L(kind="depthwise_conv2d", filter_hw=(3, 3), strides=(stride, stride), pad="same", act="relu6", out_channels=1, name="dw"),
+                  L(kind="global_avg_pool", name="pool")]
+        if integers:
+            x = si.small_integers(seed, 0, (N, H, W, 3), -2, 2)
+            layers[0].filter = si.small_integers(seed, 1, (3, 3, 3, C), -1, 1)
+            layers[0].bias = si.small_integers(seed, 2, (C,), -1, 1)
+            layers[1].filter = si.small_integers(seed, 3, (3, 3, C, 1), -2, 2)
+            layers[1].bias = si.small_integers(seed, 4, (C,), -2, 2)
+        else:
+            x = si.uniform(seed, 0, (N, H, W, 3), -1, 1)
+            si.make_model_weights(layers, 3, seed)
+        return x, layers
+
+    x, layers = build(630, True)
+    want = oracle.run_model(layers, x, keep_all=True, storage="bf16")
+    assert all(np.array_equal(a, b) for a, b in zip(want[:2], oracle.run_model(layers, x, keep_all=True)[:2]))
+    model = narrow_model(ctx, layers, x.shape)
+    model.set_keep_all(True)
+    model.run(dev(x))
+    ctx.check_device_status()
+    assert model.layer_kernels()[1] == "depthwise3x3_tma_kernel"
+    assert same_bits(host(model.layer_output_f32(1)), want[1])
+    model.close()
+
+    x, layers = build(631, False)
+    model = narrow_model(ctx, layers, x.shape)
+    model.set_keep_all(True)
+    model.run(dev(x))
+    ctx.check_device_status()
+    stem = host(model.layer_output_f32(0))
+    got = host(model.layer_output_f32(1))
+    alone = oracle.round_bf16(oracle.run_model(layers[1:2], stem, keep_all=True, storage="bf16")[0])
+    assert got.shape == alone.shape
+    assert np.all((got.view(np.uint32) & 0xFFFF) == 0)
+    steps = bf16_steps(got, alone)
+    assert steps.max() <= 1 and np.count_nonzero(steps) <= 0.01 * steps.size
+    model.close()
+
+
 def test_config3_mobilenet_025_128_narrow(ctx, oracle):
     x, layers = si.config_mobilenet(0.25, 128, 1, seed=si.CONFIG_SEEDS["mobilenet_025_128"])
     want = oracle.run_model(layers, x, keep_all=True, storage="bf16")
