@@ -364,32 +364,31 @@ struct DwVariant {
     {S, TW, DwTile<S, TW, R, D, CB, NARROW>::TH, DwTile<S, TW, R, D, CB, NARROW>::STAGE_BYTES,    \
      DwTile<S, TW, R, D, CB, NARROW>::STAGE_STRIDE, CB}
 constexpr DwVariant kDwVariants[] = {
-    DW_VARIANT(1, 16, 4, 1, 32, false),   // 0: large stride-1 images
-    DW_VARIANT(1, 16, 7, 1, 32, false),   // 1: 9..14 output rows in one tile
-    DW_VARIANT(1, 8, 2, 1, 32, false),    // 2: images up to 8 wide
-    DW_VARIANT(2, 16, 2, 1, 32, false),   // 3: stride 2
-    DW_VARIANT(2, 8, 2, 1, 32, false),    // 4: stride 2, outputs up to 8 wide
-    DW_VARIANT(1, 16, 4, 2, 32, false),   // 5: stride 1, dilation 2
-    DW_VARIANT(1, 16, 4, 4, 32, false),   // 6: stride 1, dilation 4
-    // 64 channels per tile (256-byte lines): half as many box rows for the copy unit per byte moved
-    DW_VARIANT(1, 16, 4, 1, 64, false),   // 7: as 0
-    DW_VARIANT(1, 16, 7, 1, 64, false),   // 8: as 1 (two tiles down a 14-row image)
-    DW_VARIANT(1, 8, 4, 1, 64, false),    // 9: as 2 (a whole 7 x 7 image)
-    DW_VARIANT(2, 8, 2, 1, 64, false),    // 10: stride 2, 8 outputs wide
-    // bfloat16 storage: the same tiles on 2-byte values (64 channels = one 128-byte line), then 32 channels
-    DW_VARIANT(1, 16, 4, 1, 64, true),    // 11
-    DW_VARIANT(1, 16, 7, 1, 64, true),    // 12
-    DW_VARIANT(1, 8, 4, 1, 64, true),     // 13
-    DW_VARIANT(2, 16, 2, 1, 64, true),    // 14
-    DW_VARIANT(2, 8, 2, 1, 64, true),     // 15
-    DW_VARIANT(1, 16, 4, 1, 32, true),    // 16
-    DW_VARIANT(1, 16, 7, 1, 32, true),    // 17
-    DW_VARIANT(1, 8, 2, 1, 32, true),     // 18
-    DW_VARIANT(2, 16, 2, 1, 32, true),    // 19
-    DW_VARIANT(2, 8, 2, 1, 32, true),     // 20
+    // fp32, 32 channels per tile.  Seven rows per thread for every stride-1 image wider than 8 (seven divides the
+    // heights of the usual networks, and against four rows per thread it measured [128,56,56,128] 84.0 -> 77.2 us,
+    // [128,28,28,256] 41.5 -> 39.2 us, [128,112,112,32] no change)
+    DW_VARIANT(1, 16, 7, 1, 32, false),   // 0: stride 1
+    DW_VARIANT(1, 8, 2, 1, 32, false),    // 1: stride 1, images up to 8 wide
+    DW_VARIANT(2, 16, 2, 1, 32, false),   // 2: stride 2
+    DW_VARIANT(2, 8, 2, 1, 32, false),    // 3: stride 2, 8 outputs wide
+    DW_VARIANT(1, 16, 4, 2, 32, false),   // 4: stride 1, dilation 2
+    DW_VARIANT(1, 16, 4, 4, 32, false),   // 5: stride 1, dilation 4
+    // fp32, 64 channels per tile (256-byte lines): half as many box rows for the copy unit per byte moved
+    DW_VARIANT(1, 16, 7, 1, 64, false),   // 6: stride 1
+    DW_VARIANT(1, 8, 4, 1, 64, false),    // 7: stride 1, images up to 8 wide (a whole 7 x 7 image per tile)
+    DW_VARIANT(2, 8, 2, 1, 64, false),    // 8: stride 2, 8 outputs wide
+    // bfloat16 storage: the same tiles on 2-byte values, 64 channels (one 128-byte line) then 32
+    DW_VARIANT(1, 16, 7, 1, 64, true),    // 9
+    DW_VARIANT(1, 8, 4, 1, 64, true),     // 10
+    DW_VARIANT(2, 16, 2, 1, 64, true),    // 11
+    DW_VARIANT(2, 8, 2, 1, 64, true),     // 12
+    DW_VARIANT(1, 16, 7, 1, 32, true),    // 13
+    DW_VARIANT(1, 8, 2, 1, 32, true),     // 14
+    DW_VARIANT(2, 16, 2, 1, 32, true),    // 15
+    DW_VARIANT(2, 8, 2, 1, 32, true),     // 16
 };
 #undef DW_VARIANT
-constexpr int DW_FIRST_NARROW = 11;
+constexpr int DW_FIRST_NARROW = 9;
 constexpr int DW_SMEM_BUDGET = 113 * 1024;  // two CTAs per SM
 
 template <int S, int TW, int R, int D = 1, int CB = DW_CB, bool NARROW = false>
@@ -407,27 +406,23 @@ cudaError_t launch_tma_variant(const DepthwisePlan& plan, const float* f, const 
                                const ConvGeom& g, unsigned int* dev_status, cudaStream_t s) {
 #define DW_CASE(V, ...) case V: return launch_tma_instance<__VA_ARGS__>(plan, f, bias, act, y, y_f32, g, dev_status, s)
     switch (plan.variant) {
-        DW_CASE(0, 1, 16, 4, 1, 32, false);
-        DW_CASE(1, 1, 16, 7, 1, 32, false);
-        DW_CASE(2, 1, 8, 2, 1, 32, false);
-        DW_CASE(3, 2, 16, 2, 1, 32, false);
-        DW_CASE(4, 2, 8, 2, 1, 32, false);
-        DW_CASE(5, 1, 16, 4, 2, 32, false);
-        DW_CASE(6, 1, 16, 4, 4, 32, false);
-        DW_CASE(7, 1, 16, 4, 1, 64, false);
-        DW_CASE(8, 1, 16, 7, 1, 64, false);
-        DW_CASE(9, 1, 8, 4, 1, 64, false);
-        DW_CASE(10, 2, 8, 2, 1, 64, false);
-        DW_CASE(11, 1, 16, 4, 1, 64, true);
-        DW_CASE(12, 1, 16, 7, 1, 64, true);
-        DW_CASE(13, 1, 8, 4, 1, 64, true);
-        DW_CASE(14, 2, 16, 2, 1, 64, true);
-        DW_CASE(15, 2, 8, 2, 1, 64, true);
-        DW_CASE(16, 1, 16, 4, 1, 32, true);
-        DW_CASE(17, 1, 16, 7, 1, 32, true);
-        DW_CASE(18, 1, 8, 2, 1, 32, true);
-        DW_CASE(19, 2, 16, 2, 1, 32, true);
-        DW_CASE(20, 2, 8, 2, 1, 32, true);
+        DW_CASE(0, 1, 16, 7, 1, 32, false);
+        DW_CASE(1, 1, 8, 2, 1, 32, false);
+        DW_CASE(2, 2, 16, 2, 1, 32, false);
+        DW_CASE(3, 2, 8, 2, 1, 32, false);
+        DW_CASE(4, 1, 16, 4, 2, 32, false);
+        DW_CASE(5, 1, 16, 4, 4, 32, false);
+        DW_CASE(6, 1, 16, 7, 1, 64, false);
+        DW_CASE(7, 1, 8, 4, 1, 64, false);
+        DW_CASE(8, 2, 8, 2, 1, 64, false);
+        DW_CASE(9, 1, 16, 7, 1, 64, true);
+        DW_CASE(10, 1, 8, 4, 1, 64, true);
+        DW_CASE(11, 2, 16, 2, 1, 64, true);
+        DW_CASE(12, 2, 8, 2, 1, 64, true);
+        DW_CASE(13, 1, 16, 7, 1, 32, true);
+        DW_CASE(14, 1, 8, 2, 1, 32, true);
+        DW_CASE(15, 2, 16, 2, 1, 32, true);
+        DW_CASE(16, 2, 8, 2, 1, 32, true);
         default: return cudaErrorInvalidValue;
     }
 #undef DW_CASE
@@ -449,23 +444,21 @@ tfjsb_status depthwise_plan(tfjsb_ctx* ctx, const void* x, const ConvGeom& g, De
                           (g.sh == 1 || g.sh == 2) && (g.C % 4 == 0) && g.C >= DW_CB;
     if (!shape_ok || !ctx->encode_tiled) return TFJSB_OK;
     if (narrow && (dilated || g.C % 8 != 0)) return TFJSB_OK;  // 16-byte row pitches; no dilated instances in this format
+    // the 8-wide stride-2 tile where it wastes fewer columns than the 16-wide one
+    const bool wide8 = g.Wo <= 8 || (g.Wo + 7) / 8 * 8 < (g.Wo + 15) / 16 * 16;
     int v;
-    if (dilated) v = g.dh == 2 ? 5 : 6;
-    else if (g.sh == 1) v = g.Wo <= 8 ? 2 : ((g.Ho > 8 && g.Ho <= 14) ? 1 : 0);
-    else v = g.Wo <= 8 ? 4 : 3;
-    static const bool wide_off = std::getenv("TFJSB_DW_CB32") != nullptr;
-    // 64-channel tiles where the channel count allows.  Measured at batch 128: [112,112,64] stride 2
-    // 90.1 -> 86.9 us, [7,7,1024] 19.5 -> 15.4 us, the 14 x 14 x 512 layers unchanged; the stride-2 form is
-    // 8 outputs wide, so it is taken only where that wastes fewer columns than the 16-wide 32-channel one
-    // ([28,28,256] stride 2 ran 27.3 -> 29.1 us with it).
-    if (!dilated && g.C % 64 == 0 && !wide_off) {
-        if (g.sh == 1) v = v == 0 ? 7 : (v == 1 ? 8 : 9);
-        else if ((g.Wo + 7) / 8 * 8 < (g.Wo + 15) / 16 * 16) v = 10;
-    }
-    if (narrow) {
-        const bool wide8 = g.Wo <= 8 || (g.Wo + 7) / 8 * 8 < (g.Wo + 15) / 16 * 16;  // stride 2: the 8-wide tile wastes fewer columns
-        const int base = g.sh == 1 ? (g.Wo <= 8 ? 2 : ((g.Ho > 8 && g.Ho <= 14) ? 1 : 0)) : (wide8 ? 4 : 3);
-        v = DW_FIRST_NARROW + (g.C % 64 == 0 ? 0 : 5) + base;
+    if (dilated) v = g.dh == 2 ? 4 : 5;
+    else if (narrow) v = DW_FIRST_NARROW + (g.C % 64 == 0 ? 0 : 4) + (g.sh == 1 ? (g.Wo <= 8 ? 1 : 0) : (wide8 ? 3 : 2));
+    else {
+        v = g.sh == 1 ? (g.Wo <= 8 ? 1 : 0) : (g.Wo <= 8 ? 3 : 2);
+        // 64-channel tiles where the channel count allows.  Measured at batch 128: [112,112,64] stride 2
+        // 90.1 -> 86.9 us, [7,7,1024] 19.5 -> 15.4 us, the 14 x 14 x 512 layers unchanged; the stride-2 form is
+        // 8 outputs wide, so it is taken only where that wastes fewer columns than the 16-wide 32-channel one
+        // ([28,28,256] stride 2 ran 27.3 -> 29.1 us with it).
+        if (g.C % 64 == 0) {
+            if (g.sh == 1) v = v == 0 ? 6 : 7;
+            else if (wide8) v = 8;
+        }
     }
     const DwVariant& d = kDwVariants[v];
     const cuuint64_t eb = narrow ? 2u : 4u;
