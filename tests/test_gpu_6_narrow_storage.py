@@ -334,6 +334,35 @@ def test_fused_depthwise_pointwise_block_narrow(ctx, oracle, case):
     model.close()
 
 
+def test_depthwise_as_last_layer_narrow_writes_fp32(ctx, oracle):
+    """A bfloat16-storage model hands its result back as fp32: a depthwise layer in last place runs on the
+    pipelined kernel with bfloat16 patches and an fp32 store, without the rounding of a stored activation."""
+    L = si.Layer
+    x = si.small_integers(640, 0, (2, 15, 22, 3), -2, 2)
+    layers = [L(kind="conv2d", filter_hw=(3, 3), strides=(1, 1), pad="same", act="relu6", out_channels=64, name="stem",
+                filter=si.small_integers(640, 1, (3, 3, 3, 64), -1, 1), bias=si.small_integers(640, 2, (64,), -1, 1)),
+              L(kind="depthwise_conv2d", filter_hw=(3, 3), strides=(1, 1), pad="same", act="none", out_channels=1, name="dw",
+                filter=si.small_integers(640, 3, (3, 3, 64, 1), -2, 2), bias=si.small_integers(640, 4, (64,), -2, 2))]
+    want = oracle.run_model(layers, x, keep_all=True, storage="bf16")
+    model = narrow_model(ctx, layers, x.shape)
+    out = host(model.run(dev(x)))
+    ctx.check_device_status()
+    assert model.layer_kernels()[1] == "depthwise3x3_tma_kernel"
+    assert out.dtype == np.float32 and same_bits(out, want[1])
+    # random values: sums that a bfloat16 could not hold come back unrounded
+    x = si.uniform(641, 0, x.shape, -1, 1)
+    si.make_model_weights(layers, 3, 641)
+    model.close()
+    model = narrow_model(ctx, layers, x.shape)
+    model.set_keep_all(True)
+    out = host(model.run(dev(x)))
+    stem = host(model.layer_output_f32(0))
+    alone = oracle.run_model(layers[1:2], stem, keep_all=True, storage="bf16")[0]
+    assert rel_fro(out, alone) <= 1e-6
+    assert np.any((out.view(np.uint32) & 0xFFFF) != 0)
+    model.close()
+
+
 NARROW_DEPTHWISE = [
     # N, H, W, C, stride: one case per instance of the pipelined depthwise kernel in the narrow format
     (2, 21, 37, 128, 1),   # 64-channel tiles, large stride-1 image, ragged tiles both ways
