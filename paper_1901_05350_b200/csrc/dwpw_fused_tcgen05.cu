@@ -72,6 +72,7 @@ struct FusedArgs {
     int patch_bytes, patch_stride;   // bytes of one input patch and pitch of the patch ring
     // small-window convolution mode (CONV): the patch holds (8-1)*sh+fh rows of row_floats floats
     int cin, fw_cin, sh, sw, row_floats, k_total;
+    int rows9;                // 3 x 3 window on 3 channels with even offsets: the rows are read with 8-byte loads
     int koff[32];             // patch offset of im2col column k relative to the pixel's window origin
     const float* dw_filter;   // [3,3,C,1]
     const float* dw_bias;     // [C] or null
@@ -498,6 +499,36 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 }
                 const float* patch = patch_ptr + (size_t)ps * (args.patch_stride / 4) + origin;
                 const uint32_t row_addr = a_base + (uint32_t)as * A_STAGE_BYTES + (uint32_t)p * 128u;
+                if (args.rows9) {
+                    // 3 x 3 window on 3 channels: the nine values a filter row sees lie next to each other in the
+                    // patch, 8-byte aligned, and in im2col order, so a row is four 8-byte loads and one 4-byte load
+                    // (15 loads instead of 27, and a half-warp's 8-byte loads fall on 32 distinct banks)
+                    float v[BLOCK_K];
+#pragma unroll
+                    for (int ky = 0; ky < 3; ++ky) {
+                        const float* rowp = patch + ky * args.row_floats;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float2 t = *reinterpret_cast<const float2*>(rowp + 2 * j);
+                            v[ky * 9 + 2 * j] = t.x;
+                            v[ky * 9 + 2 * j + 1] = t.y;
+                        }
+                        v[ky * 9 + 8] = rowp[8];
+                    }
+#pragma unroll
+                    for (int e = 27; e < BLOCK_K; ++e) v[e] = 0.0f;
+#pragma unroll
+                    for (int h = 0; h < BLOCK_K / 4; ++h) {
+                        if (NARROW) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) v[4 * h + e] = __bfloat162float(__float2bfloat16_rn(v[4 * h + e]));
+                        }
+                        const uint32_t dst = row_addr + (uint32_t)((h ^ (p & 7)) << 4);
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[4 * h]), "f"(v[4 * h + 1]),
+                                     "f"(v[4 * h + 2]), "f"(v[4 * h + 3])
+                                     : "memory");
+                    }
+                } else {
 #pragma unroll
                 for (int h = 0; h < BLOCK_K / 4; ++h) {
                     float v[4];
@@ -509,6 +540,7 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     const uint32_t dst = row_addr + (uint32_t)((h ^ (p & 7)) << 4);
                     asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3])
                                  : "memory");
+                }
                 }
                 fence_async_smem();
                 __syncwarp();
@@ -831,6 +863,8 @@ cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, cons
     a.patch_bytes = plan.patch_bytes; a.patch_stride = plan.patch_stride;
     a.cin = plan.g.C; a.fw_cin = plan.g.fw * plan.g.C; a.sh = plan.g.sh; a.sw = plan.g.sw;
     a.row_floats = plan.row_floats; a.k_total = plan.g.fh * plan.g.fw * plan.g.C;
+    a.rows9 = plan.conv && plan.g.fh == 3 && a.fw_cin == 9 && (a.sw * a.cin) % 2 == 0 && plan.row_floats % 2 == 0 &&
+              !std::getenv("TFJSB_NO_ROWS9");
     for (int k = 0; k < 32; ++k) {
         const int ky = a.fw_cin > 0 ? k / a.fw_cin : 0;
         a.koff[k] = (plan.conv && k < a.k_total) ? ky * plan.row_floats + (k - ky * a.fw_cin) : 0;
