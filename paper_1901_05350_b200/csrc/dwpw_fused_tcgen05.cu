@@ -417,10 +417,25 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         int first_chunk = group;
         // round-robin over tile boundaries: a tile of n_chunks chunks moves every group's first chunk
         const int chunk_shift = EPI_GROUPS - (n_chunks & (EPI_GROUPS - 1));
+        // (image, tile row, tile column) of the CTA's tiles, stepped instead of divided out for every tile: the
+        // eight or sixteen warps of this role walk every tile, and three divisions per tile and warp were a
+        // good part of the instructions the SM issues per tile
+        int n = (int)blockIdx.x / tiles_per_image;
+        int ty = ((int)blockIdx.x - n * tiles_per_image) / args.tiles_x;
+        int tx = (int)blockIdx.x - n * tiles_per_image - ty * args.tiles_x;
+        const int step_n = (int)gridDim.x / tiles_per_image;
+        const int step_rem = (int)gridDim.x - step_n * tiles_per_image;
+        const int step_ty = step_rem / args.tiles_x, step_tx = step_rem - step_ty * args.tiles_x;
+        bool first_pass = true;
         for (int tile = blockIdx.x; tile < args.num_tiles; tile += gridDim.x) {
-            const int n = tile / tiles_per_image;
-            const int rem = tile - n * tiles_per_image;
-            const int ty = rem / args.tiles_x, tx = rem - ty * args.tiles_x;
+            if (!first_pass) {
+                tx += step_tx;
+                if (tx >= args.tiles_x) { tx -= args.tiles_x; ++ty; }
+                ty += step_ty;
+                if (ty >= args.tiles_y) { ty -= args.tiles_y; ++n; }
+                n += step_n;
+            }
+            first_pass = false;
             const bool got = bounded_wait(smem_u32(&bar_acc_full[acc]), acc_phase, abort_flag);
             if (!__all_sync(0xffffffffu, got)) {
                 if (lane == 0 && !*abort_flag) {
