@@ -29,6 +29,11 @@
  *             (valid until the next call on the context).  No CPU fallback exists: with no
  *             usable CUDA device `tfjsb_init` fails with TFJSB_ERR_CUDA.
  *   Threads   A context may be used from one host thread at a time.
+ *   Streams   The kernels are written to have the GPU to themselves: persistent grids sized to all SMs,
+ *             tensor memory and most of an SM's shared memory per CTA.  Enqueue the work of a process on one
+ *             stream at a time, or order the streams with events; kernels of two streams that run side by
+ *             side on the same SMs are not a supported configuration (copies on a second stream are fine:
+ *             `tfjsb_run_model_host_async` does that itself).
  */
 #ifndef TFJSB_H_
 #define TFJSB_H_
