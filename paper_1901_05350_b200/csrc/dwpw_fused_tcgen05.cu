@@ -878,8 +878,7 @@ cudaError_t launch_dwpw_fused(const DwPwPlan& plan, const float* dw_filter, cons
     a.patch_bytes = plan.patch_bytes; a.patch_stride = plan.patch_stride;
     a.cin = plan.g.C; a.fw_cin = plan.g.fw * plan.g.C; a.sh = plan.g.sh; a.sw = plan.g.sw;
     a.row_floats = plan.row_floats; a.k_total = plan.g.fh * plan.g.fw * plan.g.C;
-    a.rows9 = plan.conv && plan.g.fh == 3 && a.fw_cin == 9 && (a.sw * a.cin) % 2 == 0 && plan.row_floats % 2 == 0 &&
-              !std::getenv("TFJSB_NO_ROWS9");
+    a.rows9 = plan.conv && plan.g.fh == 3 && a.fw_cin == 9 && (a.sw * a.cin) % 2 == 0 && plan.row_floats % 2 == 0;
     for (int k = 0; k < 32; ++k) {
         const int ky = a.fw_cin > 0 ? k / a.fw_cin : 0;
         a.koff[k] = (plan.conv && k < a.k_total) ? ky * plan.row_floats + (k - ky * a.fw_cin) : 0;
