@@ -179,9 +179,15 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             mbar_init(smem_u32(&bar_b_full[s]), 1);
             mbar_init(smem_u32(&bar_b_empty[s]), 1);
         }
+        // only the groups that have a chunk of a tile wait for its accumulator and hand it back: with fewer chunks
+        // per tile than groups, the others skip the tile (the groups' first chunks are a permutation of
+        // 0 .. EPI_GROUPS-1 that shifts by the same amount every tile, so the number of takers is constant)
+        int nch = (args.Co + EPI_COLS - 1) / EPI_COLS;
+        if (nch > block_n * args.n_sub / EPI_COLS) nch = block_n * args.n_sub / EPI_COLS;
+        const int epi_arrivals = 4 * (nch < EPI_GROUPS ? nch : EPI_GROUPS);
         for (int s = 0; s < ACCS; ++s) {
             mbar_init(smem_u32(&bar_acc_full[s]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[s]), EPI_WARPS);
+            mbar_init(smem_u32(&bar_acc_empty[s]), (uint32_t)epi_arrivals);
         }
         mbar_init(smem_u32(&bar_drain), 1);
         abort_flag_s = 0;
@@ -436,6 +442,7 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 n += step_n;
             }
             first_pass = false;
+            if (first_chunk < n_chunks) {  // else: no chunk of this tile falls to this group
             const bool got = bounded_wait(smem_u32(&bar_acc_full[acc]), acc_phase, abort_flag);
             if (!__all_sync(0xffffffffu, got)) {
                 if (lane == 0 && !*abort_flag) {
@@ -484,6 +491,7 @@ dwpw_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
+            }
             }
             first_chunk = (first_chunk + chunk_shift) & (EPI_GROUPS - 1);
             if (++acc == args.acc_stages) { acc = 0; acc_phase ^= 1u; }
