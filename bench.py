@@ -621,13 +621,13 @@ def run_ours(args):
 # Reads are cold and equal the layer's input; writes are counted when L2 evicts them, so layers whose output is
 # smaller than L2 under-count their writes.  Keyed by (kernel, launch name); an entry is dropped when its kernel changes.
 TRAFFIC_BYTES_PER_IMAGE = {
-    ("dwpw_fused_kernel<false>", "dw1+pw1"): 4342032, ("dwpw_fused_kernel<false>", "dw3+pw3"): 2805346,
-    ("dwpw_fused_kernel<false>", "dw5+pw5"): 1185136,
-    ("depthwise3x3_tma_kernel", "dw2"): 3846820, ("depthwise3x3_tma_kernel", "dw4"): 1833092,
-    ("depthwise3x3_tma_kernel", "dw6"): 844398, ("depthwise3x3_tma_kernel", "dw7"): 431794,
-    ("depthwise3x3_tma_kernel", "dw8"): 433998, ("depthwise3x3_tma_kernel", "dw9"): 433242,
-    ("depthwise3x3_tma_kernel", "dw10"): 434022, ("depthwise3x3_tma_kernel", "dw11"): 433728,
-    ("depthwise3x3_tma_kernel", "dw12"): 401792, ("depthwise3x3_tma_kernel", "dw13"): 201170,
+    ("dwpw_fused_kernel<false>", "dw1+pw1"): 4340584, ("dwpw_fused_kernel<false>", "dw3+pw3"): 2808422,
+    ("dwpw_fused_kernel<false>", "dw5+pw5"): 1182998,
+    ("depthwise3x3_tma_kernel", "dw2"): 3846712, ("depthwise3x3_tma_kernel", "dw4"): 1830648,
+    ("depthwise3x3_tma_kernel", "dw6"): 843598, ("depthwise3x3_tma_kernel", "dw7"): 431010,
+    ("depthwise3x3_tma_kernel", "dw8"): 432776, ("depthwise3x3_tma_kernel", "dw9"): 432746,
+    ("depthwise3x3_tma_kernel", "dw10"): 432158, ("depthwise3x3_tma_kernel", "dw11"): 432582,
+    ("depthwise3x3_tma_kernel", "dw12"): 401734, ("depthwise3x3_tma_kernel", "dw13"): 201166,
 }
 
 
